@@ -1,0 +1,208 @@
+"""Float64 CPU oracle for ConQuR's orthogonal-Procrustes-update (OPU) hot path.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+library is checked against.  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import it; the product path never does.  It shares no code
+with the CUDA path and imports nothing from the package.
+
+Conventions (row-vector form, as in the paper's Appendix A, "X_hat = X R"):
+activations are the rows of X (n x d); the rotation acts on the right,
+Y = X_tilde R.  The paper's Section 3.3 writes the same thing in column form
+(R x_tilde, C = Z^T X_tilde, R <- U V^T); with R_here = R_paper^T and
+M_here = C_paper^T the update R <- polar(M) below is that update transposed.
+
+What each function follows:
+  normalise_rows      Section 3.3, x_tilde = x / ||x||_2 (also Eq. 1)
+  corner_target       Eq. 2, z = sign(R x) / sqrt(d)
+  fake_quant_sym      Appendix B, Q_sym(x) = Delta * round(x / Delta),
+                      Delta = ||x||_inf / (2^(b-1) - 1)
+  OpuOracle.step      Section 3.3 (cross-covariance Z^T X_tilde) accumulated
+                      across tensors as Section 3.4 allows; objective in the
+                      l1 form of Section 3.2
+  polar_svd           Section 3.3, C = U Sigma V^T, R <- U V^T
+  OpuOracle.update    Section 3.3 / Algorithm 1: R replaced, statistics reset
+
+Readings where the paper is silent (kept identical in the CUDA library):
+  * sign(0) = 0: a zero coordinate adds nothing to the target or objective.
+  * rows with zero or non-finite norm are skipped and counted.
+  * fake-quant: b bits, levels -(2^(b-1)-1)..(2^(b-1)-1), clip ratio 1,
+    round-half-to-even; the quantised row feeds the target and the objective,
+    the unquantised normalised row feeds the cross-covariance.
+  * prior_rel = lam_rel > 0 makes the update polar(M + lam * R_prev) with
+    lam = lam_rel * ||M||_F / sqrt(d) (a proximal Procrustes step, needed only
+    when fewer tokens than dimensions were accumulated; not in the paper).
+
+Pins: tests/test_oracle_pins.py (identities of Sections 3.1-3.3 and Appendix B,
+d = 2 brute force, an independent Newton iteration for the polar factor,
+per-element brute force).  The paper prints no worked numeric example of an
+OPU, so there is no printed value to pin against: parity unpinned by worked
+example; pinned by the identities and brute force above.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def normalise_rows(x):
+    """x_tilde_i = x_i / ||x_i||_2 (Section 3.3).  Returns (x_tilde, used_mask).
+
+    Rows whose norm is zero or not finite are dropped from the statistics
+    (the paper does not define them); their x_tilde row is zero.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    with np.errstate(over="ignore", invalid="ignore"):
+        s = np.sqrt(np.sum(x * x, axis=1))
+    used = np.isfinite(s) & (s > 0.0)
+    xt = np.zeros_like(x)
+    xt[used] = x[used] / s[used, None]
+    return xt, used
+
+
+def sgn(y):
+    """Mathematical sign with sgn(0) = 0 (also for -0.0)."""
+    return np.sign(y) + 0.0
+
+
+def corner_target(y):
+    """Eq. 2: nearest vertex of the hypercube inscribed in the unit sphere."""
+    d = y.shape[-1]
+    return sgn(y) / np.sqrt(d)
+
+
+def fake_quant_sym(y, bits):
+    """Appendix B: per-row symmetric uniform quantiser.
+
+    Returns (Q(y), integer codes q, step Delta per row).  Rows that are all
+    zero get Delta = 0 and codes 0.
+    """
+    y = np.asarray(y, dtype=np.float64)
+    levels = 2 ** (bits - 1) - 1
+    delta = np.max(np.abs(y), axis=-1) / levels
+    safe = np.where(delta > 0.0, delta, 1.0)
+    q = np.rint(y / safe[..., None])          # numpy rint = round half to even
+    q = np.clip(q, -levels, levels)
+    q = np.where(delta[..., None] > 0.0, q, 0.0)
+    return q * delta[..., None], q, delta
+
+
+def polar_svd(m):
+    """Orthogonal polar factor of m via the SVD: m = U S V^T -> U V^T (Section 3.3)."""
+    u, s, vt = np.linalg.svd(np.asarray(m, dtype=np.float64))
+    return u @ vt, s
+
+
+class OpuOracle:
+    """State machine R = OPU(R, X) with accumulate-then-update (Sections 3.3-3.4)."""
+
+    def __init__(self, d, r0=None, quant_bits=0, prior_rel=0.0):
+        self.d = int(d)
+        self.quant_bits = int(quant_bits)
+        self.prior_rel = float(prior_rel)
+        self.R = np.eye(self.d) if r0 is None else np.array(r0, dtype=np.float64)
+        assert self.R.shape == (self.d, self.d)
+        self.reset_stats()
+        self.last_S = None      # sign matrix of the last step (n x d)
+        self.last_Y = None
+        self.last_sigma = None  # singular values seen by the last update
+
+    def reset_stats(self):
+        self.M = np.zeros((self.d, self.d))
+        self.J = 0.0
+        self.N = 0
+        self.n_skipped = 0
+
+    def step(self, x, signs_override=None):
+        """Accumulate one batch with R fixed.
+
+        signs_override (n x d of -1/0/+1), if given, replaces the oracle's own
+        sign decisions in the cross-covariance (used for tie-aware parity:
+        the objective still uses the oracle's own arithmetic).
+        """
+        d = self.d
+        xt, used = normalise_rows(x)                     # Section 3.3
+        y = xt @ self.R                                  # Eq. 1 in row form
+        if self.quant_bits == 0:
+            s = sgn(y)                                   # Eq. 2
+            a = np.abs(y)                                # |y| summed -> l1 objective
+        else:
+            qy, q, delta = fake_quant_sym(y, self.quant_bits)   # Appendix B
+            s = sgn(q)
+            a = np.abs(qy)
+        s[~used] = 0.0
+        a[~used] = 0.0
+        s_used = s if signs_override is None else np.asarray(signs_override, dtype=np.float64)
+        c = s_used / np.sqrt(d)                          # Eq. 2 scale
+        self.M += xt.T @ c                               # Section 3.3 cross-covariance
+        self.J += float(np.sum(a)) / np.sqrt(d)          # Section 3.2 l1 form
+        self.N += int(np.count_nonzero(used))
+        self.n_skipped += int(np.count_nonzero(~used))
+        self.last_S = s
+        self.last_Y = y
+        return self
+
+    def effective_m(self):
+        """M, plus the proximal term lam * R_prev when prior_rel > 0."""
+        if self.prior_rel > 0.0:
+            lam = self.prior_rel * np.linalg.norm(self.M) / np.sqrt(self.d)
+            return self.M + lam * self.R
+        return self.M
+
+    def update(self):
+        """R <- polar(M_eff); statistics reset (Algorithm 1)."""
+        if self.N == 0:
+            raise ValueError("update with no accumulated tokens")
+        m_eff = self.effective_m()
+        r_new, sigma = polar_svd(m_eff)
+        tol = sigma[0] * self.d * np.finfo(np.float64).eps
+        if not (sigma[-1] > tol):
+            raise np.linalg.LinAlgError("cross-covariance is rank deficient: polar factor not unique")
+        self.last_sigma = sigma
+        self.R = r_new
+        self.reset_stats()
+        return self
+
+    # derived quantities of Section 3.2
+    def objective_per_token(self):
+        return self.J / self.N
+
+    def corner_distance(self):
+        """sum_i ||x_tilde_i R - c_i||^2 = 2N - 2J."""
+        return 2.0 * self.N - 2.0 * self.J
+
+
+def corner_distance_direct(x, r):
+    """Left side of the identity of Section 3.2, evaluated literally."""
+    xt, used = normalise_rows(x)
+    y = xt[used] @ np.asarray(r, dtype=np.float64)
+    z = corner_target(y)
+    return float(np.sum((y - z) ** 2))
+
+
+def procrustes_value(r, m):
+    """<R, M>_F = tr(R^T M): the linear objective of the Procrustes subproblem."""
+    return float(np.sum(np.asarray(r, dtype=np.float64) * np.asarray(m, dtype=np.float64)))
+
+
+def run_stream(d, batches, r0, update_every, quant_bits=0, prior_rel=0.0):
+    """Drive an oracle over an iterable of batches; returns (oracle, per-update log)."""
+    orc = OpuOracle(d, r0, quant_bits, prior_rel)
+    log = []
+    for b, x in enumerate(batches):
+        orc.step(x)
+        if (b + 1) % update_every == 0:
+            log.append({"J": orc.J, "N": orc.N, "J_per_token": orc.objective_per_token()})
+            orc.update()
+    return orc, log
+
+
+def run_batched(d, xs, r0s, quant_bits=0, prior_rel=0.0):
+    """Independent problems (one Procrustes problem per head): one step + one update each."""
+    out = []
+    for x, r0 in zip(xs, r0s):
+        orc = OpuOracle(d, r0, quant_bits, prior_rel)
+        orc.step(x)
+        j, n = orc.J, orc.N
+        m = orc.M.copy()
+        orc.update()
+        out.append({"R": orc.R, "J": j, "N": n, "M": m})
+    return out
