@@ -1,0 +1,195 @@
+/*
+ * conqur.h -- C ABI of the ConQuR online rotation-calibration hot path (B200, sm_100a).
+ *
+ * One context holds one orthogonal Procrustes problem of size d (or P independent
+ * problems of size d, the per-head case): the current rotation R (d x d), the
+ * accumulated cross-covariance M (d x d) and the objective sums J, N.
+ *
+ * Row-vector convention (the paper's Appendix A, "X_hat = X R"): activations are
+ * the ROWS of X (n x d, row-major), the rotation acts on the right.  The paper's
+ * Section 3.3 states the same update in column form; with R_here = R_paper^T and
+ * M_here = (Z^T X_tilde)^T the two are the same matrices transposed.
+ *
+ * Memory: every pointer named *_dev is DEVICE memory owned by the caller,
+ * including the workspace.  The library allocates no device memory.  Pointers
+ * without that suffix are HOST memory.  All matrices are dense row-major.
+ *
+ * Ordering: conqur_step / conqur_step_batched / conqur_update only ENQUEUE work on
+ * the context's stream and return; X must stay valid until that work has run.
+ * The conqur_get_* calls synchronise the stream.  A context is not thread-safe.
+ *
+ * Errors: every call returns CONQUR_OK (0) or a negative conqur_status.  Errors
+ * found on the host change nothing.  Conditions found on the device (non-finite
+ * input, Newton-Schulz not converged) are latched in a device status word and
+ * returned by the next synchronising call; conqur_get_stats reports and clears it.
+ */
+#ifndef CONQUR_H_
+#define CONQUR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct conqur_ctx conqur_ctx;
+
+typedef enum {
+  CONQUR_OK = 0,
+  CONQUR_ERR_INVALID_ARG = -1,
+  CONQUR_ERR_WORKSPACE_TOO_SMALL = -2,
+  CONQUR_ERR_NOT_ORTHOGONAL_INPUT = -3,
+  CONQUR_ERR_EMPTY_UPDATE = -4,     /* update with no accumulated tokens */
+  CONQUR_ERR_RANK_DEFICIENT = -5,   /* fewer tokens than dimensions and prior_rel == 0 */
+  CONQUR_ERR_NS_NOT_CONVERGED = -6, /* previous R kept, M not cleared */
+  CONQUR_ERR_NONFINITE_INPUT = -7,  /* a row of X held NaN/Inf (that row was skipped) */
+  CONQUR_ERR_TIMEOUT = -8,          /* a bounded device-side wait expired */
+  CONQUR_ERR_CUDA = -9,
+  CONQUR_ERR_UNSUPPORTED = -10
+} conqur_status;
+
+enum { CONQUR_F32 = 0, CONQUR_BF16 = 1 };            /* storage type of X */
+enum { CONQUR_EXACT_F32 = 0, CONQUR_TC_BF16 = 1 };   /* arithmetic mode */
+
+/*
+ * mode CONQUR_EXACT_F32: fp32 CUDA-core contractions throughout (parity anchor).
+ * mode CONQUR_TC_BF16:   bf16 operands, fp32 accumulation on the tcgen05 tensor
+ *                        cores; fp32 X is rounded to bf16 on the way in; the
+ *                        Newton-Schulz products use a two-term bf16 split of each
+ *                        operand (three tensor-core products per matrix product).
+ */
+typedef struct {
+  uint32_t struct_size;     /* = sizeof(conqur_config) */
+  int32_t  in_dtype;        /* CONQUR_F32 | CONQUR_BF16 */
+  int32_t  mode;            /* CONQUR_EXACT_F32 | CONQUR_TC_BF16 */
+  int32_t  quant_bits;      /* 0: corner target on the rotated row (Eq. 2);
+                               b in 2..8: per-token symmetric b-bit fake-quantisation of the
+                               rotated row first (Appendix B, Q_sym), levels -(2^(b-1)-1)..(2^(b-1)-1),
+                               round half to even */
+  int32_t  ns_steps;        /* Newton-Schulz steps planned before the re-projection loop;
+                               0 = derive from ns_sigma_min_rel */
+  int32_t  ns_max_steps;    /* hard cap on Newton-Schulz steps per update; 0 = default 40 */
+  float    orth_tol;        /* accept R when max|R^T R - I| <= orth_tol; 0 = default 1e-4 */
+  float    prior_rel;       /* lam_rel >= 0: update is polar(M + lam R_prev),
+                               lam = lam_rel * ||M||_F / sqrt(d); 0 = the paper's update */
+  float    ns_sigma_min_rel;/* assumed lower bound on sigma_min(M)/||M||_F used to plan the
+                               polynomial schedule; 0 = default 1e-7 */
+  int64_t  n_max;           /* largest n of any step call (sizes the workspace) */
+  int32_t  batch;           /* P >= 1 independent problems of size d */
+} conqur_config;
+
+typedef struct {
+  uint32_t struct_size;     /* = sizeof(conqur_stats) */
+  int32_t  status;          /* latched device status (a conqur_status), cleared by the call */
+  int32_t  ns_steps_used;   /* Newton-Schulz steps of the last update (max over problems) */
+  int32_t  updates;         /* updates committed so far */
+  float    orth_err;        /* max|X^T X - I| measured when the last update accepted R */
+  float    orth_fro;        /* ||X^T X - I||_F at that point */
+  float    scale;           /* ||M_eff||_F the last update divided by (M without the 1/sqrt(d)) */
+  int64_t  n_skipped;       /* rows skipped (zero or non-finite norm) since init */
+  double   last_J;          /* objective sum and token count consumed by the last update */
+  int64_t  last_N;
+} conqur_stats;
+
+/* Bytes of device workspace conqur_init needs for (d, cfg).  Pure function; 0 on invalid arguments. */
+size_t conqur_workspace_bytes(int32_t d, const conqur_config* cfg);
+
+/*
+ * Create a context: R <- I, M <- 0, J = N = 0 (Algorithm 1 takes the initial
+ * rotations as inputs; use conqur_set_R to supply them).
+ *   out            host: receives the context
+ *   d              feature dimension, >= 2 (tensor-core mode: a multiple of 128)
+ *   cfg            host
+ *   workspace_dev  device, 256-byte aligned, >= conqur_workspace_bytes(d, cfg); owned by the
+ *                  caller, must outlive the context, contents are the library's
+ *   cuda_stream    a cudaStream_t (0 = default stream); all work of this context runs on it
+ */
+int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg,
+                void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+
+/* Release the host object (the workspace stays the caller's). */
+int conqur_destroy(conqur_ctx* ctx);
+
+/*
+ * Replace the rotation(s).  R_dev: device fp32, batch x d x d, row-major, acting as
+ * X_tilde @ R.  Must be orthogonal: max|R^T R - I| <= 1e-3 is checked (synchronises);
+ * otherwise CONQUR_ERR_NOT_ORTHOGONAL_INPUT and the old R is kept.  Does not touch M, J, N.
+ */
+int conqur_set_R(conqur_ctx* ctx, const float* R_dev);
+
+/*
+ * One streamed batch with R fixed (Sections 3.3-3.4: normalise each row, rotate,
+ * take the corner target of Eq. 2 -- after Q_sym when quant_bits > 0 -- and add
+ * this batch's cross-covariance and objective to M, J, N):
+ *   x_tilde_i = x_i / ||x_i||_2 ;  y_i = x_tilde_i R ;  c_i = sgn(y_i)/sqrt(d)
+ *   M += X_tilde^T C ;  J += sum_i ||y_i||_1 / sqrt(d) ;  N += rows used
+ * sgn(0) = 0.  Rows with zero or non-finite norm are skipped and counted.
+ *   X_dev  device, n rows of d elements of cfg.in_dtype, row stride ld elements
+ *          (tensor-core mode: X_dev 16-byte aligned and ld*sizeof(element) a multiple of 16)
+ *   n      1..cfg.n_max (n = 0 is a no-op)
+ * Single-problem contexts only (cfg.batch == 1).
+ */
+int conqur_step(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld);
+
+/*
+ * The per-head form (Section 3.4, "a Procrustes problem per head"): problem p of
+ * cfg.batch reads its n rows at X_dev + p*problem_stride + i*ld (elements), each
+ * row normalised by its own d-slice norm.  problem_stride = d, ld = P*d is the
+ * head-interleaved layout; problem_stride = n*ld is stacked problems.
+ */
+int conqur_step_batched(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld,
+                        int64_t problem_stride);
+
+/*
+ * R <- polar(M_eff) = U V^T of the SVD M_eff = U S V^T (Section 3.3), computed by
+ * Newton-Schulz iterations and accepted only when max|R^T R - I| <= orth_tol;
+ * then M, J, N <- 0 (Algorithm 1 starts every mini-batch with empty statistics).
+ * Host errors: CONQUR_ERR_EMPTY_UPDATE (no step since the last update),
+ * CONQUR_ERR_RANK_DEFICIENT (tokens enqueued < d and prior_rel == 0).
+ * If the iteration does not converge within ns_max_steps the old R and M are kept
+ * and CONQUR_ERR_NS_NOT_CONVERGED is latched.
+ */
+int conqur_update(conqur_ctx* ctx);
+
+/* Copy out the current rotation(s): device fp32 batch x d x d.  Synchronises. */
+int conqur_get_R(conqur_ctx* ctx, float* R_out_dev);
+
+/*
+ * Objective accumulated since the last update, at the R those steps used:
+ * J_sum[p] = sum_i ||y_i||_1/sqrt(d) (Section 3.2: the corner distance is 2N - 2J),
+ * n_tokens[p] = rows used.  Host arrays of cfg.batch entries.  Synchronises.
+ */
+int conqur_get_objective(conqur_ctx* ctx, double* J_sum, int64_t* n_tokens);
+
+/* Cross-covariance accumulated since the last update, including the 1/sqrt(d):
+ * device fp32 batch x d x d.  Synchronises. */
+int conqur_get_M(conqur_ctx* ctx, float* M_out_dev);
+
+/* Overwrite the accumulated cross-covariance (same scaling as conqur_get_M) and the sums:
+ * resume / teacher forcing.  J_sum, n_tokens: host arrays of cfg.batch entries. */
+int conqur_set_M(conqur_ctx* ctx, const float* M_dev, const double* J_sum, const int64_t* n_tokens);
+
+/* Sign decisions of the last conqur_step: device int8, n x d row-major, values -1/0/+1
+ * (0 also for skipped rows).  Single-problem contexts.  Synchronises. */
+int conqur_debug_get_signs(conqur_ctx* ctx, int8_t* S_out_dev);
+
+/* Counters of the last update and the latched device status (cleared).  Synchronises. */
+int conqur_get_stats(conqur_ctx* ctx, conqur_stats* out);
+
+/*
+ * Host-only introspection of the Newton-Schulz plan (no device needed): the odd quintics
+ * p_k(x) = a x + b x^3 + c x^5 an update applies, in order, for a spectrum assumed to lie in
+ * [sigma_min_rel, 1] after scaling (ns_steps > 0 instead plans for exactly that many steps).
+ * abc_out: host, 3*max_steps doubles.  Returns the number of steps written, or a negative status.
+ * No counterpart in the paper, which takes R <- U V^T from an SVD (Section 3.3); the polynomials
+ * are this library's route to the same polar factor.
+ */
+int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out, int32_t max_steps);
+
+const char* conqur_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONQUR_H_ */

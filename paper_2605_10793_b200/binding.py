@@ -1,0 +1,275 @@
+"""Thin ctypes binding of libconqur.so (argument marshalling only).
+
+Function names mirror the C ABI in ``include/conqur.h``.  PyTorch supplies device
+memory and the stream; every step of the path runs in the library's kernels.
+The library is required: there is no fallback if it is missing or no GPU exists.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libconqur.so")
+_lib = None
+
+CONQUR_F32, CONQUR_BF16 = 0, 1
+CONQUR_EXACT_F32, CONQUR_TC_BF16 = 0, 1
+
+EXPORTS = [
+    "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
+    "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
+    "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_strerror",
+]
+
+
+class conqur_config(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("in_dtype", C.c_int32), ("mode", C.c_int32), ("quant_bits", C.c_int32),
+        ("ns_steps", C.c_int32), ("ns_max_steps", C.c_int32), ("orth_tol", C.c_float), ("prior_rel", C.c_float),
+        ("ns_sigma_min_rel", C.c_float), ("n_max", C.c_int64), ("batch", C.c_int32),
+    ]
+
+
+class conqur_stats(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("status", C.c_int32), ("ns_steps_used", C.c_int32), ("updates", C.c_int32),
+        ("orth_err", C.c_float), ("orth_fro", C.c_float), ("scale", C.c_float), ("n_skipped", C.c_int64),
+        ("last_J", C.c_double), ("last_N", C.c_int64),
+    ]
+
+
+class ConqurError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+def load() -> C.CDLL:
+    """Load libconqur.so (built in-tree by paper_2605_10793_b200.build); fail loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2605_10793_b200.build` "
+                           "(the CUDA library is the only implementation; there is no fallback)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int32
+    lib.conqur_workspace_bytes.restype = C.c_size_t
+    lib.conqur_workspace_bytes.argtypes = [i32, C.POINTER(conqur_config)]
+    lib.conqur_init.restype = C.c_int
+    lib.conqur_init.argtypes = [C.POINTER(vp), i32, C.POINTER(conqur_config), vp, C.c_size_t, vp]
+    lib.conqur_destroy.restype = C.c_int
+    lib.conqur_destroy.argtypes = [vp]
+    lib.conqur_set_R.restype = C.c_int
+    lib.conqur_set_R.argtypes = [vp, vp]
+    lib.conqur_step.restype = C.c_int
+    lib.conqur_step.argtypes = [vp, vp, i64, i64]
+    lib.conqur_step_batched.restype = C.c_int
+    lib.conqur_step_batched.argtypes = [vp, vp, i64, i64, i64]
+    lib.conqur_update.restype = C.c_int
+    lib.conqur_update.argtypes = [vp]
+    lib.conqur_get_R.restype = C.c_int
+    lib.conqur_get_R.argtypes = [vp, vp]
+    lib.conqur_get_objective.restype = C.c_int
+    lib.conqur_get_objective.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.conqur_get_M.restype = C.c_int
+    lib.conqur_get_M.argtypes = [vp, vp]
+    lib.conqur_set_M.restype = C.c_int
+    lib.conqur_set_M.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.conqur_debug_get_signs.restype = C.c_int
+    lib.conqur_debug_get_signs.argtypes = [vp, vp]
+    lib.conqur_get_stats.restype = C.c_int
+    lib.conqur_get_stats.argtypes = [vp, C.POINTER(conqur_stats)]
+    lib.conqur_plan_schedule.restype = C.c_int
+    lib.conqur_plan_schedule.argtypes = [C.c_double, i32, C.POINTER(C.c_double), i32]
+    lib.conqur_strerror.restype = C.c_char_p
+    lib.conqur_strerror.argtypes = [C.c_int]
+    _lib = lib
+    return lib
+
+
+def strerror(status: int) -> str:
+    return load().conqur_strerror(int(status)).decode()
+
+
+def make_config(*, in_dtype=CONQUR_BF16, mode=CONQUR_TC_BF16, quant_bits=0, ns_steps=0, ns_max_steps=0,
+                orth_tol=0.0, prior_rel=0.0, ns_sigma_min_rel=0.0, n_max=1, batch=1) -> conqur_config:
+    return conqur_config(C.sizeof(conqur_config), in_dtype, mode, quant_bits, ns_steps, ns_max_steps, orth_tol,
+                         prior_rel, ns_sigma_min_rel, n_max, batch)
+
+
+# ---- the C calls, one to one -------------------------------------------------------------------
+
+def conqur_workspace_bytes(d: int, cfg: conqur_config) -> int:
+    return int(load().conqur_workspace_bytes(d, C.byref(cfg)))
+
+
+def conqur_init(d: int, cfg: conqur_config, workspace_ptr: int, workspace_bytes: int, stream_ptr: int) -> int:
+    h = C.c_void_p()
+    rc = load().conqur_init(C.byref(h), d, C.byref(cfg), workspace_ptr, workspace_bytes, stream_ptr)
+    if rc != 0:
+        raise ConqurError(rc, "conqur_init")
+    return h.value
+
+
+def conqur_destroy(h: int) -> int:
+    return load().conqur_destroy(h)
+
+
+def conqur_set_R(h: int, r_ptr: int) -> int:
+    return load().conqur_set_R(h, r_ptr)
+
+
+def conqur_step(h: int, x_ptr: int, n: int, ld: int) -> int:
+    return load().conqur_step(h, x_ptr, n, ld)
+
+
+def conqur_step_batched(h: int, x_ptr: int, n: int, ld: int, problem_stride: int) -> int:
+    return load().conqur_step_batched(h, x_ptr, n, ld, problem_stride)
+
+
+def conqur_update(h: int) -> int:
+    return load().conqur_update(h)
+
+
+def conqur_get_R(h: int, out_ptr: int) -> int:
+    return load().conqur_get_R(h, out_ptr)
+
+
+def conqur_get_objective(h: int, batch: int) -> Tuple[int, np.ndarray, np.ndarray]:
+    j = (C.c_double * batch)()
+    n = (C.c_int64 * batch)()
+    rc = load().conqur_get_objective(h, j, n)
+    return rc, np.array(j[:], dtype=np.float64), np.array(n[:], dtype=np.int64)
+
+
+def conqur_get_M(h: int, out_ptr: int) -> int:
+    return load().conqur_get_M(h, out_ptr)
+
+
+def conqur_set_M(h: int, m_ptr: int, j_sum, n_tokens) -> int:
+    j_sum = np.atleast_1d(np.asarray(j_sum, dtype=np.float64))
+    n_tokens = np.atleast_1d(np.asarray(n_tokens, dtype=np.int64))
+    j = (C.c_double * j_sum.size)(*j_sum.tolist())
+    n = (C.c_int64 * n_tokens.size)(*n_tokens.tolist())
+    return load().conqur_set_M(h, m_ptr, j, n)
+
+
+def conqur_debug_get_signs(h: int, out_ptr: int) -> int:
+    return load().conqur_debug_get_signs(h, out_ptr)
+
+
+def conqur_get_stats(h: int) -> Tuple[int, conqur_stats]:
+    st = conqur_stats()
+    st.struct_size = C.sizeof(conqur_stats)
+    rc = load().conqur_get_stats(h, C.byref(st))
+    return rc, st
+
+
+def conqur_plan_schedule(sigma_min_rel: float = 0.0, ns_steps: int = 0, max_steps: int = 100) -> np.ndarray:
+    buf = (C.c_double * (3 * max_steps))()
+    n = load().conqur_plan_schedule(sigma_min_rel, ns_steps, buf, max_steps)
+    if n < 0:
+        raise ConqurError(n, "conqur_plan_schedule")
+    return np.array(buf[: 3 * n], dtype=np.float64).reshape(n, 3)
+
+
+# ---- convenience wrapper: owns the workspace tensor, checks status codes ------------------------
+
+class Context:
+    """One calibration context on the current CUDA device / current torch stream."""
+
+    def __init__(self, d: int, n_max: int, *, in_dtype="bf16", mode="tc", quant_bits=0, batch=1, prior_rel=0.0,
+                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("conqur needs a CUDA device (B200); there is no CPU path")
+        self.torch = torch
+        self.d, self.n_max, self.batch = int(d), int(n_max), int(batch)
+        self.in_dtype = {"f32": CONQUR_F32, "bf16": CONQUR_BF16}[in_dtype]
+        self.mode = {"exact": CONQUR_EXACT_F32, "tc": CONQUR_TC_BF16}[mode]
+        self.cfg = make_config(in_dtype=self.in_dtype, mode=self.mode, quant_bits=quant_bits, ns_steps=ns_steps,
+                               ns_max_steps=ns_max_steps, orth_tol=orth_tol, prior_rel=prior_rel,
+                               ns_sigma_min_rel=ns_sigma_min_rel, n_max=n_max, batch=batch)
+        nbytes = conqur_workspace_bytes(self.d, self.cfg)
+        if nbytes == 0:
+            raise ConqurError(-1, "conqur_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) // 256 * 256
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.h = conqur_init(self.d, self.cfg, self._ws_ptr, nbytes, self.stream.cuda_stream)
+
+    def _chk(self, rc: int, where: str):
+        if rc != 0:
+            raise ConqurError(rc, where)
+
+    def _x_dtype(self):
+        return self.torch.float32 if self.in_dtype == CONQUR_F32 else self.torch.bfloat16
+
+    def set_R(self, r):
+        assert r.is_cuda and r.dtype == self.torch.float32 and r.is_contiguous()
+        assert r.numel() == self.batch * self.d * self.d
+        self._chk(conqur_set_R(self.h, r.data_ptr()), "conqur_set_R")
+
+    def step(self, x):
+        assert x.is_cuda and x.dtype == self._x_dtype() and x.dim() == 2 and x.stride(1) == 1
+        self._chk(conqur_step(self.h, x.data_ptr(), x.shape[0], x.stride(0)), "conqur_step")
+
+    def step_batched(self, x, n: int, ld: int, problem_stride: int):
+        assert x.is_cuda and x.dtype == self._x_dtype()
+        self._chk(conqur_step_batched(self.h, x.data_ptr(), n, ld, problem_stride), "conqur_step_batched")
+
+    def update(self):
+        self._chk(conqur_update(self.h), "conqur_update")
+
+    def get_R(self, check=True):
+        shape = (self.d, self.d) if self.batch == 1 else (self.batch, self.d, self.d)
+        out = self.torch.empty(shape, dtype=self.torch.float32, device="cuda")
+        rc = conqur_get_R(self.h, out.data_ptr())
+        if check:
+            self._chk(rc, "conqur_get_R")
+        return out
+
+    def get_M(self, check=True):
+        shape = (self.d, self.d) if self.batch == 1 else (self.batch, self.d, self.d)
+        out = self.torch.empty(shape, dtype=self.torch.float32, device="cuda")
+        rc = conqur_get_M(self.h, out.data_ptr())
+        if check:
+            self._chk(rc, "conqur_get_M")
+        return out
+
+    def set_M(self, m, j_sum, n_tokens):
+        assert m.is_cuda and m.dtype == self.torch.float32 and m.is_contiguous()
+        self._chk(conqur_set_M(self.h, m.data_ptr(), j_sum, n_tokens), "conqur_set_M")
+
+    def get_objective(self, check=True):
+        rc, j, n = conqur_get_objective(self.h, self.batch)
+        if check:
+            self._chk(rc, "conqur_get_objective")
+        return (float(j[0]), int(n[0])) if self.batch == 1 else (j, n)
+
+    def debug_get_signs(self, n: int):
+        out = self.torch.empty((n, self.d), dtype=self.torch.int8, device="cuda")
+        self._chk(conqur_debug_get_signs(self.h, out.data_ptr()), "conqur_debug_get_signs")
+        return out
+
+    def get_stats(self) -> conqur_stats:
+        rc, st = conqur_get_stats(self.h)
+        self._chk(rc, "conqur_get_stats")
+        return st
+
+    def close(self):
+        if getattr(self, "h", None):
+            conqur_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,549 @@
+// Host side of the C ABI: argument checks, workspace carving, launch sequencing.
+// Every step of the path runs in the kernels of conqur_simt.cuh / conqur_tc.cuh; this file only
+// enqueues them.  There is no CPU fallback: without a CUDA device every entry point fails.
+#include "../../include/conqur.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "conqur_internal.h"
+#include "conqur_simt.cuh"
+#include "conqur_tc.cuh"
+#include "ns_schedule.h"
+
+using namespace conqur;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+inline int cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+struct Layout {
+  size_t state, flags_agg, R, M, rnorm, rowmax, part_d, part_f, sched;
+  size_t C;                 // exact: fp32 C' / Y (P x n_max x d); TC quant mode: fp32 Y
+  size_t Xa, Xb, E, B;      // Newton-Schulz fp32 matrices (P x d x d each)
+  size_t splitk;            // exact accumulate split-K partials
+  TcLayout tc;              // tensor-core mode buffers
+  size_t total;
+  int64_t max_partials;
+  int acc_splits;
+};
+
+struct Cfg {
+  int d, P, in_dtype, mode, quant_bits, ns_max_steps;
+  int64_t n_max;
+  float orth_tol, prior_rel, fro_tol, margin;
+};
+
+int pick_acc_splits(int d, int P, int64_t n_max) {
+  const int tiles = cdiv(d, SG_BM) * cdiv(d, SG_BN) * P;
+  if (tiles >= 148) return 1;
+  int s = std::min<int64_t>(16, std::max<int64_t>(1, 148 / tiles));
+  s = (int)std::min<int64_t>(s, std::max<int64_t>(1, n_max / 256));
+  return std::max(1, s);
+}
+
+bool make_layout(int d, const conqur_config* c, Layout* L) {
+  if (!c || c->struct_size != sizeof(conqur_config)) return false;
+  if (d < 2 || d > 32768 || c->n_max < 1 || c->batch < 1 || c->batch > 65535) return false;
+  if (c->in_dtype != CONQUR_F32 && c->in_dtype != CONQUR_BF16) return false;
+  if (c->mode != CONQUR_EXACT_F32 && c->mode != CONQUR_TC_BF16) return false;
+  if (c->quant_bits != 0 && (c->quant_bits < 2 || c->quant_bits > 8)) return false;
+  if (c->prior_rel < 0.f || c->orth_tol < 0.f || c->ns_sigma_min_rel < 0.f || c->ns_steps < 0 || c->ns_max_steps < 0)
+    return false;
+  if (c->mode == CONQUR_TC_BF16 && !tc_supported_shape(d, c->batch)) return false;
+  const int64_t P = c->batch, n = c->n_max;
+  const size_t dd = (size_t)d * d;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L->state = take(sizeof(DevState) * P);
+  L->flags_agg = take(sizeof(int) * 4);
+  L->R = take(sizeof(float) * dd * P);
+  L->M = take(sizeof(float) * dd * P);
+  L->rnorm = take(sizeof(float) * n * P);
+  L->rowmax = take(sizeof(unsigned) * n * P);
+  int64_t mp = std::max<int64_t>((int64_t)cdiv(n, 128) * cdiv(d, 128), (int64_t)cdiv(d, 128) * cdiv(d, 128));
+  mp = std::max<int64_t>(mp, cdiv(n, 8));
+  mp = std::max<int64_t>(mp, 1024);
+  L->max_partials = mp;
+  L->part_d = take(sizeof(double) * mp * P);
+  L->part_f = take(sizeof(float) * mp * P);
+  L->sched = take(sizeof(float) * 3 * 128);
+  L->acc_splits = 1;
+  L->C = L->splitk = 0;
+  L->Xa = take(sizeof(float) * dd * P);
+  L->Xb = take(sizeof(float) * dd * P);
+  L->E = take(sizeof(float) * dd * P);
+  L->B = take(sizeof(float) * dd * P);
+  if (c->mode == CONQUR_EXACT_F32) {
+    L->C = take(sizeof(float) * (size_t)n * d * P);
+    L->acc_splits = pick_acc_splits(d, (int)P, n);
+    if (L->acc_splits > 1) L->splitk = take(sizeof(float) * dd * P * L->acc_splits);
+  } else {
+    if (c->quant_bits) L->C = take(sizeof(float) * (size_t)n * d * P);
+    tc_make_layout(d, (int)P, n, c->quant_bits, &L->tc, take);
+  }
+  L->total = off;
+  return true;
+}
+
+}  // namespace
+
+struct conqur_ctx {
+  Cfg cfg;
+  Layout L;
+  char* ws;
+  cudaStream_t stream;
+  int64_t tokens_since_update;
+  int64_t last_n;            // rows of the last step (for debug_get_signs)
+  int n_sched, restart_idx;
+  std::vector<NsStep> sched;
+  TcHost tc;                 // tensor maps etc. of the tensor-core mode
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  DevState* state() const { return at<DevState>(L.state); }
+};
+
+namespace {
+
+int cuda_fail(const char* what, cudaError_t e) {
+  std::fprintf(stderr, "conqur: %s: %s\n", what, cudaGetErrorString(e));
+  return CONQUR_ERR_CUDA;
+}
+#define CQ_CUDA(expr)                                        \
+  do {                                                       \
+    cudaError_t e__ = (expr);                                \
+    if (e__ != cudaSuccess) return cuda_fail(#expr, e__);    \
+  } while (0)
+#define CQ_LAUNCH_CHECK() CQ_CUDA(cudaGetLastError())
+
+__global__ void or_flags_kernel(const DevState* st, int P, int* agg) {
+  int f = 0;
+  for (int i = threadIdx.x; i < P; i += blockDim.x) f |= st[i].status_flags;
+  for (int o = 16; o > 0; o >>= 1) f |= __shfl_xor_sync(0xffffffffu, f, o);
+  if ((threadIdx.x & 31) == 0 && f) atomicOr(agg, f);
+}
+__global__ void clear_flags_kernel(DevState* st, int P, int* agg) {
+  for (int i = threadIdx.x; i < P; i += blockDim.x) st[i].status_flags = 0;
+  if (threadIdx.x == 0) *agg = 0;
+}
+__global__ void arm_check_kernel(DevState* st, int P) {
+  for (int i = threadIdx.x; i < P; i += blockDim.x) { st[i].ns_done = 0; st[i].ns_steps_used = 0; }
+}
+__global__ void set_sums_kernel(DevState* st, const double* J, const long long* N, int P) {
+  for (int i = threadIdx.x; i < P; i += blockDim.x) { st[i].J = J[i]; st[i].N = N[i]; }
+}
+
+int flags_to_status(int f) {
+  if (f & STATUS_FLAG_TIMEOUT) return CONQUR_ERR_TIMEOUT;
+  if (f & STATUS_FLAG_NS_FAILED) return CONQUR_ERR_NS_NOT_CONVERGED;
+  if (f & STATUS_FLAG_NONFINITE) return CONQUR_ERR_NONFINITE_INPUT;
+  return CONQUR_OK;
+}
+
+// Synchronise and return the latched device status (not cleared).
+int sync_status(conqur_ctx* c) {
+  int* agg = c->at<int>(c->L.flags_agg);
+  CQ_CUDA(cudaMemsetAsync(agg, 0, sizeof(int), c->stream));
+  or_flags_kernel<<<1, 256, 0, c->stream>>>(c->state(), c->cfg.P, agg);
+  CQ_LAUNCH_CHECK();
+  int f = 0;
+  CQ_CUDA(cudaMemcpyAsync(&f, agg, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  return flags_to_status(f);
+}
+
+int ew_blocks(int64_t count) { return (int)std::min<int64_t>(148 * 8, (count + 255) / 256); }
+
+// ---------------------------------------------------------------- exact-mode step
+template <typename TIn>
+int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstride) {
+  const Cfg& g = c->cfg;
+  const int d = g.d, P = g.P;
+  DevState* st = c->state();
+  float* rnorm = c->at<float>(c->L.rnorm);
+  float* C = c->at<float>(c->L.C);
+  double* part = c->at<double>(c->L.part_d);
+  const int64_t c_ps = (int64_t)g.n_max * d;
+  rownorm_kernel<TIn><<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(X, n, d, ld, pstride, rnorm, g.n_max, st, 1);
+  CQ_LAUNCH_CHECK();
+  const dim3 grid1(cdiv(d, SG_BN), cdiv(n, SG_BM), P);
+  int per_problem;
+  if (g.quant_bits == 0) {
+    rotate_target_exact_kernel<TIn, false><<<grid1, SG_THREADS, 0, c->stream>>>(
+        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, part);
+    CQ_LAUNCH_CHECK();
+    per_problem = grid1.x * grid1.y;
+  } else {
+    unsigned* rowmax = c->at<unsigned>(c->L.rowmax);
+    CQ_CUDA(cudaMemsetAsync(rowmax, 0, sizeof(unsigned) * g.n_max * P, c->stream));
+    rotate_target_exact_kernel<TIn, true><<<grid1, SG_THREADS, 0, c->stream>>>(
+        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, part);
+    CQ_LAUNCH_CHECK();
+    const int levels = (1 << (g.quant_bits - 1)) - 1;
+    quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, levels,
+                                                                    part, nullptr, 0);
+    CQ_LAUNCH_CHECK();
+    per_problem = cdiv(n, 8);
+  }
+  finalize_step_kernel<<<P, 256, 0, c->stream>>>(st, part, per_problem, n, 1.0 / std::sqrt((double)d));
+  CQ_LAUNCH_CHECK();
+  const int S = c->L.acc_splits;
+  accumulate_exact_kernel<TIn><<<dim3(cdiv(d, SG_BN), cdiv(d, SG_BM), P * S), SG_THREADS, 0, c->stream>>>(
+      X, ld, pstride, C, c_ps, rnorm, g.n_max, (int)n, d, S, c->at<float>(c->L.M),
+      S > 1 ? c->at<float>(c->L.splitk) : nullptr);
+  CQ_LAUNCH_CHECK();
+  if (S > 1) {
+    splitk_reduce_add_kernel<<<dim3(ew_blocks((int64_t)d * d), P), 256, 0, c->stream>>>(
+        c->at<float>(c->L.M), c->at<float>(c->L.splitk), (int64_t)d * d, S);
+    CQ_LAUNCH_CHECK();
+  }
+  return CONQUR_OK;
+}
+
+// ---------------------------------------------------------------- update (both modes share the control flow)
+// residual check of the fp32 matrix X (P x d x d) into E; fills the partials.
+int launch_residual(conqur_ctx* c, const float* X, int buf) {
+  const Cfg& g = c->cfg;
+  const int T = cdiv(g.d, SG_BM);
+  if (g.mode == CONQUR_EXACT_F32) {
+    ns_gemm_exact_kernel<EPI_RESIDUAL><<<dim3(T, T, g.P), SG_THREADS, 0, c->stream>>>(
+        X, X, nullptr, c->at<float>(c->L.E), g.d, c->state(), c->at<float>(c->L.part_f), c->at<double>(c->L.part_d));
+    CQ_LAUNCH_CHECK();
+    return CONQUR_OK;
+  }
+  return tc_ns_residual(c->tc, c->stream, buf);
+}
+int ns_parts(const conqur_ctx* c) {
+  if (c->cfg.mode == CONQUR_EXACT_F32) { const int T = cdiv(c->cfg.d, SG_BM); return T * T; }
+  return tc_ns_parts(c->tc);
+}
+
+int update_impl(conqur_ctx* c) {
+  const Cfg& g = c->cfg;
+  const int d = g.d, P = g.P;
+  const int64_t dd = (int64_t)d * d;
+  DevState* st = c->state();
+  float* M = c->at<float>(c->L.M);
+  float* R = c->at<float>(c->L.R);
+  float* Xa = c->at<float>(c->L.Xa);
+  float* Xb = c->at<float>(c->L.Xb);
+  float* E = c->at<float>(c->L.E);
+  float* B = c->at<float>(c->L.B);
+  double* pd = c->at<double>(c->L.part_d);
+  float* pf = c->at<float>(c->L.part_f);
+  const float* sched = c->at<float>(c->L.sched);
+  const int nb = (int)std::min<int64_t>(1024, (dd + 1023) / 1024);
+  const float isd = (float)(1.0 / std::sqrt((double)d));
+
+  sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
+  CQ_LAUNCH_CHECK();
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin);
+  CQ_LAUNCH_CHECK();
+  if (g.prior_rel > 0.f) {
+    sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 1, pd);
+    CQ_LAUNCH_CHECK();
+  }
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin);
+  CQ_LAUNCH_CHECK();
+  ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
+  CQ_LAUNCH_CHECK();
+  if (g.mode == CONQUR_TC_BF16) { int rc = tc_ns_begin(c->tc, c->stream); if (rc) return rc; }
+
+  const int T = cdiv(d, SG_BM);
+  const int parts = ns_parts(c);
+  for (int k = 0; k <= g.ns_max_steps; ++k) {
+    const int cur = k & 1;
+    float* X = cur ? Xb : Xa;
+    float* Xn = cur ? Xa : Xb;
+    int rc = launch_residual(c, X, cur);
+    if (rc) return rc;
+    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, parts, k, sched, c->n_sched, c->restart_idx, g.orth_tol,
+                                                g.fro_tol, cur, g.ns_max_steps);
+    CQ_LAUNCH_CHECK();
+    if (k == g.ns_max_steps) break;
+    if (g.mode == CONQUR_EXACT_F32) {
+      ns_gemm_exact_kernel<EPI_POLY><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(E, E, E, B, d, st, nullptr, nullptr);
+      CQ_LAUNCH_CHECK();
+      ns_gemm_exact_kernel<EPI_NEXT><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(X, B, X, Xn, d, st, nullptr, nullptr);
+      CQ_LAUNCH_CHECK();
+    } else {
+      rc = tc_ns_poly_next(c->tc, c->stream, cur);
+      if (rc) return rc;
+    }
+  }
+  ns_commit_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(st, Xa, Xb, R, M, dd);
+  CQ_LAUNCH_CHECK();
+  if (g.mode == CONQUR_TC_BF16) { int rc = tc_refresh_R(c->tc, c->stream, /*only_if_converged=*/1); if (rc) return rc; }
+  ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st);
+  CQ_LAUNCH_CHECK();
+  return CONQUR_OK;
+}
+
+}  // namespace
+
+// ================================================================== C ABI
+
+extern "C" size_t conqur_workspace_bytes(int32_t d, const conqur_config* cfg) {
+  Layout L;
+  if (!make_layout(d, cfg, &L)) return 0;
+  return L.total;
+}
+
+extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg, void* workspace_dev,
+                           size_t workspace_bytes, void* cuda_stream) {
+  if (!out) return CONQUR_ERR_INVALID_ARG;
+  *out = nullptr;
+  Layout L;
+  if (!make_layout(d, cfg, &L)) return CONQUR_ERR_INVALID_ARG;
+  if (!workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) % ALIGN) != 0) return CONQUR_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return CONQUR_ERR_WORKSPACE_TOO_SMALL;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    std::fprintf(stderr, "conqur: no CUDA device; there is no CPU fallback\n");
+    return CONQUR_ERR_CUDA;
+  }
+  conqur_ctx* c = new (std::nothrow) conqur_ctx();
+  if (!c) return CONQUR_ERR_INVALID_ARG;
+  c->L = L;
+  c->ws = static_cast<char*>(workspace_dev);
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->tokens_since_update = 0;
+  c->last_n = 0;
+  Cfg& g = c->cfg;
+  g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
+  g.n_max = cfg->n_max;
+  g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 40;
+  g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
+  g.prior_rel = cfg->prior_rel;
+  g.fro_tol = 0.1f;
+  g.margin = 1e-3f;
+  const double l0 = cfg->ns_sigma_min_rel > 0.f ? cfg->ns_sigma_min_rel : 1e-7;
+  const double final_err = 1e-6;
+  c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(cfg->ns_steps, g.margin, final_err)
+                               : plan_schedule(l0, g.margin, final_err, 100);
+  c->n_sched = (int)c->sched.size();
+  c->restart_idx = 0;
+  for (int i = 0; i < c->n_sched; ++i)
+    if (c->sched[i].l >= 1e-3) { c->restart_idx = i; break; }
+  if (c->restart_idx >= c->n_sched) c->restart_idx = c->n_sched - 1;
+  std::vector<float> coef(3 * 128, 0.f);
+  for (int i = 0; i < c->n_sched && i < 128; ++i) {
+    const NsStep& s = c->sched[i];
+    coef[3 * i + 0] = (float)(s.a + s.b + s.c);
+    coef[3 * i + 1] = (float)(s.b + 2.0 * s.c);
+    coef[3 * i + 2] = (float)s.c;
+  }
+  auto fail = [&](int rc) { delete c; return rc; };
+  if (cudaMemsetAsync(c->ws, 0, L.R, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);   // state + flags
+  if (cudaMemsetAsync(c->ws + L.M, 0, sizeof(float) * (size_t)d * d * g.P, c->stream) != cudaSuccess)
+    return fail(CONQUR_ERR_CUDA);
+  if (cudaMemcpyAsync(c->ws + L.sched, coef.data(), sizeof(float) * 3 * 128, cudaMemcpyHostToDevice, c->stream) !=
+      cudaSuccess)
+    return fail(CONQUR_ERR_CUDA);
+  set_identity_kernel<<<ew_blocks((int64_t)d * d * g.P), 256, 0, c->stream>>>(c->at<float>(L.R), d, g.P);
+  if (cudaGetLastError() != cudaSuccess) return fail(CONQUR_ERR_CUDA);
+  if (g.mode == CONQUR_TC_BF16) {
+    int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
+                     c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
+                     c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f));
+    if (rc) return fail(rc);
+    rc = tc_refresh_R(c->tc, c->stream, 0);
+    if (rc) return fail(rc);
+  }
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);   // coef is a local
+  *out = c;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_destroy(conqur_ctx* ctx) {
+  if (!ctx) return CONQUR_ERR_INVALID_ARG;
+  cudaStreamSynchronize(ctx->stream);
+  delete ctx;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_set_R(conqur_ctx* c, const float* R_dev) {
+  if (!c || !R_dev) return CONQUR_ERR_INVALID_ARG;
+  const Cfg& g = c->cfg;
+  const int64_t dd = (int64_t)g.d * g.d;
+  // check orthogonality with the exact fp32 residual product, whatever the mode
+  float* Xa = c->at<float>(c->L.Xa);
+  CQ_CUDA(cudaMemcpyAsync(Xa, R_dev, sizeof(float) * dd * g.P, cudaMemcpyDeviceToDevice, c->stream));
+  arm_check_kernel<<<1, 256, 0, c->stream>>>(c->state(), g.P);
+  CQ_LAUNCH_CHECK();
+  const int T = cdiv(g.d, SG_BM);
+  ns_gemm_exact_kernel<EPI_RESIDUAL><<<dim3(T, T, g.P), SG_THREADS, 0, c->stream>>>(
+      Xa, Xa, nullptr, c->at<float>(c->L.E), g.d, c->state(), c->at<float>(c->L.part_f), c->at<double>(c->L.part_d));
+  CQ_LAUNCH_CHECK();
+  std::vector<float> pm((size_t)T * T * g.P);
+  CQ_CUDA(cudaMemcpyAsync(pm.data(), c->at<float>(c->L.part_f), sizeof(float) * pm.size(), cudaMemcpyDeviceToHost,
+                          c->stream));
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  float mx = 0.f;
+  for (float v : pm) mx = (v == v) ? std::max(mx, v) : INFINITY;
+  if (!(mx <= 1e-3f)) return CONQUR_ERR_NOT_ORTHOGONAL_INPUT;
+  CQ_CUDA(cudaMemcpyAsync(c->at<float>(c->L.R), R_dev, sizeof(float) * dd * g.P, cudaMemcpyDeviceToDevice, c->stream));
+  if (g.mode == CONQUR_TC_BF16) return tc_refresh_R(c->tc, c->stream, 0);
+  return CONQUR_OK;
+}
+
+static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int64_t pstride) {
+  if (!c || !X) return CONQUR_ERR_INVALID_ARG;
+  const Cfg& g = c->cfg;
+  if (n < 0 || n > g.n_max || ld < g.d || pstride < 0) return CONQUR_ERR_INVALID_ARG;
+  if (n == 0) return CONQUR_OK;
+  int rc;
+  if (g.mode == CONQUR_EXACT_F32) {
+    rc = (g.in_dtype == CONQUR_F32) ? step_exact<float>(c, static_cast<const float*>(X), n, ld, pstride)
+                                    : step_exact<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(X), n, ld, pstride);
+  } else {
+    rc = tc_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride);
+  }
+  if (rc == CONQUR_OK) { c->tokens_since_update += n; c->last_n = n; }
+  return rc;
+}
+
+extern "C" int conqur_step(conqur_ctx* c, const void* X_dev, int64_t n, int64_t ld) {
+  if (!c || c->cfg.P != 1) return CONQUR_ERR_INVALID_ARG;
+  return step_common(c, X_dev, n, ld, 0);
+}
+
+extern "C" int conqur_step_batched(conqur_ctx* c, const void* X_dev, int64_t n, int64_t ld, int64_t problem_stride) {
+  if (!c) return CONQUR_ERR_INVALID_ARG;
+  return step_common(c, X_dev, n, ld, problem_stride);
+}
+
+extern "C" int conqur_update(conqur_ctx* c) {
+  if (!c) return CONQUR_ERR_INVALID_ARG;
+  if (c->tokens_since_update == 0) return CONQUR_ERR_EMPTY_UPDATE;
+  if (c->tokens_since_update < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
+  const int rc = update_impl(c);
+  if (rc == CONQUR_OK) c->tokens_since_update = 0;
+  return rc;
+}
+
+extern "C" int conqur_get_R(conqur_ctx* c, float* R_out_dev) {
+  if (!c || !R_out_dev) return CONQUR_ERR_INVALID_ARG;
+  const size_t bytes = sizeof(float) * (size_t)c->cfg.d * c->cfg.d * c->cfg.P;
+  CQ_CUDA(cudaMemcpyAsync(R_out_dev, c->at<float>(c->L.R), bytes, cudaMemcpyDeviceToDevice, c->stream));
+  return sync_status(c);
+}
+
+extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tokens) {
+  if (!c || !J_sum || !n_tokens) return CONQUR_ERR_INVALID_ARG;
+  const int P = c->cfg.P;
+  std::vector<DevState> h(P);
+  CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
+  const int rc = sync_status(c);
+  for (int p = 0; p < P; ++p) { J_sum[p] = h[p].J; n_tokens[p] = h[p].N; }
+  return rc;
+}
+
+extern "C" int conqur_get_M(conqur_ctx* c, float* M_out_dev) {
+  if (!c || !M_out_dev) return CONQUR_ERR_INVALID_ARG;
+  const int64_t count = (int64_t)c->cfg.d * c->cfg.d * c->cfg.P;
+  scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(c->at<float>(c->L.M), M_out_dev, count,
+                                                             (float)(1.0 / std::sqrt((double)c->cfg.d)));
+  CQ_LAUNCH_CHECK();
+  return sync_status(c);
+}
+
+extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_sum, const int64_t* n_tokens) {
+  if (!c || !M_dev || !J_sum || !n_tokens) return CONQUR_ERR_INVALID_ARG;
+  const int P = c->cfg.P;
+  const int64_t count = (int64_t)c->cfg.d * c->cfg.d * P;
+  scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(M_dev, c->at<float>(c->L.M), count,
+                                                             (float)std::sqrt((double)c->cfg.d));
+  CQ_LAUNCH_CHECK();
+  // stage the sums through the partials buffer
+  double* dJ = c->at<double>(c->L.part_d);
+  long long* dN = reinterpret_cast<long long*>(dJ + P);
+  std::vector<long long> n64(n_tokens, n_tokens + P);
+  CQ_CUDA(cudaMemcpyAsync(dJ, J_sum, sizeof(double) * P, cudaMemcpyHostToDevice, c->stream));
+  CQ_CUDA(cudaMemcpyAsync(dN, n64.data(), sizeof(long long) * P, cudaMemcpyHostToDevice, c->stream));
+  set_sums_kernel<<<1, 256, 0, c->stream>>>(c->state(), dJ, dN, P);
+  CQ_LAUNCH_CHECK();
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  int64_t tot = 0;
+  for (int p = 0; p < P; ++p) tot = std::max<int64_t>(tot, n_tokens[p]);
+  c->tokens_since_update = tot;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_debug_get_signs(conqur_ctx* c, int8_t* S_out_dev) {
+  if (!c || !S_out_dev || c->cfg.P != 1) return CONQUR_ERR_INVALID_ARG;
+  if (c->last_n == 0) return CONQUR_ERR_INVALID_ARG;
+  const int64_t total = c->last_n * c->cfg.d;
+  if (c->cfg.mode == CONQUR_EXACT_F32) {
+    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(c->at<float>(c->L.C), nullptr, 0, c->last_n,
+                                                                 c->cfg.d, S_out_dev);
+  } else {
+    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(nullptr, tc_ct_ptr(c->tc), tc_ct_ld(c->tc),
+                                                                 c->last_n, c->cfg.d, S_out_dev);
+  }
+  CQ_LAUNCH_CHECK();
+  return sync_status(c);
+}
+
+extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
+  if (!c || !out || out->struct_size != sizeof(conqur_stats)) return CONQUR_ERR_INVALID_ARG;
+  const int P = c->cfg.P;
+  std::vector<DevState> h(P);
+  CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
+  const int rc = sync_status(c);
+  if (rc == CONQUR_ERR_CUDA) return rc;
+  clear_flags_kernel<<<1, 256, 0, c->stream>>>(c->state(), P, c->at<int>(c->L.flags_agg));
+  CQ_LAUNCH_CHECK();
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  out->status = rc;
+  out->ns_steps_used = 0; out->orth_err = 0.f; out->orth_fro = 0.f; out->n_skipped = 0;
+  out->last_J = 0.0; out->last_N = 0;
+  out->updates = h[0].updates; out->scale = h[0].scale;
+  for (int p = 0; p < P; ++p) {
+    out->ns_steps_used = std::max(out->ns_steps_used, h[p].ns_steps_used);
+    out->orth_err = std::max(out->orth_err, h[p].last_orth);
+    out->orth_fro = std::max(out->orth_fro, h[p].last_fro);
+    out->n_skipped += h[p].n_skipped;
+    out->last_J += h[p].last_J;
+    out->last_N += h[p].last_N;
+    out->updates = std::min(out->updates, h[p].updates);
+  }
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out, int32_t max_steps) {
+  if (!abc_out || max_steps < 1 || sigma_min_rel < 0.0 || sigma_min_rel >= 1.0 || ns_steps < 0)
+    return CONQUR_ERR_INVALID_ARG;
+  const double l0 = sigma_min_rel > 0.0 ? sigma_min_rel : 1e-7;
+  const std::vector<NsStep> s = ns_steps > 0 ? plan_schedule_for_steps(ns_steps, 1e-3, 1e-6)
+                                             : plan_schedule(l0, 1e-3, 1e-6, 100);
+  const int n = std::min<int>((int)s.size(), max_steps);
+  for (int i = 0; i < n; ++i) { abc_out[3 * i] = s[i].a; abc_out[3 * i + 1] = s[i].b; abc_out[3 * i + 2] = s[i].c; }
+  return n;
+}
+
+extern "C" const char* conqur_strerror(int s) {
+  switch (s) {
+    case CONQUR_OK: return "ok";
+    case CONQUR_ERR_INVALID_ARG: return "invalid argument";
+    case CONQUR_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CONQUR_ERR_NOT_ORTHOGONAL_INPUT: return "rotation passed to set_R is not orthogonal";
+    case CONQUR_ERR_EMPTY_UPDATE: return "update with no accumulated tokens";
+    case CONQUR_ERR_RANK_DEFICIENT: return "fewer tokens than dimensions and prior_rel == 0";
+    case CONQUR_ERR_NS_NOT_CONVERGED: return "Newton-Schulz did not converge; previous rotation kept";
+    case CONQUR_ERR_NONFINITE_INPUT: return "non-finite input row (skipped)";
+    case CONQUR_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case CONQUR_ERR_CUDA: return "CUDA error";
+    case CONQUR_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown status";
+  }
+}

@@ -1,0 +1,586 @@
+// fp32 CUDA-core kernels: the exact mode of every step of the path, and the
+// reductions / element-wise passes both modes share.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "conqur_internal.h"
+
+namespace conqur {
+
+// ------------------------------------------------------------------ small helpers
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Block-wide sum in double, fixed order (lane tree, then warp 0 over the warp results).
+template <int THREADS>
+__device__ __forceinline__ double block_sum_d(double v, double* smem /* THREADS/32 */) {
+  v = warp_sum_d(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) smem[w] = v;
+  __syncthreads();
+  double r = 0.0;
+  if (w == 0) {
+    r = (l < THREADS / 32) ? smem[l] : 0.0;
+    r = warp_sum_d(r);
+  }
+  __syncthreads();
+  return r;  // valid in warp 0
+}
+template <int THREADS>
+__device__ __forceinline__ float block_max_f(float v, float* smem) {
+  v = warp_max(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) smem[w] = v;
+  __syncthreads();
+  float r = 0.f;
+  if (w == 0) {
+    r = (l < THREADS / 32) ? smem[l] : 0.f;
+    r = warp_max(r);
+  }
+  __syncthreads();
+  return r;
+}
+
+__device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+__device__ __forceinline__ void ld4_as_float(const float* p, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void ld4_as_float(const __nv_bfloat16* p, float (&v)[4]) {
+  const uint2 t = *reinterpret_cast<const uint2*>(p);
+  v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+  v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
+__device__ __forceinline__ float sgnf(float v) { return (v > 0.f) ? 1.f : ((v < 0.f) ? -1.f : 0.f); }
+
+// ------------------------------------------------------------------ a1: row norms
+// One warp per row: rnorm_i = 1/||x_i||_2 in fp32.  Rows whose sum of squares is zero
+// or not finite get rnorm = 0 (they then contribute nothing anywhere) and are counted.
+template <typename TIn>
+__global__ void __launch_bounds__(256) rownorm_kernel(const TIn* __restrict__ X, int64_t n, int d, int64_t ld,
+                                                      int64_t problem_stride, float* __restrict__ rnorm,
+                                                      int64_t rnorm_stride, DevState* st, int state_stride_problems) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int p = blockIdx.y;
+  if (row >= n) return;
+  const TIn* x = X + (int64_t)p * problem_stride + row * ld;
+  float ss = 0.f;
+  const bool vec = ((d & 3) == 0) && ((reinterpret_cast<uintptr_t>(x) & (sizeof(TIn) * 4 - 1)) == 0);
+  if (vec) {
+    for (int k = lane * 4; k < d; k += 128) {
+      float v[4];
+      ld4_as_float(x + k, v);
+      ss = fmaf(v[0], v[0], ss); ss = fmaf(v[1], v[1], ss); ss = fmaf(v[2], v[2], ss); ss = fmaf(v[3], v[3], ss);
+    }
+  } else {
+    for (int k = lane; k < d; k += 32) {
+      const float v = ld_as_float(x + k);
+      ss = fmaf(v, v, ss);
+    }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) {
+    float r = 0.f;
+    DevState* s = st + (state_stride_problems ? p : 0);
+    if (ss > 0.f && ss <= 3.0e38f) {
+      r = 1.0f / sqrtf(ss);
+    } else {
+      atomicAdd(reinterpret_cast<unsigned long long*>(&s->step_skipped), 1ull);
+      if (!(ss == 0.f)) atomicOr(&s->status_flags, STATUS_FLAG_NONFINITE);
+    }
+    rnorm[(int64_t)p * rnorm_stride + row] = r;
+  }
+}
+
+// ------------------------------------------------------------------ generic SIMT GEMM main loop
+// acc[i][j] = sum_k A(m_i, k) * B(k, n_j) over a 128 x 128 tile, BK = 16, 256 threads.
+// A(m,k) lives at A[m*lda + k] (A_M_CONTIG = false) or A[k*lda + m] (true);
+// B(k,n) lives at B[k*ldb + n] (B_N_CONTIG = true) or B[n*ldb + k] (false).
+// Thread (tx, ty) owns rows {ty*4+i, 64+ty*4+i}, cols {tx*4+j, 64+tx*4+j}, i,j in 0..3.
+constexpr int SG_BM = 128, SG_BN = 128, SG_BK = 16, SG_THREADS = 256, SG_PAD = 4;
+
+// kmask (optional, MN_CONTIG only): rows k with kmask[k] == 0 are read as zeros (skipped tokens).
+template <typename T, bool MN_CONTIG>
+__device__ __forceinline__ void sg_load_tile(const T* __restrict__ P, int64_t ld, int mn0, int k0, int MN, int K,
+                                             float (*S)[SG_BM + SG_PAD], const float* __restrict__ kmask = nullptr) {
+  const int t = threadIdx.x;
+  const bool aligned = ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(P) & (sizeof(T) * 4 - 1)) == 0);
+  if (MN_CONTIG) {
+    // element (mn, k) at P[k*ld + mn]; 4 consecutive mn per thread
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int k = (t >> 5) + 8 * r;
+      const int mn = (t & 31) * 4;
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+      const int gk = k0 + k, gmn = mn0 + mn;
+      if (gk < K && (kmask == nullptr || kmask[gk] > 0.f)) {
+        const T* src = P + (int64_t)gk * ld + gmn;
+        if (aligned && gmn + 3 < MN && ((gmn & 3) == 0)) {
+          ld4_as_float(src, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (gmn + j < MN) v[j] = ld_as_float(src + j);
+        }
+      }
+      *reinterpret_cast<float4*>(&S[k][mn]) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+  } else {
+    // element (mn, k) at P[mn*ld + k]; 4 consecutive k per thread, stored transposed
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int mn = (t >> 2) + 64 * r;
+      const int k = (t & 3) * 4;
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+      const int gk = k0 + k, gmn = mn0 + mn;
+      if (gmn < MN) {
+        const T* src = P + (int64_t)gmn * ld + gk;
+        if (aligned && gk + 3 < K && ((gk & 3) == 0)) {
+          ld4_as_float(src, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (gk + j < K) v[j] = ld_as_float(src + j);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) S[k + j][mn] = v[j];
+    }
+  }
+}
+
+template <typename TA, bool A_M_CONTIG, typename TB, bool B_N_CONTIG>
+__device__ __forceinline__ void sg_mainloop(const TA* __restrict__ A, int64_t lda, const TB* __restrict__ B,
+                                            int64_t ldb, int M, int N, int k_begin, int k_end, int m0, int n0,
+                                            float (&acc)[8][8], const float* __restrict__ kmask = nullptr) {
+  __shared__ __align__(16) float As[SG_BK][SG_BM + SG_PAD];
+  __shared__ __align__(16) float Bs[SG_BK][SG_BN + SG_PAD];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+  for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
+    sg_load_tile<TA, A_M_CONTIG>(A, lda, m0, k0, M, k_end, As, kmask);
+    sg_load_tile<TB, B_N_CONTIG>(B, ldb, n0, k0, N, k_end, Bs);
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < SG_BK; ++k) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ int sg_row(int i) { return ((threadIdx.x >> 4) * 4) + (i & 3) + ((i >> 2) * 64); }
+__device__ __forceinline__ int sg_col(int j) { return ((threadIdx.x & 15) * 4) + (j & 3) + ((j >> 2) * 64); }
+
+// ------------------------------------------------------------------ a2-a4 exact: Y = X R, target, objective
+// grid (ceil(d/128), ceil(n/128), P).  Plain mode: writes C'[i][j] = sgn(y_ij) * rnorm_i (fp32) and one
+// objective partial per CTA (sum |acc_ij| * rnorm_i).  Quant mode: writes the raw products Y and the
+// per-row max |acc| (integer atomicMax on the bit pattern: exact and order independent).
+template <typename TIn, bool QUANT>
+__global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
+    const TIn* __restrict__ X, int64_t ld, int64_t x_pstride, const float* __restrict__ R, int n, int d,
+    const float* __restrict__ rnorm, int64_t rnorm_pstride, float* __restrict__ Cp /* n x d */,
+    int64_t c_pstride, unsigned int* __restrict__ rowmax_bits, double* __restrict__ partials) {
+  const int p = blockIdx.z;
+  const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+  float acc[8][8];
+  sg_mainloop<TIn, false, float, true>(X + (int64_t)p * x_pstride, ld, R + (int64_t)p * d * d, d, n, d, 0, d, m0,
+                                        n0, acc);
+  const float* rn = rnorm + (int64_t)p * rnorm_pstride;
+  float* C = Cp + (int64_t)p * c_pstride;
+  double asum = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = m0 + sg_row(i);
+    if (row >= n) continue;
+    const float r = rn[row];
+    float rs = 0.f, rmax = 0.f;
+#pragma unroll
+    for (int jh = 0; jh < 2; ++jh) {
+      const int col = n0 + sg_col(jh * 4);
+      float o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float v = acc[i][jh * 4 + j];
+        if (QUANT) {
+          o[j] = v;
+          rmax = fmaxf(rmax, fabsf(v));
+        } else {
+          o[j] = sgnf(v) * r;
+          rs += fabsf(v);
+        }
+      }
+      float* dst = C + (int64_t)row * d + col;
+      if (col + 3 < d && ((d & 3) == 0)) {
+        *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (col + j < d) dst[j] = o[j];
+      }
+    }
+    if (QUANT) {
+      if (r > 0.f) atomicMax(rowmax_bits + (int64_t)p * rnorm_pstride + row, __float_as_uint(rmax));
+    } else {
+      if (r > 0.f) asum += (double)(rs * r);
+    }
+  }
+  if (!QUANT) {
+    __shared__ double red[SG_THREADS / 32];
+    const double tot = block_sum_d<SG_THREADS>(asum, red);
+    if (threadIdx.x == 0)
+      partials[((int64_t)p * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = tot;
+  }
+}
+
+// Quant mode, second pass (Appendix B, Q_sym per token).  One warp per row:
+// Delta_raw = rowmax/L, q = rint(acc / Delta_raw) clipped to +-L, C' = sgn(q) * rnorm,
+// objective partial = rnorm * Delta_raw * sum_j |q_j|.  Works in place: Y and C' share the buffer.
+// out_t (optional): bf16 transposed copy C'^T (d x ldt) for the tensor-core accumulate.
+__global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
+                                                           int64_t c_pstride, const float* __restrict__ rnorm,
+                                                           int64_t rnorm_pstride,
+                                                           const unsigned int* __restrict__ rowmax_bits, int levels,
+                                                           double* __restrict__ partials /* per block */,
+                                                           __nv_bfloat16* __restrict__ out_t, int64_t ldt) {
+  const int p = blockIdx.y;
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  double contrib = 0.0;
+  if (row < n) {
+    const float r = rnorm[(int64_t)p * rnorm_pstride + row];
+    const float mx = __uint_as_float(rowmax_bits[(int64_t)p * rnorm_pstride + row]);
+    float* y = YC + (int64_t)p * c_pstride + row * d;
+    const float L = (float)levels;
+    const bool live = (r > 0.f) && (mx > 0.f);
+    const float inv = live ? (L / mx) : 0.f;
+    float qs = 0.f;
+    for (int j = lane; j < d; j += 32) {
+      float q = rintf(y[j] * inv);
+      q = fminf(fmaxf(q, -L), L);
+      qs += fabsf(q);
+      const float c = live ? sgnf(q) * r : 0.f;
+      y[j] = c;
+      if (out_t) out_t[(int64_t)j * ldt + row] = __float2bfloat16(c);
+    }
+    qs = warp_sum(qs);
+    if (live) contrib = (double)(r * (mx / L)) * (double)qs;
+  }
+  __shared__ double red[8];
+  if (lane == 0) red[threadIdx.x >> 5] = contrib;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    partials[(int64_t)p * gridDim.x + blockIdx.x] = t;
+  }
+}
+
+// ------------------------------------------------------------------ a5 exact: M_raw (+)= X^T C'
+// grid (ceil(d/128), ceil(d/128), splits*P).  splits == 1: read-modify-write of M.  splits > 1: each
+// split writes its own partial; splitk_reduce_add_kernel adds them to M in a fixed order.
+template <typename TIn>
+__global__ void __launch_bounds__(SG_THREADS) accumulate_exact_kernel(const TIn* __restrict__ X, int64_t ld,
+                                                                      int64_t x_pstride,
+                                                                      const float* __restrict__ Cp,
+                                                                      int64_t c_pstride,
+                                                                      const float* __restrict__ rnorm,
+                                                                      int64_t rnorm_pstride, int n, int d,
+                                                                      int splits,
+                                                                      float* __restrict__ M,
+                                                                      float* __restrict__ partial) {
+  const int p = blockIdx.z / splits, s = blockIdx.z % splits;
+  const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+  int chunk = (n + splits - 1) / splits;
+  chunk = (chunk + SG_BK - 1) / SG_BK * SG_BK;
+  const int kb = min(n, s * chunk), ke = min(n, kb + chunk);
+  float acc[8][8];
+  sg_mainloop<TIn, true, float, true>(X + (int64_t)p * x_pstride, ld, Cp + (int64_t)p * c_pstride, d, d, d, kb, ke,
+                                       m0, n0, acc, rnorm + (int64_t)p * rnorm_pstride);
+  float* dst = (splits == 1) ? (M + (int64_t)p * d * d) : (partial + ((int64_t)p * splits + s) * d * d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = m0 + sg_row(i);
+    if (row >= d) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int col = n0 + sg_col(j);
+      if (col >= d) continue;
+      float* q = dst + (int64_t)row * d + col;
+      if (splits == 1) *q += acc[i][j]; else *q = acc[i][j];
+    }
+  }
+}
+
+__global__ void splitk_reduce_add_kernel(float* __restrict__ M, const float* __restrict__ partial, int64_t dd,
+                                         int splits) {
+  const int p = blockIdx.y;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd; i += (int64_t)gridDim.x * blockDim.x) {
+    float v = M[p * dd + i];
+    for (int s = 0; s < splits; ++s) v += partial[((int64_t)p * splits + s) * dd + i];
+    M[p * dd + i] = v;
+  }
+}
+
+// Adds the step's objective partials (fixed order) and token counts to the running sums.
+__global__ void finalize_step_kernel(DevState* st, const double* __restrict__ partials, int per_problem, int64_t n,
+                                     double inv_sqrt_d) {
+  const int p = blockIdx.x;
+  __shared__ double red[8];
+  double v = 0.0;
+  for (int i = threadIdx.x; i < per_problem; i += 256) v += partials[(int64_t)p * per_problem + i];
+  const double tot = block_sum_d<256>(v, red);
+  if (threadIdx.x == 0) {
+    DevState* s = st + p;
+    s->J += tot * inv_sqrt_d;
+    s->N += n - s->step_skipped;
+    s->n_skipped += s->step_skipped;
+    s->step_skipped = 0;
+  }
+}
+
+// ------------------------------------------------------------------ a6/a7 exact: Newton-Schulz products
+enum { EPI_RESIDUAL = 0, EPI_POLY = 1, EPI_NEXT = 2 };
+
+// EPI_RESIDUAL: D = X^T X - I, plus per-CTA max|D| and sum D^2            (A = B = X, contraction over rows)
+// EPI_POLY:     D = beta2 * (E E) + beta1 * E                             (A = B = Cin = E)
+// EPI_NEXT:     D = X B + gamma * X                                       (A = Cin = X)
+// All early-exit when the problem's iteration has finished.
+template <int EPI>
+__global__ void __launch_bounds__(SG_THREADS) ns_gemm_exact_kernel(const float* __restrict__ A,
+                                                                   const float* __restrict__ B,
+                                                                   const float* __restrict__ Cin,
+                                                                   float* __restrict__ D, int d, DevState* st,
+                                                                   float* __restrict__ part_max,
+                                                                   double* __restrict__ part_sq) {
+  const int p = blockIdx.z;
+  const DevState* s = st + p;
+  if (s->ns_done) return;
+  const int64_t off = (int64_t)p * d * d;
+  const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+  float acc[8][8];
+  if constexpr (EPI == EPI_RESIDUAL)
+    sg_mainloop<float, true, float, true>(A + off, d, B + off, d, d, d, 0, d, m0, n0, acc);
+  else
+    sg_mainloop<float, false, float, true>(A + off, d, B + off, d, d, d, 0, d, m0, n0, acc);
+  const float c0 = s->coef[0], c1 = s->coef[1], c2 = s->coef[2];  // gamma, beta1, beta2
+  float mx = 0.f;
+  double sq = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = m0 + sg_row(i);
+    if (row >= d) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int col = n0 + sg_col(j);
+      if (col >= d) continue;
+      const int64_t idx = off + (int64_t)row * d + col;
+      float v = acc[i][j];
+      if (EPI == EPI_RESIDUAL) {
+        v -= (row == col) ? 1.f : 0.f;
+        mx = fmaxf(mx, fabsf(v));
+        sq += (double)v * (double)v;
+      } else if (EPI == EPI_POLY) {
+        v = fmaf(c2, v, c1 * Cin[idx]);
+      } else {
+        v = fmaf(c0, Cin[idx], v);
+      }
+      D[idx] = v;
+    }
+  }
+  if (EPI == EPI_RESIDUAL) {
+    __shared__ double redd[SG_THREADS / 32];
+    __shared__ float redf[SG_THREADS / 32];
+    const double tsq = block_sum_d<SG_THREADS>(sq, redd);
+    const float tmx = block_max_f<SG_THREADS>(mx, redf);
+    if (threadIdx.x == 0) {
+      const int64_t slot = ((int64_t)p * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+      part_max[slot] = tmx;
+      part_sq[slot] = tsq;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ update: scalar control + element-wise
+// sum of squares of M (optionally of M + lam*R) -> per-block double partials
+__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ M, const float* __restrict__ R,
+                                                    int64_t dd, const DevState* st, int use_lam,
+                                                    double* __restrict__ partials) {
+  const int p = blockIdx.y;
+  const float lam = use_lam ? st[p].lam : 0.f;
+  double v = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < dd; i += (int64_t)gridDim.x * 256) {
+    float t = M[p * dd + i];
+    if (use_lam) t = fmaf(lam, R[p * dd + i], t);
+    v += (double)t * (double)t;
+  }
+  __shared__ double red[8];
+  const double tot = block_sum_d<256>(v, red);
+  if (threadIdx.x == 0) partials[(int64_t)p * gridDim.x + blockIdx.x] = tot;
+}
+
+// phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
+// phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
+__global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
+                                float prior_rel, float inv_sqrt_d, float margin) {
+  const int p = blockIdx.x;
+  __shared__ double red[8];
+  double v = 0.0;
+  for (int i = threadIdx.x; i < nblocks; i += 256) v += partials[(int64_t)p * nblocks + i];
+  const double tot = block_sum_d<256>(v, red);
+  if (threadIdx.x == 0) {
+    DevState* s = st + p;
+    const float fro = (float)sqrt(tot);
+    if (phase == 0) {
+      s->lam = prior_rel * fro * inv_sqrt_d;
+    } else {
+      s->scale = fro;
+      const bool ok = (fro > 0.f) && (fro <= 3.0e38f) && (s->N > 0);
+      s->x0_scale = ok ? 1.0f / (fro * (1.0f + margin)) : 0.f;
+      s->ns_done = ok ? 0 : NS_DONE_FAILED;
+      s->ns_steps_used = 0;
+      s->ns_final_buf = 0;
+    }
+  }
+}
+
+// X0 = (M_raw + lam R) * x0_scale
+__global__ void ns_x0_kernel(const float* __restrict__ M, const float* __restrict__ R, float* __restrict__ X0,
+                             int64_t dd, const DevState* st) {
+  const int p = blockIdx.y;
+  const float lam = st[p].lam, sc = st[p].x0_scale;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd; i += (int64_t)gridDim.x * blockDim.x)
+    X0[p * dd + i] = fmaf(lam, R[p * dd + i], M[p * dd + i]) * sc;
+}
+
+// After the residual product of step k: reduce the per-CTA partials, decide convergence, pick the
+// polynomial of this step.  sched: n_sched entries of (gamma, beta1, beta2); restart_idx: where the
+// schedule re-enters when it ran out without convergence.
+__global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
+                                  const double* __restrict__ part_sq, int nparts, int k,
+                                  const float* __restrict__ sched, int n_sched, int restart_idx, float tol,
+                                  float fro_tol, int cur_buf, int max_steps) {
+  const int p = blockIdx.x;
+  DevState* s = st + p;
+  if (s->ns_done) return;
+  __shared__ double redd[8];
+  __shared__ float redf[8];
+  double sq = 0.0;
+  float mx = 0.f;
+  for (int i = threadIdx.x; i < nparts; i += 256) {
+    sq += part_sq[(int64_t)p * nparts + i];
+    mx = fmaxf(mx, part_max[(int64_t)p * nparts + i]);
+  }
+  const double tsq = block_sum_d<256>(sq, redd);
+  const float tmx = block_max_f<256>(mx, redf);
+  if (threadIdx.x == 0) {
+    const float fro = (float)sqrt(tsq);
+    s->e_max = tmx;
+    s->e_fro = fro;
+    if (!(tmx == tmx) || !(fro == fro)) {
+      s->ns_done = NS_DONE_FAILED;
+    } else if (tmx <= tol && fro <= fro_tol) {
+      s->ns_done = NS_DONE_CONVERGED;
+      s->ns_final_buf = cur_buf;
+    } else if (k >= max_steps) {
+      s->ns_done = NS_DONE_FAILED;
+    } else {
+      int idx = k;
+      if (idx >= n_sched) idx = restart_idx + (k - n_sched) % (n_sched - restart_idx);
+      s->coef[0] = sched[idx * 3 + 0];
+      s->coef[1] = sched[idx * 3 + 1];
+      s->coef[2] = sched[idx * 3 + 2];
+      s->ns_steps_used = k + 1;
+    }
+  }
+}
+
+// Accept or reject the update.  On success: R <- X_final, M <- 0, sums <- 0.
+__global__ void ns_commit_kernel(DevState* st, const float* __restrict__ Xa, const float* __restrict__ Xb,
+                                 float* __restrict__ R, float* __restrict__ M, int64_t dd) {
+  const int p = blockIdx.y;
+  DevState* s = st + p;
+  if (s->ns_done != NS_DONE_CONVERGED) return;
+  const float* X = (s->ns_final_buf ? Xb : Xa) + p * dd;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd; i += (int64_t)gridDim.x * blockDim.x) {
+    R[p * dd + i] = X[i];
+    M[p * dd + i] = 0.f;
+  }
+}
+__global__ void ns_commit_state_kernel(DevState* st) {
+  DevState* s = st + blockIdx.x;
+  if (threadIdx.x != 0) return;
+  if (s->ns_done == NS_DONE_CONVERGED) {
+    s->last_J = s->J;
+    s->last_N = s->N;
+    s->J = 0.0;
+    s->N = 0;
+    s->updates += 1;
+    s->last_orth = s->e_max;
+    s->last_fro = s->e_fro;
+  } else {
+    atomicOr(&s->status_flags, STATUS_FLAG_NS_FAILED);
+  }
+}
+
+// ------------------------------------------------------------------ misc element-wise
+__global__ void scale_copy_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t count, float f) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = src[i] * f;
+}
+__global__ void set_identity_kernel(float* __restrict__ R, int d, int P) {
+  const int64_t dd = (int64_t)d * d;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd * P; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t e = i % dd;
+    R[i] = ((e / d) == (e % d)) ? 1.f : 0.f;
+  }
+}
+// sign matrix of the last step from the fp32 C' (n x d) or the transposed bf16 C'^T (d x ldt)
+__global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Ct, int64_t ldt,
+                                    int64_t n, int d, int8_t* __restrict__ S) {
+  const int64_t total = n * d;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    float v;
+    if (C) {
+      v = C[i];
+    } else {
+      const int64_t row = i / d, col = i % d;
+      v = __bfloat162float(Ct[col * ldt + row]);
+    }
+    S[i] = (v > 0.f) ? 1 : ((v < 0.f) ? -1 : 0);
+  }
+}
+
+}  // namespace conqur

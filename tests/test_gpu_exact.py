@@ -1,0 +1,228 @@
+"""GPU parity, exact mode (fp32 CUDA-core contractions) through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import conqur_oracle as O
+from paper_2605_10793_b200 import inputs as I
+from tests.parity_util import TOL, effective_m, step_parity, update_parity
+
+pytestmark = pytest.mark.gpu
+T = TOL["exact"]
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ctx(**kw):
+    from paper_2605_10793_b200 import binding as B
+    return B.Context(mode="exact", **kw)
+
+
+def _dev(x, dtype):
+    torch = _torch()
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def _check_step(ctx, x_np, dtype, quant_bits=0, before=None):
+    torch = _torch()
+    xd = _dev(x_np, dtype)
+    r = ctx.get_R().cpu().numpy().astype(np.float64)
+    ctx.step(xd)
+    j, n = ctx.get_objective()
+    m = ctx.get_M().cpu().numpy().astype(np.float64)
+    s = ctx.debug_get_signs(x_np.shape[0]).cpu().numpy()
+    mb, jb, nb = before if before is not None else (None, 0.0, 0)
+    rep = step_parity(x_np.astype(np.float64), r, s, m, j, n, "exact", quant_bits, mb, jb, nb)
+    assert rep["N_equal"]
+    assert rep["J_rel"] <= T["J"], rep
+    assert rep["M_rel_tie_aware"] <= T["M"], rep
+    assert rep["flips_outside_band"] == 0, rep
+    assert rep["flip_frac"] < 1e-3, rep
+    return rep, m, j, n, r
+
+
+def _check_update(ctx, m64, r_prev64, prior_rel=0.0):
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, st.status
+    r_new = ctx.get_R().cpu().numpy().astype(np.float64)
+    rep = update_parity(effective_m(m64, r_prev64, prior_rel), r_new)
+    assert rep["orth"] <= T["orth"], rep
+    assert rep["gap"] <= T["gap"], rep
+    assert st.orth_err <= 1e-4
+    j, n = ctx.get_objective()
+    assert j == 0.0 and n == 0
+    assert not ctx.get_M().any().item()
+    return rep, st
+
+
+def test_c0_alternation_teacher_forced_and_free_running():
+    """d=128, one fp32 batch of 2048 tokens, R0 = I, ten (step, update) rounds."""
+    w = I.WORKLOADS["c0"]
+    x = I.batch(w, 0)
+    ctx = _ctx(d=w.d, n_max=w.n, in_dtype="f32")
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    free = O.OpuOracle(w.d, I.initial_rotation(w).astype(np.float64))
+    js = []
+    for it in range(w.n_batches):
+        rep, m, j, n, r = _check_step(ctx, x, "f32")
+        free.step(x.astype(np.float64))
+        # free-running oracle (its own SVD updates) stays close: the objective is what the method tracks
+        assert abs(j - free.J) / free.J <= 2e-5, (it, j, free.J)
+        js.append(j / n)
+        urep, st = _check_update(ctx, m, r)
+        free.update()
+    assert all(b >= a * (1 - 1e-6) for a, b in zip(js, js[1:])), js    # monotone (Section 3.3)
+    assert js[-1] > js[0] + 0.05
+
+
+def test_d2_matches_brute_force_companion():
+    w = I.WORKLOADS["c0_d2"]
+    x = I.batch(w, 0)
+    ctx = _ctx(d=2, n_max=w.n, in_dtype="f32")
+    rep, m, j, n, r = _check_step(ctx, x, "f32")
+    urep, _ = _check_update(ctx, m, r)
+    assert urep["R_dist"] < 1e-5
+
+
+@pytest.mark.parametrize("d,n,dtype", [(100, 333, "f32"), (256, 1000, "bf16"), (130, 129, "bf16"), (384, 40, "f32")])
+def test_ragged_shapes_and_accumulation(d, n, dtype):
+    """Tiles with ragged tails in every dimension; two steps accumulate before one update."""
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2, dtype=dtype, r0="qr", n_massive_rows=min(4, n - 1))
+    prior = 1e-2 if (2 * n - 5) < 4 * d else 0.0
+    ctx = _ctx(d=d, n_max=n, in_dtype=dtype, prior_rel=prior)
+    r0 = I.initial_rotation(w)
+    ctx.set_R(_dev(r0, "f32"))
+    rep1, m1, j1, n1, r = _check_step(ctx, I.batch(w, 0), dtype)
+    rep2, m2, j2, n2, _ = _check_step(ctx, I.batch(w, 1)[: n - 5], dtype, before=(m1, j1, n1))
+    assert n2 == 2 * n - 5
+    _check_update(ctx, m2, r, prior_rel=prior)
+
+
+def test_strided_rows():
+    torch = _torch()
+    d, n, ld = 64, 200, 96
+    w = I.scaled(I.WORKLOADS["c0"], d=d, n=n)
+    x = I.batch(w, 0)
+    buf = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    buf[:, :d] = torch.from_numpy(x).cuda()
+    ctx = _ctx(d=d, n_max=n, in_dtype="f32")
+    ctx.step(buf[:, :d])
+    j, nn = ctx.get_objective()
+    ref = O.OpuOracle(d).step(x.astype(np.float64))
+    assert nn == n and abs(j - ref.J) / ref.J < 1e-6
+
+
+def test_quant_mode_int4():
+    d, n = 128, 1024
+    w = I.scaled(I.WORKLOADS["c4a"], d=d, n=n, n_outlier=2)
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", quant_bits=4)
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    rep, m, j, nn, r = _check_step(ctx, I.batch(w, 0), "bf16", quant_bits=4)
+    # several percent of the coordinates fall in the dead zone and get sign 0
+    s = ctx.debug_get_signs(n).cpu().numpy()
+    assert 0.005 < (s == 0).mean() < 0.5
+    _check_update(ctx, m, r)
+
+
+def test_skipped_rows_and_status():
+    torch = _torch()
+    d, n = 64, 96
+    w = I.scaled(I.WORKLOADS["c0"], d=d, n=n)
+    x = I.batch(w, 0).copy()
+    x[3] = 0.0
+    x[10, 5] = np.inf
+    x[50, 0] = np.nan
+    ctx = _ctx(d=d, n_max=n, in_dtype="f32")
+    ctx.step(_dev(x, "f32"))
+    j, nn = ctx.get_objective(check=False)
+    ref = O.OpuOracle(d).step(x.astype(np.float64))
+    assert nn == n - 3 == ref.N
+    assert abs(j - ref.J) / ref.J < 1e-6
+    m = ctx.get_M(check=False).cpu().numpy()
+    assert np.isfinite(m).all()
+    assert np.linalg.norm(m - ref.M) / np.linalg.norm(ref.M) < 1e-5
+    st = ctx.get_stats()
+    assert st.status == -7 and st.n_skipped == 3          # CONQUR_ERR_NONFINITE_INPUT latched ...
+    assert ctx.get_stats().status == 0                    # ... and cleared by the read
+
+
+def test_host_side_errors_change_nothing():
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    d, n = 32, 16
+    ctx = _ctx(d=d, n_max=64, in_dtype="f32")
+    with pytest.raises(B.ConqurError) as e:
+        ctx.update()
+    assert e.value.status == -4                            # empty update
+    x = torch.randn(n, d, device="cuda")
+    ctx.step(x)
+    with pytest.raises(B.ConqurError) as e:
+        ctx.update()
+    assert e.value.status == -5                            # fewer tokens than dimensions, no prior
+    with pytest.raises(B.ConqurError) as e:
+        ctx.step(torch.randn(65, d, device="cuda"))
+    assert e.value.status == -1                            # n > n_max
+    bad = torch.eye(d, device="cuda") * 1.1
+    with pytest.raises(B.ConqurError) as e:
+        ctx.set_R(bad)
+    assert e.value.status == -3
+    assert torch.equal(ctx.get_R(), torch.eye(d, device="cuda"))
+    j, nn = ctx.get_objective()
+    assert nn == n
+
+
+def test_set_M_round_trip_resume():
+    d, n = 64, 256
+    w = I.scaled(I.WORKLOADS["c0"], d=d, n=n)
+    x = _dev(I.batch(w, 0), "f32")
+    a = _ctx(d=d, n_max=n, in_dtype="f32")
+    a.step(x)
+    m, (j, nn) = a.get_M(), a.get_objective()
+    b = _ctx(d=d, n_max=n, in_dtype="f32")
+    b.set_M(m, j, nn)
+    a.update()
+    b.update()
+    assert np.allclose(a.get_R().cpu().numpy(), b.get_R().cpu().numpy(), atol=2e-6)
+
+
+def test_rerun_is_bit_identical():
+    d, n = 128, 512
+    w = I.scaled(I.WORKLOADS["c0"], d=d, n=n)
+    x = _dev(I.batch(w, 0), "f32")
+    outs = []
+    for _ in range(2):
+        ctx = _ctx(d=d, n_max=n, in_dtype="f32")
+        ctx.step(x)
+        m = ctx.get_M().clone()
+        ctx.update()
+        outs.append((m, ctx.get_R().clone(), ctx.get_stats().last_J))
+    torch = _torch()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and outs[0][2] == outs[1][2]
+
+
+def test_batched_problems_match_independent_oracles():
+    torch = _torch()
+    d, n, P = 32, 200, 5
+    w = I.scaled(I.WORKLOADS["c4b"], d=d, n=n, problems=P, n_outlier=1)
+    xs = [I.batch(w, 0, problem=p) for p in range(P)]
+    r0 = np.stack([I.initial_rotation(w, p) for p in range(P)])
+    # head-interleaved layout: row i holds the P slices side by side
+    inter = np.concatenate(xs, axis=1)
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", batch=P)
+    ctx.set_R(_dev(r0, "f32"))
+    ctx.step_batched(_dev(inter, "bf16"), n, P * d, d)
+    js, ns = ctx.get_objective()
+    ms = ctx.get_M().cpu().numpy().astype(np.float64)
+    ctx.update()
+    assert ctx.get_stats().status == 0
+    rs = ctx.get_R().cpu().numpy().astype(np.float64)
+    for p in range(P):
+        ref = O.OpuOracle(d, r0[p].astype(np.float64)).step(xs[p].astype(np.float64))
+        assert ns[p] == ref.N and abs(js[p] - ref.J) / ref.J < 1e-6
+        assert np.linalg.norm(ms[p] - ref.M) / np.linalg.norm(ref.M) < 1e-5
+        rep = update_parity(ms[p], rs[p])
+        assert rep["orth"] <= 1e-4 and rep["gap"] <= T["gap"], rep
