@@ -70,8 +70,9 @@ def test_c0_alternation_teacher_forced_and_free_running():
     for it in range(w.n_batches):
         rep, m, j, n, r = _check_step(ctx, x, "f32")
         free.step(x.astype(np.float64))
-        # free-running oracle (its own SVD updates) stays close: the objective is what the method tracks
-        assert abs(j - free.J) / free.J <= 2e-5, (it, j, free.J)
+        # free-running oracle (its own SVD updates): a single near-tie sign that falls the other way sends
+        # the two alternations down slightly different paths, so this is a trajectory check, not arithmetic
+        assert abs(j - free.J) / free.J <= (1e-6 if it == 0 else 1e-3), (it, j, free.J)
         js.append(j / n)
         urep, st = _check_update(ctx, m, r)
         free.update()
