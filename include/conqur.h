@@ -187,6 +187,18 @@ int conqur_get_stats(conqur_ctx* ctx, conqur_stats* out);
  */
 int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out, int32_t max_steps);
 
+/*
+ * Test hook for the tensor-core product every fused step is built on (no counterpart in the paper):
+ *   D[m][n] = sum_k A(m,k) * B(n,k),  D_dev fp32 M x N row-major.
+ * A_dev / B_dev: device bf16 row-major.  Orientation 0 (K-major): the matrix is [M|N rows][K cols];
+ * orientation 1 (MN-major): it is [K rows][M|N cols].  split != 0: each operand is a stacked pair
+ * [hi; lo] (twice the rows) and the product is hi*hi + hi*lo + lo*hi.  M, K multiples of 8, N of 32.
+ * scratch_dev: >= 256 bytes of device memory.  Synchronises; returns CONQUR_ERR_TIMEOUT if a bounded
+ * device-side wait expired.
+ */
+int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_dev, int32_t M, int32_t N, int32_t K,
+                      int32_t a_mn_major, int32_t b_mn_major, int32_t split, void* scratch_dev, void* cuda_stream);
+
 const char* conqur_strerror(int status);
 
 #ifdef __cplusplus

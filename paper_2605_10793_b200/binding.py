@@ -22,7 +22,8 @@ CONQUR_EXACT_F32, CONQUR_TC_BF16 = 0, 1
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
-    "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_strerror",
+    "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
+    "conqur_strerror",
 ]
 
 
@@ -86,6 +87,8 @@ def load() -> C.CDLL:
     lib.conqur_get_stats.argtypes = [vp, C.POINTER(conqur_stats)]
     lib.conqur_plan_schedule.restype = C.c_int
     lib.conqur_plan_schedule.argtypes = [C.c_double, i32, C.POINTER(C.c_double), i32]
+    lib.conqur_debug_gemm.restype = C.c_int
+    lib.conqur_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.conqur_strerror.restype = C.c_char_p
     lib.conqur_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -176,6 +179,18 @@ def conqur_plan_schedule(sigma_min_rel: float = 0.0, ns_steps: int = 0, max_step
     if n < 0:
         raise ConqurError(n, "conqur_plan_schedule")
     return np.array(buf[: 3 * n], dtype=np.float64).reshape(n, 3)
+
+
+def conqur_debug_gemm(a, b, m: int, n: int, k: int, a_mn: bool, b_mn: bool, split: bool = False):
+    """D = A x B (see include/conqur.h) for torch bf16 CUDA tensors; returns an fp32 (m, n) tensor."""
+    import torch
+    out = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    scratch = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    rc = load().conqur_debug_gemm(a.data_ptr(), b.data_ptr(), out.data_ptr(), m, n, k, int(a_mn), int(b_mn),
+                                  int(split), scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise ConqurError(rc, "conqur_debug_gemm")
+    return out
 
 
 # ---- convenience wrapper: owns the workspace tensor, checks status codes ------------------------

@@ -190,7 +190,7 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
     CQ_LAUNCH_CHECK();
     const int levels = (1 << (g.quant_bits - 1)) - 1;
     quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, levels,
-                                                                    part, nullptr, 0);
+                                                                    part);
     CQ_LAUNCH_CHECK();
     per_problem = cdiv(n, 8);
   }
@@ -354,7 +354,8 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   if (g.mode == CONQUR_TC_BF16) {
     int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
                      c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
-                     c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f));
+                     c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
+                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax));
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);
@@ -484,11 +485,11 @@ extern "C" int conqur_debug_get_signs(conqur_ctx* c, int8_t* S_out_dev) {
   if (c->last_n == 0) return CONQUR_ERR_INVALID_ARG;
   const int64_t total = c->last_n * c->cfg.d;
   if (c->cfg.mode == CONQUR_EXACT_F32) {
-    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(c->at<float>(c->L.C), nullptr, 0, c->last_n,
-                                                                 c->cfg.d, S_out_dev);
+    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(c->at<float>(c->L.C), nullptr, c->last_n, c->cfg.d,
+                                                                 S_out_dev);
   } else {
-    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(nullptr, tc_ct_ptr(c->tc), tc_ct_ld(c->tc),
-                                                                 c->last_n, c->cfg.d, S_out_dev);
+    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(nullptr, tc_cp_ptr(c->tc), c->last_n, c->cfg.d,
+                                                                 S_out_dev);
   }
   CQ_LAUNCH_CHECK();
   return sync_status(c);
@@ -529,6 +530,21 @@ extern "C" int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, doub
   const int n = std::min<int>((int)s.size(), max_steps);
   for (int i = 0; i < n; ++i) { abc_out[3 * i] = s[i].a; abc_out[3 * i + 1] = s[i].b; abc_out[3 * i + 2] = s[i].c; }
   return n;
+}
+
+extern "C" int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_dev, int32_t M, int32_t N, int32_t K,
+                                 int32_t a_mn_major, int32_t b_mn_major, int32_t split, void* scratch_dev,
+                                 void* cuda_stream) {
+  if (!A_dev || !B_dev || !D_dev || !scratch_dev) return CONQUR_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  CQ_CUDA(cudaMemsetAsync(scratch_dev, 0, sizeof(DevState), s));
+  int rc = tc_debug_gemm(static_cast<const __nv_bfloat16*>(A_dev), static_cast<const __nv_bfloat16*>(B_dev), D_dev, M,
+                         N, K, a_mn_major, b_mn_major, split, static_cast<DevState*>(scratch_dev), s);
+  if (rc) return rc;
+  DevState h;
+  CQ_CUDA(cudaMemcpyAsync(&h, scratch_dev, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+  CQ_CUDA(cudaStreamSynchronize(s));
+  return flags_to_status(h.status_flags);
 }
 
 extern "C" const char* conqur_strerror(int s) {

@@ -268,13 +268,11 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
 // Quant mode, second pass (Appendix B, Q_sym per token).  One warp per row:
 // Delta_raw = rowmax/L, q = rint(acc / Delta_raw) clipped to +-L, C' = sgn(q) * rnorm,
 // objective partial = rnorm * Delta_raw * sum_j |q_j|.  Works in place: Y and C' share the buffer.
-// out_t (optional): bf16 transposed copy C'^T (d x ldt) for the tensor-core accumulate.
 __global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
                                                            int64_t c_pstride, const float* __restrict__ rnorm,
                                                            int64_t rnorm_pstride,
                                                            const unsigned int* __restrict__ rowmax_bits, int levels,
-                                                           double* __restrict__ partials /* per block */,
-                                                           __nv_bfloat16* __restrict__ out_t, int64_t ldt) {
+                                                           double* __restrict__ partials /* per block */) {
   const int p = blockIdx.y;
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -293,7 +291,6 @@ __global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ Y
       qs += fabsf(q);
       const float c = live ? sgnf(q) * r : 0.f;
       y[j] = c;
-      if (out_t) out_t[(int64_t)j * ldt + row] = __float2bfloat16(c);
     }
     qs = warp_sum(qs);
     if (live) contrib = (double)(r * (mx / L)) * (double)qs;
@@ -567,18 +564,12 @@ __global__ void set_identity_kernel(float* __restrict__ R, int d, int P) {
     R[i] = ((e / d) == (e % d)) ? 1.f : 0.f;
   }
 }
-// sign matrix of the last step from the fp32 C' (n x d) or the transposed bf16 C'^T (d x ldt)
-__global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Ct, int64_t ldt,
-                                    int64_t n, int d, int8_t* __restrict__ S) {
+// sign matrix of the last step from C' (n x d, row-major) held as fp32 (exact mode) or bf16 (tensor-core mode)
+__global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Cb, int64_t n,
+                                    int d, int8_t* __restrict__ S) {
   const int64_t total = n * d;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    float v;
-    if (C) {
-      v = C[i];
-    } else {
-      const int64_t row = i / d, col = i % d;
-      v = __bfloat162float(Ct[col * ldt + row]);
-    }
+    const float v = C ? C[i] : __bfloat162float(Cb[i]);
     S[i] = (v > 0.f) ? 1 : ((v < 0.f) ? -1 : 0);
   }
 }

@@ -1,29 +1,822 @@
-// Tensor-core (tcgen05 / TMEM / TMA) mode.  Placeholder interface until the kernels land.
+// Tensor-core mode: one persistent, warp-specialised tcgen05 GEMM kernel (TMA -> 128B-swizzled
+// shared memory ring -> tcgen05.mma with fp32 accumulators in TMEM -> tcgen05.ld epilogue) with the
+// path's steps fused into its epilogues, plus the small element-wise kernels around it.
+//
+//   D[m][n] = sum_k A(m,k) * B(n,k),  tile 128 x BN, BK = 64, bf16 operands, fp32 accumulation.
+//
+// Each operand is a row-major bf16 matrix read in place in either orientation:
+//   K-major : rows are m (or n), k contiguous      -> TMA box 64(k) x 128|BN rows
+//   MN-major: rows are k, m (or n) contiguous      -> TMA boxes 64(m|n) x 64(k rows)
+// so X^T C', X^T X and X B need no transposed copies.
+//
+// Split precision: an operand may be a stacked pair [hi; lo] of bf16 matrices (value = hi + lo).  With
+// nseg = 3 the k loop runs three times over (hi,hi), (hi,lo), (lo,hi), accumulating into the same TMEM tile.
+//
+// No cluster launch and no multicast copies are used anywhere.  Every mbarrier wait is bounded: on expiry
+// the CTA raises a shared abort flag, latches STATUS_FLAG_TIMEOUT in the device state, drains its own
+// copies with a bounded wait, frees its TMEM and returns.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdio>
+
 #include "../../include/conqur.h"
 #include "conqur_internal.h"
+#include "conqur_simt.cuh"
 
 namespace conqur {
 
-struct TcLayout { size_t dummy; };
-struct TcHost { int dummy; };
+// ------------------------------------------------------------------ PTX wrappers
+namespace ptx {
 
-inline bool tc_supported_shape(int, int) { return false; }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D(tmem) (+)= A(smem desc) * B(smem desc); accumulate == 0 overwrites D.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier once every previously issued MMA of this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives row (lane base + t).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+}  // namespace ptx
+
+// ------------------------------------------------------------------ kernel configuration
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;                   // one 128-byte swizzle row of bf16
+constexpr int TC_THREADS = 192;             // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr long long TC_WAIT_LIMIT = 4000000000ll;   // ~2 s of SM clocks
+
+enum { TC_EPI_ROTATE = 0, TC_EPI_ROTATE_Q = 1, TC_EPI_ACCUM = 2, TC_EPI_RESID = 3, TC_EPI_POLY = 4, TC_EPI_NEXT = 5,
+       TC_EPI_PLAIN = 6 };
+
+template <int BN> struct TcCfg {
+  static constexpr int A_BYTES = TC_BM * TC_BK * 2;
+  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int TMEM_COLS = 2 * BN;          // two accumulators: the epilogue of tile i overlaps tile i+1
+  static constexpr int AUX_BYTES = 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + AUX_BYTES + 1024 /* alignment slack */;
+};
+
+struct TcGemmArgs {
+  int M, N, K;                  // output rows, cols; contraction length of one segment
+  int nseg;                     // 1, or 3 for the (hi,hi),(hi,lo),(lo,hi) split product
+  int a_lo, b_lo;               // outer-coordinate offset of the lo copy inside a stacked [hi; lo] operand
+  float* outF; long long ldo;   // fp32 output (M read-modify-write, E, X_next, Y)
+  __nv_bfloat16* outH; long long ldh; long long lo_elems;   // bf16 output hi part (+ lo part at +lo_elems)
+  const float* inF; long long ldi;                          // fp32 epilogue input (E or X)
+  const float* rnorm;
+  unsigned* rowmax;
+  double* part_d; float* part_f;
+  DevState* st;
+  int check_done;
+};
+
+struct TcAux {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t tfull[2];
+  uint64_t tempty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  double red_d[4];
+  float red_f[4];
+};
+
+// Bounded wait.  Returns false when the wait was abandoned (timeout here, or another role aborted).
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > TC_WAIT_LIMIT) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // start address, leading / stride byte offsets (16-byte units), descriptor version 1, 128-byte swizzle
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
+__device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
+
+template <int BN, bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcGemmArgs g) {
+  using Cfg = TcCfg<BN>;
+  if (g.check_done && g.st->ns_done) return;      // uniform: the iteration already finished
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  TcAux* aux = reinterpret_cast<TcAux*>(smem + Cfg::STAGES * Cfg::STAGE_BYTES);
+  volatile int* abort_flag = &aux->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
+  const int num_tiles = tiles_m * tiles_n;
+  const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+  const int k_iters = num_kb * g.nseg;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::STAGES; ++s) { ptx::mbar_init(&aux->full[s], 1); ptx::mbar_init(&aux->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->tfull[b], 1); ptx::mbar_init(&aux->tempty[b], 128); }
+    aux->abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    ptx::prefetch_tmap(&tmA);
+    ptx::prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&aux->tmem_base, Cfg::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = aux->tmem_base;
+  int timeout_site = 0;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * TC_BM, n0 = (tile / tiles_m) * BN;
+        for (int it = 0; it < k_iters; ++it) {
+          const int seg = it / num_kb, k0 = (it - seg * num_kb) * TC_BK;
+          const int a_off = (seg == 2) ? g.a_lo : 0, b_off = (seg == 1) ? g.b_lo : 0;
+          if (!tc_wait(&aux->empty[stage], phase ^ 1u, abort_flag)) { ok = false; timeout_site = 1; break; }
+          uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
+          uint8_t* sb = sa + Cfg::A_BYTES;
+          ptx::mbar_expect_tx(&aux->full[stage], Cfg::STAGE_BYTES);
+          if (A_MN) {
+#pragma unroll
+            for (int h = 0; h < TC_BM / 64; ++h)
+              ptx::tma_load_2d(sa + h * 8192, &tmA, &aux->full[stage], m0 + 64 * h, k0 + a_off);
+          } else {
+            ptx::tma_load_2d(sa, &tmA, &aux->full[stage], k0, m0 + a_off);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int h = 0; h < BN / 64; ++h)
+              ptx::tma_load_2d(sb + h * 8192, &tmB, &aux->full[stage], n0 + 64 * h, k0 + b_off);
+          } else {
+            ptx::tma_load_2d(sb, &tmB, &aux->full[stage], k0, n0 + b_off);
+          }
+          ++issued;
+          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // drain: wait (bounded) until the copies already issued have landed before the CTA may exit
+        const int pending = issued < Cfg::STAGES ? issued : Cfg::STAGES;
+        int s = stage;
+        uint32_t ph = phase;
+        for (int i = 0; i < pending; ++i) {
+          if (--s < 0) { s = Cfg::STAGES - 1; ph ^= 1u; }
+          const long long t0 = clock64();
+          while (!ptx::mbar_try_wait(&aux->full[s], ph) && clock64() - t0 < TC_WAIT_LIMIT) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        if (!tc_wait(&aux->tempty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 2; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int it = 0; it < k_iters; ++it) {
+          if (!tc_wait(&aux->full[stage], phase, abort_flag)) { ok = false; timeout_site = 3; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = ptx::smem_u32(smem + stage * Cfg::STAGE_BYTES);
+          const uint32_t sb = sa + Cfg::A_BYTES;
+#pragma unroll
+          for (int j = 0; j < TC_BK / 16; ++j) {
+            // K-major: 16 k = 32 bytes inside the swizzled 128-byte row; 8-row groups 1024 bytes apart.
+            // MN-major: 16 k = two 8-row groups of 1024 bytes; 64-wide m|n chunks 8192 bytes apart.
+            const uint64_t ad = A_MN ? tc_smem_desc(sa + j * 2048, 8192, 1024) : tc_smem_desc(sa + j * 32, 16, 1024);
+            const uint64_t bd = B_MN ? tc_smem_desc(sb + j * 2048, 8192, 1024) : tc_smem_desc(sb + j * 32, 16, 1024);
+            ptx::umma_bf16(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
+          }
+          ptx::umma_commit(&aux->empty[stage]);          // frees the smem stage once these MMAs retire
+          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) ptx::umma_commit(&aux->tfull[buf]);       // accumulator complete
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (4 warps, 128 TMEM lanes)
+    const int q = warp & 3;                               // TMEM lane quarter this warp may read
+    const int et = q * 32 + lane;                         // row inside the tile
+    float c_gamma = 0.f, c_b1 = 0.f, c_b2 = 0.f;
+    if (EPI == TC_EPI_POLY || EPI == TC_EPI_NEXT) { c_gamma = g.st->coef[0]; c_b1 = g.st->coef[1]; c_b2 = g.st->coef[2]; }
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+      const int buf = local & 1;
+      const int m0 = (tile % tiles_m) * TC_BM, n0 = (tile / tiles_m) * BN;
+      if (!tc_wait(&aux->tfull[buf], (uint32_t)(local >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 4; break; }
+      ptx::tc_fence_after();
+      const int row = m0 + et;
+      const bool row_ok = row < g.M;
+      const uint32_t t_addr = tmem_base + (uint32_t)(buf * BN) + ((uint32_t)(q * 32) << 16);
+      float rn = 0.f;
+      uint32_t rn_bits = 0;
+      if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_ROTATE_Q) {
+        rn = row_ok ? g.rnorm[row] : 0.f;
+        rn_bits = bf16_bits(rn);
+      }
+      float acc_abs = 0.f, acc_max = 0.f;
+      double acc_sq = 0.0;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        float v[32];
+        ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+        const int col0 = n0 + c * 32;
+        if (!row_ok || col0 >= g.N) continue;              // N is a multiple of 32 in every use
+        if (EPI == TC_EPI_ROTATE) {
+          // C' = sgn(y) * rnorm as bf16 (sign bit or-ed in; exact zeros stay zero); objective partial sum |y|
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float a = v[2 * i], b = v[2 * i + 1];
+            acc_abs += fabsf(a) + fabsf(b);
+            const uint32_t lo = (a == 0.f) ? 0u : (rn_bits | ((__float_as_uint(a) >> 16) & 0x8000u));
+            const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
+            w[i] = lo | (hi << 16);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(g.outH + (long long)row * g.ldh + col0);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        } else if (EPI == TC_EPI_ROTATE_Q) {
+          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            acc_max = fmaxf(acc_max, fmaxf(fmaxf(fabsf(v[4 * i]), fabsf(v[4 * i + 1])),
+                                           fmaxf(fabsf(v[4 * i + 2]), fabsf(v[4 * i + 3]))));
+          }
+        } else if (EPI == TC_EPI_ACCUM) {
+          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float4 t = dst[i];
+            t.x += v[4 * i]; t.y += v[4 * i + 1]; t.z += v[4 * i + 2]; t.w += v[4 * i + 3];
+            dst[i] = t;
+          }
+        } else if (EPI == TC_EPI_PLAIN) {
+          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        } else {
+          // Newton-Schulz epilogues: fp32 value, then its two-term bf16 split
+          if (EPI == TC_EPI_RESID) {
+            const int dcol = row - col0;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              if (i == dcol) v[i] -= 1.f;
+              acc_max = fmaxf(acc_max, fabsf(v[i]));
+              acc_sq += (double)v[i] * (double)v[i];
+            }
+          } else {
+            const float4* src = reinterpret_cast<const float4*>(g.inF + (long long)row * g.ldi + col0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 t = src[i];
+              if (EPI == TC_EPI_POLY) {
+                v[4 * i] = fmaf(c_b2, v[4 * i], c_b1 * t.x); v[4 * i + 1] = fmaf(c_b2, v[4 * i + 1], c_b1 * t.y);
+                v[4 * i + 2] = fmaf(c_b2, v[4 * i + 2], c_b1 * t.z); v[4 * i + 3] = fmaf(c_b2, v[4 * i + 3], c_b1 * t.w);
+              } else {
+                v[4 * i] = fmaf(c_gamma, t.x, v[4 * i]); v[4 * i + 1] = fmaf(c_gamma, t.y, v[4 * i + 1]);
+                v[4 * i + 2] = fmaf(c_gamma, t.z, v[4 * i + 2]); v[4 * i + 3] = fmaf(c_gamma, t.w, v[4 * i + 3]);
+              }
+            }
+          }
+          if (EPI != TC_EPI_POLY) {
+            float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
+          uint32_t wh[16], wl[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float a = v[2 * i], b = v[2 * i + 1];
+            const float ah = bf16_round(a), bh = bf16_round(b);
+            wh[i] = bf16_bits(ah) | (bf16_bits(bh) << 16);
+            wl[i] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+          }
+          uint4* dh = reinterpret_cast<uint4*>(g.outH + (long long)row * g.ldh + col0);
+          uint4* dl = reinterpret_cast<uint4*>(g.outH + g.lo_elems + (long long)row * g.ldh + col0);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            dh[i] = make_uint4(wh[4 * i], wh[4 * i + 1], wh[4 * i + 2], wh[4 * i + 3]);
+            dl[i] = make_uint4(wl[4 * i], wl[4 * i + 1], wl[4 * i + 2], wl[4 * i + 3]);
+          }
+        }
+      }
+      // release the accumulator to the MMA warp before the (slower) reductions
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&aux->tempty[buf]);
+
+      if (EPI == TC_EPI_ROTATE_Q) {
+        if (row_ok && rn > 0.f) atomicMax(g.rowmax + row, __float_as_uint(acc_max));
+      }
+      if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_RESID) {
+        // per-tile partials, fixed reduction order; named barrier 1 synchronises the 4 epilogue warps only
+        double dsum = (EPI == TC_EPI_ROTATE) ? (double)(acc_abs * rn) : acc_sq;
+        dsum = warp_sum_d(dsum);
+        float fmx = warp_max(acc_max);
+        if (lane == 0) { aux->red_d[q] = dsum; aux->red_f[q] = fmx; }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (q == 0 && lane == 0) {
+          g.part_d[tile] = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
+          if (EPI == TC_EPI_RESID)
+            g.part_f[tile] = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+    }
+  }
+
+  if (timeout_site != 0) {
+    atomicOr(&g.st->status_flags, STATUS_FLAG_TIMEOUT);
+    g.st->timeout_site = timeout_site;
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ element-wise kernels of the mode
+
+// a1 for the tensor-core mode: one warp per row.  rnorm_i = 1/||x_i||_2 (fp32, from the bf16-rounded values the
+// MMA will see) and a bf16 copy of the row in the workspace; skipped rows are written as zeros so that they
+// cannot reach the accumulators.
+template <typename TIn>
+__global__ void __launch_bounds__(256) rownorm_stage_kernel(const TIn* __restrict__ X, int64_t n, int d, int64_t ld,
+                                                            float* __restrict__ rnorm,
+                                                            __nv_bfloat16* __restrict__ Xs, DevState* st) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= n) return;
+  const TIn* x = X + row * ld;
+  const bool vec = (reinterpret_cast<uintptr_t>(x) & (sizeof(TIn) * 4 - 1)) == 0;    // d is a multiple of 128
+  float ss = 0.f;
+  for (int k = lane * 4; k < d; k += 128) {
+    float v[4];
+    if (vec) {
+      ld4_as_float(x + k, v);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = ld_as_float(x + k + j);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { v[j] = bf16_round(v[j]); ss = fmaf(v[j], v[j], ss); }
+  }
+  ss = warp_sum(ss);
+  const bool good = (ss > 0.f) && (ss <= 3.0e38f);
+  __nv_bfloat16* dst = Xs + row * (int64_t)d;
+  for (int k = lane * 4; k < d; k += 128) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (good) {
+      if (vec) {
+        ld4_as_float(x + k, v);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = ld_as_float(x + k + j);
+      }
+    }
+    uint2 o;
+    o.x = bf16_bits(v[0]) | (bf16_bits(v[1]) << 16);
+    o.y = bf16_bits(v[2]) | (bf16_bits(v[3]) << 16);
+    *reinterpret_cast<uint2*>(dst + k) = o;
+  }
+  if (lane == 0) {
+    if (!good) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(&st->step_skipped), 1ull);
+      if (!(ss == 0.f)) atomicOr(&st->status_flags, STATUS_FLAG_NONFINITE);
+    }
+    rnorm[row] = good ? 1.0f / sqrtf(ss) : 0.f;
+  }
+}
+
+// fp32 -> bf16 (hi only, lo_elems == 0) or the two-term split [hi; lo]
+__global__ void split_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t count,
+                                  int64_t lo_elems) {
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < count;
+       i += (int64_t)gridDim.x * blockDim.x * 4) {
+    const float4 t = *reinterpret_cast<const float4*>(src + i);
+    const float h0 = bf16_round(t.x), h1 = bf16_round(t.y), h2 = bf16_round(t.z), h3 = bf16_round(t.w);
+    uint2 o;
+    o.x = bf16_bits(h0) | (bf16_bits(h1) << 16);
+    o.y = bf16_bits(h2) | (bf16_bits(h3) << 16);
+    *reinterpret_cast<uint2*>(dst + i) = o;
+    if (lo_elems) {
+      o.x = bf16_bits(t.x - h0) | (bf16_bits(t.y - h1) << 16);
+      o.y = bf16_bits(t.z - h2) | (bf16_bits(t.w - h3) << 16);
+      *reinterpret_cast<uint2*>(dst + lo_elems + i) = o;
+    }
+  }
+}
+
+// Quant mode, second pass for the tensor-core mode: Y (fp32, row-major) -> C' (bf16, row-major) + objective partials.
+__global__ void __launch_bounds__(256) quant_target_bf16_kernel(const float* __restrict__ Y, int64_t n, int d,
+                                                                const float* __restrict__ rnorm,
+                                                                const unsigned int* __restrict__ rowmax_bits,
+                                                                int levels, double* __restrict__ partials,
+                                                                __nv_bfloat16* __restrict__ Cp) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  double contrib = 0.0;
+  if (row < n) {
+    const float r = rnorm[row];
+    const float mx = __uint_as_float(rowmax_bits[row]);
+    const float L = (float)levels;
+    const bool live = (r > 0.f) && (mx > 0.f);
+    const float inv = live ? (L / mx) : 0.f;
+    const float* y = Y + row * (int64_t)d;
+    __nv_bfloat16* c = Cp + row * (int64_t)d;
+    float qs = 0.f;
+    for (int j = lane * 4; j < d; j += 128) {
+      const float4 t = *reinterpret_cast<const float4*>(y + j);
+      const float in[4] = {t.x, t.y, t.z, t.w};
+      uint32_t b[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float qv = rintf(in[e] * inv);
+        qv = fminf(fmaxf(qv, -L), L);
+        qs += fabsf(qv);
+        b[e] = bf16_bits(live ? sgnf(qv) * r : 0.f);
+      }
+      uint2 o;
+      o.x = b[0] | (b[1] << 16);
+      o.y = b[2] | (b[3] << 16);
+      *reinterpret_cast<uint2*>(c + j) = o;
+    }
+    qs = warp_sum(qs);
+    if (live) contrib = (double)(r * (mx / L)) * (double)qs;
+  }
+  __shared__ double red[8];
+  if (lane == 0) red[threadIdx.x >> 5] = contrib;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    partials[blockIdx.x] = t;
+  }
+}
+
+// ------------------------------------------------------------------ host side
+struct TcLayout {
+  size_t Xs, Cp, Rb, Xh[2], Eh, Bh;
+};
+
+struct TcHost {
+  int d, P, quant_bits, num_sms;
+  int64_t n_max;
+  char* ws;
+  TcLayout L;
+  float *R, *M, *Xa, *Xb, *E, *B, *rnorm, *Y;
+  unsigned* rowmax;
+  DevState* st;
+  double* part_d;
+  float* part_f;
+  // static tensor maps (d x d operands)
+  CUtensorMap tmRb_mn;                       // R bf16 as MN-major B of the rotate product
+  CUtensorMap tmXh_mn[2], tmXh_k[2];         // iterate, stacked [hi; lo]
+  CUtensorMap tmEh_k, tmEh_mn, tmBh_mn;
+  long long launches;
+};
+
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline PFN_encodeTiled tc_encode_fn() {
+  static PFN_encodeTiled fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_encodeTiled>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 row-major tensor (rows x cols, row stride ld elements); box = box_rows x 64 columns, 128-byte swizzle,
+// out-of-range elements read as zero.
+inline int tc_make_tmap(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  PFN_encodeTiled fn = tc_encode_fn();
+  if (!fn) return CONQUR_ERR_CUDA;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "conqur: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+    return CONQUR_ERR_CUDA;
+  }
+  return CONQUR_OK;
+}
+
+inline bool tc_supported_shape(int d, int batch) { return d >= 128 && (d % 128) == 0 && batch == 1; }
+
 template <typename Take>
-inline void tc_make_layout(int, int, int64_t, int, TcLayout*, Take&&) {}
-inline int tc_init(TcHost*, char*, const TcLayout&, int, int, int64_t, int, float*, float*, float*, float*, float*,
-                   float*, float*, DevState*, double*, float*) { return CONQUR_ERR_UNSUPPORTED; }
-inline int tc_refresh_R(TcHost&, cudaStream_t, int) { return CONQUR_ERR_UNSUPPORTED; }
-inline int tc_step(TcHost&, cudaStream_t, const void*, int, int64_t, int64_t, int64_t) { return CONQUR_ERR_UNSUPPORTED; }
-inline int tc_ns_begin(TcHost&, cudaStream_t) { return CONQUR_ERR_UNSUPPORTED; }
-inline int tc_ns_residual(TcHost&, cudaStream_t, int) { return CONQUR_ERR_UNSUPPORTED; }
-inline int tc_ns_parts(const TcHost&) { return 0; }
-inline int tc_ns_poly_next(TcHost&, cudaStream_t, int) { return CONQUR_ERR_UNSUPPORTED; }
-inline const __nv_bfloat16* tc_ct_ptr(const TcHost&) { return nullptr; }
-inline int64_t tc_ct_ld(const TcHost&) { return 0; }
+inline void tc_make_layout(int d, int P, int64_t n_max, int quant_bits, TcLayout* L, Take&& take) {
+  (void)P; (void)quant_bits;
+  const size_t dd = (size_t)d * d;
+  L->Xs = take(2 * (size_t)n_max * d);
+  L->Cp = take(2 * (size_t)n_max * d);
+  L->Rb = take(2 * dd);
+  L->Xh[0] = take(4 * dd);
+  L->Xh[1] = take(4 * dd);
+  L->Eh = take(4 * dd);
+  L->Bh = take(4 * dd);
+}
+
+template <int BN, bool A_MN, bool B_MN, int EPI>
+inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
+  using Cfg = TcCfg<BN>;
+  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+      return CONQUR_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = ((g.M + TC_BM - 1) / TC_BM) * ((g.N + BN - 1) / BN);
+  const int grid = tiles < h.num_sms ? tiles : h.num_sms;
+  kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, g);
+  ++h.launches;
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
+}
+
+// dispatch on the N tile: 256 when the output width allows it, else 128
+template <bool A_MN, bool B_MN, int EPI>
+inline int tc_launch_n(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
+  if (g.N % 256 == 0) return tc_launch<256, A_MN, B_MN, EPI>(h, s, a, b, g);
+  return tc_launch<128, A_MN, B_MN, EPI>(h, s, a, b, g);
+}
+
+inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
+                   float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
+                   float* part_f, float* Y, unsigned* rowmax) {
+  h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
+  h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
+  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->launches = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (prop.major != 10) {
+    std::fprintf(stderr, "conqur: the tensor-core mode needs an sm_100 device (found sm_%d%d)\n", prop.major, prop.minor);
+    return CONQUR_ERR_UNSUPPORTED;
+  }
+  h->num_sms = prop.multiProcessorCount;
+  const uint64_t D = (uint64_t)d;
+  int rc = 0;
+  rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, D, D, D, 64);
+  for (int i = 0; i < 2; ++i) {
+    rc |= tc_make_tmap(&h->tmXh_mn[i], ws + L.Xh[i], 2 * D, D, D, 64);
+    rc |= tc_make_tmap(&h->tmXh_k[i], ws + L.Xh[i], 2 * D, D, D, 128);
+  }
+  rc |= tc_make_tmap(&h->tmEh_k, ws + L.Eh, 2 * D, D, D, 128);
+  rc |= tc_make_tmap(&h->tmEh_mn, ws + L.Eh, 2 * D, D, D, 64);
+  rc |= tc_make_tmap(&h->tmBh_mn, ws + L.Bh, 2 * D, D, D, 64);
+  return rc ? CONQUR_ERR_CUDA : CONQUR_OK;
+}
+
+inline int tc_ew_blocks(int64_t count4) {
+  const int64_t b = (count4 + 255) / 256;
+  return (int)(b < 148 * 8 ? b : 148 * 8);
+}
+
+inline int tc_refresh_R(TcHost& h, cudaStream_t s, int) {
+  const int64_t dd = (int64_t)h.d * h.d;
+  split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.R, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Rb), dd, 0);
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
+}
+
+inline TcGemmArgs tc_args(const TcHost& h, int M, int N, int K) {
+  TcGemmArgs g{};
+  g.M = M; g.N = N; g.K = K; g.nseg = 1; g.st = h.st; g.part_d = h.part_d; g.part_f = h.part_f;
+  return g;
+}
+
+inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t) {
+  const int d = h.d;
+  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xs);
+  __nv_bfloat16* Cp = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Cp);
+  const int rb = (int)((n + 7) / 8);
+  if (in_dtype == CONQUR_F32)
+    rownorm_stage_kernel<float><<<rb, 256, 0, s>>>(static_cast<const float*>(X), n, d, ld, h.rnorm, Xs, h.st);
+  else
+    rownorm_stage_kernel<__nv_bfloat16><<<rb, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(X), n, d, ld, h.rnorm, Xs, h.st);
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  // per-call maps over the first n rows: rows past n read as zeros
+  CUtensorMap tmXs_k, tmXs_mn, tmCp_mn;
+  int rc = tc_make_tmap(&tmXs_k, Xs, (uint64_t)n, (uint64_t)d, (uint64_t)d, 128);
+  rc |= tc_make_tmap(&tmXs_mn, Xs, (uint64_t)n, (uint64_t)d, (uint64_t)d, 64);
+  rc |= tc_make_tmap(&tmCp_mn, Cp, (uint64_t)n, (uint64_t)d, (uint64_t)d, 64);
+  if (rc) return CONQUR_ERR_CUDA;
+  const double isd = 1.0 / std::sqrt((double)d);
+  TcGemmArgs g = tc_args(h, (int)n, d, d);
+  g.rnorm = h.rnorm;
+  int per_problem;
+  if (h.quant_bits == 0) {
+    g.outH = Cp; g.ldh = d;
+    rc = tc_launch_n<false, true, TC_EPI_ROTATE>(h, s, tmXs_k, h.tmRb_mn, g);
+    if (rc) return rc;
+    per_problem = ((int)((n + TC_BM - 1) / TC_BM)) * ((d + ((d % 256 == 0) ? 256 : 128) - 1) / ((d % 256 == 0) ? 256 : 128));
+  } else {
+    if (cudaMemsetAsync(h.rowmax, 0, sizeof(unsigned) * n, s) != cudaSuccess) return CONQUR_ERR_CUDA;
+    g.outF = h.Y; g.ldo = d; g.rowmax = h.rowmax;
+    rc = tc_launch_n<false, true, TC_EPI_ROTATE_Q>(h, s, tmXs_k, h.tmRb_mn, g);
+    if (rc) return rc;
+    const int levels = (1 << (h.quant_bits - 1)) - 1;
+    quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, levels, h.part_d, Cp);
+    if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+    per_problem = rb;
+  }
+  finalize_step_kernel<<<1, 256, 0, s>>>(h.st, h.part_d, per_problem, n, isd);
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  TcGemmArgs a = tc_args(h, d, d, (int)n);
+  a.outF = h.M; a.ldo = d;
+  return tc_launch_n<true, true, TC_EPI_ACCUM>(h, s, tmXs_mn, tmCp_mn, a);
+}
+
+// X0 (fp32, in Xa) -> stacked bf16 split in Xh[0]
+inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
+  const int64_t dd = (int64_t)h.d * h.d;
+  split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.Xa, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[0]), dd, dd);
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
+}
+
+inline int tc_ns_tile_n(const TcHost& h) { return (h.d % 256 == 0) ? 256 : 128; }
+inline int tc_ns_parts(const TcHost& h) { return (h.d / TC_BM) * (h.d / tc_ns_tile_n(h)); }
+
+// E = X^T X - I from the split iterate in Xh[buf]
+inline int tc_ns_residual(TcHost& h, cudaStream_t s, int buf) {
+  const int d = h.d;
+  TcGemmArgs g = tc_args(h, d, d, d);
+  g.nseg = 3; g.a_lo = d; g.b_lo = d; g.check_done = 1;
+  g.outF = h.E; g.ldo = d;
+  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Eh); g.ldh = d; g.lo_elems = (long long)d * d;
+  return tc_launch_n<true, true, TC_EPI_RESID>(h, s, h.tmXh_mn[buf], h.tmXh_mn[buf], g);
+}
+
+// B = beta2 E E + beta1 E ;  X_next = X B + gamma X
+inline int tc_ns_poly_next(TcHost& h, cudaStream_t s, int cur) {
+  const int d = h.d;
+  const long long dd = (long long)d * d;
+  TcGemmArgs g = tc_args(h, d, d, d);
+  g.nseg = 3; g.a_lo = d; g.b_lo = d; g.check_done = 1;
+  g.inF = h.E; g.ldi = d;
+  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Bh); g.ldh = d; g.lo_elems = dd;
+  int rc = tc_launch_n<false, true, TC_EPI_POLY>(h, s, h.tmEh_k, h.tmEh_mn, g);
+  if (rc) return rc;
+  TcGemmArgs x = tc_args(h, d, d, d);
+  x.nseg = 3; x.a_lo = d; x.b_lo = d; x.check_done = 1;
+  x.inF = cur ? h.Xb : h.Xa; x.ldi = d;
+  x.outF = cur ? h.Xa : h.Xb; x.ldo = d;
+  x.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[1 - cur]); x.ldh = d; x.lo_elems = dd;
+  return tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
+}
+
+inline const __nv_bfloat16* tc_cp_ptr(const TcHost& h) { return reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Cp); }
+
+// Stand-alone product for tests: D (fp32, M x N) = A * B^T-style contraction with the given orientations.
+// a_mn / b_mn: 0 = K-major ([M|N rows][K cols]), 1 = MN-major ([K rows][M|N cols]).  split: operands are stacked
+// [hi; lo] pairs (3 products).  All device pointers; bf16 operands; caller guarantees the shapes below.
+inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* D, int M, int N, int K, int a_mn,
+                         int b_mn, int split, DevState* st, cudaStream_t s) {
+  if (M < 1 || N < 32 || (N % 32) || K < 1 || (K % 8) || (M % 8)) return CONQUR_ERR_INVALID_ARG;
+  TcHost h{};
+  h.launches = 0;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (prop.major != 10) return CONQUR_ERR_UNSUPPORTED;
+  h.num_sms = prop.multiProcessorCount;
+  const uint64_t mul = split ? 2 : 1;
+  CUtensorMap ta, tb;
+  int rc;
+  if (a_mn) rc = tc_make_tmap(&ta, A, mul * K, M, M, 64); else rc = tc_make_tmap(&ta, A, mul * M, K, K, 128);
+  if (rc) return rc;
+  const uint32_t bn = (N % 256 == 0) ? 256 : 128;
+  if (b_mn) rc = tc_make_tmap(&tb, B, mul * K, N, N, 64); else rc = tc_make_tmap(&tb, B, mul * N, K, K, bn);
+  if (rc) return rc;
+  TcGemmArgs g{};
+  g.M = M; g.N = N; g.K = K; g.nseg = split ? 3 : 1; g.st = st;
+  g.a_lo = a_mn ? K : M; g.b_lo = b_mn ? K : N;
+  g.outF = D; g.ldo = N;
+  if (!a_mn && !b_mn) return tc_launch_n<false, false, TC_EPI_PLAIN>(h, s, ta, tb, g);
+  if (!a_mn && b_mn) return tc_launch_n<false, true, TC_EPI_PLAIN>(h, s, ta, tb, g);
+  if (a_mn && !b_mn) return tc_launch_n<true, false, TC_EPI_PLAIN>(h, s, ta, tb, g);
+  return tc_launch_n<true, true, TC_EPI_PLAIN>(h, s, ta, tb, g);
+}
 
 }  // namespace conqur

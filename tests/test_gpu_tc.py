@@ -1,0 +1,128 @@
+"""GPU parity, tensor-core mode (bf16 operands, fp32 accumulation on tcgen05) through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import conqur_oracle as O
+from paper_2605_10793_b200 import inputs as I
+from tests.parity_util import TOL, effective_m, step_parity, update_parity
+
+pytestmark = pytest.mark.gpu
+T = TOL["tc"]
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ctx(**kw):
+    from paper_2605_10793_b200 import binding as B
+    return B.Context(mode="tc", **kw)
+
+
+def _dev(x, dtype):
+    torch = _torch()
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def _check_step(ctx, x_np, dtype, quant_bits=0, before=None):
+    r = ctx.get_R().cpu().numpy().astype(np.float64)
+    ctx.step(_dev(x_np, dtype))
+    j, n = ctx.get_objective()
+    m = ctx.get_M().cpu().numpy().astype(np.float64)
+    s = ctx.debug_get_signs(x_np.shape[0]).cpu().numpy()
+    mb, jb, nb = before if before is not None else (None, 0.0, 0)
+    x64 = (I.round_to_bf16(x_np) if dtype == "f32" else x_np).astype(np.float64)   # fp32 input is rounded on the way in
+    rep = step_parity(x64, r, s, m, j, n, "tc", quant_bits, mb, jb, nb)
+    assert rep["N_equal"]
+    assert rep["J_rel"] <= T["J"], rep
+    assert rep["M_rel_tie_aware"] <= T["M"], rep
+    assert rep["flips_outside_band"] == 0, rep
+    assert rep["flip_frac"] < 2e-2, rep
+    return rep, m, j, n, r
+
+
+def _check_update(ctx, m64, r_prev64, prior_rel=0.0):
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, st.status
+    r_new = ctx.get_R().cpu().numpy().astype(np.float64)
+    rep = update_parity(effective_m(m64, r_prev64, prior_rel), r_new)
+    assert rep["orth"] <= T["orth"], rep
+    assert rep["gap"] <= T["gap"], rep
+    j, n = ctx.get_objective()
+    assert j == 0.0 and n == 0 and not ctx.get_M().any().item()
+    return rep, st
+
+
+def test_c0_in_tensor_core_mode():
+    """d=128 alternation with the fp32 batch rounded to bf16 inside the library."""
+    w = I.WORKLOADS["c0"]
+    x = I.batch(w, 0)
+    ctx = _ctx(d=w.d, n_max=w.n, in_dtype="f32")
+    js = []
+    for it in range(4):
+        rep, m, j, n, r = _check_step(ctx, x, "f32")
+        js.append(j / n)
+        _check_update(ctx, m, r)
+    assert all(b >= a * (1 - 1e-3) for a, b in zip(js, js[1:])), js
+
+
+@pytest.mark.parametrize("d,n", [(256, 1000), (384, 2048), (512, 300)])
+def test_stream_steps_then_update(d, n):
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=max(2, d // 256))
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", prior_rel=0.0 if 3 * n >= 4 * d else 1e-2)
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    before = None
+    r = None
+    for b in range(3):
+        rep, m, j, nn, r = _check_step(ctx, I.batch(w, b), "bf16", before=before)
+        before = (m, j, nn)
+    _check_update(ctx, before[0], r, prior_rel=ctx.cfg.prior_rel)
+
+
+def test_quant_mode_int4_tc():
+    d, n = 256, 1024
+    w = I.scaled(I.WORKLOADS["c4a"], d=d, n=n, n_outlier=2)
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", quant_bits=4)
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    rep, m, j, nn, r = _check_step(ctx, I.batch(w, 0), "bf16", quant_bits=4)
+    _check_update(ctx, m, r)
+
+
+def test_skipped_rows_tc():
+    d, n = 128, 200
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2)
+    x = I.batch(w, 0).copy()
+    x[7] = 0.0
+    x[100, 3] = np.nan
+    x[150, 100] = -np.inf
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16")
+    ctx.step(_dev(x, "bf16"))
+    j, nn = ctx.get_objective(check=False)
+    ref = O.OpuOracle(d).step(x.astype(np.float64))
+    assert nn == n - 3 == ref.N and abs(j - ref.J) / ref.J < 1e-3
+    m = ctx.get_M(check=False).cpu().numpy()
+    assert np.isfinite(m).all()
+    st = ctx.get_stats()
+    assert st.status == -7 and st.n_skipped == 3
+
+
+def test_tc_matches_exact_mode_of_the_library():
+    """Both arithmetic modes of the library on the same stream end at rotations with the same objective."""
+    from paper_2605_10793_b200 import binding as B
+    d, n = 256, 2048
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2)
+    r0 = _dev(I.initial_rotation(w), "f32")
+    out = {}
+    for mode in ("exact", "tc"):
+        ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode=mode)
+        ctx.set_R(r0)
+        for b in range(2):
+            ctx.step(_dev(I.batch(w, b), "bf16"))
+        ctx.update()
+        ctx.step(_dev(I.batch(w, 2), "bf16"))
+        out[mode] = ctx.get_objective()
+    assert out["exact"][1] == out["tc"][1]
+    assert abs(out["exact"][0] - out["tc"][0]) / out["exact"][0] < 1e-3
