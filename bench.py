@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the ConQuR calibration hot path on B200.
+
+One "step" = one update cycle of the headline workload (d = 4096, batches of 2048 bf16 tokens, polar
+update every 8 batches): 8 x conqur_step + 1 x conqur_update = 16384 tokens through every stage of the
+path (row norms, rotate + corner target, cross-covariance accumulate, Newton-Schulz polar update with
+its orthogonality check).  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1 (torchrun): N independent replicas, one per GPU, no data-path collective ("weak" scaling).
+--impl reference: times the float64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_10793_b200 import dist as D          # noqa: E402
+from paper_2605_10793_b200 import inputs as I        # noqa: E402
+
+METRIC = "calibration tokens/sec at d=4096 (whole path incl. polar update every 8 batches)"
+WORKLOAD = "c2"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            j = json.load(fh)
+        return {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops"],
+                "bf16_tflops_sustained": j.get("bf16_tflops_sustained", j["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def _gen_one(args):
+    name, b, problem = args
+    w = I.WORKLOADS[name]
+    return I.to_bf16_bits(I.batch(w, b, problem=problem))
+
+
+def generate_batches(name: str, count: int, replica: int, workers: int):
+    """bf16 payloads (uint16, n x d) of the first `count` batches of the stream."""
+    jobs = [(name, b, replica) for b in range(count)]
+    if workers <= 1:
+        return [_gen_one(j) for j in jobs]
+    import multiprocessing as mp
+    with mp.get_context("fork").Pool(workers) as pool:
+        return pool.map(_gen_one, jobs, chunksize=1)
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(power)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def cpu_oracle_sample(w, cycles: int = 1):
+    """Time the float64 oracle, as it stands, on one update cycle of the workload (steps + one SVD update)."""
+    from oracle import conqur_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count()])
+    except Exception:
+        threads = os.cpu_count()
+    orc = O.OpuOracle(w.d, I.initial_rotation(w).astype(np.float64), quant_bits=w.quant_bits, prior_rel=w.prior_rel)
+    t_step = t_upd = 0.0
+    for c in range(cycles):
+        for b in range(w.update_every):
+            x = I.batch(w, c * w.update_every + b).astype(np.float64)      # generation is not timed
+            t0 = time.perf_counter()
+            orc.step(x)
+            t_step += time.perf_counter() - t0
+        t0 = time.perf_counter()
+        orc.update()
+        t_upd += time.perf_counter() - t0
+    cycle_s = (t_step + t_upd) / cycles
+    return {"value": w.update_every * w.n / cycle_s, "unit": "tokens/s", "cores": int(threads), "kind": "oracle",
+            "sample": f"{cycles} update cycle(s): {w.update_every} oracle steps of {w.n}x{w.d} "
+                      f"({t_step / cycles:.2f} s) + 1 SVD update of {w.d}x{w.d} ({t_upd / cycles:.2f} s)",
+            "step_s": t_step / (cycles * w.update_every), "update_s": t_upd / cycles}
+
+
+def run_reference(args):
+    g = D.Group(int(os.environ.get("RANK", "0")), 0, int(os.environ.get("WORLD_SIZE", "1")), False)
+    if g.rank != 0:
+        return 0
+    w = I.WORKLOADS[WORKLOAD]
+    # each reference "step" is a bounded sample of the cycle; keep the run within minutes
+    steps = max(1, min(args.steps, 2))
+    warm = 1 if args.warmup > 0 else 0
+    if warm:
+        cpu_oracle_sample(I.scaled(w, d=512, n=512), 1)
+    samples = [cpu_oracle_sample(w, 1) for _ in range(steps)]
+    best = max(samples, key=lambda s: s["value"])
+    val = float(np.mean([s["value"] for s in samples]))
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": 1e3 * w.update_every * w.n / val, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": _workload_desc(w), "note": "float64 numpy oracle on host cores; bounded sample per step"},
+        "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    out["cpu_baseline"]["value"] = val
+    print(json.dumps(out))
+    return 0
+
+
+def _workload_desc(w):
+    return (f"{w.name}: d={w.d}, {w.n_batches} batches x {w.n} tokens, bf16 Student-t(3) with {w.n_outlier} outlier "
+            f"channels x{w.outlier_scale:g}, {w.n_massive_rows} massive tokens x{w.massive_scale:g}/batch, "
+            f"R0=randomised Hadamard, polar update every {w.update_every} batches")
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--distinct-cycles", type=int, default=0, help="cycles of distinct batches kept resident (0=all)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2605_10793_b200 import binding as B
+    g = D.init()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    torch.cuda.set_device(g.local_rank)
+    B.load()
+    w = I.WORKLOADS[args.workload]
+    K, W = args.steps, max(args.warmup, 3)
+    cyc = w.update_every
+    total_cycles = w.n_batches // cyc
+    distinct = min(total_cycles, args.distinct_cycles or total_cycles, max(K, 1))
+    n_batches = distinct * cyc
+    workers = max(1, min(16, (os.cpu_count() or 2) // max(1, g.world)))
+    t_gen = time.perf_counter()
+    bits = generate_batches(w.name, n_batches, g.rank, workers)
+    t_gen = time.perf_counter() - t_gen
+
+    # inputs: pinned host copies (for the end-to-end leg) and resident device copies (for the device-timed leg)
+    host = [torch.from_numpy(b.view(np.int16)).pin_memory() for b in bits]
+    dev = [h.cuda(non_blocking=True).view(torch.bfloat16) for h in host]
+    torch.cuda.synchronize()
+    resident_bytes = sum(t.numel() * 2 for t in dev)
+    r0 = torch.from_numpy(I.initial_rotation(w)).cuda()
+
+    ctx = B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel)
+    ctx.set_R(r0)
+
+    def cycle_resident(c):
+        base = (c % distinct) * cyc
+        for b in range(cyc):
+            ctx.step(dev[base + b])
+        ctx.update()
+
+    for c in range(W):
+        cycle_resident(c)
+    st = ctx.get_stats()
+    if st.status != 0:
+        raise SystemExit(f"warm-up failed: {B.strerror(st.status)}")
+    ctx.set_R(r0)
+
+    # ---------------- device-timed leg: inputs resident in HBM
+    ctx.set_profiling(False)                     # resets the launch counters
+    sampler = ClockSampler(g.local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    D.barrier(g)
+    torch.cuda.synchronize()
+    ev0.record()
+    for c in range(K):
+        cycle_resident(c)
+    ev1.record()
+    torch.cuda.synchronize()
+    D.barrier(g)
+    ms_local = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    launches = ctx.get_profile()["total_launches"]
+    st = ctx.get_stats()
+    j_last, n_last = st.last_J, st.last_N
+    ms = D.max_over_ranks(g, ms_local)
+    tokens = K * cyc * w.n
+    value = g.world * tokens / (ms * 1e-3)
+
+    # ---------------- end-to-end leg: host buffers, H2D inside the timed region, objective read back each cycle
+    e2e = None
+    if not args.no_e2e:
+        ctx.set_R(r0)
+        ring = 2 * cyc
+        stage = [torch.empty((w.n, w.d), dtype=torch.bfloat16, device="cuda") for _ in range(ring)]
+        copy_stream = torch.cuda.Stream()
+        ready = [torch.cuda.Event() for _ in range(ring)]
+        freed = [torch.cuda.Event() for _ in range(ring)]
+        main_stream = torch.cuda.current_stream()
+
+        def enqueue_copy(i):
+            slot = i % ring
+            with torch.cuda.stream(copy_stream):
+                if i >= ring:
+                    copy_stream.wait_event(freed[slot])
+                stage[slot].view(torch.int16).copy_(host[i % n_batches], non_blocking=True)
+                ready[slot].record(copy_stream)
+
+        total_b = K * cyc
+        D.barrier(g)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_wall = time.perf_counter()
+        e0.record()
+        issued = 0
+        while issued < min(ring, total_b):
+            enqueue_copy(issued); issued += 1
+        d2h = 0
+        for i in range(total_b):
+            slot = i % ring
+            main_stream.wait_event(ready[slot])
+            ctx.step(stage[slot])
+            freed[slot].record(main_stream)
+            if issued < total_b:
+                enqueue_copy(issued); issued += 1
+            if (i + 1) % cyc == 0:
+                jj, nn = ctx.get_objective()          # device -> host read of the cycle's result (synchronises)
+                d2h += 16
+                ctx.update()
+        e1.record()
+        torch.cuda.synchronize()
+        t_wall = time.perf_counter() - t_wall
+        D.barrier(g)
+        ms_e2e = D.max_over_ranks(g, max(e0.elapsed_time(e1), 0.0))
+        e2e = {"value": g.world * tokens / (ms_e2e * 1e-3), "unit": "tokens/s",
+               "h2d_bytes_per_step": cyc * w.n * w.d * 2, "d2h_bytes_per_step": 16,
+               "ms_per_step": ms_e2e / K, "host_wall_ms_per_step": 1e3 * t_wall / K,
+               "how": "pinned host batches -> double-buffered cudaMemcpyAsync on a copy stream -> conqur_step; "
+                      "objective read back every cycle"}
+        del stage
+
+    # ---------------- roofline pass: same workload, each contraction launch bracketed by CUDA events
+    ctx.set_R(r0)
+    ctx.set_profiling(True)
+    upd_ms = []
+    for c in range(min(K, 4)):
+        base = (c % distinct) * cyc
+        for b in range(cyc):
+            ctx.step(dev[base + b])
+        u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        u0.record()
+        ctx.update()
+        u1.record()
+        torch.cuda.synchronize()
+        upd_ms.append(u0.elapsed_time(u1))
+    prof = ctx.get_profile()
+    st2 = ctx.get_stats()
+    ctx.set_profiling(False)
+    peaks = _peaks()
+    gemm_classes = ["rotate_target", "accumulate", "ns_residual", "ns_poly", "ns_next"]
+    tot_fl = sum(prof[k]["flops"] for k in gemm_classes)
+    tot_ms = sum(prof[k]["ms"] for k in gemm_classes)
+    tot_n = sum(prof[k]["timed"] for k in gemm_classes)
+    achieved = tot_fl / (tot_ms * 1e-3) / 1e12 if tot_ms > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    detail = {k: {"launches": prof[k]["timed"], "avg_ms": prof[k]["ms"] / max(1, prof[k]["timed"]),
+                  "tflops": (prof[k]["flops"] / (prof[k]["ms"] * 1e-3) / 1e12) if prof[k]["ms"] > 0 else 0.0}
+              for k in gemm_classes}
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": None, "kernel": "tc_gemm_kernel (all epilogues)", "launches": tot_n,
+                "flops_per_launch": tot_fl / max(1, tot_n), "avg_launch_ms": tot_ms / max(1, tot_n),
+                "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
+                "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+                "per_epilogue": detail}
+
+    if not g.is_main:
+        D.finish(g)
+        return 0
+
+    cpu_base = None
+    if not args.no_cpu_baseline and g.world == 1:
+        cpu_base = cpu_oracle_sample(w, 1)
+        cpu_base = {k: cpu_base[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": g.world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": _workload_desc(w), "tokens_per_step": cyc * w.n, "mode": "tc (bf16 operands, fp32 accumulate; "
+                   "Newton-Schulz products as 3-term bf16 split)", "l2": f"inputs larger than L2: {resident_bytes / 1e6:.0f} MB "
+                   f"of distinct batches resident, each read once per cycle", "replicas": g.world,
+                   "input_gen_s": round(t_gen, 1)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "cpu_baseline": cpu_base,
+        "polar_update_ms": float(np.mean(upd_ms)) if upd_ms else None,
+        "polar_update_ms_min": float(np.min(upd_ms)) if upd_ms else None,
+        "ns_steps_used": int(st2.ns_steps_used), "orth_err": float(st2.orth_err),
+        "objective_per_token_last_cycle": (j_last / n_last) if n_last else None,
+        "step_only_tokens_per_s": (cyc * w.n) / ((ms / K - float(np.mean(upd_ms))) * 1e-3) if upd_ms and ms / K > np.mean(upd_ms) else None,
+    }
+    print(json.dumps(out))
+    D.finish(g)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

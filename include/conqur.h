@@ -178,6 +178,30 @@ int conqur_debug_get_signs(conqur_ctx* ctx, int8_t* S_out_dev);
 int conqur_get_stats(conqur_ctx* ctx, conqur_stats* out);
 
 /*
+ * Launch accounting (measurement support; no counterpart in the paper).  Kernel classes:
+ * 0 row norms, 1 rotate+target, 2 accumulate, 3/4/5 the three Newton-Schulz products
+ * (residual X^T X - I, polynomial, next iterate), 6 everything else (reductions, element-wise).
+ * Launch counts are always kept.  With profiling enabled each contraction launch is bracketed by
+ * CUDA events on the context's stream and conqur_update synchronises at its end (so enable it only
+ * in a measurement pass); flops are the algorithmic 2*M*N*K of launches that did not early-exit.
+ */
+#define CONQUR_KERNEL_CLASSES 8
+typedef struct {
+  uint32_t struct_size;                          /* = sizeof(conqur_profile) */
+  int32_t  reserved;
+  int64_t  launches[CONQUR_KERNEL_CLASSES];      /* kernels launched since conqur_set_profiling */
+  int64_t  timed_launches[CONQUR_KERNEL_CLASSES];/* launches with event timing that ran to completion */
+  double   flops[CONQUR_KERNEL_CLASSES];         /* algorithmic flops of the timed launches */
+  double   ms[CONQUR_KERNEL_CLASSES];            /* summed event time of the timed launches */
+  int64_t  total_launches;
+} conqur_profile;
+
+/* Reset the counters and switch per-launch event timing on or off.  Synchronises. */
+int conqur_set_profiling(conqur_ctx* ctx, int32_t enabled);
+/* Read the counters.  Synchronises. */
+int conqur_get_profile(conqur_ctx* ctx, conqur_profile* out);
+
+/*
  * Host-only introspection of the Newton-Schulz plan (no device needed): the odd quintics
  * p_k(x) = a x + b x^3 + c x^5 an update applies, in order, for a spectrum assumed to lie in
  * [sigma_min_rel, 1] after scaling (ns_steps > 0 instead plans for exactly that many steps).

@@ -23,6 +23,7 @@ EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
+    "conqur_set_profiling", "conqur_get_profile",
     "conqur_strerror",
 ]
 
@@ -41,6 +42,17 @@ class conqur_stats(C.Structure):
         ("orth_err", C.c_float), ("orth_fro", C.c_float), ("scale", C.c_float), ("n_skipped", C.c_int64),
         ("last_J", C.c_double), ("last_N", C.c_int64),
     ]
+
+
+class conqur_profile(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("reserved", C.c_int32), ("launches", C.c_int64 * 8),
+        ("timed_launches", C.c_int64 * 8), ("flops", C.c_double * 8), ("ms", C.c_double * 8),
+        ("total_launches", C.c_int64),
+    ]
+
+
+KERNEL_CLASSES = ["rownorm", "rotate_target", "accumulate", "ns_residual", "ns_poly", "ns_next", "other", "unused"]
 
 
 class ConqurError(RuntimeError):
@@ -87,6 +99,10 @@ def load() -> C.CDLL:
     lib.conqur_get_stats.argtypes = [vp, C.POINTER(conqur_stats)]
     lib.conqur_plan_schedule.restype = C.c_int
     lib.conqur_plan_schedule.argtypes = [C.c_double, i32, C.POINTER(C.c_double), i32]
+    lib.conqur_set_profiling.restype = C.c_int
+    lib.conqur_set_profiling.argtypes = [vp, i32]
+    lib.conqur_get_profile.restype = C.c_int
+    lib.conqur_get_profile.argtypes = [vp, C.POINTER(conqur_profile)]
     lib.conqur_debug_gemm.restype = C.c_int
     lib.conqur_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.conqur_strerror.restype = C.c_char_p
@@ -171,6 +187,17 @@ def conqur_get_stats(h: int) -> Tuple[int, conqur_stats]:
     st.struct_size = C.sizeof(conqur_stats)
     rc = load().conqur_get_stats(h, C.byref(st))
     return rc, st
+
+
+def conqur_set_profiling(h: int, enabled: bool) -> int:
+    return load().conqur_set_profiling(h, int(enabled))
+
+
+def conqur_get_profile(h: int) -> Tuple[int, conqur_profile]:
+    pr = conqur_profile()
+    pr.struct_size = C.sizeof(conqur_profile)
+    rc = load().conqur_get_profile(h, C.byref(pr))
+    return rc, pr
 
 
 def conqur_plan_schedule(sigma_min_rel: float = 0.0, ns_steps: int = 0, max_steps: int = 100) -> np.ndarray:
@@ -277,6 +304,18 @@ class Context:
         rc, st = conqur_get_stats(self.h)
         self._chk(rc, "conqur_get_stats")
         return st
+
+    def set_profiling(self, enabled: bool):
+        self._chk(conqur_set_profiling(self.h, enabled), "conqur_set_profiling")
+
+    def get_profile(self) -> dict:
+        rc, pr = conqur_get_profile(self.h)
+        self._chk(rc, "conqur_get_profile")
+        out = {"total_launches": int(pr.total_launches)}
+        for i, name in enumerate(KERNEL_CLASSES[:7]):
+            out[name] = {"launches": int(pr.launches[i]), "timed": int(pr.timed_launches[i]),
+                         "flops": float(pr.flops[i]), "ms": float(pr.ms[i])}
+        return out
 
     def close(self):
         if getattr(self, "h", None):

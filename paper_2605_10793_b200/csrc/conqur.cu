@@ -107,6 +107,7 @@ struct conqur_ctx {
   int n_sched, restart_idx;
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
+  Prof prof;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   DevState* state() const { return at<DevState>(L.state); }
@@ -124,6 +125,12 @@ int cuda_fail(const char* what, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(#expr, e__);    \
   } while (0)
 #define CQ_LAUNCH_CHECK() CQ_CUDA(cudaGetLastError())
+// after a kernel launch of context c: check and count it
+#define CQ_LAUNCHED(c, cls)          \
+  do {                               \
+    CQ_CUDA(cudaGetLastError());     \
+    (c)->prof.count(cls);            \
+  } while (0)
 
 __global__ void or_flags_kernel(const DevState* st, int P, int* agg) {
   int f = 0;
@@ -154,7 +161,7 @@ int sync_status(conqur_ctx* c) {
   int* agg = c->at<int>(c->L.flags_agg);
   CQ_CUDA(cudaMemsetAsync(agg, 0, sizeof(int), c->stream));
   or_flags_kernel<<<1, 256, 0, c->stream>>>(c->state(), c->cfg.P, agg);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   int f = 0;
   CQ_CUDA(cudaMemcpyAsync(&f, agg, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CQ_CUDA(cudaStreamSynchronize(c->stream));
@@ -174,37 +181,37 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   double* part = c->at<double>(c->L.part_d);
   const int64_t c_ps = (int64_t)g.n_max * d;
   rownorm_kernel<TIn><<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(X, n, d, ld, pstride, rnorm, g.n_max, st, 1);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_ROWNORM);
   const dim3 grid1(cdiv(d, SG_BN), cdiv(n, SG_BM), P);
   int per_problem;
   if (g.quant_bits == 0) {
     rotate_target_exact_kernel<TIn, false><<<grid1, SG_THREADS, 0, c->stream>>>(
         X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, part);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_ROTATE);
     per_problem = grid1.x * grid1.y;
   } else {
     unsigned* rowmax = c->at<unsigned>(c->L.rowmax);
     CQ_CUDA(cudaMemsetAsync(rowmax, 0, sizeof(unsigned) * g.n_max * P, c->stream));
     rotate_target_exact_kernel<TIn, true><<<grid1, SG_THREADS, 0, c->stream>>>(
         X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, part);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_ROTATE);
     const int levels = (1 << (g.quant_bits - 1)) - 1;
     quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, levels,
                                                                     part);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_OTHER);
     per_problem = cdiv(n, 8);
   }
   finalize_step_kernel<<<P, 256, 0, c->stream>>>(st, part, per_problem, n, 1.0 / std::sqrt((double)d));
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   const int S = c->L.acc_splits;
   accumulate_exact_kernel<TIn><<<dim3(cdiv(d, SG_BN), cdiv(d, SG_BM), P * S), SG_THREADS, 0, c->stream>>>(
       X, ld, pstride, C, c_ps, rnorm, g.n_max, (int)n, d, S, c->at<float>(c->L.M),
       S > 1 ? c->at<float>(c->L.splitk) : nullptr);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_ACCUM);
   if (S > 1) {
     splitk_reduce_add_kernel<<<dim3(ew_blocks((int64_t)d * d), P), 256, 0, c->stream>>>(
         c->at<float>(c->L.M), c->at<float>(c->L.splitk), (int64_t)d * d, S);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_OTHER);
   }
   return CONQUR_OK;
 }
@@ -217,7 +224,7 @@ int launch_residual(conqur_ctx* c, const float* X, int buf) {
   if (g.mode == CONQUR_EXACT_F32) {
     ns_gemm_exact_kernel<EPI_RESIDUAL><<<dim3(T, T, g.P), SG_THREADS, 0, c->stream>>>(
         X, X, nullptr, c->at<float>(c->L.E), g.d, c->state(), c->at<float>(c->L.part_f), c->at<double>(c->L.part_d));
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_NS_RESID);
     return CONQUR_OK;
   }
   return tc_ns_residual(c->tc, c->stream, buf);
@@ -245,17 +252,17 @@ int update_impl(conqur_ctx* c) {
   const float isd = (float)(1.0 / std::sqrt((double)d));
 
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   if (g.prior_rel > 0.f) {
     sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 1, pd);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_OTHER);
   }
   ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   if (g.mode == CONQUR_TC_BF16) { int rc = tc_ns_begin(c->tc, c->stream); if (rc) return rc; }
 
   const int T = cdiv(d, SG_BM);
@@ -264,27 +271,36 @@ int update_impl(conqur_ctx* c) {
     const int cur = k & 1;
     float* X = cur ? Xb : Xa;
     float* Xn = cur ? Xa : Xb;
+    c->tc.ns_k = k;
     int rc = launch_residual(c, X, cur);
     if (rc) return rc;
     ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, parts, k, sched, c->n_sched, c->restart_idx, g.orth_tol,
                                                 g.fro_tol, cur, g.ns_max_steps);
-    CQ_LAUNCH_CHECK();
+    CQ_LAUNCHED(c, K_OTHER);
     if (k == g.ns_max_steps) break;
     if (g.mode == CONQUR_EXACT_F32) {
       ns_gemm_exact_kernel<EPI_POLY><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(E, E, E, B, d, st, nullptr, nullptr);
-      CQ_LAUNCH_CHECK();
+      CQ_LAUNCHED(c, K_NS_POLY);
       ns_gemm_exact_kernel<EPI_NEXT><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(X, B, X, Xn, d, st, nullptr, nullptr);
-      CQ_LAUNCH_CHECK();
+      CQ_LAUNCHED(c, K_NS_NEXT);
     } else {
       rc = tc_ns_poly_next(c->tc, c->stream, cur);
       if (rc) return rc;
     }
   }
   ns_commit_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(st, Xa, Xb, R, M, dd);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   if (g.mode == CONQUR_TC_BF16) { int rc = tc_refresh_R(c->tc, c->stream, /*only_if_converged=*/1); if (rc) return rc; }
   ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
+  c->tc.ns_k = -1;
+  if (c->prof.enabled) {
+    // profiling pass only: find out how many of the enqueued steps actually ran
+    DevState h0;
+    CQ_CUDA(cudaMemcpyAsync(&h0, st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CQ_CUDA(cudaStreamSynchronize(c->stream));
+    c->prof.fold(h0.ns_steps_used);
+  }
   return CONQUR_OK;
 }
 
@@ -355,7 +371,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
     int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
                      c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
                      c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
-                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax));
+                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), &c->prof);
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);
@@ -380,11 +396,11 @@ extern "C" int conqur_set_R(conqur_ctx* c, const float* R_dev) {
   float* Xa = c->at<float>(c->L.Xa);
   CQ_CUDA(cudaMemcpyAsync(Xa, R_dev, sizeof(float) * dd * g.P, cudaMemcpyDeviceToDevice, c->stream));
   arm_check_kernel<<<1, 256, 0, c->stream>>>(c->state(), g.P);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   const int T = cdiv(g.d, SG_BM);
   ns_gemm_exact_kernel<EPI_RESIDUAL><<<dim3(T, T, g.P), SG_THREADS, 0, c->stream>>>(
       Xa, Xa, nullptr, c->at<float>(c->L.E), g.d, c->state(), c->at<float>(c->L.part_f), c->at<double>(c->L.part_d));
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   std::vector<float> pm((size_t)T * T * g.P);
   CQ_CUDA(cudaMemcpyAsync(pm.data(), c->at<float>(c->L.part_f), sizeof(float) * pm.size(), cudaMemcpyDeviceToHost,
                           c->stream));
@@ -454,7 +470,7 @@ extern "C" int conqur_get_M(conqur_ctx* c, float* M_out_dev) {
   const int64_t count = (int64_t)c->cfg.d * c->cfg.d * c->cfg.P;
   scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(c->at<float>(c->L.M), M_out_dev, count,
                                                              (float)(1.0 / std::sqrt((double)c->cfg.d)));
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   return sync_status(c);
 }
 
@@ -464,7 +480,7 @@ extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_s
   const int64_t count = (int64_t)c->cfg.d * c->cfg.d * P;
   scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(M_dev, c->at<float>(c->L.M), count,
                                                              (float)std::sqrt((double)c->cfg.d));
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   // stage the sums through the partials buffer
   double* dJ = c->at<double>(c->L.part_d);
   long long* dN = reinterpret_cast<long long*>(dJ + P);
@@ -472,7 +488,7 @@ extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_s
   CQ_CUDA(cudaMemcpyAsync(dJ, J_sum, sizeof(double) * P, cudaMemcpyHostToDevice, c->stream));
   CQ_CUDA(cudaMemcpyAsync(dN, n64.data(), sizeof(long long) * P, cudaMemcpyHostToDevice, c->stream));
   set_sums_kernel<<<1, 256, 0, c->stream>>>(c->state(), dJ, dN, P);
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   CQ_CUDA(cudaStreamSynchronize(c->stream));
   int64_t tot = 0;
   for (int p = 0; p < P; ++p) tot = std::max<int64_t>(tot, n_tokens[p]);
@@ -491,7 +507,7 @@ extern "C" int conqur_debug_get_signs(conqur_ctx* c, int8_t* S_out_dev) {
     signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(nullptr, tc_cp_ptr(c->tc), c->last_n, c->cfg.d,
                                                                  S_out_dev);
   }
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   return sync_status(c);
 }
 
@@ -503,7 +519,7 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
   const int rc = sync_status(c);
   if (rc == CONQUR_ERR_CUDA) return rc;
   clear_flags_kernel<<<1, 256, 0, c->stream>>>(c->state(), P, c->at<int>(c->L.flags_agg));
-  CQ_LAUNCH_CHECK();
+  CQ_LAUNCHED(c, K_OTHER);
   CQ_CUDA(cudaStreamSynchronize(c->stream));
   out->status = rc;
   out->ns_steps_used = 0; out->orth_err = 0.f; out->orth_fro = 0.f; out->n_skipped = 0;
@@ -518,6 +534,29 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
     out->last_N += h[p].last_N;
     out->updates = std::min(out->updates, h[p].updates);
   }
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_set_profiling(conqur_ctx* c, int32_t enabled) {
+  if (!c) return CONQUR_ERR_INVALID_ARG;
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  c->prof.fold(1 << 30);
+  c->prof.reset();
+  c->prof.enabled = enabled != 0;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_get_profile(conqur_ctx* c, conqur_profile* out) {
+  if (!c || !out || out->struct_size != sizeof(conqur_profile)) return CONQUR_ERR_INVALID_ARG;
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  c->prof.fold(1 << 30);
+  for (int i = 0; i < CONQUR_KERNEL_CLASSES; ++i) {
+    out->launches[i] = c->prof.launches[i];
+    out->timed_launches[i] = c->prof.timed[i];
+    out->flops[i] = c->prof.flops[i];
+    out->ms[i] = c->prof.ms[i];
+  }
+  out->total_launches = c->prof.total;
   return CONQUR_OK;
 }
 

@@ -1,7 +1,10 @@
 // Internal definitions shared by the host orchestration and the kernels.
 #pragma once
+#include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
+
+#include <vector>
 
 namespace conqur {
 
@@ -31,6 +34,53 @@ struct DevState {
   float scale, x0_scale, lam;
   float coef[3];            // gamma, beta1, beta2 of the step in flight
   float pad_[2];
+};
+
+// Kernel classes for launch counting / optional per-launch timing.
+enum : int { K_ROWNORM = 0, K_ROTATE = 1, K_ACCUM = 2, K_NS_RESID = 3, K_NS_POLY = 4, K_NS_NEXT = 5, K_OTHER = 6, K_COUNT = 8 };
+
+// Host-side launch accounting.  Launch counts are always kept; when `enabled`, the contractions are bracketed by
+// CUDA events on the launching stream (events are created lazily and reused).
+struct Prof {
+  struct Rec { int cls; double flops; int ns_k; cudaEvent_t e0, e1; };
+  bool enabled = false;
+  long long launches[K_COUNT] = {0};
+  long long total = 0;
+  double flops[K_COUNT] = {0};
+  double ms[K_COUNT] = {0};
+  long long timed[K_COUNT] = {0};
+  std::vector<Rec> open;                 // records not yet folded into the sums
+  std::vector<cudaEvent_t> pool;
+
+  void count(int cls) { ++launches[cls]; ++total; }
+  cudaEvent_t get_event() {
+    if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  // Fold the finished records into the sums (call after a stream synchronise).  Newton-Schulz launches whose
+  // step index lies past `steps_used` early-exited on the device and are left out.
+  void fold(int steps_used) {
+    for (Rec& r : open) {
+      bool ran = true;
+      if (r.ns_k >= 0) ran = (r.cls == K_NS_RESID) ? (r.ns_k <= steps_used) : (r.ns_k < steps_used);
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, r.e0, r.e1) == cudaSuccess && ran) {
+        ms[r.cls] += t; flops[r.cls] += r.flops; ++timed[r.cls];
+      }
+      pool.push_back(r.e0); pool.push_back(r.e1);
+    }
+    open.clear();
+  }
+  void reset() {
+    for (int i = 0; i < K_COUNT; ++i) { launches[i] = 0; flops[i] = 0; ms[i] = 0; timed[i] = 0; }
+    total = 0;
+  }
+  ~Prof() {
+    for (Rec& r : open) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    for (cudaEvent_t e : pool) cudaEventDestroy(e);
+  }
 };
 
 }  // namespace conqur

@@ -584,7 +584,8 @@ struct TcHost {
   CUtensorMap tmRb_mn;                       // R bf16 as MN-major B of the rotate product
   CUtensorMap tmXh_mn[2], tmXh_k[2];         // iterate, stacked [hi; lo]
   CUtensorMap tmEh_k, tmEh_mn, tmBh_mn;
-  long long launches;
+  Prof* prof;
+  int ns_k;                                  // Newton-Schulz step index of the launches being enqueued (-1 outside)
 };
 
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -637,6 +638,17 @@ inline void tc_make_layout(int d, int P, int64_t n_max, int quant_bits, TcLayout
   L->Bh = take(4 * dd);
 }
 
+inline int tc_epi_class(int epi) {
+  switch (epi) {
+    case TC_EPI_ROTATE: case TC_EPI_ROTATE_Q: return K_ROTATE;
+    case TC_EPI_ACCUM: return K_ACCUM;
+    case TC_EPI_RESID: return K_NS_RESID;
+    case TC_EPI_POLY: return K_NS_POLY;
+    case TC_EPI_NEXT: return K_NS_NEXT;
+    default: return K_OTHER;
+  }
+}
+
 template <int BN, bool A_MN, bool B_MN, int EPI>
 inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
   using Cfg = TcCfg<BN>;
@@ -649,8 +661,17 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
   }
   const int tiles = ((g.M + TC_BM - 1) / TC_BM) * ((g.N + BN - 1) / BN);
   const int grid = tiles < h.num_sms ? tiles : h.num_sms;
+  const int cls = tc_epi_class(EPI);
+  Prof::Rec rec{};
+  const bool timed = h.prof && h.prof->enabled;
+  if (timed) {
+    rec.cls = cls; rec.flops = 2.0 * g.M * (double)g.N * g.K * g.nseg; rec.ns_k = h.ns_k;
+    rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
+    cudaEventRecord(rec.e0, s);
+  }
   kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, g);
-  ++h.launches;
+  if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
+  if (h.prof) h.prof->count(cls);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
@@ -663,10 +684,10 @@ inline int tc_launch_n(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CU
 
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
                    float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
-                   float* part_f, float* Y, unsigned* rowmax) {
+                   float* part_f, float* Y, unsigned* rowmax, Prof* prof) {
   h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
   h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
-  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->launches = 0;
+  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->prof = prof; h->ns_k = -1;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
   cudaDeviceProp prop;
@@ -697,6 +718,7 @@ inline int tc_ew_blocks(int64_t count4) {
 inline int tc_refresh_R(TcHost& h, cudaStream_t s, int) {
   const int64_t dd = (int64_t)h.d * h.d;
   split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.R, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Rb), dd, 0);
+  if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
@@ -716,6 +738,7 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
   else
     rownorm_stage_kernel<__nv_bfloat16><<<rb, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(X), n, d, ld, h.rnorm, Xs, h.st);
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_ROWNORM);
   // per-call maps over the first n rows: rows past n read as zeros
   CUtensorMap tmXs_k, tmXs_mn, tmCp_mn;
   int rc = tc_make_tmap(&tmXs_k, Xs, (uint64_t)n, (uint64_t)d, (uint64_t)d, 128);
@@ -739,10 +762,12 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
     const int levels = (1 << (h.quant_bits - 1)) - 1;
     quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, levels, h.part_d, Cp);
     if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (h.prof) h.prof->count(K_OTHER);
     per_problem = rb;
   }
   finalize_step_kernel<<<1, 256, 0, s>>>(h.st, h.part_d, per_problem, n, isd);
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_OTHER);
   TcGemmArgs a = tc_args(h, d, d, (int)n);
   a.outF = h.M; a.ldo = d;
   return tc_launch_n<true, true, TC_EPI_ACCUM>(h, s, tmXs_mn, tmCp_mn, a);
@@ -752,6 +777,7 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
 inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
   const int64_t dd = (int64_t)h.d * h.d;
   split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.Xa, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[0]), dd, dd);
+  if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
@@ -795,7 +821,7 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
                          int b_mn, int split, DevState* st, cudaStream_t s) {
   if (M < 1 || N < 32 || (N % 32) || K < 1 || (K % 8) || (M % 8)) return CONQUR_ERR_INVALID_ARG;
   TcHost h{};
-  h.launches = 0;
+  h.prof = nullptr; h.ns_k = -1;
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;

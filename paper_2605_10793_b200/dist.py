@@ -1,0 +1,85 @@
+"""Process-group plumbing for multi-GPU runs (one process per GPU, launched by torchrun).
+
+The calibration path of one rotation does not shard in this build (one context = one GPU), so N > 1
+means N independent replicas: no data-path collective.  The only communication is the barrier around
+the timed region and a max-reduction of the measured time.  Works with NCCL (GPU) and gloo (CPU tests).
+"""
+from __future__ import annotations
+
+import os
+from dataclasses import dataclass
+
+
+@dataclass
+class Group:
+    rank: int
+    local_rank: int
+    world: int
+    active: bool       # a process group was initialised
+
+    @property
+    def is_main(self) -> bool:
+        return self.rank == 0
+
+
+def init(backend: str | None = None) -> Group:
+    """Read RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* from the environment; single process if absent."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world <= 1:
+        return Group(0, local, 1, False)
+    import torch
+    import torch.distributed as dist
+    if backend is None:
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29511")
+    if backend == "nccl":
+        torch.cuda.set_device(local)
+        dist.init_process_group(backend, rank=rank, world_size=world, device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend, rank=rank, world_size=world)
+    return Group(rank, local, world, True)
+
+
+def barrier(g: Group) -> None:
+    if g.active:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(g: Group, value: float) -> float:
+    """The slowest rank's value (timings are reported as the max over ranks)."""
+    if not g.active:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(g: Group, value: float) -> float:
+    if not g.active:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def shard_problems(n_problems: int, g: Group) -> range:
+    """Contiguous block of independent problems owned by this rank (batched / per-head variant)."""
+    per = (n_problems + g.world - 1) // g.world
+    lo = min(n_problems, g.rank * per)
+    return range(lo, min(n_problems, lo + per))
+
+
+def finish(g: Group) -> None:
+    if g.active:
+        import torch.distributed as dist
+        dist.destroy_process_group()

@@ -71,7 +71,7 @@ def test_c0_in_tensor_core_mode():
 
 @pytest.mark.parametrize("d,n", [(256, 1000), (384, 2048), (512, 300)])
 def test_stream_steps_then_update(d, n):
-    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=max(2, d // 256))
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=max(2, d // 256), r0="hadamard" if d & (d - 1) == 0 else "qr")
     ctx = _ctx(d=d, n_max=n, in_dtype="bf16", prior_rel=0.0 if 3 * n >= 4 * d else 1e-2)
     ctx.set_R(_dev(I.initial_rotation(w), "f32"))
     before = None

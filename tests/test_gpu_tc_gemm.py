@@ -53,7 +53,7 @@ def test_ragged_m_k_and_n128(a_mn, b_mn):
 
 @pytest.mark.parametrize("a_mn,b_mn", [(False, True), (True, True), (False, False)])
 def test_split_precision_three_products(a_mn, b_mn):
-    assert _run(256, 256, 320, a_mn, b_mn, True, seed=3) < 2e-6
+    assert _run(256, 256, 320, a_mn, b_mn, True, seed=3) < 6e-6   # fp32 accumulation of 960 products
 
 
 def test_many_tiles_persistent_loop():
