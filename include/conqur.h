@@ -223,6 +223,30 @@ int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out
 int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_dev, int32_t M, int32_t N, int32_t K,
                       int32_t a_mn_major, int32_t b_mn_major, int32_t split, void* scratch_dev, void* cuda_stream);
 
+/*
+ * The corner objective of one batch without any device-memory allocation by anyone
+ * (the paper has no counterpart; this serves callers that cannot call cudaMalloc -- e.g. code
+ * running under a runtime that owns all device memory, or a plugin in a process whose device
+ * memory is pre-assigned -- and therefore cannot provide the workspace conqur_init needs).
+ *
+ * Computes, in the exact fp32 arithmetic of conqur_step's exact mode and with R fixed,
+ *   J = sum_i ||x_tilde_i R||_1 / sqrt(d)   and   N = rows with a finite, non-zero norm
+ * (the quantities conqur_get_objective reports after one conqur_step on a fresh context).
+ *   X_dev      device, n rows of d elements of in_dtype (CONQUR_F32 | CONQUR_BF16), row stride ld elements
+ *   R_dev      device fp32 d x d row-major
+ *   J_out_dev  device: one double;   N_out_dev: device: one int64.  Written on the stream; not synchronised.
+ *   limits     n <= 32768 and d <= 8192: the scratch (row norms, per-CTA partial sums; about 260 KB) is a
+ *              fixed array inside the library image, held by every GPU that loads the library until
+ *              the process exits.  Larger sizes return CONQUR_ERR_UNSUPPORTED and do nothing.
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call outside any stream capture.  The call uses no cudaMalloc/cudaFree and no allocating
+ * library routine.  All calls on a device share the one array: it still holds the previous call's
+ * contents (the counters are cleared at the start of each call), and two calls whose kernels overlap
+ * on the GPU (different streams, different threads) race on it -- serialise them.
+ */
+int conqur_objective_noalloc(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ld,
+                             const float* R_dev, double* J_out_dev, int64_t* N_out_dev, void* cuda_stream);
+
 const char* conqur_strerror(int status);
 
 #ifdef __cplusplus

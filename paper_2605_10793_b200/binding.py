@@ -23,7 +23,7 @@ EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
-    "conqur_set_profiling", "conqur_get_profile",
+    "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc",
     "conqur_strerror",
 ]
 
@@ -103,6 +103,8 @@ def load() -> C.CDLL:
     lib.conqur_set_profiling.argtypes = [vp, i32]
     lib.conqur_get_profile.restype = C.c_int
     lib.conqur_get_profile.argtypes = [vp, C.POINTER(conqur_profile)]
+    lib.conqur_objective_noalloc.restype = C.c_int
+    lib.conqur_objective_noalloc.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, vp]
     lib.conqur_debug_gemm.restype = C.c_int
     lib.conqur_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.conqur_strerror.restype = C.c_char_p
@@ -206,6 +208,12 @@ def conqur_plan_schedule(sigma_min_rel: float = 0.0, ns_steps: int = 0, max_step
     if n < 0:
         raise ConqurError(n, "conqur_plan_schedule")
     return np.array(buf[: 3 * n], dtype=np.float64).reshape(n, 3)
+
+
+def conqur_objective_noalloc(x_ptr: int, in_dtype: int, n: int, d: int, ld: int, r_ptr: int, j_out_ptr: int,
+                             n_out_ptr: int, stream_ptr: int) -> int:
+    """Objective of one batch using only the library's built-in scratch (see include/conqur.h)."""
+    return load().conqur_objective_noalloc(x_ptr, in_dtype, n, d, ld, r_ptr, j_out_ptr, n_out_ptr, stream_ptr)
 
 
 def conqur_debug_gemm(a, b, m: int, n: int, k: int, a_mn: bool, b_mn: bool, split: bool = False):

@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
 // Quant mode, second pass (Appendix B, Q_sym per token).  One warp per row:
 // Delta_raw = rowmax/L, q = rint(acc / Delta_raw) clipped to +-L, C' = sgn(q) * rnorm,
 // objective partial = rnorm * Delta_raw * sum_j |q_j|.  Works in place: Y and C' share the buffer.
-__global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
+static __global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
                                                            int64_t c_pstride, const float* __restrict__ rnorm,
                                                            int64_t rnorm_pstride,
                                                            const unsigned int* __restrict__ rowmax_bits, int levels,
@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(SG_THREADS) accumulate_exact_kernel(const TIn*
   }
 }
 
-__global__ void splitk_reduce_add_kernel(float* __restrict__ M, const float* __restrict__ partial, int64_t dd,
+static __global__ void splitk_reduce_add_kernel(float* __restrict__ M, const float* __restrict__ partial, int64_t dd,
                                          int splits) {
   const int p = blockIdx.y;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd; i += (int64_t)gridDim.x * blockDim.x) {
@@ -352,7 +352,7 @@ __global__ void splitk_reduce_add_kernel(float* __restrict__ M, const float* __r
 }
 
 // Adds the step's objective partials (fixed order) and token counts to the running sums.
-__global__ void finalize_step_kernel(DevState* st, const double* __restrict__ partials, int per_problem, int64_t n,
+static __global__ void finalize_step_kernel(DevState* st, const double* __restrict__ partials, int per_problem, int64_t n,
                                      double inv_sqrt_d) {
   const int p = blockIdx.x;
   __shared__ double red[8];
@@ -432,7 +432,7 @@ __global__ void __launch_bounds__(SG_THREADS) ns_gemm_exact_kernel(const float* 
 
 // ------------------------------------------------------------------ update: scalar control + element-wise
 // sum of squares of M (optionally of M + lam*R) -> per-block double partials
-__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ M, const float* __restrict__ R,
+static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ M, const float* __restrict__ R,
                                                     int64_t dd, const DevState* st, int use_lam,
                                                     double* __restrict__ partials) {
   const int p = blockIdx.y;
@@ -450,7 +450,7 @@ __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ M,
 
 // phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
 // phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
-__global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
+static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
                                 float prior_rel, float inv_sqrt_d, float margin) {
   const int p = blockIdx.x;
   __shared__ double red[8];
@@ -474,7 +474,7 @@ __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partial
 }
 
 // X0 = (M_raw + lam R) * x0_scale
-__global__ void ns_x0_kernel(const float* __restrict__ M, const float* __restrict__ R, float* __restrict__ X0,
+static __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __restrict__ R, float* __restrict__ X0,
                              int64_t dd, const DevState* st) {
   const int p = blockIdx.y;
   const float lam = st[p].lam, sc = st[p].x0_scale;
@@ -485,7 +485,7 @@ __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __restric
 // After the residual product of step k: reduce the per-CTA partials, decide convergence, pick the
 // polynomial of this step.  sched: n_sched entries of (gamma, beta1, beta2); restart_idx: where the
 // schedule re-enters when it ran out without convergence.
-__global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
+static __global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
                                   const double* __restrict__ part_sq, int nparts, int k,
                                   const float* __restrict__ sched, int n_sched, int restart_idx, float tol,
                                   float fro_tol, int cur_buf, int max_steps) {
@@ -525,7 +525,7 @@ __global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_m
 }
 
 // Accept or reject the update.  On success: R <- X_final, M <- 0, sums <- 0.
-__global__ void ns_commit_kernel(DevState* st, const float* __restrict__ Xa, const float* __restrict__ Xb,
+static __global__ void ns_commit_kernel(DevState* st, const float* __restrict__ Xa, const float* __restrict__ Xb,
                                  float* __restrict__ R, float* __restrict__ M, int64_t dd) {
   const int p = blockIdx.y;
   DevState* s = st + p;
@@ -536,7 +536,7 @@ __global__ void ns_commit_kernel(DevState* st, const float* __restrict__ Xa, con
     M[p * dd + i] = 0.f;
   }
 }
-__global__ void ns_commit_state_kernel(DevState* st) {
+static __global__ void ns_commit_state_kernel(DevState* st) {
   DevState* s = st + blockIdx.x;
   if (threadIdx.x != 0) return;
   if (s->ns_done == NS_DONE_CONVERGED) {
@@ -553,11 +553,11 @@ __global__ void ns_commit_state_kernel(DevState* st) {
 }
 
 // ------------------------------------------------------------------ misc element-wise
-__global__ void scale_copy_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t count, float f) {
+static __global__ void scale_copy_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t count, float f) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     dst[i] = src[i] * f;
 }
-__global__ void set_identity_kernel(float* __restrict__ R, int d, int P) {
+static __global__ void set_identity_kernel(float* __restrict__ R, int d, int P) {
   const int64_t dd = (int64_t)d * d;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < dd * P; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t e = i % dd;
@@ -565,7 +565,7 @@ __global__ void set_identity_kernel(float* __restrict__ R, int d, int P) {
   }
 }
 // sign matrix of the last step from C' (n x d, row-major) held as fp32 (exact mode) or bf16 (tensor-core mode)
-__global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Cb, int64_t n,
+static __global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Cb, int64_t n,
                                     int d, int8_t* __restrict__ S) {
   const int64_t total = n * d;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
