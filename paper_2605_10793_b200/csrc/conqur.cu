@@ -72,11 +72,12 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   L->rowmax = take(sizeof(unsigned) * n * P);
   int64_t mp = std::max<int64_t>((int64_t)cdiv(n, 128) * cdiv(d, 128), (int64_t)cdiv(d, 128) * cdiv(d, 128));
   mp = std::max<int64_t>(mp, cdiv(n, 8));
+  mp = std::max<int64_t>(mp, 2 * (int64_t)cdiv(d, 128) * cdiv(d, 128) + 64);   // two partial arrays per Newton-Schulz product
   mp = std::max<int64_t>(mp, 1024);
   L->max_partials = mp;
   L->part_d = take(sizeof(double) * mp * P);
   L->part_f = take(sizeof(float) * mp * P);
-  L->sched = take(sizeof(float) * 3 * 128);
+  L->sched = take(sizeof(SchedEntry) * NS_SCHED_MAX);
   L->acc_splits = 1;
   L->C = L->splitk = 0;
   L->Xa = take(sizeof(float) * dd * P);
@@ -104,7 +105,7 @@ struct conqur_ctx {
   cudaStream_t stream;
   int64_t tokens_since_update;
   int64_t last_n;            // rows of the last step (for debug_get_signs)
-  int n_sched, restart_idx;
+  int n_sched, first_endgame, reenter_idx;
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
   Prof prof;
@@ -247,19 +248,20 @@ int update_impl(conqur_ctx* c) {
   float* B = c->at<float>(c->L.B);
   double* pd = c->at<double>(c->L.part_d);
   float* pf = c->at<float>(c->L.part_f);
-  const float* sched = c->at<float>(c->L.sched);
+  const SchedEntry* sched = c->at<SchedEntry>(c->L.sched);
+  const int use_shift = g.mode == CONQUR_TC_BF16 ? 1 : 0;
   const int nb = (int)std::min<int64_t>(1024, (dd + 1023) / 1024);
   const float isd = (float)(1.0 / std::sqrt((double)d));
 
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
   CQ_LAUNCHED(c, K_OTHER);
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift);
   CQ_LAUNCHED(c, K_OTHER);
   if (g.prior_rel > 0.f) {
     sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 1, pd);
     CQ_LAUNCHED(c, K_OTHER);
   }
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift);
   CQ_LAUNCHED(c, K_OTHER);
   ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
   CQ_LAUNCHED(c, K_OTHER);
@@ -274,8 +276,9 @@ int update_impl(conqur_ctx* c) {
     c->tc.ns_k = k;
     int rc = launch_residual(c, X, cur);
     if (rc) return rc;
-    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, parts, k, sched, c->n_sched, c->restart_idx, g.orth_tol,
-                                                g.fro_tol, cur, g.ns_max_steps);
+    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, use_shift ? pd + parts : nullptr, parts, k, sched, c->n_sched,
+                                                c->first_endgame, c->reenter_idx, g.orth_tol, g.fro_tol, cur,
+                                                g.ns_max_steps, d, use_shift);
     CQ_LAUNCHED(c, K_OTHER);
     if (k == g.ns_max_steps) break;
     if (g.mode == CONQUR_EXACT_F32) {
@@ -299,7 +302,7 @@ int update_impl(conqur_ctx* c) {
     DevState h0;
     CQ_CUDA(cudaMemcpyAsync(&h0, st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
     CQ_CUDA(cudaStreamSynchronize(c->stream));
-    c->prof.fold(h0.ns_steps_used);
+    c->prof.fold(h0.ns_steps_used, h0.seg_log);
   }
   return CONQUR_OK;
 }
@@ -341,29 +344,29 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
   g.prior_rel = cfg->prior_rel;
   g.fro_tol = 0.1f;
-  g.margin = 1e-3f;
-  const double l0 = cfg->ns_sigma_min_rel > 0.f ? cfg->ns_sigma_min_rel : 1e-7;
-  const double final_err = 1e-6;
-  c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(cfg->ns_steps, g.margin, final_err)
-                               : plan_schedule(l0, g.margin, final_err, 100);
+  // bf16 products perturb the singular values by up to ~1e-3 per step, fp32 products by ~1e-6
+  g.margin = g.mode == CONQUR_TC_BF16 ? 2e-2f : 1e-3f;
+  NsPlanParams pp;
+  pp.l0 = cfg->ns_sigma_min_rel > 0.f ? cfg->ns_sigma_min_rel : 1e-9;
+  pp.margin = g.margin;
+  pp.d = g.mode == CONQUR_TC_BF16 ? d : 0;
+  pp.max_len = NS_SCHED_MAX;
+  c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(std::min(cfg->ns_steps, NS_SCHED_MAX), pp, &c->first_endgame)
+                               : plan_schedule(pp, &c->first_endgame);
   c->n_sched = (int)c->sched.size();
-  c->restart_idx = 0;
-  for (int i = 0; i < c->n_sched; ++i)
-    if (c->sched[i].l >= 1e-3) { c->restart_idx = i; break; }
-  if (c->restart_idx >= c->n_sched) c->restart_idx = c->n_sched - 1;
-  std::vector<float> coef(3 * 128, 0.f);
-  for (int i = 0; i < c->n_sched && i < 128; ++i) {
-    const NsStep& s = c->sched[i];
-    coef[3 * i + 0] = (float)(s.a + s.b + s.c);
-    coef[3 * i + 1] = (float)(s.b + 2.0 * s.c);
-    coef[3 * i + 2] = (float)s.c;
+  // if the schedule runs out (sigma_min below the assumed bound): two more lifting steps, then the endgame again
+  c->reenter_idx = std::max(0, c->first_endgame - 2);
+  std::vector<SchedEntry> coef(NS_SCHED_MAX);
+  for (int i = 0; i < NS_SCHED_MAX; ++i) {
+    const NsStep& s = c->sched[std::min(i, c->n_sched - 1)];
+    coef[i] = SchedEntry{(float)s.a, (float)s.b, (float)s.c, (float)s.l, s.lift, s.seg_x};
   }
   auto fail = [&](int rc) { delete c; return rc; };
   if (cudaMemsetAsync(c->ws, 0, L.R, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);   // state + flags
   if (cudaMemsetAsync(c->ws + L.M, 0, sizeof(float) * (size_t)d * d * g.P, c->stream) != cudaSuccess)
     return fail(CONQUR_ERR_CUDA);
-  if (cudaMemcpyAsync(c->ws + L.sched, coef.data(), sizeof(float) * 3 * 128, cudaMemcpyHostToDevice, c->stream) !=
-      cudaSuccess)
+  if (cudaMemcpyAsync(c->ws + L.sched, coef.data(), sizeof(SchedEntry) * NS_SCHED_MAX, cudaMemcpyHostToDevice,
+                      c->stream) != cudaSuccess)
     return fail(CONQUR_ERR_CUDA);
   set_identity_kernel<<<ew_blocks((int64_t)d * d * g.P), 256, 0, c->stream>>>(c->at<float>(L.R), d, g.P);
   if (cudaGetLastError() != cudaSuccess) return fail(CONQUR_ERR_CUDA);
@@ -563,9 +566,9 @@ extern "C" int conqur_get_profile(conqur_ctx* c, conqur_profile* out) {
 extern "C" int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out, int32_t max_steps) {
   if (!abc_out || max_steps < 1 || sigma_min_rel < 0.0 || sigma_min_rel >= 1.0 || ns_steps < 0)
     return CONQUR_ERR_INVALID_ARG;
-  const double l0 = sigma_min_rel > 0.0 ? sigma_min_rel : 1e-7;
-  const std::vector<NsStep> s = ns_steps > 0 ? plan_schedule_for_steps(ns_steps, 1e-3, 1e-6)
-                                             : plan_schedule(l0, 1e-3, 1e-6, 100);
+  NsPlanParams pp;
+  pp.l0 = sigma_min_rel > 0.0 ? sigma_min_rel : 1e-9;
+  const std::vector<NsStep> s = ns_steps > 0 ? plan_schedule_for_steps(ns_steps, pp) : plan_schedule(pp);
   const int n = std::min<int>((int)s.size(), max_steps);
   for (int i = 0; i < n; ++i) { abc_out[3 * i] = s[i].a; abc_out[3 * i + 1] = s[i].b; abc_out[3 * i + 2] = s[i].c; }
   return n;

@@ -32,9 +32,16 @@ struct DevState {
   float e_max, e_fro;       // residual norms of the last Newton-Schulz check
   float last_orth, last_fro;
   float scale, x0_scale, lam;
-  float coef[3];            // gamma, beta1, beta2 of the step in flight
-  float pad_[2];
+  float coef[4];            // gamma + kappa, beta1, beta2, kappa of the step in flight
+  float tau;                // shift of the residual: E = X^T X - tau I (1 in exact mode)
+  int ns_idx;               // next entry of the polynomial schedule
+  int seg_x;                // tensor-core mode: segments of the next-iterate product of the step in flight (1 or 2)
+  unsigned char seg_log[128];   // seg_x chosen at each step of the last update (launch accounting)
 };
+
+// One entry of the device copy of the polynomial schedule.
+struct SchedEntry { float a, b, c, l; int lift, seg_x; };
+constexpr int NS_SCHED_MAX = 128;
 
 // Kernel classes for launch counting / optional per-launch timing.
 enum : int { K_ROWNORM = 0, K_ROTATE = 1, K_ACCUM = 2, K_NS_RESID = 3, K_NS_POLY = 4, K_NS_NEXT = 5, K_OTHER = 6, K_COUNT = 8 };
@@ -42,7 +49,7 @@ enum : int { K_ROWNORM = 0, K_ROTATE = 1, K_ACCUM = 2, K_NS_RESID = 3, K_NS_POLY
 // Host-side launch accounting.  Launch counts are always kept; when `enabled`, the contractions are bracketed by
 // CUDA events on the launching stream (events are created lazily and reused).
 struct Prof {
-  struct Rec { int cls; double flops; int ns_k; cudaEvent_t e0, e1; };
+  struct Rec { int cls; double flops; int ns_k; int nseg; cudaEvent_t e0, e1; };   // nseg 0: look it up in seg_log
   bool enabled = false;
   long long launches[K_COUNT] = {0};
   long long total = 0;
@@ -61,13 +68,15 @@ struct Prof {
   }
   // Fold the finished records into the sums (call after a stream synchronise).  Newton-Schulz launches whose
   // step index lies past `steps_used` early-exited on the device and are left out.
-  void fold(int steps_used) {
+  void fold(int steps_used, const unsigned char* seg_log = nullptr) {
     for (Rec& r : open) {
       bool ran = true;
       if (r.ns_k >= 0) ran = (r.cls == K_NS_RESID) ? (r.ns_k <= steps_used) : (r.ns_k < steps_used);
       float t = 0.f;
       if (cudaEventElapsedTime(&t, r.e0, r.e1) == cudaSuccess && ran) {
-        ms[r.cls] += t; flops[r.cls] += r.flops; ++timed[r.cls];
+        int passes = r.nseg;
+        if (passes == 0) passes = (seg_log && r.ns_k >= 0 && r.ns_k < 128) ? seg_log[r.ns_k] : 1;
+        ms[r.cls] += t; flops[r.cls] += r.flops * passes; ++timed[r.cls];
       }
       pool.push_back(r.e0); pool.push_back(r.e1);
     }

@@ -451,7 +451,7 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
 // phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
 // phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
 static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
-                                float prior_rel, float inv_sqrt_d, float margin) {
+                                float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift) {
   const int p = blockIdx.x;
   __shared__ double red[8];
   double v = 0.0;
@@ -469,6 +469,10 @@ static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ 
       s->ns_done = ok ? 0 : NS_DONE_FAILED;
       s->ns_steps_used = 0;
       s->ns_final_buf = 0;
+      s->ns_idx = 0;
+      s->seg_x = 2;
+      // ||X_0||_F = 1/(1+margin): mean sigma^2 of the first iterate (the tensor-core mode shifts by it)
+      s->tau = use_shift ? 1.0f / ((1.0f + margin) * (1.0f + margin) * (float)d) : 1.0f;
     }
   }
 }
@@ -482,25 +486,35 @@ static __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __
     X0[p * dd + i] = fmaf(lam, R[p * dd + i], M[p * dd + i]) * sc;
 }
 
-// After the residual product of step k: reduce the per-CTA partials, decide convergence, pick the
-// polynomial of this step.  sched: n_sched entries of (gamma, beta1, beta2); restart_idx: where the
-// schedule re-enters when it ran out without convergence.
+// After the residual product of step k: reduce the per-tile partials (max|G - I|, sum (G - I)^2, trace G with
+// G = X^T X), decide convergence, and pick the quintic of this step from the schedule:
+//   * normally the next entry;
+//   * once ||G - I||_F < 0.7 every singular value is known to lie above sqrt(1 - ||G - I||_F), so the schedule
+//     jumps ahead to the last endgame entry fitted for an interval that still contains the spectrum;
+//   * if the schedule ran out without convergence (sigma_min was below the assumed bound) it re-enters at
+//     `reenter_idx` (lifting steps are safe to repeat: they never push a singular value below their floor).
+// The step is handed to the product kernels in shifted residual form (see ns_schedule.h): coef = (gamma + kappa,
+// beta1, beta2, kappa) where kappa = mean diagonal of beta1 E + beta2 E^2 is moved from the matrix that gets
+// rounded to bf16 into the scalar multiple of X.  use_shift == 0 (exact mode): tau = 1, kappa = 0.
 static __global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
-                                  const double* __restrict__ part_sq, int nparts, int k,
-                                  const float* __restrict__ sched, int n_sched, int restart_idx, float tol,
-                                  float fro_tol, int cur_buf, int max_steps) {
+                                  const double* __restrict__ part_sq, const double* __restrict__ part_tr,
+                                  int nparts, int k, const SchedEntry* __restrict__ sched, int n_sched,
+                                  int first_endgame, int reenter_idx, float tol, float fro_tol, int cur_buf,
+                                  int max_steps, int d, int use_shift) {
   const int p = blockIdx.x;
   DevState* s = st + p;
   if (s->ns_done) return;
   __shared__ double redd[8];
   __shared__ float redf[8];
-  double sq = 0.0;
+  double sq = 0.0, tr = 0.0;
   float mx = 0.f;
   for (int i = threadIdx.x; i < nparts; i += 256) {
     sq += part_sq[(int64_t)p * nparts + i];
     mx = fmaxf(mx, part_max[(int64_t)p * nparts + i]);
+    if (part_tr) tr += part_tr[(int64_t)p * nparts + i];
   }
   const double tsq = block_sum_d<256>(sq, redd);
+  const double ttr = block_sum_d<256>(tr, redd);
   const float tmx = block_max_f<256>(mx, redf);
   if (threadIdx.x == 0) {
     const float fro = (float)sqrt(tsq);
@@ -514,14 +528,45 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
     } else if (k >= max_steps) {
       s->ns_done = NS_DONE_FAILED;
     } else {
-      int idx = k;
-      if (idx >= n_sched) idx = restart_idx + (k - n_sched) % (n_sched - restart_idx);
-      s->coef[0] = sched[idx * 3 + 0];
-      s->coef[1] = sched[idx * 3 + 1];
-      s->coef[2] = sched[idx * 3 + 2];
+      int idx = s->ns_idx;
+      if (fro < 0.7f) {
+        const float lb = sqrtf(1.0f - fro);
+        for (int j = n_sched - 1; j >= first_endgame && j > idx; --j)
+          if (sched[j].l <= lb) { idx = j; break; }
+      }
+      if (idx >= n_sched) idx = reenter_idx;
+      const SchedEntry e = sched[idx];
+      const double a = e.a, b = e.b, c = e.c;
+      const double tau = use_shift ? (double)s->tau : 1.0;
+      const double b1 = b + 2.0 * c * tau;
+      double kappa = 0.0;
+      if (use_shift) {
+        // ||E_tau||_F^2 and tr E_tau from the statistics of G - I and tr G
+        const double dd = (double)d;
+        const double e2 = fmax(0.0, tsq + 2.0 * (1.0 - tau) * ttr + dd * (tau * tau - 1.0));
+        kappa = (c * e2 + b1 * (ttr - dd * tau)) / dd;
+      }
+      s->coef[0] = (float)(a + b * tau + c * tau * tau + kappa);
+      s->coef[1] = (float)b1;
+      s->coef[2] = (float)c;
+      s->coef[3] = (float)kappa;
+      s->seg_x = e.seg_x;
+      if (k < 128) s->seg_log[k] = (unsigned char)e.seg_x;
+      s->ns_idx = idx + 1;
       s->ns_steps_used = k + 1;
     }
   }
+}
+
+// tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode).
+static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ part_x2, int nparts, int d) {
+  DevState* s = st + blockIdx.x;
+  if (s->ns_done) return;
+  __shared__ double redd[8];
+  double v = 0.0;
+  for (int i = threadIdx.x; i < nparts; i += 256) v += part_x2[(int64_t)blockIdx.x * nparts + i];
+  const double tot = block_sum_d<256>(v, redd);
+  if (threadIdx.x == 0) s->tau = (float)(tot / (double)d);
 }
 
 // Accept or reject the update.  On success: R <- X_final, M <- 0, sums <- 0.

@@ -136,17 +136,34 @@ template <int BN> struct TcCfg {
 
 struct TcGemmArgs {
   int M, N, K;                  // output rows, cols; contraction length of one segment
-  int nseg;                     // 1, or 3 for the (hi,hi),(hi,lo),(lo,hi) split product
-  int a_lo, b_lo;               // outer-coordinate offset of the lo copy inside a stacked [hi; lo] operand
+  int nseg;                     // k-loop passes: 1, or up to 3 for split-precision products
+  int nseg_from_state;          // 1: take the number of passes from st->seg_x (chosen on the device per step)
+  int a_off[3], b_off[3];       // outer-coordinate offset of each pass's operand inside a stacked [hi; lo] pair
+  int sym;                      // 1: the output is symmetric (M == N): only tiles that touch the upper triangle are
+                                //    computed; tiles strictly above the diagonal also write their transpose
   float* outF; long long ldo;   // fp32 output (M read-modify-write, E, X_next, Y)
   __nv_bfloat16* outH; long long ldh; long long lo_elems;   // bf16 output hi part (+ lo part at +lo_elems)
   const float* inF; long long ldi;                          // fp32 epilogue input (E or X)
   const float* rnorm;
   unsigned* rowmax;
   double* part_d; float* part_f;
+  double* part_t;               // per-tile trace (residual) or sum of squares (next iterate)
   DevState* st;
   int check_done;
 };
+
+// Tiles of a symmetric product, column by column: column tn holds the row tiles 0 .. (tn+1)*BN/128 - 1.
+__host__ __device__ inline int tc_sym_tiles(int tiles_n, int BN) { return (BN / 128) * tiles_n * (tiles_n + 1) / 2; }
+template <int BN>
+__device__ __forceinline__ void tc_tile_coords(int t, int tiles_m, int sym, int& tm, int& tn) {
+  if (!sym) { tm = t % tiles_m; tn = t / tiles_m; return; }
+  constexpr int r = BN / 128;
+  int j = (int)((sqrtf(1.0f + 8.0f * (float)t / (float)r) - 1.0f) * 0.5f);
+  while (r * (j + 1) * (j + 2) / 2 <= t) ++j;
+  while (r * j * (j + 1) / 2 > t) --j;
+  tn = j;
+  tm = t - r * j * (j + 1) / 2;
+}
 
 struct TcAux {
   uint64_t full[8];
@@ -157,6 +174,7 @@ struct TcAux {
   int abort_flag;
   double red_d[4];
   float red_f[4];
+  float red_t[4];
 };
 
 // Bounded wait.  Returns false when the wait was abandoned (timeout here, or another role aborted).
@@ -198,9 +216,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
-  const int num_tiles = tiles_m * tiles_n;
+  const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, BN) : tiles_m * tiles_n;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
-  const int k_iters = num_kb * g.nseg;
+  const int nseg = g.nseg_from_state ? max(1, min(3, g.st->seg_x)) : g.nseg;
+  const int k_iters = num_kb * nseg;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { ptx::mbar_init(&aux->full[s], 1); ptx::mbar_init(&aux->empty[s], 1); }
@@ -229,10 +248,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int issued = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % tiles_m) * TC_BM, n0 = (tile / tiles_m) * BN;
+        int tm, tn;
+        tc_tile_coords<BN>(tile, tiles_m, g.sym, tm, tn);
+        const int m0 = tm * TC_BM, n0 = tn * BN;
         for (int it = 0; it < k_iters; ++it) {
           const int seg = it / num_kb, k0 = (it - seg * num_kb) * TC_BK;
-          const int a_off = (seg == 2) ? g.a_lo : 0, b_off = (seg == 1) ? g.b_lo : 0;
+          const int a_off = g.a_off[seg], b_off = g.b_off[seg];
           if (!tc_wait(&aux->empty[stage], phase ^ 1u, abort_flag)) { ok = false; timeout_site = 1; break; }
           uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
           uint8_t* sb = sa + Cfg::A_BYTES;
@@ -304,13 +325,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------------------------------------------------------- epilogue (4 warps, 128 TMEM lanes)
     const int q = warp & 3;                               // TMEM lane quarter this warp may read
     const int et = q * 32 + lane;                         // row inside the tile
-    float c_gamma = 0.f, c_b1 = 0.f, c_b2 = 0.f;
-    if (EPI == TC_EPI_POLY || EPI == TC_EPI_NEXT) { c_gamma = g.st->coef[0]; c_b1 = g.st->coef[1]; c_b2 = g.st->coef[2]; }
+    float c_gamma = 0.f, c_b1 = 0.f, c_b2 = 0.f, c_kappa = 0.f, c_tau = 1.f;
+    if (EPI == TC_EPI_POLY || EPI == TC_EPI_NEXT) {
+      c_gamma = g.st->coef[0]; c_b1 = g.st->coef[1]; c_b2 = g.st->coef[2]; c_kappa = g.st->coef[3];
+    }
+    if (EPI == TC_EPI_RESID) c_tau = g.st->tau;
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
       const int buf = local & 1;
-      const int m0 = (tile % tiles_m) * TC_BM, n0 = (tile / tiles_m) * BN;
+      int tm, tn;
+      tc_tile_coords<BN>(tile, tiles_m, g.sym, tm, tn);
+      const int m0 = tm * TC_BM, n0 = tn * BN;
+      const bool mirror = g.sym && ((tm + 1) * TC_BM <= tn * BN);     // strictly above the diagonal
       if (!tc_wait(&aux->tfull[buf], (uint32_t)(local >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 4; break; }
       ptx::tc_fence_after();
       const int row = m0 + et;
@@ -322,7 +349,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         rn = row_ok ? g.rnorm[row] : 0.f;
         rn_bits = bf16_bits(rn);
       }
-      float acc_abs = 0.f, acc_max = 0.f;
+      float acc_abs = 0.f, acc_max = 0.f, acc_tr = 0.f;
       double acc_sq = 0.0;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
@@ -365,14 +392,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         } else {
-          // Newton-Schulz epilogues: fp32 value, then its two-term bf16 split
+          // Newton-Schulz epilogues
+          const int dcol = row - col0;                      // position of the diagonal inside this chunk, if any
           if (EPI == TC_EPI_RESID) {
-            const int dcol = row - col0;
+            // statistics of G - I and of tr G; the stored residual is E = G - tau I
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              if (i == dcol) v[i] -= 1.f;
-              acc_max = fmaxf(acc_max, fabsf(v[i]));
-              acc_sq += (double)v[i] * (double)v[i];
+              float e1 = v[i];
+              if (i == dcol) { acc_tr += v[i]; e1 -= 1.f; v[i] -= c_tau; }
+              acc_max = fmaxf(acc_max, fabsf(e1));
+              acc_sq += (double)e1 * (double)e1;
             }
           } else {
             const float4* src = reinterpret_cast<const float4*>(g.inF + (long long)row * g.ldi + col0);
@@ -387,6 +416,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 v[4 * i + 2] = fmaf(c_gamma, t.z, v[4 * i + 2]); v[4 * i + 3] = fmaf(c_gamma, t.w, v[4 * i + 3]);
               }
             }
+            if (EPI == TC_EPI_POLY) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i == dcol) v[i] -= c_kappa;
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc_sq += (double)v[i] * (double)v[i];
+            }
           }
           if (EPI != TC_EPI_POLY) {
             float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
@@ -399,14 +436,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const float a = v[2 * i], b = v[2 * i + 1];
             const float ah = bf16_round(a), bh = bf16_round(b);
             wh[i] = bf16_bits(ah) | (bf16_bits(bh) << 16);
-            wl[i] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+            if (EPI == TC_EPI_NEXT) wl[i] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
           }
           uint4* dh = reinterpret_cast<uint4*>(g.outH + (long long)row * g.ldh + col0);
-          uint4* dl = reinterpret_cast<uint4*>(g.outH + g.lo_elems + (long long)row * g.ldh + col0);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            dh[i] = make_uint4(wh[4 * i], wh[4 * i + 1], wh[4 * i + 2], wh[4 * i + 3]);
-            dl[i] = make_uint4(wl[4 * i], wl[4 * i + 1], wl[4 * i + 2], wl[4 * i + 3]);
+          for (int i = 0; i < 4; ++i) dh[i] = make_uint4(wh[4 * i], wh[4 * i + 1], wh[4 * i + 2], wh[4 * i + 3]);
+          if (EPI == TC_EPI_NEXT) {
+            uint4* dl = reinterpret_cast<uint4*>(g.outH + g.lo_elems + (long long)row * g.ldh + col0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dl[i] = make_uint4(wl[4 * i], wl[4 * i + 1], wl[4 * i + 2], wl[4 * i + 3]);
+          }
+          if (EPI != TC_EPI_NEXT && mirror) {
+            // transpose of the tile: lane t holds row (m0 + 32 q + t), so for a fixed column the 32 lanes write
+            // 32 consecutive elements of one output row
+            unsigned short* oh = reinterpret_cast<unsigned short*>(g.outH);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const long long at = (long long)(col0 + i) * g.ldh + row;
+              oh[at] = (unsigned short)((i & 1) ? (wh[i >> 1] >> 16) : (wh[i >> 1] & 0xffffu));
+            }
           }
         }
       }
@@ -417,17 +465,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (EPI == TC_EPI_ROTATE_Q) {
         if (row_ok && rn > 0.f) atomicMax(g.rowmax + row, __float_as_uint(acc_max));
       }
-      if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_RESID) {
+      if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_RESID || EPI == TC_EPI_NEXT) {
         // per-tile partials, fixed reduction order; named barrier 1 synchronises the 4 epilogue warps only
         double dsum = (EPI == TC_EPI_ROTATE) ? (double)(acc_abs * rn) : acc_sq;
         dsum = warp_sum_d(dsum);
         float fmx = warp_max(acc_max);
-        if (lane == 0) { aux->red_d[q] = dsum; aux->red_f[q] = fmx; }
+        float ftr = warp_sum(acc_tr);
+        if (lane == 0) { aux->red_d[q] = dsum; aux->red_f[q] = fmx; aux->red_t[q] = ftr; }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (q == 0 && lane == 0) {
-          g.part_d[tile] = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
-          if (EPI == TC_EPI_RESID)
+          const double tot = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
+          if (EPI == TC_EPI_NEXT) {
+            g.part_t[tile] = tot;
+          } else {
+            g.part_d[tile] = mirror ? 2.0 * tot : tot;       // a mirrored tile stands for two
+          }
+          if (EPI == TC_EPI_RESID) {
             g.part_f[tile] = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
+            g.part_t[tile] = (double)aux->red_t[0] + (double)aux->red_t[1] + (double)aux->red_t[2] + (double)aux->red_t[3];
+          }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
@@ -634,8 +690,8 @@ inline void tc_make_layout(int d, int P, int64_t n_max, int quant_bits, TcLayout
   L->Rb = take(2 * dd);
   L->Xh[0] = take(4 * dd);
   L->Xh[1] = take(4 * dd);
-  L->Eh = take(4 * dd);
-  L->Bh = take(4 * dd);
+  L->Eh = take(2 * dd);
+  L->Bh = take(2 * dd);
 }
 
 inline int tc_epi_class(int epi) {
@@ -659,13 +715,16 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
       return CONQUR_ERR_CUDA;
     attr_set = true;
   }
-  const int tiles = ((g.M + TC_BM - 1) / TC_BM) * ((g.N + BN - 1) / BN);
+  const int tiles_n = (g.N + BN - 1) / BN;
+  const int tiles = g.sym ? tc_sym_tiles(tiles_n, BN) : ((g.M + TC_BM - 1) / TC_BM) * tiles_n;
   const int grid = tiles < h.num_sms ? tiles : h.num_sms;
   const int cls = tc_epi_class(EPI);
   Prof::Rec rec{};
   const bool timed = h.prof && h.prof->enabled;
   if (timed) {
-    rec.cls = cls; rec.flops = 2.0 * g.M * (double)g.N * g.K * g.nseg; rec.ns_k = h.ns_k;
+    // flops the tensor cores execute: computed tiles only, one pass (scaled by the passes taken when folded)
+    rec.cls = cls; rec.flops = 2.0 * (double)tiles * TC_BM * BN * (double)g.K; rec.ns_k = h.ns_k;
+    rec.nseg = g.nseg_from_state ? 0 : g.nseg;
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
@@ -704,9 +763,9 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
     rc |= tc_make_tmap(&h->tmXh_mn[i], ws + L.Xh[i], 2 * D, D, D, 64);
     rc |= tc_make_tmap(&h->tmXh_k[i], ws + L.Xh[i], 2 * D, D, D, 128);
   }
-  rc |= tc_make_tmap(&h->tmEh_k, ws + L.Eh, 2 * D, D, D, 128);
-  rc |= tc_make_tmap(&h->tmEh_mn, ws + L.Eh, 2 * D, D, D, 64);
-  rc |= tc_make_tmap(&h->tmBh_mn, ws + L.Bh, 2 * D, D, D, 64);
+  rc |= tc_make_tmap(&h->tmEh_k, ws + L.Eh, D, D, D, 128);
+  rc |= tc_make_tmap(&h->tmEh_mn, ws + L.Eh, D, D, D, 64);
+  rc |= tc_make_tmap(&h->tmBh_mn, ws + L.Bh, D, D, D, 64);
   return rc ? CONQUR_ERR_CUDA : CONQUR_OK;
 }
 
@@ -782,34 +841,45 @@ inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
 }
 
 inline int tc_ns_tile_n(const TcHost& h) { return (h.d % 256 == 0) ? 256 : 128; }
-inline int tc_ns_parts(const TcHost& h) { return (h.d / TC_BM) * (h.d / tc_ns_tile_n(h)); }
 
-// E = X^T X - I from the split iterate in Xh[buf]
+// Partials of the Newton-Schulz epilogues: [0, parts) sums of squares, [parts, 2 parts) traces / iterate norms.
+inline int tc_ns_parts(const TcHost& h) { return tc_sym_tiles(h.d / tc_ns_tile_n(h), tc_ns_tile_n(h)); }
+inline int tc_ns_next_parts(const TcHost& h) { return (h.d / TC_BM) * (h.d / tc_ns_tile_n(h)); }
+
+// G = X^T X from the split iterate in Xh[buf] (three passes: hi hi, hi lo, lo hi; symmetric tiles only);
+// stores E = G - tau I as fp32 and bf16, and the statistics of G - I.
 inline int tc_ns_residual(TcHost& h, cudaStream_t s, int buf) {
   const int d = h.d;
   TcGemmArgs g = tc_args(h, d, d, d);
-  g.nseg = 3; g.a_lo = d; g.b_lo = d; g.check_done = 1;
+  g.nseg = 3; g.a_off[2] = d; g.b_off[1] = d; g.check_done = 1; g.sym = 1;
   g.outF = h.E; g.ldo = d;
-  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Eh); g.ldh = d; g.lo_elems = (long long)d * d;
+  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Eh); g.ldh = d;
+  g.part_t = h.part_d + tc_ns_parts(h);
   return tc_launch_n<true, true, TC_EPI_RESID>(h, s, h.tmXh_mn[buf], h.tmXh_mn[buf], g);
 }
 
-// B = beta2 E E + beta1 E ;  X_next = X B + gamma X
+// B = beta2 E E + beta1 E - kappa I (one bf16 pass, symmetric tiles only) ;  X_next = X B + (gamma + kappa) X
+// (the iterate enters as hi, or hi + lo while small singular values are still being lifted).
 inline int tc_ns_poly_next(TcHost& h, cudaStream_t s, int cur) {
   const int d = h.d;
   const long long dd = (long long)d * d;
   TcGemmArgs g = tc_args(h, d, d, d);
-  g.nseg = 3; g.a_lo = d; g.b_lo = d; g.check_done = 1;
+  g.nseg = 1; g.check_done = 1; g.sym = 1;
   g.inF = h.E; g.ldi = d;
-  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Bh); g.ldh = d; g.lo_elems = dd;
+  g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Bh); g.ldh = d;
   int rc = tc_launch_n<false, true, TC_EPI_POLY>(h, s, h.tmEh_k, h.tmEh_mn, g);
   if (rc) return rc;
   TcGemmArgs x = tc_args(h, d, d, d);
-  x.nseg = 3; x.a_lo = d; x.b_lo = d; x.check_done = 1;
+  x.nseg = 2; x.nseg_from_state = 1; x.a_off[1] = d; x.check_done = 1;
   x.inF = cur ? h.Xb : h.Xa; x.ldi = d;
   x.outF = cur ? h.Xa : h.Xb; x.ldo = d;
   x.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[1 - cur]); x.ldh = d; x.lo_elems = dd;
-  return tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
+  x.part_t = h.part_d + tc_ns_parts(h);
+  rc = tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
+  if (rc) return rc;
+  ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d);
+  if (h.prof) h.prof->count(K_OTHER);
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
 inline const __nv_bfloat16* tc_cp_ptr(const TcHost& h) { return reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Cp); }
@@ -837,7 +907,7 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   if (rc) return rc;
   TcGemmArgs g{};
   g.M = M; g.N = N; g.K = K; g.nseg = split ? 3 : 1; g.st = st;
-  g.a_lo = a_mn ? K : M; g.b_lo = b_mn ? K : N;
+  g.a_off[2] = a_mn ? K : M; g.b_off[1] = b_mn ? K : N;
   g.outF = D; g.ldo = N;
   if (!a_mn && !b_mn) return tc_launch_n<false, false, TC_EPI_PLAIN>(h, s, ta, tb, g);
   if (!a_mn && b_mn) return tc_launch_n<false, true, TC_EPI_PLAIN>(h, s, ta, tb, g);

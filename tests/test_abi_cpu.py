@@ -61,7 +61,7 @@ def test_init_rejects_bad_arguments_without_a_device(B):
     assert B.strerror(0) == "ok" and "Newton" in B.strerror(-6)
 
 
-@pytest.mark.parametrize("l0", [1e-2, 1e-4, 1e-7])
+@pytest.mark.parametrize("l0", [1e-2, 1e-4, 1e-7, 1e-9])
 def test_planned_polynomials_drive_the_assumed_interval_to_one(B, l0):
     abc = B.conqur_plan_schedule(l0)
     x = np.concatenate([np.logspace(np.log10(l0), 0, 4000), np.linspace(l0, 1, 4000)])
@@ -71,13 +71,28 @@ def test_planned_polynomials_drive_the_assumed_interval_to_one(B, l0):
         assert x.max() <= 1.0 + 1e-9                   # never leaves [0, 1]: no divergence
         assert x.min() > lo_track                      # the bottom of the spectrum only moves up
         lo_track = x.min()
-    assert 1.0 - x.min() < 5e-6 and len(abc) <= 16
+    assert 1.0 - x.min() < 5e-6 and len(abc) <= 20
     # below the assumed bound singular values still grow monotonically (slower convergence, no failure)
     y = np.array([l0 * 1e-3])
     for a, b, c in abc:
         y2 = a * y + b * y ** 3 + c * y ** 5
         assert y2 > y
         y = y2
+
+
+def test_lifting_steps_never_push_a_large_singular_value_down(B):
+    """The repeated lifting quintic keeps everything that has reached [0.05, 1] above its floor (about 0.2), so
+    directions that already carry weight are never brought back to the rounding-noise level."""
+    abc = B.conqur_plan_schedule(1e-9)
+    a, b, c = abc[0]
+    assert np.allclose(abc[1], abc[0]) and np.allclose(abc[5], abc[0])      # the same quintic, repeated
+    x = np.linspace(0.05, 1.0, 100001)
+    p = a * x + b * x ** 3 + c * x ** 5
+    assert p.min() > 0.19 and p.max() <= 1.0 / 1.02 + 1e-9
+    x = np.logspace(-9, 0, 20001)
+    for k in range(40):                                                       # far more often than planned
+        x = a * x + b * x ** 3 + c * x ** 5
+    assert x.min() > 0.19 and x.max() <= 1.0
 
 
 def test_plan_for_a_step_budget(B):
@@ -87,15 +102,15 @@ def test_plan_for_a_step_budget(B):
     assert len(B.conqur_plan_schedule(0.0, 8)) == 8
 
 
-def test_first_polynomial_is_the_minimax_quintic(B):
-    # equioscillation: |1 - p| attains the same maximum at both ends and two interior points of [l, 1/(1+m)]
-    l0 = 1e-2
-    a, b, c = B.conqur_plan_schedule(l0)[0]
-    x = np.linspace(l0, 1.0, 200001)
+def test_lifting_polynomial_is_the_minimax_quintic(B):
+    # equioscillation: |1 - p| attains the same maximum at both ends and two interior points of [0.05, 1]
+    lf = 0.05
+    a, b, c = B.conqur_plan_schedule(1e-6)[0]
+    x = np.linspace(lf, 1.0, 200001)
     p = a * x + b * x ** 3 + c * x ** 5
     top = p.max()
     err = 1 - p / top                                  # undo the output rescaling: p/top ranges over [1-2E/(1+E), 1]
-    ext = [err[0], err.max()]
     assert abs(err[0] - err.max()) < 1e-6
-    interior_min = p[(x > 0.2) & (x < 0.95)].min()
+    assert abs(p[-1] - top) < 1e-6 * top
+    interior_min = p[(x > 0.4) & (x < 0.95)].min()
     assert abs((1 - interior_min / top) - err[0]) < 1e-6
