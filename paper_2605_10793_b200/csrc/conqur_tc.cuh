@@ -22,6 +22,7 @@
 #include <stdint.h>
 
 #include <cstdio>
+#include <cstdlib>
 
 #include "../../include/conqur.h"
 #include "conqur_internal.h"
@@ -113,6 +114,60 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// ---- CTA-pair (cta_group::2) forms: two CTAs of a cluster share one 256-row MMA
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory; the bytes are counted on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tmap, uint32_t bar_cluster_addr,
+                                                 int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far retire.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask)
+               : "memory");
+}
+
 }  // namespace ptx
 
 // ------------------------------------------------------------------ kernel configuration
@@ -124,11 +179,16 @@ constexpr long long TC_WAIT_LIMIT = 4000000000ll;   // ~2 s of SM clocks
 enum { TC_EPI_ROTATE = 0, TC_EPI_ROTATE_Q = 1, TC_EPI_ACCUM = 2, TC_EPI_RESID = 3, TC_EPI_POLY = 4, TC_EPI_NEXT = 5,
        TC_EPI_PLAIN = 6 };
 
-template <int BN> struct TcCfg {
+// PAIR: two CTAs of a cluster work on one 256 x 256 tile (each holds 128 rows of A and of the accumulator and
+// 128 of the 256 columns of B in its own shared memory); otherwise one CTA works on a 128 x BN tile.
+template <int BN, bool PAIR> struct TcCfg {
+  static_assert(!PAIR || BN == 256, "a CTA pair always computes 256 x 256 tiles");
+  static constexpr int TILE_M = PAIR ? 256 : TC_BM;
   static constexpr int A_BYTES = TC_BM * TC_BK * 2;
-  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int B_ROWS = PAIR ? 128 : BN;      // rows (n) of B this CTA loads per stage
+  static constexpr int B_BYTES = B_ROWS * TC_BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int STAGES = PAIR ? 6 : ((BN == 256) ? 4 : 6);
   static constexpr int TMEM_COLS = 2 * BN;          // two accumulators: the epilogue of tile i overlaps tile i+1
   static constexpr int AUX_BYTES = 1024;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + AUX_BYTES + 1024 /* alignment slack */;
@@ -152,17 +212,16 @@ struct TcGemmArgs {
   int check_done;
 };
 
-// Tiles of a symmetric product, column by column: column tn holds the row tiles 0 .. (tn+1)*BN/128 - 1.
-__host__ __device__ inline int tc_sym_tiles(int tiles_n, int BN) { return (BN / 128) * tiles_n * (tiles_n + 1) / 2; }
-template <int BN>
+// Tiles (TM x BN) of a symmetric product, column by column: column tn holds the row tiles 0 .. (tn+1)*BN/TM - 1.
+__host__ __device__ inline int tc_sym_tiles(int tiles_n, int r /* BN / TM */) { return r * tiles_n * (tiles_n + 1) / 2; }
+template <int R>
 __device__ __forceinline__ void tc_tile_coords(int t, int tiles_m, int sym, int& tm, int& tn) {
   if (!sym) { tm = t % tiles_m; tn = t / tiles_m; return; }
-  constexpr int r = BN / 128;
-  int j = (int)((sqrtf(1.0f + 8.0f * (float)t / (float)r) - 1.0f) * 0.5f);
-  while (r * (j + 1) * (j + 2) / 2 <= t) ++j;
-  while (r * j * (j + 1) / 2 > t) --j;
+  int j = (int)((sqrtf(1.0f + 8.0f * (float)t / (float)R) - 1.0f) * 0.5f);
+  while (R * (j + 1) * (j + 2) / 2 <= t) ++j;
+  while (R * j * (j + 1) / 2 > t) --j;
   tn = j;
-  tm = t - r * j * (j + 1) / 2;
+  tm = t - R * j * (j + 1) / 2;
 }
 
 struct TcAux {
@@ -203,11 +262,13 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_by
 __device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
 
-template <int BN, bool A_MN, bool B_MN, int EPI>
+template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcGemmArgs g) {
-  using Cfg = TcCfg<BN>;
-  if (g.check_done && g.st->ns_done) return;      // uniform: the iteration already finished
+  using Cfg = TcCfg<BN, PAIR>;
+  constexpr int TM = Cfg::TILE_M;
+  constexpr int R = BN / TM;                        // tiles per column step of a symmetric product
+  if (g.check_done && g.st->ns_done) return;      // uniform over the grid: the iteration already finished
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -215,15 +276,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile int* abort_flag = &aux->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
-  const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, BN) : tiles_m * tiles_n;
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;        // 0: the CTA that issues the pair's MMAs
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int tiles_m = (g.M + TM - 1) / TM, tiles_n = (g.N + BN - 1) / BN;
+  const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, R) : tiles_m * tiles_n;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
   const int nseg = g.nseg_from_state ? max(1, min(3, g.st->seg_x)) : g.nseg;
   const int k_iters = num_kb * nseg;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { ptx::mbar_init(&aux->full[s], 1); ptx::mbar_init(&aux->empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->tfull[b], 1); ptx::mbar_init(&aux->tempty[b], 128); }
+    // the accumulator is handed back by every epilogue thread (of both CTAs of a pair)
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->tfull[b], 1); ptx::mbar_init(&aux->tempty[b], PAIR ? 256 : 128); }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -231,11 +296,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tmap(&tmB);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&aux->tmem_base, Cfg::TMEM_COLS);
-    ptx::tmem_relinquish();
+    if (PAIR) { ptx::tmem_alloc_pair(&aux->tmem_base, Cfg::TMEM_COLS); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(&aux->tmem_base, Cfg::TMEM_COLS); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();                // the peer's barriers exist before anything is sent to them
   ptx::tc_fence_after();
   const uint32_t tmem_base = aux->tmem_base;
   int timeout_site = 0;
@@ -247,57 +313,82 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < num_tiles && ok; tile += n_workers) {
         int tm, tn;
-        tc_tile_coords<BN>(tile, tiles_m, g.sym, tm, tn);
-        const int m0 = tm * TC_BM, n0 = tn * BN;
+        tc_tile_coords<R>(tile, tiles_m, g.sym, tm, tn);
+        // a pair splits the tile: this CTA loads 128 of the 256 rows of A and 128 of the 256 columns of B
+        const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN + (PAIR ? (int)rank * Cfg::B_ROWS : 0);
         for (int it = 0; it < k_iters; ++it) {
           const int seg = it / num_kb, k0 = (it - seg * num_kb) * TC_BK;
           const int a_off = g.a_off[seg], b_off = g.b_off[seg];
           if (!tc_wait(&aux->empty[stage], phase ^ 1u, abort_flag)) { ok = false; timeout_site = 1; break; }
           uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
           uint8_t* sb = sa + Cfg::A_BYTES;
-          ptx::mbar_expect_tx(&aux->full[stage], Cfg::STAGE_BYTES);
-          if (A_MN) {
+          if (PAIR) {
+            // both CTAs' copies are counted on the barrier of CTA 0, whose MMA thread consumes the stage
+            const uint32_t bar = ptx::mapa_u32(ptx::smem_u32(&aux->full[stage]), 0);
+            if (rank == 0) ptx::mbar_expect_tx(&aux->full[stage], 2 * Cfg::STAGE_BYTES);
+            if (A_MN) {
 #pragma unroll
-            for (int h = 0; h < TC_BM / 64; ++h)
-              ptx::tma_load_2d(sa + h * 8192, &tmA, &aux->full[stage], m0 + 64 * h, k0 + a_off);
-          } else {
-            ptx::tma_load_2d(sa, &tmA, &aux->full[stage], k0, m0 + a_off);
-          }
-          if (B_MN) {
+              for (int h = 0; h < TC_BM / 64; ++h) ptx::tma_load_2d_pair(sa + h * 8192, &tmA, bar, m0 + 64 * h, k0 + a_off);
+            } else {
+              ptx::tma_load_2d_pair(sa, &tmA, bar, k0, m0 + a_off);
+            }
+            if (B_MN) {
 #pragma unroll
-            for (int h = 0; h < BN / 64; ++h)
-              ptx::tma_load_2d(sb + h * 8192, &tmB, &aux->full[stage], n0 + 64 * h, k0 + b_off);
+              for (int h = 0; h < Cfg::B_ROWS / 64; ++h) ptx::tma_load_2d_pair(sb + h * 8192, &tmB, bar, n0 + 64 * h, k0 + b_off);
+            } else {
+              ptx::tma_load_2d_pair(sb, &tmB, bar, k0, n0 + b_off);
+            }
           } else {
-            ptx::tma_load_2d(sb, &tmB, &aux->full[stage], k0, n0 + b_off);
+            ptx::mbar_expect_tx(&aux->full[stage], Cfg::STAGE_BYTES);
+            if (A_MN) {
+#pragma unroll
+              for (int h = 0; h < TC_BM / 64; ++h)
+                ptx::tma_load_2d(sa + h * 8192, &tmA, &aux->full[stage], m0 + 64 * h, k0 + a_off);
+            } else {
+              ptx::tma_load_2d(sa, &tmA, &aux->full[stage], k0, m0 + a_off);
+            }
+            if (B_MN) {
+#pragma unroll
+              for (int h = 0; h < BN / 64; ++h)
+                ptx::tma_load_2d(sb + h * 8192, &tmB, &aux->full[stage], n0 + 64 * h, k0 + b_off);
+            } else {
+              ptx::tma_load_2d(sb, &tmB, &aux->full[stage], k0, n0 + b_off);
+            }
           }
           ++issued;
           if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
-        // drain: wait (bounded) until the copies already issued have landed before the CTA may exit
-        const int pending = issued < Cfg::STAGES ? issued : Cfg::STAGES;
-        int s = stage;
-        uint32_t ph = phase;
-        for (int i = 0; i < pending; ++i) {
-          if (--s < 0) { s = Cfg::STAGES - 1; ph ^= 1u; }
+        // drain: the copies already issued must have landed before the CTA may exit
+        if (PAIR) {
+          // their completion is counted in the other CTA: give them a fixed time (far beyond any copy latency)
           const long long t0 = clock64();
-          while (!ptx::mbar_try_wait(&aux->full[s], ph) && clock64() - t0 < TC_WAIT_LIMIT) {}
+          while (clock64() - t0 < 4000000ll) {}
+        } else {
+          const int pending = issued < Cfg::STAGES ? issued : Cfg::STAGES;
+          int s = stage;
+          uint32_t ph = phase;
+          for (int i = 0; i < pending; ++i) {
+            if (--s < 0) { s = Cfg::STAGES - 1; ph ^= 1u; }
+            const long long t0 = clock64();
+            while (!ptx::mbar_try_wait(&aux->full[s], ph) && clock64() - t0 < TC_WAIT_LIMIT) {}
+          }
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // ---------------------------------------------------------------- MMA issuer (CTA 0 of a pair issues for both)
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+      for (int tile = worker; tile < num_tiles && ok; tile += n_workers, ++local) {
         const int buf = local & 1;
         if (!tc_wait(&aux->tempty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 2; break; }
         ptx::tc_fence_after();
@@ -311,14 +402,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int j = 0; j < TC_BK / 16; ++j) {
             // K-major: 16 k = 32 bytes inside the swizzled 128-byte row; 8-row groups 1024 bytes apart.
             // MN-major: 16 k = two 8-row groups of 1024 bytes; 64-wide m|n chunks 8192 bytes apart.
+            // For a pair the descriptors name this CTA's tiles; the peer's halves sit at the same offsets in its memory.
             const uint64_t ad = A_MN ? tc_smem_desc(sa + j * 2048, 8192, 1024) : tc_smem_desc(sa + j * 32, 16, 1024);
             const uint64_t bd = B_MN ? tc_smem_desc(sb + j * 2048, 8192, 1024) : tc_smem_desc(sb + j * 32, 16, 1024);
-            ptx::umma_bf16(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
+            if (PAIR) ptx::umma_bf16_pair(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
+            else ptx::umma_bf16(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
           }
-          ptx::umma_commit(&aux->empty[stage]);          // frees the smem stage once these MMAs retire
+          // frees the shared-memory stage (in both CTAs of a pair) once these MMAs retire
+          if (PAIR) ptx::umma_commit_pair(&aux->empty[stage]); else ptx::umma_commit(&aux->empty[stage]);
           if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) ptx::umma_commit(&aux->tfull[buf]);       // accumulator complete
+        if (ok) {                                         // accumulator complete
+          if (PAIR) ptx::umma_commit_pair(&aux->tfull[buf]); else ptx::umma_commit(&aux->tfull[buf]);
+        }
       }
     }
   } else {
@@ -332,12 +428,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (EPI == TC_EPI_RESID) c_tau = g.st->tau;
     int local = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+    const uint32_t tempty_addr0 = PAIR ? ptx::mapa_u32(ptx::smem_u32(&aux->tempty[0]), 0) : 0u;
+    for (int tile = worker; tile < num_tiles && ok; tile += n_workers, ++local) {
       const int buf = local & 1;
       int tm, tn;
-      tc_tile_coords<BN>(tile, tiles_m, g.sym, tm, tn);
-      const int m0 = tm * TC_BM, n0 = tn * BN;
-      const bool mirror = g.sym && ((tm + 1) * TC_BM <= tn * BN);     // strictly above the diagonal
+      tc_tile_coords<R>(tile, tiles_m, g.sym, tm, tn);
+      const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN;   // this CTA's 128 rows, all BN columns
+      const bool mirror = g.sym && ((tm + 1) * TM <= tn * BN);        // strictly above the diagonal
+      const int slot = PAIR ? 2 * tile + (int)rank : tile;            // where this CTA's per-tile partials go
       if (!tc_wait(&aux->tfull[buf], (uint32_t)(local >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 4; break; }
       ptx::tc_fence_after();
       const int row = m0 + et;
@@ -458,9 +556,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
-      // release the accumulator to the MMA warp before the (slower) reductions
+      // release the accumulator to the MMA thread before the (slower) reductions
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&aux->tempty[buf]);
+      if (PAIR) ptx::mbar_arrive_cluster(tempty_addr0 + (uint32_t)(buf * sizeof(uint64_t)));
+      else ptx::mbar_arrive(&aux->tempty[buf]);
 
       if (EPI == TC_EPI_ROTATE_Q) {
         if (row_ok && rn > 0.f) atomicMax(g.rowmax + row, __float_as_uint(acc_max));
@@ -476,13 +575,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (q == 0 && lane == 0) {
           const double tot = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
           if (EPI == TC_EPI_NEXT) {
-            g.part_t[tile] = tot;
+            g.part_t[slot] = tot;
           } else {
-            g.part_d[tile] = mirror ? 2.0 * tot : tot;       // a mirrored tile stands for two
+            g.part_d[slot] = mirror ? 2.0 * tot : tot;       // a mirrored tile stands for two
           }
           if (EPI == TC_EPI_RESID) {
-            g.part_f[tile] = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
-            g.part_t[tile] = (double)aux->red_t[0] + (double)aux->red_t[1] + (double)aux->red_t[2] + (double)aux->red_t[3];
+            g.part_f[slot] = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
+            g.part_t[slot] = (double)aux->red_t[0] + (double)aux->red_t[1] + (double)aux->red_t[2] + (double)aux->red_t[3];
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -496,9 +595,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();                // neither CTA leaves while the other may still reach into it
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS); else ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
   }
 }
 
@@ -628,6 +728,7 @@ struct TcLayout {
 
 struct TcHost {
   int d, P, quant_bits, num_sms;
+  int pair_clusters;                         // CTA pairs that can be co-resident (0: single-CTA kernels only)
   int64_t n_max;
   char* ws;
   TcLayout L;
@@ -705,40 +806,88 @@ inline int tc_epi_class(int epi) {
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, int EPI>
+// Which kernel variant a product of output width N runs with.
+//   pair : CTA pairs on 256 x 256 tiles (needs N % 256 == 0 and a device that can co-schedule the pairs)
+//   else : single CTAs on 128 x 256 (N % 256 == 0) or 128 x 128 tiles
+struct TcVariant { bool pair; int tile_m, tile_n; };
+inline TcVariant tc_variant(const TcHost& h, int N) {
+  if (N % 256 == 0) return h.pair_clusters > 0 ? TcVariant{true, 256, 256} : TcVariant{false, 128, 256};
+  return TcVariant{false, 128, 128};
+}
+// tiles the kernel computes, and per-tile partial slots it writes (a pair writes one per CTA)
+inline int tc_tiles(const TcVariant& v, int M, int N, int sym) {
+  const int tn = (N + v.tile_n - 1) / v.tile_n, tm = (M + v.tile_m - 1) / v.tile_m;
+  return sym ? tc_sym_tiles(tn, v.tile_n / v.tile_m) : tm * tn;
+}
+inline int tc_part_slots(const TcVariant& v, int M, int N, int sym) { return tc_tiles(v, M, N, sym) * (v.pair ? 2 : 1); }
+
+template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR>
 inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
-  using Cfg = TcCfg<BN>;
-  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI>;
+  using Cfg = TcCfg<BN, PAIR>;
+  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, PAIR>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
     attr_set = true;
   }
-  const int tiles_n = (g.N + BN - 1) / BN;
-  const int tiles = g.sym ? tc_sym_tiles(tiles_n, BN) : ((g.M + TC_BM - 1) / TC_BM) * tiles_n;
-  const int grid = tiles < h.num_sms ? tiles : h.num_sms;
+  const TcVariant v{PAIR, Cfg::TILE_M, BN};
+  const int tiles = tc_tiles(v, g.M, g.N, g.sym);
+  const int workers = PAIR ? h.pair_clusters : h.num_sms;
+  const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
   const int cls = tc_epi_class(EPI);
   Prof::Rec rec{};
   const bool timed = h.prof && h.prof->enabled;
   if (timed) {
     // flops the tensor cores execute: computed tiles only, one pass (scaled by the passes taken when folded)
-    rec.cls = cls; rec.flops = 2.0 * (double)tiles * TC_BM * BN * (double)g.K; rec.ns_k = h.ns_k;
+    rec.cls = cls; rec.flops = 2.0 * (double)tiles * Cfg::TILE_M * BN * (double)g.K; rec.ns_k = h.ns_k;
     rec.nseg = g.nseg_from_state ? 0 : g.nseg;
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
-  kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, g);
+  cudaError_t err;
+  if (PAIR) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = Cfg::SMEM_BYTES; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, kern, a, b, g);
+  } else {
+    kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, g);
+    err = cudaGetLastError();
+  }
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
   if (h.prof) h.prof->count(cls);
-  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
+  return err == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
-// dispatch on the N tile: 256 when the output width allows it, else 128
+// dispatch on the kernel variant (see tc_variant)
 template <bool A_MN, bool B_MN, int EPI>
 inline int tc_launch_n(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
-  if (g.N % 256 == 0) return tc_launch<256, A_MN, B_MN, EPI>(h, s, a, b, g);
-  return tc_launch<128, A_MN, B_MN, EPI>(h, s, a, b, g);
+  const TcVariant v = tc_variant(h, g.N);
+  if (v.pair) return tc_launch<256, A_MN, B_MN, EPI, true>(h, s, a, b, g);
+  if (v.tile_n == 256) return tc_launch<256, A_MN, B_MN, EPI, false>(h, s, a, b, g);
+  return tc_launch<128, A_MN, B_MN, EPI, false>(h, s, a, b, g);
+}
+
+// How many CTA pairs of the 256 x 256 kernel can be resident at once (0: use single CTAs).
+inline int tc_query_pair_clusters() {
+  const char* env = std::getenv("CONQUR_TC_SINGLE_CTA");
+  if (env && env[0] == '1') return 0;
+  using Cfg = TcCfg<256, true>;
+  auto kern = tc_gemm_kernel<256, false, true, TC_EPI_PLAIN, true>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * 1024); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n > 0 ? n : 0;
 }
 
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
@@ -756,6 +905,7 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
     return CONQUR_ERR_UNSUPPORTED;
   }
   h->num_sms = prop.multiProcessorCount;
+  h->pair_clusters = tc_query_pair_clusters();
   const uint64_t D = (uint64_t)d;
   int rc = 0;
   rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, D, D, D, 64);
@@ -812,7 +962,7 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
     g.outH = Cp; g.ldh = d;
     rc = tc_launch_n<false, true, TC_EPI_ROTATE>(h, s, tmXs_k, h.tmRb_mn, g);
     if (rc) return rc;
-    per_problem = ((int)((n + TC_BM - 1) / TC_BM)) * ((d + ((d % 256 == 0) ? 256 : 128) - 1) / ((d % 256 == 0) ? 256 : 128));
+    per_problem = tc_part_slots(tc_variant(h, d), (int)n, d, 0);
   } else {
     if (cudaMemsetAsync(h.rowmax, 0, sizeof(unsigned) * n, s) != cudaSuccess) return CONQUR_ERR_CUDA;
     g.outF = h.Y; g.ldo = d; g.rowmax = h.rowmax;
@@ -840,11 +990,10 @@ inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
-inline int tc_ns_tile_n(const TcHost& h) { return (h.d % 256 == 0) ? 256 : 128; }
 
 // Partials of the Newton-Schulz epilogues: [0, parts) sums of squares, [parts, 2 parts) traces / iterate norms.
-inline int tc_ns_parts(const TcHost& h) { return tc_sym_tiles(h.d / tc_ns_tile_n(h), tc_ns_tile_n(h)); }
-inline int tc_ns_next_parts(const TcHost& h) { return (h.d / TC_BM) * (h.d / tc_ns_tile_n(h)); }
+inline int tc_ns_parts(const TcHost& h) { return tc_part_slots(tc_variant(h, h.d), h.d, h.d, 1); }
+inline int tc_ns_next_parts(const TcHost& h) { return tc_part_slots(tc_variant(h, h.d), h.d, h.d, 0); }
 
 // G = X^T X from the split iterate in Xh[buf] (three passes: hi hi, hi lo, lo hi; symmetric tiles only);
 // stores E = G - tau I as fp32 and bf16, and the statistics of G - I.
@@ -897,12 +1046,14 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
   if (prop.major != 10) return CONQUR_ERR_UNSUPPORTED;
   h.num_sms = prop.multiProcessorCount;
+  h.pair_clusters = tc_query_pair_clusters();
   const uint64_t mul = split ? 2 : 1;
   CUtensorMap ta, tb;
   int rc;
   if (a_mn) rc = tc_make_tmap(&ta, A, mul * K, M, M, 64); else rc = tc_make_tmap(&ta, A, mul * M, K, K, 128);
   if (rc) return rc;
-  const uint32_t bn = (N % 256 == 0) ? 256 : 128;
+  const TcVariant v = tc_variant(h, N);
+  const uint32_t bn = v.pair ? 128 : (uint32_t)v.tile_n;      // rows of B one CTA loads per stage
   if (b_mn) rc = tc_make_tmap(&tb, B, mul * K, N, N, 64); else rc = tc_make_tmap(&tb, B, mul * N, K, K, bn);
   if (rc) return rc;
   TcGemmArgs g{};
