@@ -340,7 +340,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
-  g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 40;
+  g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 0;   // 0: set from the schedule below
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
   g.prior_rel = cfg->prior_rel;
   g.fro_tol = 0.1f;
@@ -354,6 +354,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(std::min(cfg->ns_steps, NS_SCHED_MAX), pp, &c->first_endgame)
                                : plan_schedule(pp, &c->first_endgame);
   c->n_sched = (int)c->sched.size();
+  if (g.ns_max_steps == 0) g.ns_max_steps = std::min(120, c->n_sched + 12);
   // if the schedule runs out (sigma_min below the assumed bound): two more lifting steps, then the endgame again
   c->reenter_idx = std::max(0, c->first_endgame - 2);
   std::vector<SchedEntry> coef(NS_SCHED_MAX);

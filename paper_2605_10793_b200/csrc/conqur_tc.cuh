@@ -175,6 +175,7 @@ constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                   // one 128-byte swizzle row of bf16
 constexpr int TC_THREADS = 192;             // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr long long TC_WAIT_LIMIT = 4000000000ll;   // ~2 s of SM clocks
+constexpr int TC_BAND = 8;                  // row tiles per band of the tile order
 
 enum { TC_EPI_ROTATE = 0, TC_EPI_ROTATE_Q = 1, TC_EPI_ACCUM = 2, TC_EPI_RESID = 3, TC_EPI_POLY = 4, TC_EPI_NEXT = 5,
        TC_EPI_PLAIN = 6 };
@@ -215,8 +216,17 @@ struct TcGemmArgs {
 // Tiles (TM x BN) of a symmetric product, column by column: column tn holds the row tiles 0 .. (tn+1)*BN/TM - 1.
 __host__ __device__ inline int tc_sym_tiles(int tiles_n, int r /* BN / TM */) { return r * tiles_n * (tiles_n + 1) / 2; }
 template <int R>
-__device__ __forceinline__ void tc_tile_coords(int t, int tiles_m, int sym, int& tm, int& tn) {
-  if (!sym) { tm = t % tiles_m; tn = t / tiles_m; return; }
+__device__ __forceinline__ void tc_tile_coords(int t, int tiles_m, int tiles_n, int sym, int& tm, int& tn) {
+  if (!sym) {
+    // bands of TC_BAND row tiles, column by column inside a band: the tiles in flight at any time cover a roughly
+    // square patch of the output, which keeps the operand blocks they share resident in L2
+    const int per_band = TC_BAND * tiles_n;
+    const int band = t / per_band, within = t - band * per_band;
+    const int rows = min(TC_BAND, tiles_m - band * TC_BAND);
+    tn = within / rows;
+    tm = band * TC_BAND + (within - tn * rows);
+    return;
+  }
   int j = (int)((sqrtf(1.0f + 8.0f * (float)t / (float)R) - 1.0f) * 0.5f);
   while (R * (j + 1) * (j + 2) / 2 <= t) ++j;
   while (R * j * (j + 1) / 2 > t) --j;
@@ -315,7 +325,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (int tile = worker; tile < num_tiles && ok; tile += n_workers) {
         int tm, tn;
-        tc_tile_coords<R>(tile, tiles_m, g.sym, tm, tn);
+        tc_tile_coords<R>(tile, tiles_m, tiles_n, g.sym, tm, tn);
         // a pair splits the tile: this CTA loads 128 of the 256 rows of A and 128 of the 256 columns of B
         const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN + (PAIR ? (int)rank * Cfg::B_ROWS : 0);
         for (int it = 0; it < k_iters; ++it) {
@@ -432,7 +442,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int tile = worker; tile < num_tiles && ok; tile += n_workers, ++local) {
       const int buf = local & 1;
       int tm, tn;
-      tc_tile_coords<R>(tile, tiles_m, g.sym, tm, tn);
+      tc_tile_coords<R>(tile, tiles_m, tiles_n, g.sym, tm, tn);
       const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN;   // this CTA's 128 rows, all BN columns
       const bool mirror = g.sym && ((tm + 1) * TM <= tn * BN);        // strictly above the diagonal
       const int slot = PAIR ? 2 * tile + (int)rank : tile;            // where this CTA's per-tile partials go
@@ -478,13 +488,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                            fmaxf(fabsf(v[4 * i + 2]), fabsf(v[4 * i + 3]))));
           }
         } else if (EPI == TC_EPI_ACCUM) {
-          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
+          // M += acc as fire-and-forget vector reductions performed at the L2: the epilogue never waits for M to
+          // arrive.  Each element of M receives exactly one addition per launch, so the result does not depend on
+          // any ordering inside the launch.
+          float* dst = g.outF + (long long)row * g.ldo + col0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float4 t = dst[i];
-            t.x += v[4 * i]; t.y += v[4 * i + 1]; t.z += v[4 * i + 2]; t.w += v[4 * i + 3];
-            dst[i] = t;
-          }
+          for (int i = 0; i < 8; ++i)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(v[4 * i]), "f"(v[4 * i + 1]),
+                         "f"(v[4 * i + 2]), "f"(v[4 * i + 3])
+                         : "memory");
         } else if (EPI == TC_EPI_PLAIN) {
           float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
 #pragma unroll
