@@ -16,6 +16,7 @@
 #include "conqur_internal.h"
 #include "conqur_simt.cuh"
 #include "conqur_tc.cuh"
+#include "conqur_tc_batched.cuh"
 #include "ns_schedule.h"
 
 using namespace conqur;
@@ -41,6 +42,7 @@ struct Cfg {
   int d, P, in_dtype, mode, quant_bits, ns_max_steps;
   int64_t n_max;
   float orth_tol, prior_rel, fro_tol, margin;
+  bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode; batched problems)
 };
 
 int pick_acc_splits(int d, int P, int64_t n_max) {
@@ -89,8 +91,8 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
     L->acc_splits = pick_acc_splits(d, (int)P, n);
     if (L->acc_splits > 1) L->splitk = take(sizeof(float) * dd * P * L->acc_splits);
   } else {
-    if (c->quant_bits) L->C = take(sizeof(float) * (size_t)n * d * P);
-    tc_make_layout(d, (int)P, n, c->quant_bits, &L->tc, take);
+    if (c->quant_bits && P == 1) L->C = take(sizeof(float) * (size_t)n * d);
+    tc_make_layout(d, (int)P, n, c->quant_bits, c->in_dtype, &L->tc, take);
   }
   L->total = off;
   return true;
@@ -222,7 +224,7 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
 int launch_residual(conqur_ctx* c, const float* X, int buf) {
   const Cfg& g = c->cfg;
   const int T = cdiv(g.d, SG_BM);
-  if (g.mode == CONQUR_EXACT_F32) {
+  if (g.simt_ns) {
     ns_gemm_exact_kernel<EPI_RESIDUAL><<<dim3(T, T, g.P), SG_THREADS, 0, c->stream>>>(
         X, X, nullptr, c->at<float>(c->L.E), g.d, c->state(), c->at<float>(c->L.part_f), c->at<double>(c->L.part_d));
     CQ_LAUNCHED(c, K_NS_RESID);
@@ -231,7 +233,7 @@ int launch_residual(conqur_ctx* c, const float* X, int buf) {
   return tc_ns_residual(c->tc, c->stream, buf);
 }
 int ns_parts(const conqur_ctx* c) {
-  if (c->cfg.mode == CONQUR_EXACT_F32) { const int T = cdiv(c->cfg.d, SG_BM); return T * T; }
+  if (c->cfg.simt_ns) { const int T = cdiv(c->cfg.d, SG_BM); return T * T; }
   return tc_ns_parts(c->tc);
 }
 
@@ -249,7 +251,7 @@ int update_impl(conqur_ctx* c) {
   double* pd = c->at<double>(c->L.part_d);
   float* pf = c->at<float>(c->L.part_f);
   const SchedEntry* sched = c->at<SchedEntry>(c->L.sched);
-  const int use_shift = g.mode == CONQUR_TC_BF16 ? 1 : 0;
+  const int use_shift = g.simt_ns ? 0 : 1;
   const int nb = (int)std::min<int64_t>(1024, (dd + 1023) / 1024);
   const float isd = (float)(1.0 / std::sqrt((double)d));
 
@@ -265,7 +267,7 @@ int update_impl(conqur_ctx* c) {
   CQ_LAUNCHED(c, K_OTHER);
   ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
   CQ_LAUNCHED(c, K_OTHER);
-  if (g.mode == CONQUR_TC_BF16) { int rc = tc_ns_begin(c->tc, c->stream); if (rc) return rc; }
+  if (!g.simt_ns) { int rc = tc_ns_begin(c->tc, c->stream); if (rc) return rc; }
 
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);
@@ -281,7 +283,7 @@ int update_impl(conqur_ctx* c) {
                                                 g.ns_max_steps, d, use_shift);
     CQ_LAUNCHED(c, K_OTHER);
     if (k == g.ns_max_steps) break;
-    if (g.mode == CONQUR_EXACT_F32) {
+    if (g.simt_ns) {
       ns_gemm_exact_kernel<EPI_POLY><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(E, E, E, B, d, st, nullptr, nullptr);
       CQ_LAUNCHED(c, K_NS_POLY);
       ns_gemm_exact_kernel<EPI_NEXT><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(X, B, X, Xn, d, st, nullptr, nullptr);
@@ -340,16 +342,17 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
+  g.simt_ns = (g.mode == CONQUR_EXACT_F32) || g.P > 1;
   g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 0;   // 0: set from the schedule below
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
   g.prior_rel = cfg->prior_rel;
   g.fro_tol = 0.1f;
   // bf16 products perturb the singular values by up to ~1e-3 per step, fp32 products by ~1e-6
-  g.margin = g.mode == CONQUR_TC_BF16 ? 2e-2f : 1e-3f;
+  g.margin = g.simt_ns ? 1e-3f : 2e-2f;
   NsPlanParams pp;
   pp.l0 = cfg->ns_sigma_min_rel > 0.f ? cfg->ns_sigma_min_rel : 1e-9;
   pp.margin = g.margin;
-  pp.d = g.mode == CONQUR_TC_BF16 ? d : 0;
+  pp.d = g.simt_ns ? 0 : d;
   pp.max_len = NS_SCHED_MAX;
   c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(std::min(cfg->ns_steps, NS_SCHED_MAX), pp, &c->first_endgame)
                                : plan_schedule(pp, &c->first_endgame);
@@ -420,14 +423,15 @@ extern "C" int conqur_set_R(conqur_ctx* c, const float* R_dev) {
 static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int64_t pstride) {
   if (!c || !X) return CONQUR_ERR_INVALID_ARG;
   const Cfg& g = c->cfg;
-  if (n < 0 || n > g.n_max || ld < g.d || pstride < 0) return CONQUR_ERR_INVALID_ARG;
+  if (n < 0 || n > g.n_max || ld < g.d || pstride < 0 || (g.P > 1 && pstride == 0)) return CONQUR_ERR_INVALID_ARG;
   if (n == 0) return CONQUR_OK;
   int rc;
   if (g.mode == CONQUR_EXACT_F32) {
     rc = (g.in_dtype == CONQUR_F32) ? step_exact<float>(c, static_cast<const float*>(X), n, ld, pstride)
                                     : step_exact<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(X), n, ld, pstride);
   } else {
-    rc = tc_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride);
+    rc = g.P > 1 ? tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride)
+                 : tc_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride);
   }
   if (rc == CONQUR_OK) { c->tokens_since_update += n; c->last_n = n; }
   return rc;

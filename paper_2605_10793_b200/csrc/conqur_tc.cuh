@@ -792,12 +792,20 @@ inline int tc_make_tmap(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_
   return CONQUR_OK;
 }
 
-inline bool tc_supported_shape(int d, int batch) { return d >= 128 && (d % 128) == 0 && batch == 1; }
+// one problem of any d that is a multiple of 128, or many problems of d = 128 (the per-head case)
+inline bool tc_supported_shape(int d, int batch) { return d >= 128 && (d % 128) == 0 && (batch == 1 || d == 128); }
 
 template <typename Take>
-inline void tc_make_layout(int d, int P, int64_t n_max, int quant_bits, TcLayout* L, Take&& take) {
-  (void)P; (void)quant_bits;
+inline void tc_make_layout(int d, int P, int64_t n_max, int quant_bits, int in_dtype, TcLayout* L, Take&& take) {
+  (void)quant_bits;
   const size_t dd = (size_t)d * d;
+  *L = TcLayout{};
+  if (P > 1) {
+    // batched (d = 128): the fused kernel keeps everything else on chip
+    if (in_dtype == CONQUR_F32) L->Xs = take(2 * (size_t)n_max * d * P);
+    L->Rb = take(2 * dd * P);
+    return;
+  }
   L->Xs = take(2 * (size_t)n_max * d);
   L->Cp = take(2 * (size_t)n_max * d);
   L->Rb = take(2 * dd);
@@ -920,6 +928,11 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
   h->pair_clusters = tc_query_pair_clusters();
   const uint64_t D = (uint64_t)d;
   int rc = 0;
+  if (P > 1) {
+    // all rotations stacked: problem p's R is rows [128 p, 128 p + 128); one box = 64 columns x all 128 rows
+    rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, (uint64_t)P * D, D, D, 128);
+    return rc ? CONQUR_ERR_CUDA : CONQUR_OK;
+  }
   rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, D, D, D, 64);
   for (int i = 0; i < 2; ++i) {
     rc |= tc_make_tmap(&h->tmXh_mn[i], ws + L.Xh[i], 2 * D, D, D, 64);
@@ -937,7 +950,7 @@ inline int tc_ew_blocks(int64_t count4) {
 }
 
 inline int tc_refresh_R(TcHost& h, cudaStream_t s, int) {
-  const int64_t dd = (int64_t)h.d * h.d;
+  const int64_t dd = (int64_t)h.d * h.d * h.P;
   split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.R, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Rb), dd, 0);
   if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;

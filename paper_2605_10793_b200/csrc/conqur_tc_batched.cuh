@@ -1,0 +1,378 @@
+// Tensor-core mode for many small problems (the per-head case, d = 128): one fused kernel per streamed batch.
+//
+// A CTA owns one problem at a time and walks its tokens in tiles of 128 rows.  Per tile
+//   TMA            X tile (128 tokens x 128, bf16)              -> shared memory (read ONCE from HBM)
+//   tcgen05.mma    Y = X_tile R                                 -> TMEM          (R: bf16, resident in shared memory)
+//   epilogue       row norms from the X tile, sign / fake-quant of Y, objective partial,
+//                  C' = sgn(.) * rnorm as bf16                   -> shared memory
+//   tcgen05.mma    M += X_tile^T C'                              -> TMEM accumulator that lives for the whole problem
+// and after the last tile the accumulator is added to the problem's fp32 M in global memory.  The X tile in
+// shared memory serves three times: K-major operand of the first product, source of the row norms, MN-major
+// operand of the second product.  Rows with a zero or non-finite norm are zeroed in shared memory before the
+// second product so that they cannot reach M.
+//
+// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue.  Every wait is bounded.
+#pragma once
+#include "conqur_tc.cuh"
+
+namespace conqur {
+
+constexpr int TCB_D = 128;                       // problem size this kernel is built for
+constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = two 64-column swizzled chunks of 16 KB
+constexpr int TCB_XSTAGES = 3;
+constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + 1024 + 1024;
+
+struct TcbAux {
+  uint64_t rfull, rempty, mfull, mempty;
+  uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
+  uint64_t yfull[2], yempty[2], cready[2], cfree[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  double red_d[4];
+  int red_i[4];
+  int red_f[4];
+};
+
+struct TcbStepArgs {
+  int n, P;
+  int levels;                 // 0: corner target of the rotated row; > 0: symmetric fake-quantisation with this many levels first
+  float* M;                   // P x 128 x 128 fp32 (without the 1/sqrt(d))
+  double* part_d;             // P objective partials (sum |y| * rnorm, or the quantised equivalent)
+  DevState* st;               // P
+};
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(ptx::smem_u32(smem_dst)), "l"(tmap), "r"(ptx::smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+// Byte offset of the 16-byte piece `c16` (0..15) of row `r` inside a 128 x 128 bf16 tile stored as two 64-column
+// chunks with the 128-byte swizzle (what TMA writes and what the MMA descriptors expect).
+__device__ __forceinline__ uint32_t tcb_piece(int r, int c16) {
+  return (uint32_t)((c16 >> 3) * 16384 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR, const TcbStepArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sR = smem;
+  uint8_t* sX = smem + TCB_TILE_BYTES;
+  uint8_t* sC = smem + TCB_TILE_BYTES * (1 + TCB_XSTAGES);
+  TcbAux* aux = reinterpret_cast<TcbAux*>(smem + TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2));
+  volatile int* abort_flag = &aux->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int T = (g.n + 127) / 128;                 // token tiles per problem
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
+    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, 128);
+    for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], 128);
+      ptx::mbar_init(&aux->cready[b], 128); ptx::mbar_init(&aux->cfree[b], 1);
+    }
+    aux->abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    ptx::prefetch_tmap(&tmX);
+    ptx::prefetch_tmap(&tmR);
+  }
+  if (warp == 1) { ptx::tmem_alloc(&aux->tmem_base, 512); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = aux->tmem_base;     // columns [0,128) and [128,256): Y buffers; [256,384): M accumulator
+  int timeout_site = 0;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int xs = 0; uint32_t xph = 0;
+      int lp = 0;
+      bool ok = true;
+      int issued = 0;
+      for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+        if (!tc_wait(&aux->rempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 11; break; }
+        ptx::mbar_expect_tx(&aux->rfull, TCB_TILE_BYTES);
+        ptx::tma_load_2d(sR, &tmR, &aux->rfull, 0, p * TCB_D);
+        ptx::tma_load_2d(sR + 16384, &tmR, &aux->rfull, 64, p * TCB_D);
+        for (int t = 0; t < T; ++t) {
+          if (!tc_wait(&aux->xempty[xs], xph ^ 1u, abort_flag)) { ok = false; timeout_site = 12; break; }
+          uint8_t* dst = sX + xs * TCB_TILE_BYTES;
+          ptx::mbar_expect_tx(&aux->xfull[xs], TCB_TILE_BYTES);
+          tma_load_3d(dst, &tmX, &aux->xfull[xs], 0, t * 128, p);
+          tma_load_3d(dst + 16384, &tmX, &aux->xfull[xs], 64, t * 128, p);
+          ++issued;
+          if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
+        }
+      }
+      if (!ok && issued > 0) {                     // let the copies in flight land before the CTA exits
+        const long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) {}
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptors: bf16 x bf16 -> fp32, M = N = 128; first product A K-major / B MN-major, second both MN-major
+      const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t idesc1 = idesc_base | (1u << 16);
+      const uint32_t idesc2 = idesc_base | (1u << 15) | (1u << 16);
+      const uint32_t sR_a = ptx::smem_u32(sR), sX_a = ptx::smem_u32(sX), sC_a = ptx::smem_u32(sC);
+      int xs = 0; uint32_t xph = 0;          // stage of the tile the first product reads
+      int xs2 = 0;                           // stage of the tile the second product reads (one tile behind)
+      int it = 0, it2 = 0;                   // tiles issued to the first / second product (over all problems)
+      int lp = 0;
+      bool ok = true;
+      auto second_product = [&](bool first_of_problem) -> bool {
+        const int cb = it2 & 1;
+        if (!tc_wait(&aux->cready[cb], ((uint32_t)it2 >> 1) & 1u, abort_flag)) { timeout_site = 23; return false; }
+        ptx::tc_fence_after();
+        const uint32_t xa = sX_a + xs2 * TCB_TILE_BYTES, ca = sC_a + cb * TCB_TILE_BYTES;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)          // 16 tokens per instruction: two 8-row groups, 2048 bytes per step
+          ptx::umma_bf16(tmem_base + 256, tc_smem_desc(xa + j * 2048, 16384, 1024), tc_smem_desc(ca + j * 2048, 16384, 1024),
+                         idesc2, (!first_of_problem || j > 0) ? 1u : 0u);
+        ptx::umma_commit(&aux->xempty[xs2]);
+        ptx::umma_commit(&aux->cfree[cb]);
+        if (++xs2 == TCB_XSTAGES) xs2 = 0;
+        ++it2;
+        return true;
+      };
+      for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+        if (!tc_wait(&aux->rfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 20; break; }
+        if (!tc_wait(&aux->mempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 21; break; }
+        for (int t = 0; t < T && ok; ++t) {
+          const int yb = it & 1;
+          if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 22; break; }
+          if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
+          ptx::tc_fence_after();
+          const uint32_t xa = sX_a + xs * TCB_TILE_BYTES;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)        // 16 features per instruction: chunk j/4, 32 bytes per step inside the swizzled row
+            ptx::umma_bf16(tmem_base + yb * 128, tc_smem_desc(xa + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024),
+                           tc_smem_desc(sR_a + j * 2048, 16384, 1024), idesc1, j > 0 ? 1u : 0u);
+          ptx::umma_commit(&aux->yfull[yb]);
+          if (t == T - 1) ptx::umma_commit(&aux->rempty);     // R may be replaced once every first product has run
+          if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
+          ++it;
+          if (t > 0) ok = second_product(t == 1);
+        }
+        if (ok) ok = second_product(T == 1);
+        if (ok) ptx::umma_commit(&aux->mfull);
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const int r = q * 32 + lane;                   // token inside the tile; later: row of M
+    const float L = (float)g.levels;
+    int it = 0, lp = 0;
+    bool ok = true;
+    for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+      double acc = 0.0;
+      int skipped = 0, nonfinite = 0;
+      for (int t = 0; t < T && ok; ++t, ++it) {
+        const int yb = it & 1, xs = it % TCB_XSTAGES;
+        const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
+        if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
+        // a1: row norm from the tile in shared memory
+        uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
+        float ss = 0.f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, c));
+          const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float a = __uint_as_float(u[e] << 16), b = __uint_as_float(u[e] & 0xffff0000u);
+            ss = fmaf(a, a, ss); ss = fmaf(b, b, ss);
+          }
+        }
+        const bool valid = (t * 128 + r) < g.n;
+        const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
+        if (valid && !good) {
+          ++skipped;
+          if (!(ss == 0.f)) nonfinite = 1;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, c)) = make_uint4(0, 0, 0, 0);
+        }
+        const float rn = good ? 1.0f / sqrtf(ss) : 0.f;
+        const uint32_t rn_bits = bf16_bits(rn);
+        if (!tc_wait(&aux->cfree[yb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
+        if (!tc_wait(&aux->yfull[yb], par2, abort_flag)) { ok = false; timeout_site = 32; break; }
+        ptx::tc_fence_after();
+        const uint32_t t_addr = tmem_base + (uint32_t)(yb * 128) + ((uint32_t)(q * 32) << 16);
+        uint8_t* crow = sC + yb * TCB_TILE_BYTES;
+        float inv = 0.f, delta = 0.f;
+        if (g.levels > 0) {
+          float mx = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float v[32];
+            ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(v[i]));
+          }
+          const bool live = good && (mx > 0.f);
+          inv = live ? (L / mx) : 0.f;
+          delta = live ? (mx / L) : 0.f;
+        }
+        float acc_t = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float a = v[2 * i], b = v[2 * i + 1];
+            if (g.levels > 0) {
+              a = fminf(fmaxf(rintf(a * inv), -L), L);
+              b = fminf(fmaxf(rintf(b * inv), -L), L);
+            }
+            acc_t += fabsf(a) + fabsf(b);
+            const uint32_t lo = (a == 0.f) ? 0u : (rn_bits | ((__float_as_uint(a) >> 16) & 0x8000u));
+            const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
+            w[i] = good ? (lo | (hi << 16)) : 0u;
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            *reinterpret_cast<uint4*>(crow + tcb_piece(r, c * 4 + k)) = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+        }
+        if (good) acc += (g.levels > 0) ? (double)(rn * delta) * (double)acc_t : (double)(acc_t * rn);
+        // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
+        ptx::tc_fence_before();
+        ptx::fence_proxy_async();
+        ptx::mbar_arrive(&aux->cready[yb]);
+        ptx::mbar_arrive(&aux->yempty[yb]);
+      }
+      if (!ok) break;
+      // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T)
+      if (!tc_wait(&aux->mfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 33; break; }
+      ptx::tc_fence_after();
+      {
+        const uint32_t t_addr = tmem_base + 256u + ((uint32_t)(q * 32) << 16);
+        float* dst = g.M + ((long long)p * TCB_D + r) * TCB_D;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+          float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float4 o = d4[i];
+            o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
+            d4[i] = o;
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&aux->mempty);
+      // per-problem reductions in a fixed order (named barrier 1: the four epilogue warps only)
+      const double wsum = warp_sum_d(acc);
+      int wsk = skipped, wnf = nonfinite;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
+      if (lane == 0) { aux->red_d[q] = wsum; aux->red_i[q] = wsk; aux->red_f[q] = wnf; }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (q == 0 && lane == 0) {
+        g.part_d[p] = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
+        const int sk = aux->red_i[0] + aux->red_i[1] + aux->red_i[2] + aux->red_i[3];
+        if (sk) g.st[p].step_skipped += sk;                      // this CTA is the only writer of problem p's state
+        if (aux->red_f[0] | aux->red_f[1] | aux->red_f[2] | aux->red_f[3]) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+  }
+
+  if (timeout_site != 0) {
+    atomicOr(&g.st[0].status_flags, STATUS_FLAG_TIMEOUT);
+    g.st[0].timeout_site = timeout_site;
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// fp32 -> bf16 staging of a batched input (problem p, row i at X + p*pstride + i*ld) into a dense P x n x 128 copy
+__global__ void tcb_stage_f32_kernel(const float* __restrict__ X, int64_t n, int64_t ld, int64_t pstride, int P,
+                                     __nv_bfloat16* __restrict__ Xs) {
+  const int64_t total4 = (int64_t)P * n * (TCB_D / 4);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += (int64_t)gridDim.x * blockDim.x) {
+    const int c4 = (int)(i % (TCB_D / 4));
+    const int64_t row = (i / (TCB_D / 4)) % n, p = i / ((TCB_D / 4) * n);
+    const float* src = X + p * pstride + row * ld + c4 * 4;
+    uint2 o;
+    o.x = bf16_bits(src[0]) | (bf16_bits(src[1]) << 16);
+    o.y = bf16_bits(src[2]) | (bf16_bits(src[3]) << 16);
+    *reinterpret_cast<uint2*>(Xs + (p * n + row) * TCB_D + c4 * 4) = o;
+  }
+}
+
+// 3-D view of a batched bf16 input: (128 features, n rows with stride ld, P problems with stride pstride); box 64 x 128 x 1.
+inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_t ld, uint64_t pstride, uint64_t P) {
+  PFN_encodeTiled fn = tc_encode_fn();
+  if (!fn) return CONQUR_ERR_CUDA;
+  const cuuint64_t dims[3] = {TCB_D, n, P};
+  const cuuint64_t strides[2] = {ld * 2, (P > 1 ? pstride : ld * n) * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "conqur: cuTensorMapEncodeTiled (batched input) failed (%d)\n", (int)r);
+    return CONQUR_ERR_INVALID_ARG;
+  }
+  return CONQUR_OK;
+}
+
+// One streamed batch for all P problems.  X: device, bf16 or fp32 (fp32 is first rounded into the staging copy).
+inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tcb_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCB_SMEM_BYTES) != cudaSuccess)
+      return CONQUR_ERR_CUDA;
+    attr_set = true;
+  }
+  const void* src = X;
+  int64_t src_ld = ld, src_ps = pstride;
+  if (in_dtype == CONQUR_F32) {
+    __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xs);
+    tcb_stage_f32_kernel<<<tc_ew_blocks((int64_t)h.P * n * (TCB_D / 4)), 256, 0, s>>>(static_cast<const float*>(X), n, ld,
+                                                                                     pstride, h.P, Xs);
+    if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (h.prof) h.prof->count(K_ROWNORM);
+    src = Xs; src_ld = TCB_D; src_ps = n * TCB_D;
+  } else if ((reinterpret_cast<uintptr_t>(X) & 15) || (ld % 8) || (pstride % 8)) {
+    return CONQUR_ERR_INVALID_ARG;            // TMA needs 16-byte aligned rows and problem bases
+  }
+  CUtensorMap tmX;
+  int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)h.P);
+  if (rc) return rc;
+  TcbStepArgs g{};
+  g.n = (int)n; g.P = h.P; g.levels = h.quant_bits ? (1 << (h.quant_bits - 1)) - 1 : 0;
+  g.M = h.M; g.part_d = h.part_d; g.st = h.st;
+  const int grid = h.P < h.num_sms ? h.P : h.num_sms;
+  Prof::Rec rec{};
+  const bool timed = h.prof && h.prof->enabled;
+  if (timed) {
+    rec.cls = K_ROTATE; rec.flops = 4.0 * (double)h.P * (double)n * TCB_D * TCB_D; rec.ns_k = -1; rec.nseg = 1;
+    rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
+    cudaEventRecord(rec.e0, s);
+  }
+  tcb_step_kernel<<<grid, TC_THREADS, TCB_SMEM_BYTES, s>>>(tmX, h.tmRb_mn, g);
+  if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_ROTATE);
+  finalize_step_kernel<<<h.P, 256, 0, s>>>(h.st, h.part_d, 1, n, 1.0 / std::sqrt((double)TCB_D));
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_OTHER);
+  return CONQUR_OK;
+}
+
+}  // namespace conqur
