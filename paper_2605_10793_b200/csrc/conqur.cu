@@ -42,7 +42,7 @@ struct Cfg {
   int d, P, in_dtype, mode, quant_bits, ns_max_steps;
   int64_t n_max;
   float orth_tol, prior_rel, fro_tol, margin;
-  bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode; batched problems)
+  bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode)
 };
 
 int pick_acc_splits(int d, int P, int64_t n_max) {
@@ -254,6 +254,12 @@ int update_impl(conqur_ctx* c) {
   const int use_shift = g.simt_ns ? 0 : 1;
   const int nb = (int)std::min<int64_t>(1024, (dd + 1023) / 1024);
   const float isd = (float)(1.0 / std::sqrt((double)d));
+  if (g.mode == CONQUR_TC_BF16 && P > 1) {
+    // many small problems: the whole iteration of a problem runs inside one CTA
+    const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->first_endgame, c->reenter_idx, g.ns_max_steps, d, 1,
+                              g.orth_tol, g.fro_tol};
+    return tcb_update(c->tc, c->stream, ncp, g.prior_rel, g.margin);
+  }
 
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
   CQ_LAUNCHED(c, K_OTHER);
@@ -271,6 +277,7 @@ int update_impl(conqur_ctx* c) {
 
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);
+  const NsControlParams ncp{sched, c->n_sched, c->first_endgame, c->reenter_idx, g.ns_max_steps, d, use_shift, g.orth_tol, g.fro_tol};
   for (int k = 0; k <= g.ns_max_steps; ++k) {
     const int cur = k & 1;
     float* X = cur ? Xb : Xa;
@@ -278,9 +285,7 @@ int update_impl(conqur_ctx* c) {
     c->tc.ns_k = k;
     int rc = launch_residual(c, X, cur);
     if (rc) return rc;
-    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, use_shift ? pd + parts : nullptr, parts, k, sched, c->n_sched,
-                                                c->first_endgame, c->reenter_idx, g.orth_tol, g.fro_tol, cur,
-                                                g.ns_max_steps, d, use_shift);
+    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, use_shift ? pd + parts : nullptr, parts, k, cur, ncp);
     CQ_LAUNCHED(c, K_OTHER);
     if (k == g.ns_max_steps) break;
     if (g.simt_ns) {
@@ -342,7 +347,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
-  g.simt_ns = (g.mode == CONQUR_EXACT_F32) || g.P > 1;
+  g.simt_ns = (g.mode == CONQUR_EXACT_F32);
   g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 0;   // 0: set from the schedule below
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
   g.prior_rel = cfg->prior_rel;

@@ -496,11 +496,58 @@ static __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __
 // The step is handed to the product kernels in shifted residual form (see ns_schedule.h): coef = (gamma + kappa,
 // beta1, beta2, kappa) where kappa = mean diagonal of beta1 E + beta2 E^2 is moved from the matrix that gets
 // rounded to bf16 into the scalar multiple of X.  use_shift == 0 (exact mode): tau = 1, kappa = 0.
+struct NsControlParams {
+  const SchedEntry* sched;
+  int n_sched, first_endgame, reenter_idx, max_steps, d, use_shift;
+  float tol, fro_tol;
+};
+
+// The decision itself (one thread): tmx = max|G - I|, tsq = ||G - I||_F^2, ttr = tr G of step k.
+__device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double tsq, double ttr, int k, int cur_buf,
+                                                  const NsControlParams& c) {
+  const float fro = (float)sqrt(tsq);
+  s->e_max = tmx;
+  s->e_fro = fro;
+  if (!(tmx == tmx) || !(fro == fro)) {
+    s->ns_done = NS_DONE_FAILED;
+  } else if (tmx <= c.tol && fro <= c.fro_tol) {
+    s->ns_done = NS_DONE_CONVERGED;
+    s->ns_final_buf = cur_buf;
+  } else if (k >= c.max_steps) {
+    s->ns_done = NS_DONE_FAILED;
+  } else {
+    int idx = s->ns_idx;
+    if (fro < 0.7f) {
+      const float lb = sqrtf(1.0f - fro);
+      for (int j = c.n_sched - 1; j >= c.first_endgame && j > idx; --j)
+        if (c.sched[j].l <= lb) { idx = j; break; }
+    }
+    if (idx >= c.n_sched) idx = c.reenter_idx;
+    const SchedEntry e = c.sched[idx];
+    const double a = e.a, b = e.b, cc = e.c;
+    const double tau = c.use_shift ? (double)s->tau : 1.0;
+    const double b1 = b + 2.0 * cc * tau;
+    double kappa = 0.0;
+    if (c.use_shift) {
+      // ||E_tau||_F^2 and tr E_tau from the statistics of G - I and tr G
+      const double dd = (double)c.d;
+      const double e2 = fmax(0.0, tsq + 2.0 * (1.0 - tau) * ttr + dd * (tau * tau - 1.0));
+      kappa = (cc * e2 + b1 * (ttr - dd * tau)) / dd;
+    }
+    s->coef[0] = (float)(a + b * tau + cc * tau * tau + kappa);
+    s->coef[1] = (float)b1;
+    s->coef[2] = (float)cc;
+    s->coef[3] = (float)kappa;
+    s->seg_x = e.seg_x;
+    if (k < 128) s->seg_log[k] = (unsigned char)e.seg_x;
+    s->ns_idx = idx + 1;
+    s->ns_steps_used = k + 1;
+  }
+}
+
 static __global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
                                   const double* __restrict__ part_sq, const double* __restrict__ part_tr,
-                                  int nparts, int k, const SchedEntry* __restrict__ sched, int n_sched,
-                                  int first_endgame, int reenter_idx, float tol, float fro_tol, int cur_buf,
-                                  int max_steps, int d, int use_shift) {
+                                  int nparts, int k, int cur_buf, const NsControlParams c) {
   const int p = blockIdx.x;
   DevState* s = st + p;
   if (s->ns_done) return;
@@ -516,46 +563,7 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
   const double tsq = block_sum_d<256>(sq, redd);
   const double ttr = block_sum_d<256>(tr, redd);
   const float tmx = block_max_f<256>(mx, redf);
-  if (threadIdx.x == 0) {
-    const float fro = (float)sqrt(tsq);
-    s->e_max = tmx;
-    s->e_fro = fro;
-    if (!(tmx == tmx) || !(fro == fro)) {
-      s->ns_done = NS_DONE_FAILED;
-    } else if (tmx <= tol && fro <= fro_tol) {
-      s->ns_done = NS_DONE_CONVERGED;
-      s->ns_final_buf = cur_buf;
-    } else if (k >= max_steps) {
-      s->ns_done = NS_DONE_FAILED;
-    } else {
-      int idx = s->ns_idx;
-      if (fro < 0.7f) {
-        const float lb = sqrtf(1.0f - fro);
-        for (int j = n_sched - 1; j >= first_endgame && j > idx; --j)
-          if (sched[j].l <= lb) { idx = j; break; }
-      }
-      if (idx >= n_sched) idx = reenter_idx;
-      const SchedEntry e = sched[idx];
-      const double a = e.a, b = e.b, c = e.c;
-      const double tau = use_shift ? (double)s->tau : 1.0;
-      const double b1 = b + 2.0 * c * tau;
-      double kappa = 0.0;
-      if (use_shift) {
-        // ||E_tau||_F^2 and tr E_tau from the statistics of G - I and tr G
-        const double dd = (double)d;
-        const double e2 = fmax(0.0, tsq + 2.0 * (1.0 - tau) * ttr + dd * (tau * tau - 1.0));
-        kappa = (c * e2 + b1 * (ttr - dd * tau)) / dd;
-      }
-      s->coef[0] = (float)(a + b * tau + c * tau * tau + kappa);
-      s->coef[1] = (float)b1;
-      s->coef[2] = (float)c;
-      s->coef[3] = (float)kappa;
-      s->seg_x = e.seg_x;
-      if (k < 128) s->seg_log[k] = (unsigned char)e.seg_x;
-      s->ns_idx = idx + 1;
-      s->ns_steps_used = k + 1;
-    }
-  }
+  if (threadIdx.x == 0) ns_control_decide(s, tmx, tsq, ttr, k, cur_buf, c);
 }
 
 // tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode).

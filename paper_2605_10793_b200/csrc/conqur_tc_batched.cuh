@@ -375,4 +375,324 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   return CONQUR_OK;
 }
 
+// ------------------------------------------------------------------ fused polar update of many 128 x 128 problems
+// One CTA runs the whole Newton-Schulz iteration of one problem at a time with everything on chip: the iterate as
+// a bf16 (hi, lo) pair in shared memory, G = X^T X and the products in TMEM, the scalar control in one thread.
+// Per step (phases are strictly sequential; 128 threads = 128 rows):
+//   G = X^T X (hi hi + hi lo + lo hi)      -> TMEM [0,128)
+//   statistics of G - I, control decision, E = G - tau I as bf16           -> shared memory
+//   E E                                     -> TMEM [128,256)
+//   B = beta2 E E + beta1 E - kappa I as bf16                              -> shared memory (over E)
+//   X B (hi, + lo while the schedule asks)  -> TMEM [0,128)
+//   X <- (gamma + kappa) X + X B, tau = ||X||_F^2 / d, split into (hi, lo) -> shared memory
+// Two CTAs fit one SM (96 KB of shared memory and 256 TMEM columns each), so one problem's element-wise phases
+// overlap the other's products.
+constexpr int TCBU_THREADS = 128;
+constexpr int TCBU_SMEM_BYTES = 3 * TCB_TILE_BYTES + 1024 + 1024;
+
+struct TcbUpdAux {
+  uint64_t mbar;
+  uint32_t tmem_base;
+  int abort_flag;
+  int done;
+  float tau, x0s, lam;
+  float coef[4];
+  int seg_x;
+  double red_d[4], red_t[4];
+  float red_f[4];
+};
+
+struct TcbUpdArgs {
+  int P;
+  float* M; float* R;          // P x 128 x 128 fp32
+  DevState* st;
+  NsControlParams ncp;
+  float prior_rel, margin;
+};
+
+__device__ __forceinline__ double tcbu_block_sum(double v, double* red, int warp, int lane) {
+  v = warp_sum_d(v);
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  const double t = red[0] + red[1] + red[2] + red[3];
+  __syncthreads();
+  return t;
+}
+
+__global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUpdArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sXh = smem;
+  uint8_t* sXl = smem + TCB_TILE_BYTES;
+  uint8_t* sEB = smem + 2 * TCB_TILE_BYTES;
+  TcbUpdAux* aux = reinterpret_cast<TcbUpdAux*>(smem + 3 * TCB_TILE_BYTES);
+  volatile int* abort_flag = &aux->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = threadIdx.x;                       // the row this thread owns everywhere
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&aux->mbar, 1);
+    aux->abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 0) { ptx::tmem_alloc(&aux->tmem_base, 256); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = aux->tmem_base;
+  const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);      // this warp's 32 TMEM lanes
+  const uint32_t aXh = ptx::smem_u32(sXh), aXl = ptx::smem_u32(sXl), aEB = ptx::smem_u32(sEB);
+  const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  const uint32_t idesc_mm = idesc_base | (1u << 15) | (1u << 16);       // both operands read "transposed" (MN-major)
+  const uint32_t idesc_km = idesc_base | (1u << 16);                    // A as stored (K-major), B MN-major
+  uint32_t mph = 0;
+  bool timed_out = false;
+  const float isd = rsqrtf((float)TCB_D);
+
+  // descriptor of k-step j (16 of the 128 contraction indices) of a 128 x 128 tile held as two swizzled 64-column chunks
+  auto desc_k = [](uint32_t base, int j) { return tc_smem_desc(base + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024); };   // contraction along columns
+  auto desc_mn = [](uint32_t base, int j) { return tc_smem_desc(base + j * 2048, 16384, 1024); };                        // contraction along rows
+  // all threads: make shared-memory writes visible to the tensor cores, then thread 0 issues `issue` and everyone waits
+  auto run_products = [&](auto issue) -> bool {
+    ptx::fence_proxy_async();
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      ptx::tc_fence_after();
+      issue();
+      ptx::umma_commit(&aux->mbar);
+    }
+    const bool okw = tc_wait(&aux->mbar, mph, abort_flag);
+    mph ^= 1u;
+    ptx::tc_fence_after();
+    return okw;
+  };
+
+  for (int p = blockIdx.x; p < g.P && !timed_out; p += gridDim.x) {
+    DevState* s = g.st + p;
+    const float* Mrow = g.M + ((long long)p * TCB_D + r) * TCB_D;
+    const float* Rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
+    // ---- scale: lam = prior_rel ||M||_F / sqrt(d), X_0 = (M + lam R) / (||M + lam R||_F (1 + margin))
+    double ssq = 0.0;
+    for (int c = 0; c < TCB_D; c += 4) {
+      const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
+      ssq += (double)m.x * m.x + (double)m.y * m.y + (double)m.z * m.z + (double)m.w * m.w;
+    }
+    double fro2 = tcbu_block_sum(ssq, aux->red_d, warp, lane);
+    const float lam = g.prior_rel * (float)sqrt(fro2) * isd;
+    if (g.prior_rel > 0.f) {
+      ssq = 0.0;
+      for (int c = 0; c < TCB_D; c += 4) {
+        const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
+        const float4 q = *reinterpret_cast<const float4*>(Rrow + c);
+        const float a = fmaf(lam, q.x, m.x), b = fmaf(lam, q.y, m.y), cc = fmaf(lam, q.z, m.z), d4 = fmaf(lam, q.w, m.w);
+        ssq += (double)a * a + (double)b * b + (double)cc * cc + (double)d4 * d4;
+      }
+      fro2 = tcbu_block_sum(ssq, aux->red_d, warp, lane);
+    }
+    if (threadIdx.x == 0) {
+      const float fro = (float)sqrt(fro2);
+      const bool ok = (fro > 0.f) && (fro <= 3.0e38f) && (s->N > 0);
+      s->lam = lam; s->scale = fro;
+      s->x0_scale = ok ? 1.0f / (fro * (1.0f + g.margin)) : 0.f;
+      s->ns_done = ok ? 0 : NS_DONE_FAILED;
+      s->ns_steps_used = 0; s->ns_final_buf = 0; s->ns_idx = 0; s->seg_x = 2;
+      s->tau = 1.0f / ((1.0f + g.margin) * (1.0f + g.margin) * (float)TCB_D);
+      aux->done = s->ns_done; aux->tau = s->tau; aux->x0s = s->x0_scale; aux->lam = lam;
+    }
+    __syncthreads();
+    if (!aux->done) {
+      const float x0s = aux->x0s;
+      for (int c16 = 0; c16 < 16; ++c16) {
+        uint32_t wh[4], wl[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int col = c16 * 8 + e * 2;
+          const float a = fmaf(lam, Rrow[col], Mrow[col]) * x0s, b = fmaf(lam, Rrow[col + 1], Mrow[col + 1]) * x0s;
+          const float ah = bf16_round(a), bh = bf16_round(b);
+          wh[e] = bf16_bits(ah) | (bf16_bits(bh) << 16);
+          wl[e] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+        }
+        *reinterpret_cast<uint4*>(sXh + tcb_piece(r, c16)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+        *reinterpret_cast<uint4*>(sXl + tcb_piece(r, c16)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+      }
+      for (int k = 0; k <= g.ncp.max_steps; ++k) {
+        // ---- G = X^T X
+        if (!run_products([&] {
+              const uint32_t aa[3] = {aXh, aXh, aXl}, bb[3] = {aXh, aXl, aXh};
+#pragma unroll
+              for (int seg = 0; seg < 3; ++seg)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                  ptx::umma_bf16(tmem_base, desc_mn(aa[seg], j), desc_mn(bb[seg], j), idesc_mm, (seg > 0 || j > 0) ? 1u : 0u);
+            })) { timed_out = true; break; }
+        // ---- statistics of G - I; E = G - tau I
+        const float tau = aux->tau;
+        float mx = 0.f, tr = 0.f;
+        double sq = 0.0;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
+          const int dcol = r - c * 32;
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float e1 = v[i];
+            if (i == dcol) { tr += v[i]; e1 -= 1.f; v[i] -= tau; }
+            mx = fmaxf(mx, fabsf(e1));
+            sq += (double)e1 * (double)e1;
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[i] = bf16_bits(v[2 * i]) | (bf16_bits(v[2 * i + 1]) << 16);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        }
+        {
+          const double wsq = warp_sum_d(sq), wtr = warp_sum_d((double)tr);
+          const float wmx = warp_max(mx);
+          if (lane == 0) { aux->red_d[warp] = wsq; aux->red_t[warp] = wtr; aux->red_f[warp] = wmx; }
+          __syncthreads();
+          if (threadIdx.x == 0) {
+            const double tsq = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
+            const double ttr = aux->red_t[0] + aux->red_t[1] + aux->red_t[2] + aux->red_t[3];
+            const float tmx = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
+            ns_control_decide(s, tmx, tsq, ttr, k, 0, g.ncp);
+            aux->done = s->ns_done;
+            aux->coef[0] = s->coef[0]; aux->coef[1] = s->coef[1]; aux->coef[2] = s->coef[2]; aux->coef[3] = s->coef[3];
+            aux->seg_x = s->seg_x;
+          }
+          __syncthreads();
+        }
+        if (aux->done) break;
+        const float cg = aux->coef[0], cb1 = aux->coef[1], cb2 = aux->coef[2], ck = aux->coef[3];
+        const int seg_x = aux->seg_x;
+        // ---- E E
+        if (!run_products([&] {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                ptx::umma_bf16(tmem_base + 128, desc_k(aEB, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
+            })) { timed_out = true; break; }
+        // ---- B = beta2 E E + beta1 E - kappa I (over E: the product that read it has finished)
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float gq[32], ee[32];
+          ptx::tmem_ld32(t_row + (uint32_t)(c * 32), gq);
+          ptx::tmem_ld32(t_row + 128u + (uint32_t)(c * 32), ee);
+          const int dcol = r - c * 32;
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float e = (i == dcol) ? gq[i] - tau : gq[i];
+            float b = fmaf(cb2, ee[i], cb1 * e);
+            if (i == dcol) b -= ck;
+            ee[i] = b;
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[i] = bf16_bits(ee[2 * i]) | (bf16_bits(ee[2 * i + 1]) << 16);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        }
+        // ---- X B
+        if (!run_products([&] {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXh, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
+              if (seg_x > 1) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXl, j), desc_mn(aEB, j), idesc_km, 1u);
+              }
+            })) { timed_out = true; break; }
+        // ---- X <- (gamma + kappa) X + X B; tau of the next step
+        double x2 = 0.0;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint32_t off = tcb_piece(r, c * 4 + q4);
+            const uint4 h4 = *reinterpret_cast<const uint4*>(sXh + off), l4 = *reinterpret_cast<const uint4*>(sXl + off);
+            const uint32_t hh[4] = {h4.x, h4.y, h4.z, h4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
+            uint32_t wh[4], wl[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float xa = __uint_as_float(hh[e] << 16) + __uint_as_float(ll[e] << 16);
+              const float xb = __uint_as_float(hh[e] & 0xffff0000u) + __uint_as_float(ll[e] & 0xffff0000u);
+              const float a = fmaf(cg, xa, v[q4 * 8 + 2 * e]), b = fmaf(cg, xb, v[q4 * 8 + 2 * e + 1]);
+              x2 += (double)a * a + (double)b * b;
+              const float ah = bf16_round(a), bh = bf16_round(b);
+              wh[e] = bf16_bits(ah) | (bf16_bits(bh) << 16);
+              wl[e] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+            }
+            *reinterpret_cast<uint4*>(sXh + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+            *reinterpret_cast<uint4*>(sXl + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+          }
+        }
+        const double tx2 = tcbu_block_sum(x2, aux->red_d, warp, lane);
+        if (threadIdx.x == 0) { s->tau = (float)(tx2 / (double)TCB_D); aux->tau = s->tau; }
+        __syncthreads();
+      }
+    }
+    if (timed_out) break;
+    // ---- commit: R <- X, M <- 0, sums <- 0; or keep everything and latch the failure
+    const bool converged = (aux->done == NS_DONE_CONVERGED);
+    if (converged) {
+      float* Ro = g.R + ((long long)p * TCB_D + r) * TCB_D;
+      float* Mo = g.M + ((long long)p * TCB_D + r) * TCB_D;
+      for (int c16 = 0; c16 < 16; ++c16) {
+        const uint32_t off = tcb_piece(r, c16);
+        const uint4 h4 = *reinterpret_cast<const uint4*>(sXh + off), l4 = *reinterpret_cast<const uint4*>(sXl + off);
+        const uint32_t hh[4] = {h4.x, h4.y, h4.z, h4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
+        float o[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          o[2 * e] = __uint_as_float(hh[e] << 16) + __uint_as_float(ll[e] << 16);
+          o[2 * e + 1] = __uint_as_float(hh[e] & 0xffff0000u) + __uint_as_float(ll[e] & 0xffff0000u);
+        }
+        *reinterpret_cast<float4*>(Ro + c16 * 8) = make_float4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<float4*>(Ro + c16 * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+        *reinterpret_cast<float4*>(Mo + c16 * 8) = make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(Mo + c16 * 8 + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    if (threadIdx.x == 0) {
+      if (converged) {
+        s->last_J = s->J; s->last_N = s->N; s->J = 0.0; s->N = 0; s->updates += 1;
+        s->last_orth = s->e_max; s->last_fro = s->e_fro;
+      } else {
+        atomicOr(&s->status_flags, STATUS_FLAG_NS_FAILED);
+      }
+    }
+    __syncthreads();                                // aux->done is rewritten by the next problem
+  }
+  if (timed_out && threadIdx.x == 0) {
+    atomicOr(&g.st[0].status_flags, STATUS_FLAG_TIMEOUT);
+    g.st[0].timeout_site = 40;
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 256);
+  }
+}
+
+inline int tcb_update(TcHost& h, cudaStream_t s, const NsControlParams& ncp, float prior_rel, float margin) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tcb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCBU_SMEM_BYTES) != cudaSuccess)
+      return CONQUR_ERR_CUDA;
+    attr_set = true;
+  }
+  TcbUpdArgs g{};
+  g.P = h.P; g.M = h.M; g.R = h.R; g.st = h.st; g.ncp = ncp; g.prior_rel = prior_rel; g.margin = margin;
+  const int grid = h.P < 2 * h.num_sms ? h.P : 2 * h.num_sms;
+  tcb_update_kernel<<<grid, TCBU_THREADS, TCBU_SMEM_BYTES, s>>>(g);
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_NS_RESID);
+  return tc_refresh_R(h, s, 0);
+}
+
 }  // namespace conqur
