@@ -11,7 +11,8 @@
 // operand of the second product.  Rows with a zero or non-finite norm are zeroed in shared memory before the
 // second product so that they cannot reach M.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue.  Every wait is bounded.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..9 = epilogue (two warps per TMEM lane quarter,
+// one per half of the 128 columns).  Every wait is bounded.
 #pragma once
 #include "conqur_tc.cuh"
 
@@ -20,6 +21,8 @@ namespace conqur {
 constexpr int TCB_D = 128;                       // problem size this kernel is built for
 constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = two 64-column swizzled chunks of 16 KB
 constexpr int TCB_XSTAGES = 3;
+constexpr int TCB_THREADS = 320;                 // 2 + 8 warps
+constexpr int TCB_EPI_THREADS = 256;
 constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + 1024 + 1024;
 
 struct TcbAux {
@@ -28,9 +31,9 @@ struct TcbAux {
   uint64_t yfull[2], yempty[2], cready[2], cfree[2];
   uint32_t tmem_base;
   int abort_flag;
-  double red_d[4];
-  int red_i[4];
-  int red_f[4];
+  double red_d[8];
+  int red_i[8];
+  int red_f[8];
 };
 
 struct TcbStepArgs {
@@ -54,7 +57,7 @@ __device__ __forceinline__ uint32_t tcb_piece(int r, int c16) {
   return (uint32_t)((c16 >> 3) * 16384 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TCB_THREADS, 1)
 tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR, const TcbStepArgs g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -68,11 +71,11 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
-    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, 128);
+    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, TCB_EPI_THREADS);
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
     for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], 128);
-      ptx::mbar_init(&aux->cready[b], 128); ptx::mbar_init(&aux->cfree[b], 1);
+      ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_THREADS);
+      ptx::mbar_init(&aux->cready[b], TCB_EPI_THREADS); ptx::mbar_init(&aux->cfree[b], 1);
     }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
@@ -164,7 +167,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   } else {
-    const int q = warp & 3;
+    const int q = warp & 3;                        // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;              // which 64 of the 128 columns this warp handles
+    const int ew = (warp - 2);                     // 0..7
     const int r = q * 32 + lane;                   // token inside the tile; later: row of M
     const float L = (float)g.levels;
     int it = 0, lp = 0;
@@ -176,7 +181,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int yb = it & 1, xs = it % TCB_XSTAGES;
         const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
-        // a1: row norm from the tile in shared memory
+        // a1: row norm from the tile in shared memory (both warps of a row form the full sum)
         uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
         float ss = 0.f;
 #pragma unroll
@@ -192,10 +197,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const bool valid = (t * 128 + r) < g.n;
         const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
         if (valid && !good) {
-          ++skipped;
-          if (!(ss == 0.f)) nonfinite = 1;
+          if (half == 0) { ++skipped; if (!(ss == 0.f)) nonfinite = 1; }
 #pragma unroll
-          for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, c)) = make_uint4(0, 0, 0, 0);
+          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, half * 8 + c)) = make_uint4(0, 0, 0, 0);
         }
         const float rn = good ? 1.0f / sqrtf(ss) : 0.f;
         const uint32_t rn_bits = bf16_bits(rn);
@@ -206,7 +210,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         uint8_t* crow = sC + yb * TCB_TILE_BYTES;
         float inv = 0.f, delta = 0.f;
         if (g.levels > 0) {
-          float mx = 0.f;
+          float mx = 0.f;                          // the per-token scale needs the whole row
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             float v[32];
@@ -220,7 +224,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
         float acc_t = 0.f;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
           uint32_t w[16];
@@ -255,7 +260,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const uint32_t t_addr = tmem_base + 256u + ((uint32_t)(q * 32) << 16);
         float* dst = g.M + ((long long)p * TCB_D + r) * TCB_D;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
           float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
@@ -269,20 +275,22 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&aux->mempty);
-      // per-problem reductions in a fixed order (named barrier 1: the four epilogue warps only)
+      // per-problem reductions in a fixed order (named barrier 1: the eight epilogue warps only)
       const double wsum = warp_sum_d(acc);
       int wsk = skipped, wnf = nonfinite;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
-      if (lane == 0) { aux->red_d[q] = wsum; aux->red_i[q] = wsk; aux->red_f[q] = wnf; }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (q == 0 && lane == 0) {
-        g.part_d[p] = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
-        const int sk = aux->red_i[0] + aux->red_i[1] + aux->red_i[2] + aux->red_i[3];
+      if (lane == 0) { aux->red_d[ew] = wsum; aux->red_i[ew] = wsk; aux->red_f[ew] = wnf; }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (ew == 0 && lane == 0) {
+        double tot = 0.0;
+        int sk = 0, nf = 0;
+        for (int i = 0; i < 8; ++i) { tot += aux->red_d[i]; sk += aux->red_i[i]; nf |= aux->red_f[i]; }
+        g.part_d[p] = tot;
         if (sk) g.st[p].step_skipped += sk;                      // this CTA is the only writer of problem p's state
-        if (aux->red_f[0] | aux->red_f[1] | aux->red_f[2] | aux->red_f[3]) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
+        if (nf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
     }
   }
 
@@ -365,7 +373,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
-  tcb_step_kernel<<<grid, TC_THREADS, TCB_SMEM_BYTES, s>>>(tmX, h.tmRb_mn, g);
+  tcb_step_kernel<<<grid, TCB_THREADS, TCB_SMEM_BYTES, s>>>(tmX, h.tmRb_mn, g);
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_ROTATE);
