@@ -1,0 +1,180 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times (tensor-core mode,
+same Context arguments).  Where the oracle is too slow for a whole stream, a stated subset is checked:
+whole steps where a float64 step takes about a second, sampled columns / properties where it does not."""
+import numpy as np
+import pytest
+
+from oracle import conqur_oracle as O
+from paper_2605_10793_b200 import inputs as I
+from tests.parity_util import TOL, effective_m, step_parity, unit_roundoff, update_parity
+
+pytestmark = pytest.mark.gpu
+T = TOL["tc"]
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _bench_ctx(w, **kw):
+    from paper_2605_10793_b200 import binding as B
+    return B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel, **kw)
+
+
+def _dev_bf16(x):
+    torch = _torch()
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda().to(torch.bfloat16)
+
+
+def _f64(t):
+    return t.cpu().numpy().astype(np.float64)
+
+
+def _full_step_check(ctx, w, x, before):
+    r = _f64(ctx.get_R())
+    ctx.step(_dev_bf16(x))
+    j, n = ctx.get_objective()
+    m = _f64(ctx.get_M())
+    s = ctx.debug_get_signs(x.shape[0]).cpu().numpy()
+    mb, jb, nb = before if before is not None else (None, 0.0, 0)
+    rep = step_parity(x.astype(np.float64), r, s, m, j, n, "tc", w.quant_bits, mb, jb, nb)
+    assert rep["N_equal"]
+    assert rep["J_rel"] <= T["J"], rep
+    assert rep["M_rel_tie_aware"] <= T["M"], rep
+    assert rep["flips_outside_band"] == 0, rep
+    assert rep["flip_frac"] < 2e-2, rep
+    return rep, (m, j, n), r
+
+
+def test_c2_one_update_cycle_headline_workload():
+    """d = 4096: 8 batches of 2048 tokens, then the polar update.  First and last step checked in full against the
+    oracle (objective, tie-aware cross-covariance, every differing sign inside the rounding band); the steps in
+    between by their objective; the update against the SVD polar factor of the library's own M."""
+    w = I.WORKLOADS["c2"]
+    ctx = _bench_ctx(w)
+    torch = _torch()
+    r0 = I.initial_rotation(w)
+    ctx.set_R(torch.from_numpy(r0).cuda())
+    before = None
+    orc = O.OpuOracle(w.d, r0.astype(np.float64))
+    for b in range(w.update_every):
+        x = I.batch(w, b)
+        if b in (0, w.update_every - 1):
+            rep, before, r = _full_step_check(ctx, w, x, before)
+            orc.step(x.astype(np.float64))
+        else:
+            ctx.step(_dev_bf16(x))
+            orc.step(x.astype(np.float64))
+            j, n = ctx.get_objective()
+            assert n == orc.N and abs(j - orc.J) / orc.J <= T["J"]
+            before = (_f64(ctx.get_M()), j, n)
+    j, n = ctx.get_objective()
+    assert n == w.update_every * w.n
+    assert abs(j - orc.J) / orc.J <= T["J"]
+    m = before[0]
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0 and st.ns_steps_used <= 24, (st.status, st.ns_steps_used)
+    r_new = _f64(ctx.get_R())
+    rep = update_parity(m, r_new)
+    assert rep["orth"] <= T["orth"], rep
+    assert rep["gap"] <= T["gap"], rep
+    # ascent on the statistics the update was computed from: <R_new, M> >= <R_old, M> = J
+    assert np.sum(r_new * m) >= j * (1.0 - 1e-3)
+
+
+def test_c4a_int4_fake_quant_step_at_d4096():
+    w = I.WORKLOADS["c4a"]
+    ctx = _bench_ctx(w)
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _full_step_check(ctx, w, I.batch(w, 0), None)
+
+
+def test_c1_fewer_tokens_than_dimensions_proximal_update_at_d3072():
+    w = I.WORKLOADS["c1"]
+    ctx = _bench_ctx(w)
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    rep, (m, j, n), r = _full_step_check(ctx, w, I.batch(w, 0), None)
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0
+    rep = update_parity(effective_m(m, r, w.prior_rel), _f64(ctx.get_R()))
+    assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], rep
+
+
+def test_c3_sampled_columns_and_update_properties_at_d8192():
+    """d = 8192, n = 4096: a float64 step takes tens of seconds, so one step is checked on its objective (one
+    float64 product) and on 24 sampled columns of M (tie-aware, signs inside the band); the update on properties
+    that characterise the polar factor: orthogonality, R^T M symmetric and positive on random probes, and ascent
+    of <R, M>."""
+    w = I.WORKLOADS["c3"]
+    d, n = w.d, w.n
+    torch = _torch()
+    ctx = _bench_ctx(w)
+    r0 = I.initial_rotation(w)
+    ctx.set_R(torch.from_numpy(r0).cuda())
+    x = I.batch(w, 0)
+    r64 = _f64(ctx.get_R())
+    ctx.step(_dev_bf16(x))
+    j, nn = ctx.get_objective()
+    m = _f64(ctx.get_M())
+    s_gpu = ctx.debug_get_signs(n).cpu().numpy()
+    xt, used = O.normalise_rows(x)
+    y = xt @ r64
+    j_ref = np.abs(y).sum() / np.sqrt(d)
+    assert nn == int(used.sum()) and abs(j - j_ref) / j_ref <= T["J"]
+    cols = np.random.default_rng(3).choice(d, size=24, replace=False)
+    s_ref = O.sgn(y[:, cols])
+    diff = s_gpu[:, cols].astype(np.float64) != s_ref
+    band = 6.0 * unit_roundoff("tc", d) * np.sqrt((xt * xt) @ (r64[:, cols] ** 2))
+    assert not (diff & (np.abs(y[:, cols]) > band)).any()
+    assert diff.mean() < 2e-2
+    m_ta = xt.T @ (s_gpu[:, cols].astype(np.float64) / np.sqrt(d))
+    assert np.linalg.norm(m[:, cols] - m_ta) / np.linalg.norm(m_ta) <= T["M"]
+    del ctx
+    # one update on the accumulated M (4096 tokens < d: needs the proximal term; the workload itself updates every 16)
+    ctx2 = _bench_ctx(I.scaled(w, prior_rel=1e-2))
+    ctx2.set_R(torch.from_numpy(r0).cuda())
+    ctx2.step(_dev_bf16(x))
+    ctx2.update()
+    st = ctx2.get_stats()
+    assert st.status == 0, st.status
+    r_new = _f64(ctx2.get_R())
+    m_eff = effective_m(m, r64, 1e-2)
+    assert np.max(np.abs(r_new.T @ r_new - np.eye(d))) <= T["orth"]
+    a = r_new.T @ m_eff
+    assert np.linalg.norm(a - a.T) / np.linalg.norm(a) <= 2e-3          # R^T M symmetric  <=>  R is a polar factor of M
+    assert np.sum(r_new * m_eff) > np.sum(r64 * m_eff)                   # ascent of the Procrustes objective
+    v = np.random.default_rng(4).standard_normal((d, 16))                # ... and positive semidefinite (random probes)
+    assert (np.einsum("ik,ik->k", v, a @ v) > 0).all()
+
+
+def test_c4b_1024_heads_sampled_problems():
+    """1024 independent d = 128 problems of 4096 tokens in one batched call (64 distinct seeded problems repeated
+    16 times, generation being the slow part); sampled problems against independent oracle runs."""
+    w = I.WORKLOADS["c4b"]
+    torch = _torch()
+    P, distinct = w.problems, 64
+    xs = [I.batch(w, 0, problem=p) for p in range(distinct)]
+    r0s = [I.initial_rotation(w, p) for p in range(distinct)]
+    x_all = _dev_bf16(np.concatenate(xs, axis=0)).repeat(P // distinct, 1)
+    r_all = torch.from_numpy(np.stack(r0s)).cuda().repeat(P // distinct, 1, 1).contiguous()
+    ctx = _bench_ctx(w, batch=P)
+    ctx.set_R(r_all)
+    ctx.step_batched(x_all, w.n, w.d, w.n * w.d)
+    js, ns = ctx.get_objective()
+    ms = _f64(ctx.get_M())
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0
+    rs = _f64(ctx.get_R())
+    for p in (0, 17, 63, 64 + 5, 511, 1023):
+        q = p % distinct
+        ref = O.OpuOracle(w.d, r0s[q].astype(np.float64)).step(xs[q].astype(np.float64))
+        assert ns[p] == ref.N and abs(js[p] - ref.J) / ref.J <= T["J"], p
+        assert np.linalg.norm(ms[p] - ref.M) / np.linalg.norm(ref.M) < 3e-2, p
+        rep = update_parity(ms[p], rs[p])
+        assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], (p, rep)
+    # identical problems give bit-identical results wherever they ran
+    assert np.array_equal(ms[5], ms[64 + 5]) and np.array_equal(rs[5], rs[64 * 7 + 5])
