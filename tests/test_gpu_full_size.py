@@ -144,7 +144,9 @@ def test_c3_sampled_columns_and_update_properties_at_d8192():
     m_eff = effective_m(m, r64, 1e-2)
     assert np.max(np.abs(r_new.T @ r_new - np.eye(d))) <= T["orth"]
     a = r_new.T @ m_eff
-    assert np.linalg.norm(a - a.T) / np.linalg.norm(a) <= 2e-3          # R^T M symmetric  <=>  R is a polar factor of M
+    # R^T M symmetric  <=>  R is a polar factor of M.  The asymmetry is first order in the rotation error w while the
+    # Procrustes gap is second order (gap ~ sum (s_i + s_j) w_ij^2 / (2 ||M||_*)): a gap of 1e-3 allows ~4e-2 here.
+    assert np.linalg.norm(a - a.T) / np.linalg.norm(a) <= 2e-2
     assert np.sum(r_new * m_eff) > np.sum(r64 * m_eff)                   # ascent of the Procrustes objective
     v = np.random.default_rng(4).standard_normal((d, 16))                # ... and positive semidefinite (random probes)
     assert (np.einsum("ik,ik->k", v, a @ v) > 0).all()
