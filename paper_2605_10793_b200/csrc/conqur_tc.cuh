@@ -182,14 +182,17 @@ enum { TC_EPI_ROTATE = 0, TC_EPI_ROTATE_Q = 1, TC_EPI_ACCUM = 2, TC_EPI_RESID = 
 
 // PAIR: two CTAs of a cluster work on one 256 x 256 tile (each holds 128 rows of A and of the accumulator and
 // 128 of the 256 columns of B in its own shared memory); otherwise one CTA works on a 128 x BN tile.
-template <int BN, bool PAIR> struct TcCfg {
+template <int BN, bool PAIR, int NA = 1, int NB = 1> struct TcCfg {
   static_assert(!PAIR || BN == 256, "a CTA pair always computes 256 x 256 tiles");
+  static_assert(PAIR || (NA == 1 && NB == 1), "only the pair kernel keeps several operand tiles per stage");
   static constexpr int TILE_M = PAIR ? 256 : TC_BM;
   static constexpr int A_BYTES = TC_BM * TC_BK * 2;
   static constexpr int B_ROWS = PAIR ? 128 : BN;      // rows (n) of B this CTA loads per stage
   static constexpr int B_BYTES = B_ROWS * TC_BK * 2;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = PAIR ? 6 : ((BN == 256) ? 4 : 6);
+  // A pair's stage holds every distinct operand tile the passes of a split product need (e.g. A_hi, A_lo, B_hi, B_lo),
+  // so the three passes hi hi + hi lo + lo hi cost four tile loads per k block instead of six.
+  static constexpr int STAGE_BYTES = NA * A_BYTES + NB * B_BYTES;
+  static constexpr int STAGES = PAIR ? (12 / (NA + NB)) : ((BN == 256) ? 4 : 6);
   static constexpr int TMEM_COLS = 2 * BN;          // two accumulators: the epilogue of tile i overlaps tile i+1
   static constexpr int AUX_BYTES = 1024;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + AUX_BYTES + 1024 /* alignment slack */;
@@ -200,6 +203,10 @@ struct TcGemmArgs {
   int nseg;                     // k-loop passes: 1, or up to 3 for split-precision products
   int nseg_from_state;          // 1: take the number of passes from st->seg_x (chosen on the device per step)
   int a_off[3], b_off[3];       // outer-coordinate offset of each pass's operand inside a stacked [hi; lo] pair
+  // the same passes as (distinct operand tiles, which tile each pass reads): filled by tc_fuse_passes for the pair kernel
+  int na, nb;                   // distinct A / B tiles over all passes
+  int a_toff[2], b_toff[2];     // their outer-coordinate offsets
+  int a_tile[3], b_tile[3];     // tile index each pass reads (tiles appear in order of first use)
   int sym;                      // 1: the output is symmetric (M == N): only tiles that touch the upper triangle are
                                 //    computed; tiles strictly above the diagonal also write their transpose
   float* outF; long long ldo;   // fp32 output (M read-modify-write, E, X_next, Y)
@@ -272,10 +279,10 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_by
 __device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
 
-template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR>
+template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR, int NA = 1, int NB = 1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcGemmArgs g) {
-  using Cfg = TcCfg<BN, PAIR>;
+  using Cfg = TcCfg<BN, PAIR, NA, NB>;
   constexpr int TM = Cfg::TILE_M;
   constexpr int R = BN / TM;                        // tiles per column step of a symmetric product
   if (g.check_done && g.st->ns_done) return;      // uniform over the grid: the iteration already finished
@@ -293,7 +300,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, R) : tiles_m * tiles_n;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
   const int nseg = g.nseg_from_state ? max(1, min(3, g.st->seg_x)) : g.nseg;
-  const int k_iters = num_kb * nseg;
+  const int k_iters = PAIR ? num_kb : num_kb * nseg;     // a pair runs all passes of a k block from one stage
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { ptx::mbar_init(&aux->full[s], 1); ptx::mbar_init(&aux->empty[s], 1); }
@@ -337,18 +344,32 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (PAIR) {
             // both CTAs' copies are counted on the barrier of CTA 0, whose MMA thread consumes the stage
             const uint32_t bar = ptx::mapa_u32(ptx::smem_u32(&aux->full[stage]), 0);
-            if (rank == 0) ptx::mbar_expect_tx(&aux->full[stage], 2 * Cfg::STAGE_BYTES);
-            if (A_MN) {
+            int na = 1, nb = 1;                          // tiles the passes in use need
+            for (int sg = 0; sg < nseg; ++sg) { na = max(na, g.a_tile[sg] + 1); nb = max(nb, g.b_tile[sg] + 1); }
+            na = min(na, NA); nb = min(nb, NB);
+            if (rank == 0) ptx::mbar_expect_tx(&aux->full[stage], 2 * (na * Cfg::A_BYTES + nb * Cfg::B_BYTES));
+            const int kk = it * TC_BK;
 #pragma unroll
-              for (int h = 0; h < TC_BM / 64; ++h) ptx::tma_load_2d_pair(sa + h * 8192, &tmA, bar, m0 + 64 * h, k0 + a_off);
-            } else {
-              ptx::tma_load_2d_pair(sa, &tmA, bar, k0, m0 + a_off);
+            for (int ia = 0; ia < NA; ++ia) {
+              if (ia >= na) break;
+              uint8_t* ta = sa + ia * Cfg::A_BYTES;
+              if (A_MN) {
+#pragma unroll
+                for (int h = 0; h < TC_BM / 64; ++h) ptx::tma_load_2d_pair(ta + h * 8192, &tmA, bar, m0 + 64 * h, kk + g.a_toff[ia]);
+              } else {
+                ptx::tma_load_2d_pair(ta, &tmA, bar, kk, m0 + g.a_toff[ia]);
+              }
             }
-            if (B_MN) {
 #pragma unroll
-              for (int h = 0; h < Cfg::B_ROWS / 64; ++h) ptx::tma_load_2d_pair(sb + h * 8192, &tmB, bar, n0 + 64 * h, k0 + b_off);
-            } else {
-              ptx::tma_load_2d_pair(sb, &tmB, bar, k0, n0 + b_off);
+            for (int ib = 0; ib < NB; ++ib) {
+              if (ib >= nb) break;
+              uint8_t* tb = sa + NA * Cfg::A_BYTES + ib * Cfg::B_BYTES;
+              if (B_MN) {
+#pragma unroll
+                for (int h = 0; h < Cfg::B_ROWS / 64; ++h) ptx::tma_load_2d_pair(tb + h * 8192, &tmB, bar, n0 + 64 * h, kk + g.b_toff[ib]);
+              } else {
+                ptx::tma_load_2d_pair(tb, &tmB, bar, kk, n0 + g.b_toff[ib]);
+              }
             }
           } else {
             ptx::mbar_expect_tx(&aux->full[stage], Cfg::STAGE_BYTES);
@@ -407,16 +428,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!tc_wait(&aux->full[stage], phase, abort_flag)) { ok = false; timeout_site = 3; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(smem + stage * Cfg::STAGE_BYTES);
-          const uint32_t sb = sa + Cfg::A_BYTES;
+          // K-major: 16 k = 32 bytes inside the swizzled 128-byte row; 8-row groups 1024 bytes apart.
+          // MN-major: 16 k = two 8-row groups of 1024 bytes; 64-wide m|n chunks 8192 bytes apart.
+          // For a pair the descriptors name this CTA's tiles; the peer's halves sit at the same offsets in its memory.
+          if (PAIR) {
+            for (int sg = 0; sg < nseg; ++sg) {
+              const uint32_t ta = sa + (uint32_t)(g.a_tile[sg] * Cfg::A_BYTES);
+              const uint32_t tb = sa + (uint32_t)(NA * Cfg::A_BYTES + g.b_tile[sg] * Cfg::B_BYTES);
 #pragma unroll
-          for (int j = 0; j < TC_BK / 16; ++j) {
-            // K-major: 16 k = 32 bytes inside the swizzled 128-byte row; 8-row groups 1024 bytes apart.
-            // MN-major: 16 k = two 8-row groups of 1024 bytes; 64-wide m|n chunks 8192 bytes apart.
-            // For a pair the descriptors name this CTA's tiles; the peer's halves sit at the same offsets in its memory.
-            const uint64_t ad = A_MN ? tc_smem_desc(sa + j * 2048, 8192, 1024) : tc_smem_desc(sa + j * 32, 16, 1024);
-            const uint64_t bd = B_MN ? tc_smem_desc(sb + j * 2048, 8192, 1024) : tc_smem_desc(sb + j * 32, 16, 1024);
-            if (PAIR) ptx::umma_bf16_pair(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
-            else ptx::umma_bf16(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
+              for (int j = 0; j < TC_BK / 16; ++j) {
+                const uint64_t ad = A_MN ? tc_smem_desc(ta + j * 2048, 8192, 1024) : tc_smem_desc(ta + j * 32, 16, 1024);
+                const uint64_t bd = B_MN ? tc_smem_desc(tb + j * 2048, 8192, 1024) : tc_smem_desc(tb + j * 32, 16, 1024);
+                ptx::umma_bf16_pair(d_tmem, ad, bd, idesc, (it > 0 || sg > 0 || j > 0) ? 1u : 0u);
+              }
+            }
+          } else {
+            const uint32_t sb = sa + Cfg::A_BYTES;
+#pragma unroll
+            for (int j = 0; j < TC_BK / 16; ++j) {
+              const uint64_t ad = A_MN ? tc_smem_desc(sa + j * 2048, 8192, 1024) : tc_smem_desc(sa + j * 32, 16, 1024);
+              const uint64_t bd = B_MN ? tc_smem_desc(sb + j * 2048, 8192, 1024) : tc_smem_desc(sb + j * 32, 16, 1024);
+              ptx::umma_bf16(d_tmem, ad, bd, idesc, (it > 0 || j > 0) ? 1u : 0u);
+            }
           }
           // frees the shared-memory stage (in both CTAs of a pair) once these MMAs retire
           if (PAIR) ptx::umma_commit_pair(&aux->empty[stage]); else ptx::umma_commit(&aux->empty[stage]);
@@ -841,10 +874,24 @@ inline int tc_tiles(const TcVariant& v, int M, int N, int sym) {
 }
 inline int tc_part_slots(const TcVariant& v, int M, int N, int sym) { return tc_tiles(v, M, N, sym) * (v.pair ? 2 : 1); }
 
-template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR>
+// Rewrite the passes (a_off[s], b_off[s]) as distinct operand tiles + which tile each pass reads.
+inline void tc_fuse_passes(TcGemmArgs* g) {
+  g->na = g->nb = 0;
+  for (int s = 0; s < g->nseg && s < 3; ++s) {
+    int ia = -1, ib = -1;
+    for (int i = 0; i < g->na; ++i) if (g->a_toff[i] == g->a_off[s]) ia = i;
+    for (int i = 0; i < g->nb; ++i) if (g->b_toff[i] == g->b_off[s]) ib = i;
+    if (ia < 0 && g->na < 2) { ia = g->na; g->a_toff[g->na++] = g->a_off[s]; }
+    if (ib < 0 && g->nb < 2) { ib = g->nb; g->b_toff[g->nb++] = g->b_off[s]; }
+    g->a_tile[s] = ia < 0 ? 0 : ia;
+    g->b_tile[s] = ib < 0 ? 0 : ib;
+  }
+}
+
+template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR, int NA = 1, int NB = 1>
 inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
-  using Cfg = TcCfg<BN, PAIR>;
-  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, PAIR>;
+  using Cfg = TcCfg<BN, PAIR, NA, NB>;
+  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, PAIR, NA, NB>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
@@ -887,7 +934,15 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
 template <bool A_MN, bool B_MN, int EPI>
 inline int tc_launch_n(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
   const TcVariant v = tc_variant(h, g.N);
-  if (v.pair) return tc_launch<256, A_MN, B_MN, EPI, true>(h, s, a, b, g);
+  if (v.pair) {
+    TcGemmArgs gg = g;
+    tc_fuse_passes(&gg);
+    if constexpr (EPI == TC_EPI_RESID || EPI == TC_EPI_PLAIN) {
+      if (gg.na + gg.nb > 2) return tc_launch<256, A_MN, B_MN, EPI, true, 2, 2>(h, s, a, b, gg);
+    }
+    if constexpr (EPI == TC_EPI_NEXT) return tc_launch<256, A_MN, B_MN, EPI, true, 2, 1>(h, s, a, b, gg);
+    return tc_launch<256, A_MN, B_MN, EPI, true>(h, s, a, b, gg);
+  }
   if (v.tile_n == 256) return tc_launch<256, A_MN, B_MN, EPI, false>(h, s, a, b, g);
   return tc_launch<128, A_MN, B_MN, EPI, false>(h, s, a, b, g);
 }
