@@ -173,7 +173,8 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
 // ------------------------------------------------------------------ kernel configuration
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                   // one 128-byte swizzle row of bf16
-constexpr int TC_THREADS = 192;             // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int TC_THREADS = 320;             // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-9: epilogue
+constexpr int TC_EPI_THREADS = 256;         // two warps per TMEM lane quarter, one per half of the tile's columns
 constexpr long long TC_WAIT_LIMIT = 4000000000ll;   // ~2 s of SM clocks
 constexpr int TC_BAND = 8;                  // row tiles per band of the tile order
 
@@ -248,9 +249,9 @@ struct TcAux {
   uint64_t tempty[2];
   uint32_t tmem_base;
   int abort_flag;
-  double red_d[4];
-  float red_f[4];
-  float red_t[4];
+  double red_d[8];
+  float red_f[8];
+  float red_t[8];
 };
 
 // Bounded wait.  Returns false when the wait was abandoned (timeout here, or another role aborted).
@@ -305,7 +306,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { ptx::mbar_init(&aux->full[s], 1); ptx::mbar_init(&aux->empty[s], 1); }
     // the accumulator is handed back by every epilogue thread (of both CTAs of a pair)
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->tfull[b], 1); ptx::mbar_init(&aux->tempty[b], PAIR ? 256 : 128); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->tfull[b], 1); ptx::mbar_init(&aux->tempty[b], PAIR ? 2 * TC_EPI_THREADS : TC_EPI_THREADS); }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -461,8 +462,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    // ---------------------------------------------------------------- epilogue (4 warps, 128 TMEM lanes)
+    // ---------------------------------------------------------------- epilogue (8 warps: 128 TMEM lanes x 2 column halves)
     const int q = warp & 3;                               // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;                     // which half of the tile's columns this warp handles
+    const int ew = warp - 2;                              // 0..7
     const int et = q * 32 + lane;                         // row inside the tile
     float c_gamma = 0.f, c_b1 = 0.f, c_b2 = 0.f, c_kappa = 0.f, c_tau = 1.f;
     if (EPI == TC_EPI_POLY || EPI == TC_EPI_NEXT) {
@@ -493,7 +496,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       float acc_abs = 0.f, acc_max = 0.f, acc_tr = 0.f;
       double acc_sq = 0.0;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
         float v[32];
         ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
         const int col0 = n0 + c * 32;
@@ -610,26 +613,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (row_ok && rn > 0.f) atomicMax(g.rowmax + row, __float_as_uint(acc_max));
       }
       if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_RESID || EPI == TC_EPI_NEXT) {
-        // per-tile partials, fixed reduction order; named barrier 1 synchronises the 4 epilogue warps only
+        // per-tile partials, fixed reduction order; named barrier 1 synchronises the 8 epilogue warps only
         double dsum = (EPI == TC_EPI_ROTATE) ? (double)(acc_abs * rn) : acc_sq;
         dsum = warp_sum_d(dsum);
         float fmx = warp_max(acc_max);
         float ftr = warp_sum(acc_tr);
-        if (lane == 0) { aux->red_d[q] = dsum; aux->red_f[q] = fmx; aux->red_t[q] = ftr; }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (q == 0 && lane == 0) {
-          const double tot = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
+        if (lane == 0) { aux->red_d[ew] = dsum; aux->red_f[ew] = fmx; aux->red_t[ew] = ftr; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (ew == 0 && lane == 0) {
+          double tot = 0.0, ttr = 0.0;
+          float tmx = 0.f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { tot += aux->red_d[i]; ttr += (double)aux->red_t[i]; tmx = fmaxf(tmx, aux->red_f[i]); }
           if (EPI == TC_EPI_NEXT) {
             g.part_t[slot] = tot;
           } else {
             g.part_d[slot] = mirror ? 2.0 * tot : tot;       // a mirrored tile stands for two
           }
           if (EPI == TC_EPI_RESID) {
-            g.part_f[slot] = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
-            g.part_t[slot] = (double)aux->red_t[0] + (double)aux->red_t[1] + (double)aux->red_t[2] + (double)aux->red_t[3];
+            g.part_f[slot] = tmx;
+            g.part_t[slot] = ttr;
           }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
       }
     }
   }
