@@ -263,13 +263,13 @@ int update_impl(conqur_ctx* c) {
 
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
   CQ_LAUNCHED(c, K_OTHER);
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau);
   CQ_LAUNCHED(c, K_OTHER);
   if (g.prior_rel > 0.f) {
     sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 1, pd);
     CQ_LAUNCHED(c, K_OTHER);
   }
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau);
   CQ_LAUNCHED(c, K_OTHER);
   ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
   CQ_LAUNCHED(c, K_OTHER);

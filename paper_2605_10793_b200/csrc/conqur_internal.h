@@ -35,8 +35,9 @@ struct DevState {
   float coef[4];            // gamma + kappa, beta1, beta2, kappa of the step in flight
   float tau;                // shift of the residual: E = X^T X - tau I (1 in exact mode)
   int ns_idx;               // next entry of the polynomial schedule
-  int seg_x;                // tensor-core mode: segments of the next-iterate product of the step in flight (1 or 2)
-  unsigned char seg_log[128];   // seg_x chosen at each step of the last update (launch accounting)
+  int seg_x;                // tensor-core mode: passes of the next-iterate product of the step in flight (1 or 2)
+  int seg_e;                // tensor-core mode: passes of the next residual product (1 while the iterate is tiny, else 3)
+  unsigned char seg_log[128];   // seg_x | seg_e << 4 of each step of the last update (launch accounting)
 };
 
 // One entry of the device copy of the polynomial schedule.
@@ -49,7 +50,7 @@ enum : int { K_ROWNORM = 0, K_ROTATE = 1, K_ACCUM = 2, K_NS_RESID = 3, K_NS_POLY
 // Host-side launch accounting.  Launch counts are always kept; when `enabled`, the contractions are bracketed by
 // CUDA events on the launching stream (events are created lazily and reused).
 struct Prof {
-  struct Rec { int cls; double flops; int ns_k; int nseg; cudaEvent_t e0, e1; };   // nseg 0: look it up in seg_log
+  struct Rec { int cls; double flops; int ns_k; int nseg; cudaEvent_t e0, e1; };   // nseg 0 / -1: seg_x / seg_e from seg_log
   bool enabled = false;
   long long launches[K_COUNT] = {0};
   long long total = 0;
@@ -75,7 +76,11 @@ struct Prof {
       float t = 0.f;
       if (cudaEventElapsedTime(&t, r.e0, r.e1) == cudaSuccess && ran) {
         int passes = r.nseg;
-        if (passes == 0) passes = (seg_log && r.ns_k >= 0 && r.ns_k < 128) ? seg_log[r.ns_k] : 1;
+        if (passes <= 0) {
+          const int lg = (seg_log && r.ns_k >= 0 && r.ns_k < 128) ? seg_log[r.ns_k] : 0x31;
+          passes = (passes == 0) ? (lg & 15) : (lg >> 4);
+          if (passes < 1) passes = 1;
+        }
         ms[r.cls] += t; flops[r.cls] += r.flops * passes; ++timed[r.cls];
       }
       pool.push_back(r.e0); pool.push_back(r.e1);

@@ -451,7 +451,7 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
 // phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
 // phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
 static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
-                                float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift) {
+                                float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift, float e1_tau) {
   const int p = blockIdx.x;
   __shared__ double red[8];
   double v = 0.0;
@@ -473,6 +473,7 @@ static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ 
       s->seg_x = 2;
       // ||X_0||_F = 1/(1+margin): mean sigma^2 of the first iterate (the tensor-core mode shifts by it)
       s->tau = use_shift ? 1.0f / ((1.0f + margin) * (1.0f + margin) * (float)d) : 1.0f;
+      s->seg_e = (use_shift && s->tau < e1_tau) ? 1 : 3;
     }
   }
 }
@@ -539,7 +540,7 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
     s->coef[2] = (float)cc;
     s->coef[3] = (float)kappa;
     s->seg_x = e.seg_x;
-    if (k < 128) s->seg_log[k] = (unsigned char)e.seg_x;
+    if (k < 128) s->seg_log[k] = (unsigned char)(e.seg_x | (s->seg_e << 4));   // seg_e: what this step's residual product used
     s->ns_idx = idx + 1;
     s->ns_steps_used = k + 1;
   }
@@ -567,14 +568,19 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
 }
 
 // tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode).
-static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ part_x2, int nparts, int d) {
+// While the iterate is tiny (tau below e1_tau) the lo part cannot matter to G = X^T X: dropping it changes G by
+// about 4.4e-3 sqrt(tau) sigma_max, so the next residual product runs one bf16 pass instead of three.
+static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ part_x2, int nparts, int d, float e1_tau) {
   DevState* s = st + blockIdx.x;
   if (s->ns_done) return;
   __shared__ double redd[8];
   double v = 0.0;
   for (int i = threadIdx.x; i < nparts; i += 256) v += part_x2[(int64_t)blockIdx.x * nparts + i];
   const double tot = block_sum_d<256>(v, redd);
-  if (threadIdx.x == 0) s->tau = (float)(tot / (double)d);
+  if (threadIdx.x == 0) {
+    s->tau = (float)(tot / (double)d);
+    s->seg_e = (s->tau < e1_tau) ? 1 : 3;
+  }
 }
 
 // Accept or reject the update.  On success: R <- X_final, M <- 0, sums <- 0.

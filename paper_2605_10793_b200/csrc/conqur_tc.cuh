@@ -202,7 +202,7 @@ template <int BN, bool PAIR, int NA = 1, int NB = 1> struct TcCfg {
 struct TcGemmArgs {
   int M, N, K;                  // output rows, cols; contraction length of one segment
   int nseg;                     // k-loop passes: 1, or up to 3 for split-precision products
-  int nseg_from_state;          // 1: take the number of passes from st->seg_x (chosen on the device per step)
+  int nseg_from_state;          // passes chosen on the device per step: 1 = st->seg_x, 2 = st->seg_e (else nseg)
   int a_off[3], b_off[3];       // outer-coordinate offset of each pass's operand inside a stacked [hi; lo] pair
   // the same passes as (distinct operand tiles, which tile each pass reads): filled by tc_fuse_passes for the pair kernel
   int na, nb;                   // distinct A / B tiles over all passes
@@ -300,7 +300,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_m = (g.M + TM - 1) / TM, tiles_n = (g.N + BN - 1) / BN;
   const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, R) : tiles_m * tiles_n;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
-  const int nseg = g.nseg_from_state ? max(1, min(3, g.st->seg_x)) : g.nseg;
+  const int nseg = g.nseg_from_state ? max(1, min(g.nseg, g.nseg_from_state == 2 ? g.st->seg_e : g.st->seg_x)) : g.nseg;
   const int k_iters = PAIR ? num_kb : num_kb * nseg;     // a pair runs all passes of a k block from one stage
 
   if (threadIdx.x == 0) {
@@ -780,6 +780,7 @@ struct TcLayout {
 struct TcHost {
   int d, P, quant_bits, num_sms;
   int pair_clusters;                         // CTA pairs that can be co-resident (0: single-CTA kernels only)
+  float e1_tau;                              // residual product runs one pass while mean sigma^2 of the iterate is below this
   int64_t n_max;
   char* ws;
   TcLayout L;
@@ -914,7 +915,7 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
   if (timed) {
     // flops the tensor cores execute: computed tiles only, one pass (scaled by the passes taken when folded)
     rec.cls = cls; rec.flops = 2.0 * (double)tiles * Cfg::TILE_M * BN * (double)g.K; rec.ns_k = h.ns_k;
-    rec.nseg = g.nseg_from_state ? 0 : g.nseg;
+    rec.nseg = g.nseg_from_state == 1 ? 0 : (g.nseg_from_state == 2 ? -1 : g.nseg);
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
@@ -987,6 +988,8 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
   }
   h->num_sms = prop.multiProcessorCount;
   h->pair_clusters = tc_query_pair_clusters();
+  h->e1_tau = 2e-3f;
+  if (const char* env = std::getenv("CONQUR_NS_E1_TAU")) h->e1_tau = (float)std::atof(env);   // tuning knob
   const uint64_t D = (uint64_t)d;
   int rc = 0;
   if (P > 1) {
@@ -1086,7 +1089,7 @@ inline int tc_ns_next_parts(const TcHost& h) { return tc_part_slots(tc_variant(h
 inline int tc_ns_residual(TcHost& h, cudaStream_t s, int buf) {
   const int d = h.d;
   TcGemmArgs g = tc_args(h, d, d, d);
-  g.nseg = 3; g.a_off[2] = d; g.b_off[1] = d; g.check_done = 1; g.sym = 1;
+  g.nseg = 3; g.nseg_from_state = 2; g.a_off[2] = d; g.b_off[1] = d; g.check_done = 1; g.sym = 1;
   g.outF = h.E; g.ldo = d;
   g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Eh); g.ldh = d;
   g.part_t = h.part_d + tc_ns_parts(h);
@@ -1112,7 +1115,7 @@ inline int tc_ns_poly_next(TcHost& h, cudaStream_t s, int cur) {
   x.part_t = h.part_d + tc_ns_parts(h);
   rc = tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
   if (rc) return rc;
-  ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d);
+  ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d, h.e1_tau);
   if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
