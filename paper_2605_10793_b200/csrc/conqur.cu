@@ -9,6 +9,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -111,6 +112,12 @@ struct conqur_ctx {
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
   Prof prof;
+  // The update enqueues the same ~150 launches every time (same buffers, same order; which of them do work is
+  // decided on the device), so after the first update it is captured once into a CUDA graph and replayed.
+  cudaStream_t cap_stream = nullptr;       // side stream used only to capture
+  cudaGraphExec_t upd_graph = nullptr;
+  int updates_enqueued = 0;
+  long long graph_launches[K_COUNT] = {0};
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   DevState* state() const { return at<DevState>(L.state); }
@@ -314,6 +321,46 @@ int update_impl(conqur_ctx* c) {
   return CONQUR_OK;
 }
 
+// Enqueue one update: directly the first time (kernel attributes get set), then through a captured graph.
+int update_enqueue(conqur_ctx* c) {
+  static const bool no_graph = [] { const char* e = std::getenv("CONQUR_NO_GRAPH"); return e && e[0] == '1'; }();
+  const bool eligible = !no_graph && c->cfg.mode == CONQUR_TC_BF16 && c->cfg.P == 1 && !c->prof.enabled;
+  if (!eligible || c->updates_enqueued++ == 0) return update_impl(c);
+  if (!c->upd_graph) {
+    if (!c->cap_stream && cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaGetLastError();
+      return update_impl(c);
+    }
+    long long before[K_COUNT];
+    for (int i = 0; i < K_COUNT; ++i) before[i] = c->prof.launches[i];
+    const long long total_before = c->prof.total;
+    if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      return update_impl(c);
+    }
+    cudaStream_t user = c->stream;
+    c->stream = c->cap_stream;
+    const int rc = update_impl(c);
+    c->stream = user;
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
+    for (int i = 0; i < K_COUNT; ++i) { c->graph_launches[i] = c->prof.launches[i] - before[i]; c->prof.launches[i] = before[i]; }
+    c->prof.total = total_before;
+    if (rc != CONQUR_OK || e != cudaSuccess || !graph ||
+        cudaGraphInstantiate(&c->upd_graph, graph, 0) != cudaSuccess) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      c->upd_graph = nullptr;
+      c->updates_enqueued = -(1 << 30);          // stay on direct launches
+      return update_impl(c);
+    }
+    cudaGraphDestroy(graph);
+  }
+  CQ_CUDA(cudaGraphLaunch(c->upd_graph, c->stream));
+  for (int i = 0; i < K_COUNT; ++i) { c->prof.launches[i] += c->graph_launches[i]; c->prof.total += c->graph_launches[i]; }
+  return CONQUR_OK;
+}
+
 }  // namespace
 
 // ================================================================== C ABI
@@ -396,6 +443,8 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
 extern "C" int conqur_destroy(conqur_ctx* ctx) {
   if (!ctx) return CONQUR_ERR_INVALID_ARG;
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->upd_graph) cudaGraphExecDestroy(ctx->upd_graph);
+  if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   delete ctx;
   return CONQUR_OK;
 }
@@ -456,7 +505,7 @@ extern "C" int conqur_update(conqur_ctx* c) {
   if (!c) return CONQUR_ERR_INVALID_ARG;
   if (c->tokens_since_update == 0) return CONQUR_ERR_EMPTY_UPDATE;
   if (c->tokens_since_update < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
-  const int rc = update_impl(c);
+  const int rc = update_enqueue(c);
   if (rc == CONQUR_OK) c->tokens_since_update = 0;
   return rc;
 }
