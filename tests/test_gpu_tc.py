@@ -164,3 +164,27 @@ def test_batched_heads_fused_kernel(layout, n, P, quant_bits, dtype):
         assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], (p, rep)
     j2, n2 = ctx.get_objective()
     assert not n2.any() and not ctx.get_M().any().item()
+
+
+def test_tensor_core_rerun_is_bit_identical():
+    """Same stream twice (steps + update, graph-replayed second update included): identical M, R and objective.
+    The accumulate epilogue adds with L2 reductions, but every element of M receives exactly one addition per launch."""
+    torch = _torch()
+    d, n = 512, 1024
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2)
+    xs = [_dev(I.batch(w, b), "bf16") for b in range(4)]
+    outs = []
+    for rep in range(2):
+        ctx = _ctx(d=d, n_max=n, in_dtype="bf16")
+        ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+        trace = []
+        for cyc in range(3):
+            for x in xs[:2] if cyc % 2 == 0 else xs[2:]:
+                ctx.step(x)
+            trace.append(ctx.get_M().clone())
+            ctx.update()
+            trace.append(ctx.get_R().clone())
+        st = ctx.get_stats()
+        assert st.status == 0 and st.updates == 3
+        outs.append((trace, st.last_J))
+    assert all(torch.equal(a, b) for a, b in zip(outs[0][0], outs[1][0])) and outs[0][1] == outs[1][1]
