@@ -217,11 +217,22 @@ int conqur_plan_schedule(double sigma_min_rel, int32_t ns_steps, double* abc_out
  * A_dev / B_dev: device bf16 row-major.  Orientation 0 (K-major): the matrix is [M|N rows][K cols];
  * orientation 1 (MN-major): it is [K rows][M|N cols].  split != 0: each operand is a stacked pair
  * [hi; lo] (twice the rows) and the product is hi*hi + hi*lo + lo*hi.  M, K multiples of 8, N of 32.
- * scratch_dev: >= 256 bytes of device memory.  Synchronises; returns CONQUR_ERR_TIMEOUT if a bounded
+ * scratch_dev: >= 512 bytes of device memory.  Synchronises; returns CONQUR_ERR_TIMEOUT if a bounded
  * device-side wait expired.
  */
 int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_dev, int32_t M, int32_t N, int32_t K,
                       int32_t a_mn_major, int32_t b_mn_major, int32_t split, void* scratch_dev, void* cuda_stream);
+
+/*
+ * Test hook for the bounded device-side waits (no counterpart in the paper).  Every wait of the tensor-core kernels
+ * (on a TMA completion, on the MMA pipeline, on a peer CTA) gives up after a cycle limit, latches
+ * CONQUR_ERR_TIMEOUT and lets the kernel end normally, so that a protocol error can never hang the GPU.  This call
+ * runs that mechanism on purpose: one thread waits, for at most limit_cycles SM clocks (1 .. 2e9), on a barrier
+ * that nothing arrives at.  Returns CONQUR_ERR_TIMEOUT when the wait gave up as designed (the expected result),
+ * CONQUR_OK if it did not.  scratch_dev: >= 512 bytes of device memory.  Synchronises the stream; the context
+ * of the process stays usable.
+ */
+int conqur_debug_wait_timeout(void* scratch_dev, int64_t limit_cycles, void* cuda_stream);
 
 /*
  * The corner objective of one batch without any device-memory allocation by anyone

@@ -23,7 +23,7 @@ EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
-    "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc",
+    "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
     "conqur_strerror",
 ]
 
@@ -107,6 +107,8 @@ def load() -> C.CDLL:
     lib.conqur_objective_noalloc.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, vp]
     lib.conqur_debug_gemm.restype = C.c_int
     lib.conqur_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.conqur_debug_wait_timeout.restype = C.c_int
+    lib.conqur_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.conqur_strerror.restype = C.c_char_p
     lib.conqur_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -216,11 +218,18 @@ def conqur_objective_noalloc(x_ptr: int, in_dtype: int, n: int, d: int, ld: int,
     return load().conqur_objective_noalloc(x_ptr, in_dtype, n, d, ld, r_ptr, j_out_ptr, n_out_ptr, stream_ptr)
 
 
+def conqur_debug_wait_timeout(limit_cycles: int) -> int:
+    """Run the bounded-wait probe (see include/conqur.h); returns the status code (-8 = the wait gave up as designed)."""
+    import torch
+    scratch = torch.zeros(512, dtype=torch.uint8, device="cuda")
+    return load().conqur_debug_wait_timeout(scratch.data_ptr(), int(limit_cycles), torch.cuda.current_stream().cuda_stream)
+
+
 def conqur_debug_gemm(a, b, m: int, n: int, k: int, a_mn: bool, b_mn: bool, split: bool = False):
     """D = A x B (see include/conqur.h) for torch bf16 CUDA tensors; returns an fp32 (m, n) tensor."""
     import torch
     out = torch.empty((m, n), dtype=torch.float32, device="cuda")
-    scratch = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    scratch = torch.zeros(512, dtype=torch.uint8, device="cuda")
     rc = load().conqur_debug_gemm(a.data_ptr(), b.data_ptr(), out.data_ptr(), m, n, k, int(a_mn), int(b_mn),
                                   int(split), scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
     if rc != 0:

@@ -648,6 +648,18 @@ extern "C" int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_
   return flags_to_status(h.status_flags);
 }
 
+extern "C" int conqur_debug_wait_timeout(void* scratch_dev, int64_t limit_cycles, void* cuda_stream) {
+  if (!scratch_dev || limit_cycles < 1 || limit_cycles > 2000000000ll) return CONQUR_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  CQ_CUDA(cudaMemsetAsync(scratch_dev, 0, sizeof(DevState), s));
+  tc_wait_probe_kernel<<<1, 32, 0, s>>>(static_cast<DevState*>(scratch_dev), (long long)limit_cycles);
+  CQ_CUDA(cudaGetLastError());
+  DevState h;
+  CQ_CUDA(cudaMemcpyAsync(&h, scratch_dev, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+  CQ_CUDA(cudaStreamSynchronize(s));
+  return flags_to_status(h.status_flags);
+}
+
 extern "C" const char* conqur_strerror(int s) {
   switch (s) {
     case CONQUR_OK: return "ok";

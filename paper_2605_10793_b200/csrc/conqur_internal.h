@@ -40,6 +40,8 @@ struct DevState {
   unsigned char seg_log[128];   // seg_x | seg_e << 4 of each step of the last update (launch accounting)
 };
 
+static_assert(sizeof(DevState) <= 512, "scratch buffers of the test hooks are documented as 512 bytes");
+
 // One entry of the device copy of the polynomial schedule.
 struct SchedEntry { float a, b, c, l; int lift, seg_x; };
 constexpr int NS_SCHED_MAX = 128;

@@ -255,14 +255,15 @@ struct TcAux {
 };
 
 // Bounded wait.  Returns false when the wait was abandoned (timeout here, or another role aborted).
-__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                        long long limit = TC_WAIT_LIMIT) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!ptx::mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > TC_WAIT_LIMIT) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         return false;
       }
@@ -279,6 +280,23 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_by
 
 __device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
+
+// Exercises the bounded wait on purpose: one thread waits on a barrier that nothing will ever arrive at, gives up after
+// `limit_cycles`, and latches TIMEOUT exactly as the product kernels do.  The kernel then ends normally.
+static __global__ void tc_wait_probe_kernel(DevState* st, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && !tc_wait(&bar, 0u, &abort_flag, limit_cycles)) {
+    atomicOr(&st->status_flags, STATUS_FLAG_TIMEOUT);
+    st->timeout_site = 99;
+  }
+}
 
 template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR, int NA = 1, int NB = 1>
 __global__ void __launch_bounds__(TC_THREADS, 1)

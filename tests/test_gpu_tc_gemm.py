@@ -59,3 +59,12 @@ def test_split_precision_three_products(a_mn, b_mn):
 def test_many_tiles_persistent_loop():
     # more tiles than SMs: every CTA walks several tiles through both accumulator buffers
     assert _run(128 * 40, 256 * 5, 192, False, True, False, seed=4) < 2e-5
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """A wait on a barrier nothing arrives at ends after its cycle limit with CONQUR_ERR_TIMEOUT; the kernel returns
+    normally and the device keeps working (a product right after it is still correct)."""
+    from paper_2605_10793_b200 import binding as B
+    assert B.conqur_debug_wait_timeout(2_000_000) == -8          # about 1 ms of SM clocks
+    assert "wait" in B.strerror(-8)
+    test_single_tile_k_major()
