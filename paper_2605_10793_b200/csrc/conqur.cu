@@ -305,8 +305,13 @@ int update_impl(conqur_ctx* c) {
       if (rc) return rc;
     }
   }
-  ns_commit_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(st, Xa, Xb, R, M, dd);
-  CQ_LAUNCHED(c, K_OTHER);
+  if (g.simt_ns) {
+    ns_commit_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(st, Xa, Xb, R, M, dd);
+    CQ_LAUNCHED(c, K_OTHER);
+  } else {
+    int rc = tc_ns_commit(c->tc, c->stream);
+    if (rc) return rc;
+  }
   if (g.mode == CONQUR_TC_BF16) { int rc = tc_refresh_R(c->tc, c->stream, /*only_if_converged=*/1); if (rc) return rc; }
   ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st);
   CQ_LAUNCHED(c, K_OTHER);

@@ -196,7 +196,8 @@ template <int BN, bool PAIR, int NA = 1, int NB = 1> struct TcCfg {
   static constexpr int STAGES = PAIR ? (12 / (NA + NB)) : ((BN == 256) ? 4 : 6);
   static constexpr int TMEM_COLS = 2 * BN;          // two accumulators: the epilogue of tile i overlaps tile i+1
   static constexpr int AUX_BYTES = 1024;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + AUX_BYTES + 1024 /* alignment slack */;
+  static constexpr int EPI_STAGE_BYTES = 8 * 4096;   // one 32 x 32 fp32 transposition buffer per epilogue warp
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + AUX_BYTES + EPI_STAGE_BYTES + 1024 /* alignment slack */;
 };
 
 struct TcGemmArgs {
@@ -212,7 +213,7 @@ struct TcGemmArgs {
                                 //    computed; tiles strictly above the diagonal also write their transpose
   float* outF; long long ldo;   // fp32 output (M read-modify-write, E, X_next, Y)
   __nv_bfloat16* outH; long long ldh; long long lo_elems;   // bf16 output hi part (+ lo part at +lo_elems)
-  const float* inF; long long ldi;                          // fp32 epilogue input (E or X)
+  const __nv_bfloat16* inH;                                 // bf16 pair epilogue input (the old iterate; same ld / lo_elems as outH)
   const float* rnorm;
   unsigned* rowmax;
   double* part_d; float* part_f;
@@ -280,6 +281,58 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_by
 
 __device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
+
+// Epilogue stores.  A thread holds 32 consecutive columns of ONE row (TMEM lane = row), so a direct 16-byte store
+// per thread touches 32 different lines per instruction and only half a sector of each.  The warp's 32 x 32 block
+// goes through a private, swizzled shared-memory buffer instead and leaves as full 128-byte (fp32) or 64-byte (bf16)
+// row segments.  All 32 lanes must call these; rows >= rows_ok are not written.
+__device__ __forceinline__ void tc_store_block_f32(uint8_t* stg, int lane, const float (&v)[32], float* out, long long ld,
+                                                   int rows_ok) {
+#pragma unroll
+  for (int p = 0; p < 8; ++p)
+    *reinterpret_cast<float4*>(stg + lane * 128 + ((p ^ (lane & 7)) << 4)) = make_float4(v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = i * 4 + (lane >> 3), c = lane & 7;
+    const float4 t = *reinterpret_cast<const float4*>(stg + r * 128 + ((c ^ (r & 7)) << 4));
+    if (r < rows_ok) __stcs(reinterpret_cast<float4*>(out + (long long)r * ld + c * 4), t);   // streaming: keep operand tiles in L2
+  }
+  __syncwarp();
+}
+// The same block added into `out` with vector reductions (fire-and-forget, performed at the L2).
+__device__ __forceinline__ void tc_red_block_f32(uint8_t* stg, int lane, const float (&v)[32], float* out, long long ld,
+                                                 int rows_ok) {
+#pragma unroll
+  for (int p = 0; p < 8; ++p)
+    *reinterpret_cast<float4*>(stg + lane * 128 + ((p ^ (lane & 7)) << 4)) = make_float4(v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = i * 4 + (lane >> 3), c = lane & 7;
+    const float4 t = *reinterpret_cast<const float4*>(stg + r * 128 + ((c ^ (r & 7)) << 4));
+    if (r < rows_ok)
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + (long long)r * ld + c * 4), "f"(t.x), "f"(t.y),
+                   "f"(t.z), "f"(t.w)
+                   : "memory");
+  }
+  __syncwarp();
+}
+// 32 rows x 32 bf16 (w[16] = the thread's row as packed pairs) -> 64-byte row segments.
+__device__ __forceinline__ void tc_store_block_bf16(uint8_t* stg, int lane, const uint32_t (&w)[16], __nv_bfloat16* out,
+                                                    long long ld, int rows_ok) {
+#pragma unroll
+  for (int p = 0; p < 4; ++p)
+    *reinterpret_cast<uint4*>(stg + lane * 64 + ((p ^ ((lane >> 1) & 3)) << 4)) = make_uint4(w[4 * p], w[4 * p + 1], w[4 * p + 2], w[4 * p + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), c = lane & 3;
+    const uint4 t = *reinterpret_cast<const uint4*>(stg + r * 64 + ((c ^ ((r >> 1) & 3)) << 4));
+    if (r < rows_ok) __stcs(reinterpret_cast<uint4*>(out + (long long)r * ld + c * 8), t);
+  }
+  __syncwarp();
+}
 
 // Exercises the bounded wait on purpose: one thread waits on a barrier that nothing will ever arrive at, gives up after
 // `limit_cycles`, and latches TIMEOUT exactly as the product kernels do.  The kernel then ends normally.
@@ -485,6 +538,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;                     // which half of the tile's columns this warp handles
     const int ew = warp - 2;                              // 0..7
     const int et = q * 32 + lane;                         // row inside the tile
+    uint8_t* stg = smem + Cfg::STAGES * Cfg::STAGE_BYTES + Cfg::AUX_BYTES + ew * 4096;   // this warp's transposition buffer
     float c_gamma = 0.f, c_b1 = 0.f, c_b2 = 0.f, c_kappa = 0.f, c_tau = 1.f;
     if (EPI == TC_EPI_POLY || EPI == TC_EPI_NEXT) {
       c_gamma = g.st->coef[0]; c_b1 = g.st->coef[1]; c_b2 = g.st->coef[2]; c_kappa = g.st->coef[3];
@@ -518,7 +572,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         float v[32];
         ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
         const int col0 = n0 + c * 32;
-        if (!row_ok || col0 >= g.N) continue;              // N is a multiple of 32 in every use
+        if (col0 >= g.N) continue;                         // N is a multiple of 32 in every use (uniform over the warp)
+        const int wrow0 = m0 + q * 32;                     // first row of this warp's 32 x 32 block
+        const int rows_ok = min(32, max(0, g.M - wrow0));  // rows of it inside the matrix
+        if (rows_ok == 0) continue;
+        if (!row_ok) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;         // rows past the end take part in the stores with nothing to say
+        }
         if (EPI == TC_EPI_ROTATE) {
           // C' = sgn(y) * rnorm as bf16 (sign bit or-ed in; exact zeros stay zero); objective partial sum |y|
           uint32_t w[16];
@@ -530,31 +591,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
             w[i] = lo | (hi << 16);
           }
-          uint4* dst = reinterpret_cast<uint4*>(g.outH + (long long)row * g.ldh + col0);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          tc_store_block_bf16(stg, lane, w, g.outH + (long long)wrow0 * g.ldh + col0, g.ldh, rows_ok);
         } else if (EPI == TC_EPI_ROTATE_Q) {
-          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-            acc_max = fmaxf(acc_max, fmaxf(fmaxf(fabsf(v[4 * i]), fabsf(v[4 * i + 1])),
-                                           fmaxf(fabsf(v[4 * i + 2]), fabsf(v[4 * i + 3]))));
-          }
+          for (int i = 0; i < 32; ++i) acc_max = fmaxf(acc_max, fabsf(v[i]));
+          tc_store_block_f32(stg, lane, v, g.outF + (long long)wrow0 * g.ldo + col0, g.ldo, rows_ok);
         } else if (EPI == TC_EPI_ACCUM) {
           // M += acc as fire-and-forget vector reductions performed at the L2: the epilogue never waits for M to
           // arrive.  Each element of M receives exactly one addition per launch, so the result does not depend on
           // any ordering inside the launch.
-          float* dst = g.outF + (long long)row * g.ldo + col0;
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * i), "f"(v[4 * i]), "f"(v[4 * i + 1]),
-                         "f"(v[4 * i + 2]), "f"(v[4 * i + 3])
-                         : "memory");
+          tc_red_block_f32(stg, lane, v, g.outF + (long long)wrow0 * g.ldo + col0, g.ldo, rows_ok);
         } else if (EPI == TC_EPI_PLAIN) {
-          float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          tc_store_block_f32(stg, lane, v, g.outF + (long long)wrow0 * g.ldo + col0, g.ldo, rows_ok);
         } else {
           // Newton-Schulz epilogues
           const int dcol = row - col0;                      // position of the diagonal inside this chunk, if any
@@ -568,16 +616,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               acc_sq += (double)e1 * (double)e1;
             }
           } else {
-            const float4* src = reinterpret_cast<const float4*>(g.inF + (long long)row * g.ldi + col0);
+            if (EPI == TC_EPI_POLY) {
+              // beta1 E from the bf16 copy of E this product streams as its operands: the difference to fp32 E is a
+              // symmetric relative perturbation of the size of B's own rounding to bf16
+              const uint4* se = reinterpret_cast<const uint4*>(g.inH + (long long)(row_ok ? row : wrow0) * g.ldh + col0);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float4 t = src[i];
-              if (EPI == TC_EPI_POLY) {
-                v[4 * i] = fmaf(c_b2, v[4 * i], c_b1 * t.x); v[4 * i + 1] = fmaf(c_b2, v[4 * i + 1], c_b1 * t.y);
-                v[4 * i + 2] = fmaf(c_b2, v[4 * i + 2], c_b1 * t.z); v[4 * i + 3] = fmaf(c_b2, v[4 * i + 3], c_b1 * t.w);
-              } else {
-                v[4 * i] = fmaf(c_gamma, t.x, v[4 * i]); v[4 * i + 1] = fmaf(c_gamma, t.y, v[4 * i + 1]);
-                v[4 * i + 2] = fmaf(c_gamma, t.z, v[4 * i + 2]); v[4 * i + 3] = fmaf(c_gamma, t.w, v[4 * i + 3]);
+              for (int i = 0; i < 4; ++i) {
+                const uint4 e4 = se[i];
+                const uint32_t ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  v[8 * i + 2 * e] = fmaf(c_b2, v[8 * i + 2 * e], c_b1 * __uint_as_float(ee[e] << 16));
+                  v[8 * i + 2 * e + 1] = fmaf(c_b2, v[8 * i + 2 * e + 1], c_b1 * __uint_as_float(ee[e] & 0xffff0000u));
+                }
+              }
+            } else {
+              // the old iterate is its bf16 pair hi + lo (the same tiles this product streams as operand A)
+              const long long at = (long long)(row_ok ? row : wrow0) * g.ldh + col0;
+              const uint4* sh = reinterpret_cast<const uint4*>(g.inH + at);
+              const uint4* sl = reinterpret_cast<const uint4*>(g.inH + g.lo_elems + at);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint4 h4 = sh[i], l4 = sl[i];
+                const uint32_t hh[4] = {h4.x, h4.y, h4.z, h4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float xa = __uint_as_float(hh[e] << 16) + __uint_as_float(ll[e] << 16);
+                  const float xb = __uint_as_float(hh[e] & 0xffff0000u) + __uint_as_float(ll[e] & 0xffff0000u);
+                  v[8 * i + 2 * e] = fmaf(c_gamma, xa, v[8 * i + 2 * e]);
+                  v[8 * i + 2 * e + 1] = fmaf(c_gamma, xb, v[8 * i + 2 * e + 1]);
+                }
               }
             }
             if (EPI == TC_EPI_POLY) {
@@ -589,11 +657,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int i = 0; i < 32; ++i) acc_sq += (double)v[i] * (double)v[i];
             }
           }
-          if (EPI != TC_EPI_POLY) {
-            float4* dst = reinterpret_cast<float4*>(g.outF + (long long)row * g.ldo + col0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          }
           uint32_t wh[16], wl[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -602,15 +665,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             wh[i] = bf16_bits(ah) | (bf16_bits(bh) << 16);
             if (EPI == TC_EPI_NEXT) wl[i] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
           }
-          uint4* dh = reinterpret_cast<uint4*>(g.outH + (long long)row * g.ldh + col0);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dh[i] = make_uint4(wh[4 * i], wh[4 * i + 1], wh[4 * i + 2], wh[4 * i + 3]);
-          if (EPI == TC_EPI_NEXT) {
-            uint4* dl = reinterpret_cast<uint4*>(g.outH + g.lo_elems + (long long)row * g.ldh + col0);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dl[i] = make_uint4(wl[4 * i], wl[4 * i + 1], wl[4 * i + 2], wl[4 * i + 3]);
-          }
-          if (EPI != TC_EPI_NEXT && mirror) {
+          tc_store_block_bf16(stg, lane, wh, g.outH + (long long)wrow0 * g.ldh + col0, g.ldh, rows_ok);
+          if (EPI == TC_EPI_NEXT)
+            tc_store_block_bf16(stg, lane, wl, g.outH + g.lo_elems + (long long)wrow0 * g.ldh + col0, g.ldh, rows_ok);
+          if (EPI != TC_EPI_NEXT && mirror && row_ok) {
             // transpose of the tile: lane t holds row (m0 + 32 q + t), so for a fixed column the 32 lanes write
             // 32 consecutive elements of one output row
             unsigned short* oh = reinterpret_cast<unsigned short*>(g.outH);
@@ -1108,7 +1166,6 @@ inline int tc_ns_residual(TcHost& h, cudaStream_t s, int buf) {
   const int d = h.d;
   TcGemmArgs g = tc_args(h, d, d, d);
   g.nseg = 3; g.nseg_from_state = 2; g.a_off[2] = d; g.b_off[1] = d; g.check_done = 1; g.sym = 1;
-  g.outF = h.E; g.ldo = d;
   g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Eh); g.ldh = d;
   g.part_t = h.part_d + tc_ns_parts(h);
   return tc_launch_n<true, true, TC_EPI_RESID>(h, s, h.tmXh_mn[buf], h.tmXh_mn[buf], g);
@@ -1121,19 +1178,40 @@ inline int tc_ns_poly_next(TcHost& h, cudaStream_t s, int cur) {
   const long long dd = (long long)d * d;
   TcGemmArgs g = tc_args(h, d, d, d);
   g.nseg = 1; g.check_done = 1; g.sym = 1;
-  g.inF = h.E; g.ldi = d;
+  g.inH = reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Eh);
   g.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Bh); g.ldh = d;
   int rc = tc_launch_n<false, true, TC_EPI_POLY>(h, s, h.tmEh_k, h.tmEh_mn, g);
   if (rc) return rc;
   TcGemmArgs x = tc_args(h, d, d, d);
   x.nseg = 2; x.nseg_from_state = 1; x.a_off[1] = d; x.check_done = 1;
-  x.inF = cur ? h.Xb : h.Xa; x.ldi = d;
-  x.outF = cur ? h.Xa : h.Xb; x.ldo = d;
+  x.inH = reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Xh[cur]);
   x.outH = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[1 - cur]); x.ldh = d; x.lo_elems = dd;
   x.part_t = h.part_d + tc_ns_parts(h);
   rc = tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
   if (rc) return rc;
   ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d, h.e1_tau);
+  if (h.prof) h.prof->count(K_OTHER);
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
+}
+
+// Accept the update in tensor-core mode: R <- hi + lo of the final iterate, M <- 0.
+static __global__ void tc_commit_kernel(DevState* st, const __nv_bfloat16* __restrict__ X0, const __nv_bfloat16* __restrict__ X1,
+                                        float* __restrict__ R, float* __restrict__ M, int64_t dd) {
+  if (st->ns_done != NS_DONE_CONVERGED) return;
+  const __nv_bfloat16* X = st->ns_final_buf ? X1 : X0;
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < dd; i += (int64_t)gridDim.x * blockDim.x * 2) {
+    const uint32_t hb = *reinterpret_cast<const uint32_t*>(X + i), lb = *reinterpret_cast<const uint32_t*>(X + dd + i);
+    float2 o;
+    o.x = __uint_as_float(hb << 16) + __uint_as_float(lb << 16);
+    o.y = __uint_as_float(hb & 0xffff0000u) + __uint_as_float(lb & 0xffff0000u);
+    *reinterpret_cast<float2*>(R + i) = o;
+    *reinterpret_cast<float2*>(M + i) = make_float2(0.f, 0.f);
+  }
+}
+inline int tc_ns_commit(TcHost& h, cudaStream_t s) {
+  const int64_t dd = (int64_t)h.d * h.d;
+  tc_commit_kernel<<<tc_ew_blocks(dd / 2), 256, 0, s>>>(h.st, reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Xh[0]),
+                                                       reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Xh[1]), h.R, h.M, dd);
   if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
