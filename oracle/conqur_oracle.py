@@ -16,6 +16,10 @@ What each function follows:
   corner_target       Eq. 2, z = sign(R x) / sqrt(d)
   fake_quant_sym      Appendix B, Q_sym(x) = Delta * round(x / Delta),
                       Delta = ||x||_inf / (2^(b-1) - 1)
+  fake_quant_zp       Appendix B, Q_zp(x) = Delta * (round(x / Delta + zeta) - zeta),
+                      Delta = (max x - min x) / (2^b - 1), zeta the integer zero-point
+                      that puts min x on the lower end of the grid; with the clipping
+                      ratio of Appendix C (0.9 for activations) applied to the range
   OpuOracle.step      Section 3.3 (cross-covariance Z^T X_tilde) accumulated
                       across tensors as Section 3.4 allows; objective in the
                       l1 form of Section 3.2
@@ -28,6 +32,11 @@ Readings where the paper is silent (kept identical in the CUDA library):
   * fake-quant: b bits, levels -(2^(b-1)-1)..(2^(b-1)-1), clip ratio 1,
     round-half-to-even; the quantised row feeds the target and the objective,
     the unquantised normalised row feeds the cross-covariance.
+  * zero-point fake-quant (quant_mode = "zp"): the range is [c min x, c max x] with
+    clipping ratio c (Appendix C; the paper does not say how the ratio enters: it
+    scales both ends, as in the evaluation code bases it follows), zeta =
+    -round(c min x / Delta), codes are clamped to 0..2^b-1 (only matters for c < 1),
+    round-half-to-even; a constant row (max = min) quantises to zero.
   * prior_rel = lam_rel > 0 makes the update polar(M + lam * R_prev) with
     lam = lam_rel * ||M||_F / sqrt(d) (a proximal Procrustes step, needed only
     when fewer tokens than dimensions were accumulated; not in the paper).
@@ -85,6 +94,25 @@ def fake_quant_sym(y, bits):
     return q * delta[..., None], q, delta
 
 
+def fake_quant_zp(y, bits, clip_ratio=1.0):
+    """Appendix B: per-row asymmetric (zero-point) uniform quantiser, range scaled by clip_ratio (Appendix C).
+
+    Returns (Q(y), codes minus zero-point k = q - zeta, step Delta per row).
+    """
+    y = np.asarray(y, dtype=np.float64)
+    levels = 2 ** bits - 1
+    lo = clip_ratio * np.min(y, axis=-1)
+    hi = clip_ratio * np.max(y, axis=-1)
+    delta = (hi - lo) / levels
+    ok = delta > 0.0
+    safe = np.where(ok, delta, 1.0)
+    zeta = -np.rint(lo / safe)                             # integer zero-point: round(lo/Delta + zeta) = 0
+    q = np.rint(y / safe[..., None]) + zeta[..., None]     # round(y/Delta + zeta), zeta integer
+    q = np.clip(q, 0.0, float(levels))
+    k = np.where(ok[..., None], q - zeta[..., None], 0.0)
+    return k * delta[..., None], k, delta
+
+
 def polar_svd(m):
     """Orthogonal polar factor of m via the SVD: m = U S V^T -> U V^T (Section 3.3)."""
     u, s, vt = np.linalg.svd(np.asarray(m, dtype=np.float64))
@@ -94,9 +122,11 @@ def polar_svd(m):
 class OpuOracle:
     """State machine R = OPU(R, X) with accumulate-then-update (Sections 3.3-3.4)."""
 
-    def __init__(self, d, r0=None, quant_bits=0, prior_rel=0.0):
+    def __init__(self, d, r0=None, quant_bits=0, prior_rel=0.0, quant_mode="sym", clip_ratio=1.0):
         self.d = int(d)
         self.quant_bits = int(quant_bits)
+        self.quant_mode = quant_mode
+        self.clip_ratio = float(clip_ratio)
         self.prior_rel = float(prior_rel)
         self.R = np.eye(self.d) if r0 is None else np.array(r0, dtype=np.float64)
         assert self.R.shape == (self.d, self.d)
@@ -124,8 +154,12 @@ class OpuOracle:
         if self.quant_bits == 0:
             s = sgn(y)                                   # Eq. 2
             a = np.abs(y)                                # |y| summed -> l1 objective
-        else:
+        elif self.quant_mode == "sym":
             qy, q, delta = fake_quant_sym(y, self.quant_bits)   # Appendix B
+            s = sgn(q)
+            a = np.abs(qy)
+        else:
+            qy, q, delta = fake_quant_zp(y, self.quant_bits, self.clip_ratio)   # Appendix B / C
             s = sgn(q)
             a = np.abs(qy)
         s[~used] = 0.0

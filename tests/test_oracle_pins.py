@@ -407,3 +407,66 @@ def test_reflections_are_allowed():
     m = np.diag([3.0, 2.0, -1.0])
     r, _ = O.polar_svd(m)
     assert np.isclose(np.linalg.det(r), -1.0) and np.allclose(r, np.diag([1.0, 1.0, -1.0]))
+
+
+# ---- zero-point quantiser (Appendix B, Q_zp; clipping ratio of Appendix C)
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_zero_point_quantiser_error_bounds_and_grid(bits):
+    rng = np.random.default_rng(40 + bits)
+    y = rng.standard_normal((50, 64)) * np.exp(rng.standard_normal((50, 1))) + 0.3 * rng.standard_normal((50, 1))
+    qy, k, delta = O.fake_quant_zp(y, bits)
+    levels = 2 ** bits - 1
+    assert np.allclose(delta, (y.max(axis=1) - y.min(axis=1)) / levels)
+    assert np.all(np.abs(qy - y) <= delta[:, None] / 2 + 1e-12)                    # rounding error <= Delta/2 per coordinate
+    assert np.all(np.sum((qy - y) ** 2, axis=1) <= y.shape[1] * delta ** 2 / 4 + 1e-12)   # the printed MSE bound
+    assert np.all(y.max(axis=1) - y.min(axis=1) <= 2 * np.abs(y).max(axis=1) + 1e-15)     # range <= 2 ||x||_inf
+    assert np.all(k.max(axis=1) - k.min(axis=1) == levels)                         # min and max sit on the two grid ends
+    assert np.all(k == np.rint(k))                                                 # integer codes
+
+
+def test_zero_point_quantiser_brute_force_and_clipping():
+    rng = np.random.default_rng(7)
+    y = rng.standard_normal((6, 17))
+    for clip in (1.0, 0.9):
+        qy, k, delta = O.fake_quant_zp(y, 4, clip)
+        for i in range(y.shape[0]):
+            lo, hi = clip * min(y[i]), clip * max(y[i])
+            dl = (hi - lo) / 15.0
+            z = -int(np.rint(lo / dl))
+            for j in range(y.shape[1]):
+                q = min(max(int(np.rint(y[i, j] / dl)) + z, 0), 15)
+                assert q - z == k[i, j] and abs(dl * (q - z) - qy[i, j]) < 1e-15
+    # with a clipping ratio the extremes saturate at the ends of the grid and lose more than Delta/2
+    qy, k, delta = O.fake_quant_zp(y, 4, 0.9)
+    imax = np.argmax(y, axis=1)
+    assert np.allclose(qy[np.arange(6), imax], 0.9 * y.max(axis=1), atol=delta.max())      # clamped to the top of the clipped range
+    assert np.all(y[np.arange(6), imax] - qy[np.arange(6), imax] > 0) and np.all(k.max(axis=1) - k.min(axis=1) == 15)
+    # a constant row quantises to zero; many bits reproduce the plain signs
+    assert not O.fake_quant_zp(np.full((1, 8), 0.3), 4)[0].any()
+    qy16, k16, _ = O.fake_quant_zp(y, 16)
+    assert np.array_equal(O.sgn(k16), O.sgn(y)) and np.allclose(qy16, y, atol=1e-4)
+
+
+def test_zero_point_mode_statistics_and_shift_sensitivity():
+    """OPU statistics in zero-point mode: brute force on a small case; and, unlike the symmetric quantiser, the
+    dead zone follows the signed range (max - min)/(2^b - 1), not ||y||_inf."""
+    d, n = 8, 30
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((n, d))
+    r = np.linalg.qr(rng.standard_normal((d, d)))[0]
+    orc = O.OpuOracle(d, r, quant_bits=4, quant_mode="zp", clip_ratio=0.9).step(x)
+    m = np.zeros((d, d)); j = 0.0
+    for i in range(n):
+        xt = x[i] / np.linalg.norm(x[i])
+        y = xt @ r
+        lo, hi = 0.9 * y.min(), 0.9 * y.max()
+        dl = (hi - lo) / 15.0
+        z = -np.rint(lo / dl)
+        k = np.clip(np.rint(y / dl) + z, 0, 15) - z
+        j += dl * np.abs(k).sum() / np.sqrt(d)
+        m += np.outer(xt, np.sign(k) / np.sqrt(d))
+    assert abs(orc.J - j) < 1e-12 and np.allclose(orc.M, m, atol=1e-14) and orc.N == n
+    # scale invariance of the codes: a positive row scale changes nothing
+    orc2 = O.OpuOracle(d, r, quant_bits=4, quant_mode="zp", clip_ratio=0.9).step(x * np.exp(rng.standard_normal((n, 1))))
+    assert abs(orc2.J - orc.J) < 1e-12 and np.allclose(orc2.M, orc.M, atol=1e-13)
