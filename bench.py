@@ -124,7 +124,8 @@ def cpu_oracle_sample(w, cycles: int = 1):
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count()])
     except Exception:
         threads = os.cpu_count()
-    orc = O.OpuOracle(w.d, I.initial_rotation(w).astype(np.float64), quant_bits=w.quant_bits, prior_rel=w.prior_rel)
+    orc = O.OpuOracle(w.d, I.initial_rotation(w).astype(np.float64), quant_bits=w.quant_bits, prior_rel=w.prior_rel,
+                      quant_mode=w.quant_mode, clip_ratio=w.clip_ratio)
     t_step = t_upd = 0.0
     for c in range(cycles):
         for b in range(w.update_every):
@@ -214,7 +215,8 @@ def main():
     resident_bytes = sum(t.numel() * 2 for t in dev)
     r0 = torch.from_numpy(I.initial_rotation(w)).cuda()
 
-    ctx = B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel)
+    ctx = B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel,
+                    quant_mode=w.quant_mode, clip_ratio=w.clip_ratio)
     ctx.set_R(r0)
 
     def cycle_resident(c):

@@ -51,6 +51,7 @@ typedef enum {
 
 enum { CONQUR_F32 = 0, CONQUR_BF16 = 1 };            /* storage type of X */
 enum { CONQUR_EXACT_F32 = 0, CONQUR_TC_BF16 = 1 };   /* arithmetic mode */
+enum { CONQUR_QUANT_SYMMETRIC = 0, CONQUR_QUANT_ZEROPOINT = 1 };   /* fake-quantiser applied when quant_bits > 0 */
 
 /*
  * mode CONQUR_EXACT_F32: fp32 CUDA-core contractions throughout (parity anchor).
@@ -77,6 +78,10 @@ typedef struct {
                                polynomial schedule; 0 = default 1e-7 */
   int64_t  n_max;           /* largest n of any step call (sizes the workspace) */
   int32_t  batch;           /* P >= 1 independent problems of size d */
+  int32_t  quant_mode;      /* CONQUR_QUANT_SYMMETRIC: Q_sym of Appendix B (delta = max|y| / (2^(b-1)-1));
+                               CONQUR_QUANT_ZEROPOINT: Q_zp of Appendix B (delta = c (max y - min y) / (2^b - 1), integer
+                               zero-point, codes clamped to 0..2^b-1), the quantiser the paper's evaluation uses */
+  float    clip_ratio;      /* c in (0, 1] for the zero-point quantiser (Appendix C uses 0.9 for activations); 0 = 1 */
 } conqur_config;
 
 typedef struct {

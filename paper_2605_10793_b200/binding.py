@@ -18,6 +18,7 @@ _lib = None
 
 CONQUR_F32, CONQUR_BF16 = 0, 1
 CONQUR_EXACT_F32, CONQUR_TC_BF16 = 0, 1
+CONQUR_QUANT_SYMMETRIC, CONQUR_QUANT_ZEROPOINT = 0, 1
 
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
@@ -33,6 +34,7 @@ class conqur_config(C.Structure):
         ("struct_size", C.c_uint32), ("in_dtype", C.c_int32), ("mode", C.c_int32), ("quant_bits", C.c_int32),
         ("ns_steps", C.c_int32), ("ns_max_steps", C.c_int32), ("orth_tol", C.c_float), ("prior_rel", C.c_float),
         ("ns_sigma_min_rel", C.c_float), ("n_max", C.c_int64), ("batch", C.c_int32),
+        ("quant_mode", C.c_int32), ("clip_ratio", C.c_float),
     ]
 
 
@@ -120,9 +122,10 @@ def strerror(status: int) -> str:
 
 
 def make_config(*, in_dtype=CONQUR_BF16, mode=CONQUR_TC_BF16, quant_bits=0, ns_steps=0, ns_max_steps=0,
-                orth_tol=0.0, prior_rel=0.0, ns_sigma_min_rel=0.0, n_max=1, batch=1) -> conqur_config:
+                orth_tol=0.0, prior_rel=0.0, ns_sigma_min_rel=0.0, n_max=1, batch=1, quant_mode=CONQUR_QUANT_SYMMETRIC,
+                clip_ratio=0.0) -> conqur_config:
     return conqur_config(C.sizeof(conqur_config), in_dtype, mode, quant_bits, ns_steps, ns_max_steps, orth_tol,
-                         prior_rel, ns_sigma_min_rel, n_max, batch)
+                         prior_rel, ns_sigma_min_rel, n_max, batch, quant_mode, clip_ratio)
 
 
 # ---- the C calls, one to one -------------------------------------------------------------------
@@ -243,7 +246,7 @@ class Context:
     """One calibration context on the current CUDA device / current torch stream."""
 
     def __init__(self, d: int, n_max: int, *, in_dtype="bf16", mode="tc", quant_bits=0, batch=1, prior_rel=0.0,
-                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None):
+                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None, quant_mode="sym", clip_ratio=0.0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("conqur needs a CUDA device (B200); there is no CPU path")
@@ -253,7 +256,9 @@ class Context:
         self.mode = {"exact": CONQUR_EXACT_F32, "tc": CONQUR_TC_BF16}[mode]
         self.cfg = make_config(in_dtype=self.in_dtype, mode=self.mode, quant_bits=quant_bits, ns_steps=ns_steps,
                                ns_max_steps=ns_max_steps, orth_tol=orth_tol, prior_rel=prior_rel,
-                               ns_sigma_min_rel=ns_sigma_min_rel, n_max=n_max, batch=batch)
+                               ns_sigma_min_rel=ns_sigma_min_rel, n_max=n_max, batch=batch,
+                               quant_mode={"sym": CONQUR_QUANT_SYMMETRIC, "zp": CONQUR_QUANT_ZEROPOINT}[quant_mode],
+                               clip_ratio=clip_ratio)
         nbytes = conqur_workspace_bytes(self.d, self.cfg)
         if nbytes == 0:
             raise ConqurError(-1, "conqur_workspace_bytes")

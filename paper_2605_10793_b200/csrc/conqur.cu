@@ -41,6 +41,7 @@ struct Layout {
 
 struct Cfg {
   int d, P, in_dtype, mode, quant_bits, ns_max_steps;
+  QuantSpec qs;
   int64_t n_max;
   float orth_tol, prior_rel, fro_tol, margin;
   bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode)
@@ -60,6 +61,8 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   if (c->in_dtype != CONQUR_F32 && c->in_dtype != CONQUR_BF16) return false;
   if (c->mode != CONQUR_EXACT_F32 && c->mode != CONQUR_TC_BF16) return false;
   if (c->quant_bits != 0 && (c->quant_bits < 2 || c->quant_bits > 8)) return false;
+  if (c->quant_mode != CONQUR_QUANT_SYMMETRIC && c->quant_mode != CONQUR_QUANT_ZEROPOINT) return false;
+  if (c->clip_ratio < 0.f || c->clip_ratio > 1.f) return false;
   if (c->prior_rel < 0.f || c->orth_tol < 0.f || c->ns_sigma_min_rel < 0.f || c->ns_steps < 0 || c->ns_max_steps < 0)
     return false;
   if (c->mode == CONQUR_TC_BF16 && !tc_supported_shape(d, c->batch)) return false;
@@ -72,7 +75,7 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   L->R = take(sizeof(float) * dd * P);
   L->M = take(sizeof(float) * dd * P);
   L->rnorm = take(sizeof(float) * n * P);
-  L->rowmax = take(sizeof(unsigned) * n * P);
+  L->rowmax = take(sizeof(unsigned) * 2 * n * P);   // per row: ordered max, then ordered min (quant modes)
   int64_t mp = std::max<int64_t>((int64_t)cdiv(n, 128) * cdiv(d, 128), (int64_t)cdiv(d, 128) * cdiv(d, 128));
   mp = std::max<int64_t>(mp, cdiv(n, 8));
   mp = std::max<int64_t>(mp, 2 * (int64_t)cdiv(d, 128) * cdiv(d, 128) + 64);   // two partial arrays per Newton-Schulz product
@@ -196,17 +199,18 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   int per_problem;
   if (g.quant_bits == 0) {
     rotate_target_exact_kernel<TIn, false><<<grid1, SG_THREADS, 0, c->stream>>>(
-        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, part);
+        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, nullptr, part);
     CQ_LAUNCHED(c, K_ROTATE);
     per_problem = grid1.x * grid1.y;
   } else {
     unsigned* rowmax = c->at<unsigned>(c->L.rowmax);
+    unsigned* rowmin = rowmax + g.n_max * P;
     CQ_CUDA(cudaMemsetAsync(rowmax, 0, sizeof(unsigned) * g.n_max * P, c->stream));
+    CQ_CUDA(cudaMemsetAsync(rowmin, 0xff, sizeof(unsigned) * g.n_max * P, c->stream));
     rotate_target_exact_kernel<TIn, true><<<grid1, SG_THREADS, 0, c->stream>>>(
-        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, part);
+        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, rowmin, part);
     CQ_LAUNCHED(c, K_ROTATE);
-    const int levels = (1 << (g.quant_bits - 1)) - 1;
-    quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, levels,
+    quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, rowmin, g.qs,
                                                                     part);
     CQ_LAUNCHED(c, K_OTHER);
     per_problem = cdiv(n, 8);
@@ -399,6 +403,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
+  g.qs = QuantSpec{cfg->quant_bits, cfg->quant_mode, cfg->clip_ratio > 0.f ? cfg->clip_ratio : 1.0f};
   g.simt_ns = (g.mode == CONQUR_EXACT_F32);
   g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 0;   // 0: set from the schedule below
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
@@ -435,7 +440,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
     int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
                      c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
                      c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
-                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), &c->prof);
+                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), g.qs, &c->prof);
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);

@@ -72,6 +72,40 @@ __device__ __forceinline__ void ld4_as_float(const __nv_bfloat16* p, float (&v)[
 
 __device__ __forceinline__ float sgnf(float v) { return (v > 0.f) ? 1.f : ((v < 0.f) ? -1.f : 0.f); }
 
+// Order-preserving map float -> unsigned, so that integer atomicMax / atomicMin give an exact, order-independent
+// row maximum / minimum of signed values.
+__device__ __forceinline__ unsigned f2ord(float f) {
+  const unsigned b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ord2f(unsigned u) { return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u); }
+
+// Per-token fake-quantiser (Appendix B), as a rule "k = clamp(rint(y * inv), klo, khi); Q(y) = delta * k":
+//   symmetric : delta = max|y| / (2^(b-1) - 1), k in [-(2^(b-1)-1), 2^(b-1)-1]
+//   zero-point: delta = c (max y - min y) / (2^b - 1), zeta = -rint(c min y / delta), k = q - zeta in [-zeta, 2^b - 1 - zeta]
+// (c = clipping ratio of Appendix C).  The same rule works on the un-normalised products (a positive row scale
+// changes neither k nor zeta); the caller multiplies delta by the row's 1/norm.
+struct QuantSpec { int bits, mode; float clip; };          // bits == 0: no fake-quantisation
+struct RowQuant { float inv, delta, klo, khi; };
+__device__ __forceinline__ RowQuant row_quant(const QuantSpec q, float vmax, float vmin, bool good) {
+  RowQuant r{0.f, 0.f, 0.f, 0.f};
+  if (q.mode == 0) {
+    const float L = (float)((1 << (q.bits - 1)) - 1);
+    const float mx = fmaxf(fabsf(vmax), fabsf(vmin));
+    if (good && mx > 0.f) { r.inv = L / mx; r.delta = mx / L; r.klo = -L; r.khi = L; }
+  } else {
+    const float L = (float)((1 << q.bits) - 1);
+    const float lo = q.clip * vmin, hi = q.clip * vmax;
+    const float range = hi - lo;
+    if (good && range > 0.f) {
+      r.inv = L / range; r.delta = range / L;
+      const float zeta = -rintf(lo * r.inv);
+      r.klo = -zeta; r.khi = L - zeta;
+    }
+  }
+  return r;
+}
+
 // ------------------------------------------------------------------ a1: row norms
 // One warp per row: rnorm_i = 1/||x_i||_2 in fp32.  Rows whose sum of squares is zero
 // or not finite get rnorm = 0 (they then contribute nothing anywhere) and are counted.
@@ -212,7 +246,8 @@ template <typename TIn, bool QUANT>
 __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
     const TIn* __restrict__ X, int64_t ld, int64_t x_pstride, const float* __restrict__ R, int n, int d,
     const float* __restrict__ rnorm, int64_t rnorm_pstride, float* __restrict__ Cp /* n x d */,
-    int64_t c_pstride, unsigned int* __restrict__ rowmax_bits, double* __restrict__ partials) {
+    int64_t c_pstride, unsigned int* __restrict__ rowmax_ord, unsigned int* __restrict__ rowmin_ord,
+    double* __restrict__ partials) {
   const int p = blockIdx.z;
   const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
   float acc[8][8];
@@ -226,7 +261,7 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
     const int row = m0 + sg_row(i);
     if (row >= n) continue;
     const float r = rn[row];
-    float rs = 0.f, rmax = 0.f;
+    float rs = 0.f, rmax = -3.0e38f, rmin = 3.0e38f;
 #pragma unroll
     for (int jh = 0; jh < 2; ++jh) {
       const int col = n0 + sg_col(jh * 4);
@@ -236,7 +271,7 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
         const float v = acc[i][jh * 4 + j];
         if (QUANT) {
           o[j] = v;
-          rmax = fmaxf(rmax, fabsf(v));
+          if (col + j < d) { rmax = fmaxf(rmax, v); rmin = fminf(rmin, v); }
         } else {
           o[j] = sgnf(v) * r;
           rs += fabsf(v);
@@ -252,7 +287,10 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
       }
     }
     if (QUANT) {
-      if (r > 0.f) atomicMax(rowmax_bits + (int64_t)p * rnorm_pstride + row, __float_as_uint(rmax));
+      if (r > 0.f) {
+        atomicMax(rowmax_ord + (int64_t)p * rnorm_pstride + row, f2ord(rmax));
+        atomicMin(rowmin_ord + (int64_t)p * rnorm_pstride + row, f2ord(rmin));
+      }
     } else {
       if (r > 0.f) asum += (double)(rs * r);
     }
@@ -265,13 +303,13 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
   }
 }
 
-// Quant mode, second pass (Appendix B, Q_sym per token).  One warp per row:
-// Delta_raw = rowmax/L, q = rint(acc / Delta_raw) clipped to +-L, C' = sgn(q) * rnorm,
-// objective partial = rnorm * Delta_raw * sum_j |q_j|.  Works in place: Y and C' share the buffer.
+// Quant mode, second pass (Appendix B, per token).  One warp per row: k = clamp(rint(acc * inv), klo, khi),
+// C' = sgn(k) * rnorm, objective partial = rnorm * delta * sum_j |k_j|.  Works in place: Y and C' share the buffer.
 static __global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
                                                            int64_t c_pstride, const float* __restrict__ rnorm,
                                                            int64_t rnorm_pstride,
-                                                           const unsigned int* __restrict__ rowmax_bits, int levels,
+                                                           const unsigned int* __restrict__ rowmax_ord,
+                                                           const unsigned int* __restrict__ rowmin_ord, QuantSpec qs,
                                                            double* __restrict__ partials /* per block */) {
   const int p = blockIdx.y;
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -279,21 +317,17 @@ static __global__ void __launch_bounds__(256) quant_target_kernel(float* __restr
   double contrib = 0.0;
   if (row < n) {
     const float r = rnorm[(int64_t)p * rnorm_pstride + row];
-    const float mx = __uint_as_float(rowmax_bits[(int64_t)p * rnorm_pstride + row]);
+    const RowQuant rq = row_quant(qs, ord2f(rowmax_ord[(int64_t)p * rnorm_pstride + row]),
+                                  ord2f(rowmin_ord[(int64_t)p * rnorm_pstride + row]), r > 0.f);
     float* y = YC + (int64_t)p * c_pstride + row * d;
-    const float L = (float)levels;
-    const bool live = (r > 0.f) && (mx > 0.f);
-    const float inv = live ? (L / mx) : 0.f;
-    float qs = 0.f;
+    float qsum = 0.f;
     for (int j = lane; j < d; j += 32) {
-      float q = rintf(y[j] * inv);
-      q = fminf(fmaxf(q, -L), L);
-      qs += fabsf(q);
-      const float c = live ? sgnf(q) * r : 0.f;
-      y[j] = c;
+      const float k = fminf(fmaxf(rintf(y[j] * rq.inv), rq.klo), rq.khi);
+      qsum += fabsf(k);
+      y[j] = (rq.inv > 0.f) ? sgnf(k) * r : 0.f;
     }
-    qs = warp_sum(qs);
-    if (live) contrib = (double)(r * (mx / L)) * (double)qs;
+    qsum = warp_sum(qsum);
+    contrib = (double)(r * rq.delta) * (double)qsum;
   }
   __shared__ double red[8];
   if (lane == 0) red[threadIdx.x >> 5] = contrib;

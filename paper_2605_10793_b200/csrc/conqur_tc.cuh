@@ -215,7 +215,7 @@ struct TcGemmArgs {
   __nv_bfloat16* outH; long long ldh; long long lo_elems;   // bf16 output hi part (+ lo part at +lo_elems)
   const __nv_bfloat16* inH;                                 // bf16 pair epilogue input (the old iterate; same ld / lo_elems as outH)
   const float* rnorm;
-  unsigned* rowmax;
+  unsigned* rowmax; unsigned* rowmin;   // per-row ordered max / min of the raw products (quant modes)
   double* part_d; float* part_f;
   double* part_t;               // per-tile trace (residual) or sum of squares (next iterate)
   DevState* st;
@@ -565,7 +565,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         rn = row_ok ? g.rnorm[row] : 0.f;
         rn_bits = bf16_bits(rn);
       }
-      float acc_abs = 0.f, acc_max = 0.f, acc_tr = 0.f;
+      float acc_abs = 0.f, acc_max = 0.f, acc_tr = 0.f, acc_vmax = -3.0e38f, acc_vmin = 3.0e38f;
       double acc_sq = 0.0;
 #pragma unroll 1
       for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
@@ -594,7 +594,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_store_block_bf16(stg, lane, w, g.outH + (long long)wrow0 * g.ldh + col0, g.ldh, rows_ok);
         } else if (EPI == TC_EPI_ROTATE_Q) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc_max = fmaxf(acc_max, fabsf(v[i]));
+          for (int i = 0; i < 32; ++i) { acc_vmax = fmaxf(acc_vmax, v[i]); acc_vmin = fminf(acc_vmin, v[i]); }
           tc_store_block_f32(stg, lane, v, g.outF + (long long)wrow0 * g.ldo + col0, g.ldo, rows_ok);
         } else if (EPI == TC_EPI_ACCUM) {
           // M += acc as fire-and-forget vector reductions performed at the L2: the epilogue never waits for M to
@@ -686,7 +686,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       else ptx::mbar_arrive(&aux->tempty[buf]);
 
       if (EPI == TC_EPI_ROTATE_Q) {
-        if (row_ok && rn > 0.f) atomicMax(g.rowmax + row, __float_as_uint(acc_max));
+        if (row_ok && rn > 0.f) { atomicMax(g.rowmax + row, f2ord(acc_vmax)); atomicMin(g.rowmin + row, f2ord(acc_vmin)); }
       }
       if (EPI == TC_EPI_ROTATE || EPI == TC_EPI_RESID || EPI == TC_EPI_NEXT) {
         // per-tile partials, fixed reduction order; named barrier 1 synchronises the 8 epilogue warps only
@@ -804,39 +804,37 @@ __global__ void split_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* 
 // Quant mode, second pass for the tensor-core mode: Y (fp32, row-major) -> C' (bf16, row-major) + objective partials.
 __global__ void __launch_bounds__(256) quant_target_bf16_kernel(const float* __restrict__ Y, int64_t n, int d,
                                                                 const float* __restrict__ rnorm,
-                                                                const unsigned int* __restrict__ rowmax_bits,
-                                                                int levels, double* __restrict__ partials,
+                                                                const unsigned int* __restrict__ rowmax_ord,
+                                                                const unsigned int* __restrict__ rowmin_ord,
+                                                                QuantSpec qs, double* __restrict__ partials,
                                                                 __nv_bfloat16* __restrict__ Cp) {
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   double contrib = 0.0;
   if (row < n) {
     const float r = rnorm[row];
-    const float mx = __uint_as_float(rowmax_bits[row]);
-    const float L = (float)levels;
-    const bool live = (r > 0.f) && (mx > 0.f);
-    const float inv = live ? (L / mx) : 0.f;
+    const RowQuant rq = row_quant(qs, ord2f(rowmax_ord[row]), ord2f(rowmin_ord[row]), r > 0.f);
+    const bool live = rq.inv > 0.f;
     const float* y = Y + row * (int64_t)d;
     __nv_bfloat16* c = Cp + row * (int64_t)d;
-    float qs = 0.f;
+    float qsum = 0.f;
     for (int j = lane * 4; j < d; j += 128) {
       const float4 t = *reinterpret_cast<const float4*>(y + j);
       const float in[4] = {t.x, t.y, t.z, t.w};
       uint32_t b[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float qv = rintf(in[e] * inv);
-        qv = fminf(fmaxf(qv, -L), L);
-        qs += fabsf(qv);
-        b[e] = bf16_bits(live ? sgnf(qv) * r : 0.f);
+        const float k = fminf(fmaxf(rintf(in[e] * rq.inv), rq.klo), rq.khi);
+        qsum += fabsf(k);
+        b[e] = bf16_bits(live ? sgnf(k) * r : 0.f);
       }
       uint2 o;
       o.x = b[0] | (b[1] << 16);
       o.y = b[2] | (b[3] << 16);
       *reinterpret_cast<uint2*>(c + j) = o;
     }
-    qs = warp_sum(qs);
-    if (live) contrib = (double)(r * (mx / L)) * (double)qs;
+    qsum = warp_sum(qsum);
+    contrib = (double)(r * rq.delta) * (double)qsum;
   }
   __shared__ double red[8];
   if (lane == 0) red[threadIdx.x >> 5] = contrib;
@@ -862,6 +860,7 @@ struct TcHost {
   TcLayout L;
   float *R, *M, *Xa, *Xb, *E, *B, *rnorm, *Y;
   unsigned* rowmax;
+  QuantSpec qs;
   DevState* st;
   double* part_d;
   float* part_f;
@@ -1050,10 +1049,10 @@ inline int tc_query_pair_clusters() {
 
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
                    float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
-                   float* part_f, float* Y, unsigned* rowmax, Prof* prof) {
+                   float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, Prof* prof) {
   h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
   h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
-  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->prof = prof; h->ns_k = -1;
+  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->qs = qs; h->prof = prof; h->ns_k = -1;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
   cudaDeviceProp prop;
@@ -1129,12 +1128,13 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
     if (rc) return rc;
     per_problem = tc_part_slots(tc_variant(h, d), (int)n, d, 0);
   } else {
+    unsigned* rowmin = h.rowmax + h.n_max;
     if (cudaMemsetAsync(h.rowmax, 0, sizeof(unsigned) * n, s) != cudaSuccess) return CONQUR_ERR_CUDA;
-    g.outF = h.Y; g.ldo = d; g.rowmax = h.rowmax;
+    if (cudaMemsetAsync(rowmin, 0xff, sizeof(unsigned) * n, s) != cudaSuccess) return CONQUR_ERR_CUDA;
+    g.outF = h.Y; g.ldo = d; g.rowmax = h.rowmax; g.rowmin = rowmin;
     rc = tc_launch_n<false, true, TC_EPI_ROTATE_Q>(h, s, tmXs_k, h.tmRb_mn, g);
     if (rc) return rc;
-    const int levels = (1 << (h.quant_bits - 1)) - 1;
-    quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, levels, h.part_d, Cp);
+    quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, rowmin, h.qs, h.part_d, Cp);
     if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
     if (h.prof) h.prof->count(K_OTHER);
     per_problem = rb;

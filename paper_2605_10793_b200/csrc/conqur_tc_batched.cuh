@@ -38,7 +38,7 @@ struct TcbAux {
 
 struct TcbStepArgs {
   int n, P;
-  int levels;                 // 0: corner target of the rotated row; > 0: symmetric fake-quantisation with this many levels first
+  QuantSpec qs;               // bits == 0: corner target of the rotated row; else per-token fake-quantisation first
   float* M;                   // P x 128 x 128 fp32 (without the 1/sqrt(d))
   double* part_d;             // P objective partials (sum |y| * rnorm, or the quantised equivalent)
   DevState* st;               // P
@@ -171,7 +171,6 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int half = (warp - 2) >> 2;              // which 64 of the 128 columns this warp handles
     const int ew = (warp - 2);                     // 0..7
     const int r = q * 32 + lane;                   // token inside the tile; later: row of M
-    const float L = (float)g.levels;
     int it = 0, lp = 0;
     bool ok = true;
     for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
@@ -208,20 +207,19 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ptx::tc_fence_after();
         const uint32_t t_addr = tmem_base + (uint32_t)(yb * 128) + ((uint32_t)(q * 32) << 16);
         uint8_t* crow = sC + yb * TCB_TILE_BYTES;
-        float inv = 0.f, delta = 0.f;
-        if (g.levels > 0) {
-          float mx = 0.f;                          // the per-token scale needs the whole row
+        RowQuant rq{0.f, 0.f, 0.f, 0.f};
+        if (g.qs.bits > 0) {
+          float vmax = -3.0e38f, vmin = 3.0e38f;   // the per-token scale needs the whole row
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             float v[32];
             ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(v[i]));
+            for (int i = 0; i < 32; ++i) { vmax = fmaxf(vmax, v[i]); vmin = fminf(vmin, v[i]); }
           }
-          const bool live = good && (mx > 0.f);
-          inv = live ? (L / mx) : 0.f;
-          delta = live ? (mx / L) : 0.f;
+          rq = row_quant(g.qs, vmax, vmin, good);
         }
+        const bool live = (g.qs.bits == 0) ? good : (rq.inv > 0.f);
         float acc_t = 0.f;
 #pragma unroll 1
         for (int cc = 0; cc < 2; ++cc) {
@@ -232,20 +230,20 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             float a = v[2 * i], b = v[2 * i + 1];
-            if (g.levels > 0) {
-              a = fminf(fmaxf(rintf(a * inv), -L), L);
-              b = fminf(fmaxf(rintf(b * inv), -L), L);
+            if (g.qs.bits > 0) {
+              a = fminf(fmaxf(rintf(a * rq.inv), rq.klo), rq.khi);
+              b = fminf(fmaxf(rintf(b * rq.inv), rq.klo), rq.khi);
             }
             acc_t += fabsf(a) + fabsf(b);
             const uint32_t lo = (a == 0.f) ? 0u : (rn_bits | ((__float_as_uint(a) >> 16) & 0x8000u));
             const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
-            w[i] = good ? (lo | (hi << 16)) : 0u;
+            w[i] = live ? (lo | (hi << 16)) : 0u;
           }
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             *reinterpret_cast<uint4*>(crow + tcb_piece(r, c * 4 + k)) = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
         }
-        if (good) acc += (g.levels > 0) ? (double)(rn * delta) * (double)acc_t : (double)(acc_t * rn);
+        if (live) acc += (g.qs.bits > 0) ? (double)(rn * rq.delta) * (double)acc_t : (double)(acc_t * rn);
         // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
         ptx::tc_fence_before();
         ptx::fence_proxy_async();
@@ -363,7 +361,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)h.P);
   if (rc) return rc;
   TcbStepArgs g{};
-  g.n = (int)n; g.P = h.P; g.levels = h.quant_bits ? (1 << (h.quant_bits - 1)) - 1 : 0;
+  g.n = (int)n; g.P = h.P; g.qs = h.qs;
   g.M = h.M; g.part_d = h.part_d; g.st = h.st;
   const int grid = h.P < h.num_sms ? h.P : h.num_sms;
   Prof::Rec rec{};

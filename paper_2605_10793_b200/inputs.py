@@ -74,6 +74,8 @@ class Workload:
     prior_rel: float = 0.0     # proximal weight for rank-deficient updates
     problems: int = 1          # independent problems (batched variant)
     same_batch: bool = False   # every step sees batch 0 (alternation on a fixed batch)
+    quant_mode: str = "sym"    # "sym": symmetric per-token quantiser; "zp": zero-point quantiser
+    clip_ratio: float = 1.0    # range clipping ratio of the zero-point quantiser
 
 
 WORKLOADS: Dict[str, Workload] = {
@@ -95,6 +97,9 @@ WORKLOADS: Dict[str, Workload] = {
     # c2 with per-token symmetric INT4 fake-quantisation of the rotated rows
     "c4a": Workload("c4a", 4, 4096, 2048, 128, 8, "bf16", "student_t3", 16, 100.0, 0.5, 4, 1000.0,
                     "hadamard", quant_bits=4),
+    # c2 with the quantiser the paper's evaluation uses: per-token zero-point INT4, clipping ratio 0.9
+    "c4a_zp": Workload("c4a_zp", 6, 4096, 2048, 128, 8, "bf16", "student_t3", 16, 100.0, 0.5, 4, 1000.0,
+                       "hadamard", quant_bits=4, quant_mode="zp", clip_ratio=0.9),
     # per-head problems: 1024 independent d=128 problems, one step + one update each
     "c4b": Workload("c4b", 5, 128, 4096, 1, 1, "bf16", "student_t3", 2, 100.0, 0.5, 1, 1000.0,
                     "hadamard", problems=1024),

@@ -29,16 +29,17 @@ def unit_roundoff(mode: str, d: int) -> float:
 
 def step_parity(x64: np.ndarray, r64: np.ndarray, s_gpu: np.ndarray, m_gpu: np.ndarray, j_gpu: float, n_gpu: int,
                 mode: str, quant_bits: int = 0, m_before: np.ndarray | None = None, j_before: float = 0.0,
-                n_before: int = 0) -> dict:
+                n_before: int = 0, quant_mode: str = "sym", clip_ratio: float = 1.0) -> dict:
     """Compare one library step against the oracle.  Returns a report dict (asserts nothing)."""
     d = x64.shape[1]
-    orc = O.OpuOracle(d, r64, quant_bits=quant_bits).step(x64)
+    qkw = dict(quant_bits=quant_bits, quant_mode=quant_mode, clip_ratio=clip_ratio)
+    orc = O.OpuOracle(d, r64, **qkw).step(x64)
     s_ref = orc.last_S
     y = orc.last_Y
     m_ref = orc.M + (0.0 if m_before is None else m_before)
     j_ref = orc.J + j_before
     # tie-aware M: the oracle's arithmetic with the library's sign decisions
-    ta = O.OpuOracle(d, r64, quant_bits=quant_bits).step(x64, signs_override=s_gpu.astype(np.float64))
+    ta = O.OpuOracle(d, r64, **qkw).step(x64, signs_override=s_gpu.astype(np.float64))
     m_ta = ta.M + (0.0 if m_before is None else m_before)
     diff = s_gpu.astype(np.float64) != s_ref
     flip_frac = float(diff.mean())
@@ -48,13 +49,21 @@ def step_parity(x64: np.ndarray, r64: np.ndarray, s_gpu: np.ndarray, m_gpu: np.n
     u = unit_roundoff(mode, d)
     if quant_bits == 0:
         dist = np.abs(y)
-    else:
+    elif quant_mode == "sym":
         levels = 2 ** (quant_bits - 1) - 1
         delta = np.max(np.abs(y), axis=1, keepdims=True) / levels
         # distance to the dead-zone edge |y| = Delta/2; Delta itself carries the band of the row maximum
         dist = np.abs(np.abs(y) - delta / 2)
         row_arg = np.argmax(np.abs(y), axis=1)
         scale = scale + 0.5 * scale[np.arange(y.shape[0]), row_arg][:, None] / levels
+    else:
+        levels = 2 ** quant_bits - 1
+        delta = clip_ratio * (np.max(y, axis=1, keepdims=True) - np.min(y, axis=1, keepdims=True)) / levels
+        # sgn(q - zeta) = sgn(rint(y / Delta)): the same dead zone |y| < Delta/2, Delta from the row's max and min
+        dist = np.abs(np.abs(y) - delta / 2)
+        rows = np.arange(y.shape[0])
+        ends = scale[rows, np.argmax(y, axis=1)] + scale[rows, np.argmin(y, axis=1)]
+        scale = scale + 0.5 * clip_ratio * ends[:, None] / levels
     band = 6.0 * u * scale
     outside = diff & (dist > band) & used[:, None]
     rep = {

@@ -227,3 +227,21 @@ def test_batched_problems_match_independent_oracles():
         assert np.linalg.norm(ms[p] - ref.M) / np.linalg.norm(ref.M) < 1e-5
         rep = update_parity(ms[p], rs[p])
         assert rep["orth"] <= 1e-4 and rep["gap"] <= T["gap"], rep
+
+
+@pytest.mark.parametrize("d,n,clip", [(128, 600, 0.9), (100, 257, 1.0)])
+def test_zero_point_quant_mode_int4(d, n, clip):
+    """Per-token zero-point fake-quantisation (Appendix B, clipping ratio of Appendix C) before the target."""
+    w = I.scaled(I.WORKLOADS["c4a_zp"], d=d, n=n, n_outlier=2, r0="hadamard" if d & (d - 1) == 0 else "qr")
+    x = I.batch(w, 0)
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", quant_bits=4, quant_mode="zp", clip_ratio=clip)
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    r = ctx.get_R().cpu().numpy().astype(np.float64)
+    ctx.step(_dev(x, "bf16"))
+    j, nn = ctx.get_objective()
+    m = ctx.get_M().cpu().numpy().astype(np.float64)
+    s = ctx.debug_get_signs(n).cpu().numpy()
+    rep = step_parity(x.astype(np.float64), r, s, m, j, nn, "exact", 4, quant_mode="zp", clip_ratio=clip)
+    assert rep["N_equal"] and rep["J_rel"] <= 1e-5, rep          # a tie in the zero-point moves a clamped code by one
+    assert rep["M_rel_tie_aware"] <= T["M"] and rep["flips_outside_band"] == 0 and rep["flip_frac"] < 1e-3, rep
+    _check_update(ctx, m, r)

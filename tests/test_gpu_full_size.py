@@ -19,7 +19,8 @@ def _torch():
 
 def _bench_ctx(w, **kw):
     from paper_2605_10793_b200 import binding as B
-    return B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel, **kw)
+    return B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel,
+                     quant_mode=w.quant_mode, clip_ratio=w.clip_ratio, **kw)
 
 
 def _dev_bf16(x):
@@ -38,7 +39,7 @@ def _full_step_check(ctx, w, x, before):
     m = _f64(ctx.get_M())
     s = ctx.debug_get_signs(x.shape[0]).cpu().numpy()
     mb, jb, nb = before if before is not None else (None, 0.0, 0)
-    rep = step_parity(x.astype(np.float64), r, s, m, j, n, "tc", w.quant_bits, mb, jb, nb)
+    rep = step_parity(x.astype(np.float64), r, s, m, j, n, "tc", w.quant_bits, mb, jb, nb, w.quant_mode, w.clip_ratio)
     assert rep["N_equal"]
     assert rep["J_rel"] <= T["J"], rep
     assert rep["M_rel_tie_aware"] <= T["M"], rep
@@ -86,6 +87,14 @@ def test_c2_one_update_cycle_headline_workload():
 
 def test_c4a_int4_fake_quant_step_at_d4096():
     w = I.WORKLOADS["c4a"]
+    ctx = _bench_ctx(w)
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _full_step_check(ctx, w, I.batch(w, 0), None)
+
+
+def test_c4a_zero_point_int4_clip09_step_at_d4096():
+    """The quantiser the paper's evaluation uses (zero-point, clipping ratio 0.9) at the headline size."""
+    w = I.WORKLOADS["c4a_zp"]
     ctx = _bench_ctx(w)
     ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
     _full_step_check(ctx, w, I.batch(w, 0), None)

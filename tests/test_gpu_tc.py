@@ -188,3 +188,35 @@ def test_tensor_core_rerun_is_bit_identical():
         assert st.status == 0 and st.updates == 3
         outs.append((trace, st.last_J))
     assert all(torch.equal(a, b) for a, b in zip(outs[0][0], outs[1][0])) and outs[0][1] == outs[1][1]
+
+
+def test_zero_point_quant_mode_tc_and_batched():
+    """Zero-point INT4 with clipping ratio 0.9 in tensor-core mode: one large problem and the fused per-head kernel."""
+    d, n = 256, 1024
+    w = I.scaled(I.WORKLOADS["c4a_zp"], d=d, n=n, n_outlier=2)
+    x = I.batch(w, 0)
+    ctx = _ctx(d=d, n_max=n, in_dtype="bf16", quant_bits=4, quant_mode="zp", clip_ratio=0.9)
+    ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+    r = ctx.get_R().cpu().numpy().astype(np.float64)
+    ctx.step(_dev(x, "bf16"))
+    j, nn = ctx.get_objective()
+    m = ctx.get_M().cpu().numpy().astype(np.float64)
+    s = ctx.debug_get_signs(n).cpu().numpy()
+    rep = step_parity(x.astype(np.float64), r, s, m, j, nn, "tc", 4, quant_mode="zp", clip_ratio=0.9)
+    assert rep["N_equal"] and rep["J_rel"] <= T["J"], rep
+    assert rep["M_rel_tie_aware"] <= T["M"] and rep["flips_outside_band"] == 0 and rep["flip_frac"] < 2e-2, rep
+    _check_update(ctx, m, r)
+    # per-head problems
+    P, n2 = 4, 300
+    wb = I.scaled(I.WORKLOADS["c4b"], n=n2, problems=P)
+    xs = [I.batch(wb, 0, problem=p) for p in range(P)]
+    r0 = np.stack([I.initial_rotation(wb, p) for p in range(P)])
+    cb = _ctx(d=128, n_max=n2, in_dtype="bf16", batch=P, quant_bits=4, quant_mode="zp", clip_ratio=0.9)
+    cb.set_R(_dev(r0, "f32"))
+    cb.step_batched(_dev(np.concatenate(xs, axis=0), "bf16"), n2, 128, n2 * 128)
+    js, ns = cb.get_objective()
+    ms = cb.get_M().cpu().numpy().astype(np.float64)
+    for p in range(P):
+        ref = O.OpuOracle(128, r0[p].astype(np.float64), quant_bits=4, quant_mode="zp", clip_ratio=0.9).step(xs[p].astype(np.float64))
+        assert ns[p] == ref.N and abs(js[p] - ref.J) / ref.J < T["J"], (p, js[p], ref.J)
+        assert np.linalg.norm(ms[p] - ref.M) / np.linalg.norm(ref.M) < 3e-2, p
