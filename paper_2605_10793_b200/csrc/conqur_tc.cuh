@@ -209,6 +209,8 @@ struct TcGemmArgs {
   int na, nb;                   // distinct A / B tiles over all passes
   int a_toff[2], b_toff[2];     // their outer-coordinate offsets
   int a_tile[3], b_tile[3];     // tile index each pass reads (tiles appear in order of first use)
+  int full_tiles;               // pair kernel, non-symmetric products: tiles [0, full_tiles) are worked on whole, the
+                                //   remaining ones as two half-width items each (fills the last, partial wave)
   int sym;                      // 1: the output is symmetric (M == N): only tiles that touch the upper triangle are
                                 //    computed; tiles strictly above the diagonal also write their transpose
   float* outF; long long ldo;   // fp32 output (M read-modify-write, E, X_next, Y)
@@ -370,6 +372,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int tiles_m = (g.M + TM - 1) / TM, tiles_n = (g.N + BN - 1) / BN;
   const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, R) : tiles_m * tiles_n;
+  // work items: whole tiles, then (pair kernel only) the tail tiles as two half-width items each
+  const int full_tiles = (PAIR && B_MN && !g.sym) ? min(max(g.full_tiles, 0), num_tiles) : num_tiles;
+  const int num_items = full_tiles + 2 * (num_tiles - full_tiles);
+  auto decode_item = [&](int item, int& tm, int& tn, int& nt, int& ncol0) {
+    int tile = item; nt = BN; ncol0 = 0;
+    if (item >= full_tiles) { const int hh = item - full_tiles; tile = full_tiles + (hh >> 1); nt = BN / 2; ncol0 = (hh & 1) * (BN / 2); }
+    tc_tile_coords<R>(tile, tiles_m, tiles_n, g.sym, tm, tn);
+  };
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
   const int nseg = g.nseg_from_state ? max(1, min(g.nseg, g.nseg_from_state == 2 ? g.st->seg_e : g.st->seg_x)) : g.nseg;
   const int k_iters = PAIR ? num_kb : num_kb * nseg;     // a pair runs all passes of a k block from one stage
@@ -402,11 +412,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
-      for (int tile = worker; tile < num_tiles && ok; tile += n_workers) {
-        int tm, tn;
-        tc_tile_coords<R>(tile, tiles_m, tiles_n, g.sym, tm, tn);
-        // a pair splits the tile: this CTA loads 128 of the 256 rows of A and 128 of the 256 columns of B
-        const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN + (PAIR ? (int)rank * Cfg::B_ROWS : 0);
+      for (int tile = worker; tile < num_items && ok; tile += n_workers) {
+        int tm, tn, nt, ncol0;
+        decode_item(tile, tm, tn, nt, ncol0);
+        // a pair splits the item: this CTA loads 128 of the 256 rows of A and half of the item's columns of B
+        const int b_rows = PAIR ? nt / 2 : BN;
+        const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN + ncol0 + (PAIR ? (int)rank * b_rows : 0);
         for (int it = 0; it < k_iters; ++it) {
           const int seg = it / num_kb, k0 = (it - seg * num_kb) * TC_BK;
           const int a_off = g.a_off[seg], b_off = g.b_off[seg];
@@ -419,7 +430,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int na = 1, nb = 1;                          // tiles the passes in use need
             for (int sg = 0; sg < nseg; ++sg) { na = max(na, g.a_tile[sg] + 1); nb = max(nb, g.b_tile[sg] + 1); }
             na = min(na, NA); nb = min(nb, NB);
-            if (rank == 0) ptx::mbar_expect_tx(&aux->full[stage], 2 * (na * Cfg::A_BYTES + nb * Cfg::B_BYTES));
+            if (rank == 0) ptx::mbar_expect_tx(&aux->full[stage], 2 * (na * Cfg::A_BYTES + nb * b_rows * TC_BK * 2));
             const int kk = it * TC_BK;
 #pragma unroll
             for (int ia = 0; ia < NA; ++ia) {
@@ -438,7 +449,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               uint8_t* tb = sa + NA * Cfg::A_BYTES + ib * Cfg::B_BYTES;
               if (B_MN) {
 #pragma unroll
-                for (int h = 0; h < Cfg::B_ROWS / 64; ++h) ptx::tma_load_2d_pair(tb + h * 8192, &tmB, bar, n0 + 64 * h, kk + g.b_toff[ib]);
+                for (int h = 0; h < Cfg::B_ROWS / 64; ++h) {
+                  if (h * 64 >= b_rows) break;
+                  ptx::tma_load_2d_pair(tb + h * 8192, &tmB, bar, n0 + 64 * h, kk + g.b_toff[ib]);
+                }
               } else {
                 ptx::tma_load_2d_pair(tb, &tmB, bar, kk, n0 + g.b_toff[ib]);
               }
@@ -491,8 +505,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = worker; tile < num_tiles && ok; tile += n_workers, ++local) {
+      const uint32_t idesc_half = (idesc & ~(0x3fu << 17)) | ((uint32_t)((BN / 2) >> 3) << 17);   // N = BN / 2
+      for (int tile = worker; tile < num_items && ok; tile += n_workers, ++local) {
         const int buf = local & 1;
+        const uint32_t idesc_t = (tile >= full_tiles) ? idesc_half : idesc;
         if (!tc_wait(&aux->tempty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 2; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
@@ -511,7 +527,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int j = 0; j < TC_BK / 16; ++j) {
                 const uint64_t ad = A_MN ? tc_smem_desc(ta + j * 2048, 8192, 1024) : tc_smem_desc(ta + j * 32, 16, 1024);
                 const uint64_t bd = B_MN ? tc_smem_desc(tb + j * 2048, 8192, 1024) : tc_smem_desc(tb + j * 32, 16, 1024);
-                ptx::umma_bf16_pair(d_tmem, ad, bd, idesc, (it > 0 || sg > 0 || j > 0) ? 1u : 0u);
+                ptx::umma_bf16_pair(d_tmem, ad, bd, idesc_t, (it > 0 || sg > 0 || j > 0) ? 1u : 0u);
               }
             }
           } else {
@@ -547,11 +563,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int local = 0;
     bool ok = true;
     const uint32_t tempty_addr0 = PAIR ? ptx::mapa_u32(ptx::smem_u32(&aux->tempty[0]), 0) : 0u;
-    for (int tile = worker; tile < num_tiles && ok; tile += n_workers, ++local) {
+    for (int tile = worker; tile < num_items && ok; tile += n_workers, ++local) {
       const int buf = local & 1;
-      int tm, tn;
-      tc_tile_coords<R>(tile, tiles_m, tiles_n, g.sym, tm, tn);
-      const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN;   // this CTA's 128 rows, all BN columns
+      int tm, tn, nt, ncol0;
+      decode_item(tile, tm, tn, nt, ncol0);
+      const int m0 = tm * TM + (PAIR ? (int)rank * TC_BM : 0), n0 = tn * BN + ncol0;   // this CTA's 128 rows, all nt columns
       const bool mirror = g.sym && ((tm + 1) * TM <= tn * BN);        // strictly above the diagonal
       const int slot = PAIR ? 2 * tile + (int)rank : tile;            // where this CTA's per-tile partials go
       if (!tc_wait(&aux->tfull[buf], (uint32_t)(local >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 4; break; }
@@ -568,7 +584,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       float acc_abs = 0.f, acc_max = 0.f, acc_tr = 0.f, acc_vmax = -3.0e38f, acc_vmin = 3.0e38f;
       double acc_sq = 0.0;
 #pragma unroll 1
-      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+      for (int c = half * (nt / 64); c < (half + 1) * (nt / 64); ++c) {
         float v[32];
         ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
         const int col0 = n0 + c * 32;
@@ -949,12 +965,28 @@ inline TcVariant tc_variant(const TcHost& h, int N) {
   if (N % 256 == 0) return h.pair_clusters > 0 ? TcVariant{true, 256, 256} : TcVariant{false, 128, 256};
   return TcVariant{false, 128, 128};
 }
-// tiles the kernel computes, and per-tile partial slots it writes (a pair writes one per CTA)
+// tiles the kernel computes
 inline int tc_tiles(const TcVariant& v, int M, int N, int sym) {
   const int tn = (N + v.tile_n - 1) / v.tile_n, tm = (M + v.tile_m - 1) / v.tile_m;
   return sym ? tc_sym_tiles(tn, v.tile_n / v.tile_m) : tm * tn;
 }
-inline int tc_part_slots(const TcVariant& v, int M, int N, int sym) { return tc_tiles(v, M, N, sym) * (v.pair ? 2 : 1); }
+// Work items of a launch (B operand MN-major): the pair kernel works on the tiles of its last, partial wave as two
+// half-width items each when that lets them all run at once (e.g. 256 tiles on 74 pairs: 3 waves + 34 tiles ->
+// 3 waves + 68 half tiles, i.e. 3.5 instead of 4 tile times).  *full_tiles: tiles worked on whole.
+inline int tc_items(const TcHost& h, const TcVariant& v, int M, int N, int sym, int* full_tiles = nullptr) {
+  const int tiles = tc_tiles(v, M, N, sym);
+  int full = tiles;
+  if (v.pair && !sym && h.pair_clusters > 0) {
+    const int r = tiles % h.pair_clusters;
+    if (r > 0 && 2 * r <= h.pair_clusters) full = tiles - r;
+  }
+  if (full_tiles) *full_tiles = full;
+  return full + 2 * (tiles - full);
+}
+// per-item partial slots a launch writes (a pair writes one per CTA)
+inline int tc_part_slots(const TcHost& h, const TcVariant& v, int M, int N, int sym) {
+  return tc_items(h, v, M, N, sym) * (v.pair ? 2 : 1);
+}
 
 // Rewrite the passes (a_off[s], b_off[s]) as distinct operand tiles + which tile each pass reads.
 inline void tc_fuse_passes(TcGemmArgs* g) {
@@ -982,8 +1014,11 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
   }
   const TcVariant v{PAIR, Cfg::TILE_M, BN};
   const int tiles = tc_tiles(v, g.M, g.N, g.sym);
+  TcGemmArgs gl = g;
+  gl.full_tiles = tiles;
+  const int items = B_MN ? tc_items(h, v, g.M, g.N, g.sym, &gl.full_tiles) : tiles;
   const int workers = PAIR ? h.pair_clusters : h.num_sms;
-  const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
+  const int grid = (items < workers ? items : workers) * (PAIR ? 2 : 1);
   const int cls = tc_epi_class(EPI);
   Prof::Rec rec{};
   const bool timed = h.prof && h.prof->enabled;
@@ -1002,9 +1037,9 @@ inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUte
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    err = cudaLaunchKernelEx(&cfg, kern, a, b, g);
+    err = cudaLaunchKernelEx(&cfg, kern, a, b, gl);
   } else {
-    kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, g);
+    kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(a, b, gl);
     err = cudaGetLastError();
   }
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
@@ -1126,7 +1161,7 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
     g.outH = Cp; g.ldh = d;
     rc = tc_launch_n<false, true, TC_EPI_ROTATE>(h, s, tmXs_k, h.tmRb_mn, g);
     if (rc) return rc;
-    per_problem = tc_part_slots(tc_variant(h, d), (int)n, d, 0);
+    per_problem = tc_part_slots(h, tc_variant(h, d), (int)n, d, 0);
   } else {
     unsigned* rowmin = h.rowmax + h.n_max;
     if (cudaMemsetAsync(h.rowmax, 0, sizeof(unsigned) * n, s) != cudaSuccess) return CONQUR_ERR_CUDA;
@@ -1157,8 +1192,8 @@ inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
 
 
 // Partials of the Newton-Schulz epilogues: [0, parts) sums of squares, [parts, 2 parts) traces / iterate norms.
-inline int tc_ns_parts(const TcHost& h) { return tc_part_slots(tc_variant(h, h.d), h.d, h.d, 1); }
-inline int tc_ns_next_parts(const TcHost& h) { return tc_part_slots(tc_variant(h, h.d), h.d, h.d, 0); }
+inline int tc_ns_parts(const TcHost& h) { return tc_part_slots(h, tc_variant(h, h.d), h.d, h.d, 1); }
+inline int tc_ns_next_parts(const TcHost& h) { return tc_part_slots(h, tc_variant(h, h.d), h.d, h.d, 0); }
 
 // G = X^T X from the split iterate in Xh[buf] (three passes: hi hi, hi lo, lo hi; symmetric tiles only);
 // stores E = G - tau I as fp32 and bf16, and the statistics of G - I.
