@@ -209,7 +209,7 @@ struct TcGemmArgs {
   int na, nb;                   // distinct A / B tiles over all passes
   int a_toff[2], b_toff[2];     // their outer-coordinate offsets
   int a_tile[3], b_tile[3];     // tile index each pass reads (tiles appear in order of first use)
-  int full_tiles;               // pair kernel, non-symmetric products: tiles [0, full_tiles) are worked on whole, the
+  int full_tiles;               // pair kernel: tiles [0, full_tiles) are worked on whole, the
                                 //   remaining ones as two half-width items each (fills the last, partial wave)
   int sym;                      // 1: the output is symmetric (M == N): only tiles that touch the upper triangle are
                                 //    computed; tiles strictly above the diagonal also write their transpose
@@ -373,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_m = (g.M + TM - 1) / TM, tiles_n = (g.N + BN - 1) / BN;
   const int num_tiles = g.sym ? tc_sym_tiles(tiles_n, R) : tiles_m * tiles_n;
   // work items: whole tiles, then (pair kernel only) the tail tiles as two half-width items each
-  const int full_tiles = (PAIR && B_MN && !g.sym) ? min(max(g.full_tiles, 0), num_tiles) : num_tiles;
+  const int full_tiles = (PAIR && B_MN) ? min(max(g.full_tiles, 0), num_tiles) : num_tiles;
   const int num_items = full_tiles + 2 * (num_tiles - full_tiles);
   auto decode_item = [&](int item, int& tm, int& tn, int& nt, int& ncol0) {
     int tile = item; nt = BN; ncol0 = 0;
@@ -976,7 +976,7 @@ inline int tc_tiles(const TcVariant& v, int M, int N, int sym) {
 inline int tc_items(const TcHost& h, const TcVariant& v, int M, int N, int sym, int* full_tiles = nullptr) {
   const int tiles = tc_tiles(v, M, N, sym);
   int full = tiles;
-  if (v.pair && !sym && h.pair_clusters > 0) {
+  if (v.pair && h.pair_clusters > 0) {
     const int r = tiles % h.pair_clusters;
     if (r > 0 && 2 * r <= h.pair_clusters) full = tiles - r;
   }
