@@ -220,3 +220,41 @@ def test_zero_point_quant_mode_tc_and_batched():
         ref = O.OpuOracle(128, r0[p].astype(np.float64), quant_bits=4, quant_mode="zp", clip_ratio=0.9).step(xs[p].astype(np.float64))
         assert ns[p] == ref.N and abs(js[p] - ref.J) / ref.J < T["J"], (p, js[p], ref.J)
         assert np.linalg.norm(ms[p] - ref.M) / np.linalg.norm(ref.M) < 3e-2, p
+
+
+@pytest.mark.parametrize("mode", ["tc", "exact"])
+@pytest.mark.parametrize("spectrum", ["gauss", "log1e4", "near_orth", "spiky1e8", "below_bound"])
+def test_update_on_synthetic_spectra(mode, spectrum):
+    """The polar update on cross-covariances with prescribed singular values (loaded through conqur_set_M):
+    well conditioned, log-spaced, already orthogonal, a few dominant directions over a 1e-8 tail, and a spectrum whose
+    smallest singular value lies below the bound the schedule was planned for (the iteration must re-enter and
+    still deliver)."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    d = 512
+    rng = np.random.default_rng(5)
+    u, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    v, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    kw = {}
+    if spectrum == "gauss":
+        m = rng.standard_normal((d, d))
+    elif spectrum == "log1e4":
+        m = (u * np.logspace(0, -4, d)) @ v.T
+    elif spectrum == "near_orth":
+        m = u @ v.T + 1e-3 * rng.standard_normal((d, d)) / np.sqrt(d)
+    elif spectrum == "spiky1e8":
+        m = (u * np.concatenate([np.ones(8), np.logspace(-3, -8, d - 8)])) @ v.T
+    else:
+        m = (u * np.concatenate([np.ones(8), np.logspace(-2, -6, d - 8)])) @ v.T
+        kw = dict(ns_sigma_min_rel=1e-3, ns_max_steps=40)        # planned for a far better conditioned matrix
+    m32 = m.astype(np.float32)
+    ctx = B.Context(d=d, n_max=128, in_dtype="bf16", mode=mode, **kw)
+    ctx.set_M(torch.from_numpy(m32).cuda(), 1.0, d)
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, (st.status, st.ns_steps_used)
+    r = ctx.get_R().cpu().numpy().astype(np.float64)
+    rep = update_parity(m32.astype(np.float64), r)
+    tol = TOL[mode]
+    assert rep["orth"] <= tol["orth"], rep
+    assert rep["gap"] <= tol["gap"], (rep["gap"], st.ns_steps_used)
