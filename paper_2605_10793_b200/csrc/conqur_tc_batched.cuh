@@ -393,8 +393,8 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
 //   X <- (gamma + kappa) X + X B, tau = ||X||_F^2 / d, split into (hi, lo) -> shared memory
 // Two CTAs fit one SM (96 KB of shared memory and 256 TMEM columns each), so one problem's element-wise phases
 // overlap the other's products.
-constexpr int TCBU_THREADS = 128;
-constexpr int TCBU_SMEM_BYTES = 3 * TCB_TILE_BYTES + 1024 + 1024;
+constexpr int TCBU_THREADS = 256;            // 128 rows x 2 column halves
+constexpr int TCBU_SMEM_BYTES = 3 * TCB_TILE_BYTES + 4096 + 1024;
 
 struct TcbUpdAux {
   uint64_t mbar;
@@ -404,8 +404,10 @@ struct TcbUpdAux {
   float tau, x0s, lam;
   float coef[4];
   int seg_x;
-  double red_d[4], red_t[4];
-  float red_f[4];
+  double red_d[8], red_t[8];
+  float red_f[8];
+  DevState state;                    // the problem's state while it is being iterated (written back once at the end)
+  SchedEntry sched[NS_SCHED_MAX];    // the polynomial schedule (copied once per CTA)
 };
 
 struct TcbUpdArgs {
@@ -420,7 +422,7 @@ __device__ __forceinline__ double tcbu_block_sum(double v, double* red, int warp
   v = warp_sum_d(v);
   if (lane == 0) red[warp] = v;
   __syncthreads();
-  const double t = red[0] + red[1] + red[2] + red[3];
+  const double t = ((red[0] + red[1]) + (red[2] + red[3])) + ((red[4] + red[5]) + (red[6] + red[7]));
   __syncthreads();
   return t;
 }
@@ -434,7 +436,8 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
   TcbUpdAux* aux = reinterpret_cast<TcbUpdAux*>(smem + 3 * TCB_TILE_BYTES);
   volatile int* abort_flag = &aux->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = threadIdx.x;                       // the row this thread owns everywhere
+  const int r = threadIdx.x & 127;                 // the row this thread works on everywhere
+  const int half = threadIdx.x >> 7;               // ... and which 64 of its 128 columns
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->mbar, 1);
     aux->abort_flag = 0;
@@ -442,11 +445,14 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     ptx::fence_proxy_async();
   }
   if (warp == 0) { ptx::tmem_alloc(&aux->tmem_base, 256); ptx::tmem_relinquish(); }
+  for (int i = threadIdx.x; i < g.ncp.n_sched && i < NS_SCHED_MAX; i += TCBU_THREADS) aux->sched[i] = g.ncp.sched[i];
+  NsControlParams ncp = g.ncp;
+  ncp.sched = aux->sched;                          // control decisions read the shared-memory copy
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = aux->tmem_base;
-  const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);      // this warp's 32 TMEM lanes
+  const uint32_t t_row = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);      // this warp's 32 TMEM lanes
   const uint32_t aXh = ptx::smem_u32(sXh), aXl = ptx::smem_u32(sXl), aEB = ptx::smem_u32(sEB);
   const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   const uint32_t idesc_mm = idesc_base | (1u << 15) | (1u << 16);       // both operands read "transposed" (MN-major)
@@ -475,12 +481,14 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
   };
 
   for (int p = blockIdx.x; p < g.P && !timed_out; p += gridDim.x) {
-    DevState* s = g.st + p;
+    DevState* const sg = g.st + p;                 // global copy: read once, written back once
+    DevState* const s = &aux->state;
+    if (threadIdx.x == 0) *s = *sg;
     const float* Mrow = g.M + ((long long)p * TCB_D + r) * TCB_D;
     const float* Rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
     // ---- scale: lam = prior_rel ||M||_F / sqrt(d), X_0 = (M + lam R) / (||M + lam R||_F (1 + margin))
     double ssq = 0.0;
-    for (int c = 0; c < TCB_D; c += 4) {
+    for (int c = half * 64; c < half * 64 + 64; c += 4) {
       const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
       ssq += (double)m.x * m.x + (double)m.y * m.y + (double)m.z * m.z + (double)m.w * m.w;
     }
@@ -488,7 +496,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     const float lam = g.prior_rel * (float)sqrt(fro2) * isd;
     if (g.prior_rel > 0.f) {
       ssq = 0.0;
-      for (int c = 0; c < TCB_D; c += 4) {
+      for (int c = half * 64; c < half * 64 + 64; c += 4) {
         const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
         const float4 q = *reinterpret_cast<const float4*>(Rrow + c);
         const float a = fmaf(lam, q.x, m.x), b = fmaf(lam, q.y, m.y), cc = fmaf(lam, q.z, m.z), d4 = fmaf(lam, q.w, m.w);
@@ -509,7 +517,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     __syncthreads();
     if (!aux->done) {
       const float x0s = aux->x0s;
-      for (int c16 = 0; c16 < 16; ++c16) {
+      for (int c16 = half * 8; c16 < half * 8 + 8; ++c16) {
         uint32_t wh[4], wl[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -522,7 +530,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         *reinterpret_cast<uint4*>(sXh + tcb_piece(r, c16)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
         *reinterpret_cast<uint4*>(sXl + tcb_piece(r, c16)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
       }
-      for (int k = 0; k <= g.ncp.max_steps; ++k) {
+      for (int k = 0; k <= ncp.max_steps; ++k) {
         // ---- G = X^T X
         if (!run_products([&] {
               const uint32_t aa[3] = {aXh, aXh, aXl}, bb[3] = {aXh, aXl, aXh};
@@ -537,7 +545,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         float mx = 0.f, tr = 0.f;
         double sq = 0.0;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
           float v[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
           const int dcol = r - c * 32;
@@ -561,10 +569,10 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           if (lane == 0) { aux->red_d[warp] = wsq; aux->red_t[warp] = wtr; aux->red_f[warp] = wmx; }
           __syncthreads();
           if (threadIdx.x == 0) {
-            const double tsq = aux->red_d[0] + aux->red_d[1] + aux->red_d[2] + aux->red_d[3];
-            const double ttr = aux->red_t[0] + aux->red_t[1] + aux->red_t[2] + aux->red_t[3];
-            const float tmx = fmaxf(fmaxf(aux->red_f[0], aux->red_f[1]), fmaxf(aux->red_f[2], aux->red_f[3]));
-            ns_control_decide(s, tmx, tsq, ttr, k, 0, g.ncp);
+            double tsq = 0.0, ttr = 0.0;
+            float tmx = 0.f;
+            for (int i = 0; i < 8; ++i) { tsq += aux->red_d[i]; ttr += aux->red_t[i]; tmx = fmaxf(tmx, aux->red_f[i]); }
+            ns_control_decide(s, tmx, tsq, ttr, k, 0, ncp);
             aux->done = s->ns_done;
             aux->coef[0] = s->coef[0]; aux->coef[1] = s->coef[1]; aux->coef[2] = s->coef[2]; aux->coef[3] = s->coef[3];
             aux->seg_x = s->seg_x;
@@ -582,7 +590,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
             })) { timed_out = true; break; }
         // ---- B = beta2 E E + beta1 E - kappa I (over E: the product that read it has finished)
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
           float gq[32], ee[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), gq);
           ptx::tmem_ld32(t_row + 128u + (uint32_t)(c * 32), ee);
@@ -613,7 +621,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         // ---- X <- (gamma + kappa) X + X B; tau of the next step
         double x2 = 0.0;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
           float v[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
 #pragma unroll
@@ -647,7 +655,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     if (converged) {
       float* Ro = g.R + ((long long)p * TCB_D + r) * TCB_D;
       float* Mo = g.M + ((long long)p * TCB_D + r) * TCB_D;
-      for (int c16 = 0; c16 < 16; ++c16) {
+      for (int c16 = half * 8; c16 < half * 8 + 8; ++c16) {
         const uint32_t off = tcb_piece(r, c16);
         const uint4 h4 = *reinterpret_cast<const uint4*>(sXh + off), l4 = *reinterpret_cast<const uint4*>(sXl + off);
         const uint32_t hh[4] = {h4.x, h4.y, h4.z, h4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
@@ -668,8 +676,9 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         s->last_J = s->J; s->last_N = s->N; s->J = 0.0; s->N = 0; s->updates += 1;
         s->last_orth = s->e_max; s->last_fro = s->e_fro;
       } else {
-        atomicOr(&s->status_flags, STATUS_FLAG_NS_FAILED);
+        s->status_flags |= STATUS_FLAG_NS_FAILED;
       }
+      *sg = *s;                                     // this CTA is the only writer of problem p's state during the update
     }
     __syncthreads();                                // aux->done is rewritten by the next problem
   }
