@@ -283,6 +283,17 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_by
 
 __device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16(v)); }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16(v)); }
+// Two floats -> packed bf16 pair (first in the low half) with one conversion instruction.
+__device__ __forceinline__ uint32_t bf16x2_pack(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// Two-term split of a pair of floats: wh = packed round-to-nearest bf16, wl = packed bf16 of the remainders.
+__device__ __forceinline__ void bf16x2_split(float a, float b, uint32_t& wh, uint32_t& wl) {
+  wh = bf16x2_pack(a, b);
+  wl = bf16x2_pack(a - __uint_as_float(wh << 16), b - __uint_as_float(wh & 0xffff0000u));
+}
 
 // Epilogue stores.  A thread holds 32 consecutive columns of ONE row (TMEM lane = row), so a direct 16-byte store
 // per thread touches 32 different lines per instruction and only half a sector of each.  The warp's 32 x 32 block
@@ -624,13 +635,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int dcol = row - col0;                      // position of the diagonal inside this chunk, if any
           if (EPI == TC_EPI_RESID) {
             // statistics of G - I and of tr G; the stored residual is E = G - tau I
+            float sq32 = 0.f;                              // 32 terms in fp32, then one double add per chunk
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               float e1 = v[i];
               if (i == dcol) { acc_tr += v[i]; e1 -= 1.f; v[i] -= c_tau; }
               acc_max = fmaxf(acc_max, fabsf(e1));
-              acc_sq += (double)e1 * (double)e1;
+              sq32 = fmaf(e1, e1, sq32);
             }
+            acc_sq += (double)sq32;
           } else {
             if (EPI == TC_EPI_POLY) {
               // beta1 E from the bf16 copy of E this product streams as its operands: the difference to fp32 E is a
@@ -669,17 +682,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int i = 0; i < 32; ++i)
                 if (i == dcol) v[i] -= c_kappa;
             } else {
+              float sq32 = 0.f;
 #pragma unroll
-              for (int i = 0; i < 32; ++i) acc_sq += (double)v[i] * (double)v[i];
+              for (int i = 0; i < 32; ++i) sq32 = fmaf(v[i], v[i], sq32);
+              acc_sq += (double)sq32;
             }
           }
           uint32_t wh[16], wl[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float a = v[2 * i], b = v[2 * i + 1];
-            const float ah = bf16_round(a), bh = bf16_round(b);
-            wh[i] = bf16_bits(ah) | (bf16_bits(bh) << 16);
-            if (EPI == TC_EPI_NEXT) wl[i] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+            if (EPI == TC_EPI_NEXT) bf16x2_split(v[2 * i], v[2 * i + 1], wh[i], wl[i]);
+            else wh[i] = bf16x2_pack(v[2 * i], v[2 * i + 1]);
           }
           tc_store_block_bf16(stg, lane, wh, g.outH + (long long)wrow0 * g.ldh + col0, g.ldh, rows_ok);
           if (EPI == TC_EPI_NEXT)
@@ -768,8 +781,13 @@ __global__ void __launch_bounds__(256) rownorm_stage_kernel(const TIn* __restric
 #pragma unroll
       for (int j = 0; j < 4; ++j) v[j] = ld_as_float(x + k + j);
     }
+    if (sizeof(TIn) == 4) {                            // fp32 input: the norm of what the MMA will see (bf16 values are exact already)
+      const uint32_t p0 = bf16x2_pack(v[0], v[1]), p1 = bf16x2_pack(v[2], v[3]);
+      v[0] = __uint_as_float(p0 << 16); v[1] = __uint_as_float(p0 & 0xffff0000u);
+      v[2] = __uint_as_float(p1 << 16); v[3] = __uint_as_float(p1 & 0xffff0000u);
+    }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { v[j] = bf16_round(v[j]); ss = fmaf(v[j], v[j], ss); }
+    for (int j = 0; j < 4; ++j) ss = fmaf(v[j], v[j], ss);
   }
   ss = warp_sum(ss);
   const bool good = (ss > 0.f) && (ss <= 3.0e38f);
@@ -785,8 +803,8 @@ __global__ void __launch_bounds__(256) rownorm_stage_kernel(const TIn* __restric
       }
     }
     uint2 o;
-    o.x = bf16_bits(v[0]) | (bf16_bits(v[1]) << 16);
-    o.y = bf16_bits(v[2]) | (bf16_bits(v[3]) << 16);
+    o.x = bf16x2_pack(v[0], v[1]);
+    o.y = bf16x2_pack(v[2], v[3]);
     *reinterpret_cast<uint2*>(dst + k) = o;
   }
   if (lane == 0) {
@@ -804,16 +822,11 @@ __global__ void split_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* 
   for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < count;
        i += (int64_t)gridDim.x * blockDim.x * 4) {
     const float4 t = *reinterpret_cast<const float4*>(src + i);
-    const float h0 = bf16_round(t.x), h1 = bf16_round(t.y), h2 = bf16_round(t.z), h3 = bf16_round(t.w);
-    uint2 o;
-    o.x = bf16_bits(h0) | (bf16_bits(h1) << 16);
-    o.y = bf16_bits(h2) | (bf16_bits(h3) << 16);
+    uint2 o, l;
+    bf16x2_split(t.x, t.y, o.x, l.x);
+    bf16x2_split(t.z, t.w, o.y, l.y);
     *reinterpret_cast<uint2*>(dst + i) = o;
-    if (lo_elems) {
-      o.x = bf16_bits(t.x - h0) | (bf16_bits(t.y - h1) << 16);
-      o.y = bf16_bits(t.z - h2) | (bf16_bits(t.w - h3) << 16);
-      *reinterpret_cast<uint2*>(dst + lo_elems + i) = o;
-    }
+    if (lo_elems) *reinterpret_cast<uint2*>(dst + lo_elems + i) = l;
   }
 }
 

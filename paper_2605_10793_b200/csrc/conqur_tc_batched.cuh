@@ -523,9 +523,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         for (int e = 0; e < 4; ++e) {
           const int col = c16 * 8 + e * 2;
           const float a = fmaf(lam, Rrow[col], Mrow[col]) * x0s, b = fmaf(lam, Rrow[col + 1], Mrow[col + 1]) * x0s;
-          const float ah = bf16_round(a), bh = bf16_round(b);
-          wh[e] = bf16_bits(ah) | (bf16_bits(bh) << 16);
-          wl[e] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+          bf16x2_split(a, b, wh[e], wl[e]);
         }
         *reinterpret_cast<uint4*>(sXh + tcb_piece(r, c16)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
         *reinterpret_cast<uint4*>(sXl + tcb_piece(r, c16)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
@@ -550,15 +548,17 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
           const int dcol = r - c * 32;
           uint32_t w[16];
+          float sq32 = 0.f;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             float e1 = v[i];
             if (i == dcol) { tr += v[i]; e1 -= 1.f; v[i] -= tau; }
             mx = fmaxf(mx, fabsf(e1));
-            sq += (double)e1 * (double)e1;
+            sq32 = fmaf(e1, e1, sq32);
           }
+          sq += (double)sq32;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) w[i] = bf16_bits(v[2 * i]) | (bf16_bits(v[2 * i + 1]) << 16);
+          for (int i = 0; i < 16; ++i) w[i] = bf16x2_pack(v[2 * i], v[2 * i + 1]);
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
             *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
@@ -604,7 +604,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
             ee[i] = b;
           }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) w[i] = bf16_bits(ee[2 * i]) | (bf16_bits(ee[2 * i + 1]) << 16);
+          for (int i = 0; i < 16; ++i) w[i] = bf16x2_pack(ee[2 * i], ee[2 * i + 1]);
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
             *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
@@ -624,6 +624,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         for (int c = half * 2; c < half * 2 + 2; ++c) {
           float v[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
+          float x2f = 0.f;
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             const uint32_t off = tcb_piece(r, c * 4 + q4);
@@ -635,14 +636,13 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
               const float xa = __uint_as_float(hh[e] << 16) + __uint_as_float(ll[e] << 16);
               const float xb = __uint_as_float(hh[e] & 0xffff0000u) + __uint_as_float(ll[e] & 0xffff0000u);
               const float a = fmaf(cg, xa, v[q4 * 8 + 2 * e]), b = fmaf(cg, xb, v[q4 * 8 + 2 * e + 1]);
-              x2 += (double)a * a + (double)b * b;
-              const float ah = bf16_round(a), bh = bf16_round(b);
-              wh[e] = bf16_bits(ah) | (bf16_bits(bh) << 16);
-              wl[e] = bf16_bits(a - ah) | (bf16_bits(b - bh) << 16);
+              x2f = fmaf(a, a, fmaf(b, b, x2f));
+              bf16x2_split(a, b, wh[e], wl[e]);
             }
             *reinterpret_cast<uint4*>(sXh + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
             *reinterpret_cast<uint4*>(sXl + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
           }
+          x2 += (double)x2f;
         }
         const double tx2 = tcbu_block_sum(x2, aux->red_d, warp, lane);
         if (threadIdx.x == 0) { s->tau = (float)(tx2 / (double)TCB_D); aux->tau = s->tau; }
