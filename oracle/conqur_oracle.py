@@ -23,6 +23,10 @@ What each function follows:
   OpuOracle.step      Section 3.3 (cross-covariance Z^T X_tilde) accumulated
                       across tensors as Section 3.4 allows; objective in the
                       l1 form of Section 3.2
+  token_diagnostics   Section 4 diagnostics of the rotated rows: normalised participation ratio
+                      PR(y)/d = ||y||_2^4 / (d ||y||_4^4), dynamic-range ratio
+                      rho(y) = ||y||_inf^2 / ||y||_2^2 (Appendix B), and the relative squared
+                      quantisation error ||X R - Q(X R)||_F^2 / ||X||_F^2 (on un-normalised rows)
   polar_svd           Section 3.3, C = U Sigma V^T, R <- U V^T
   OpuOracle.update    Section 3.3 / Algorithm 1: R replaced, statistics reset
 
@@ -111,6 +115,23 @@ def fake_quant_zp(y, bits, clip_ratio=1.0):
     q = np.clip(q, 0.0, float(levels))
     k = np.where(ok[..., None], q - zeta[..., None], 0.0)
     return k * delta[..., None], k, delta
+
+
+def token_diagnostics(x, r, quant_bits=0, quant_mode="sym", clip_ratio=1.0):
+    """Sums over the used rows of x of PR(y)/d and rho(y) for y = x R, and numerator / denominator of the relative
+    squared quantisation error (Section 4).  Returns (sum_pr_over_d, sum_rho, qerr_num, qerr_den, rows_used)."""
+    x = np.asarray(x, dtype=np.float64)
+    _, used = normalise_rows(x)
+    y = x[used] @ np.asarray(r, dtype=np.float64)          # un-normalised: PR and rho do not depend on the row scale
+    d = y.shape[1]
+    n2 = np.sum(y * y, axis=1)
+    pr = n2 * n2 / (d * np.sum(y ** 4, axis=1))
+    rho = np.max(np.abs(y), axis=1) ** 2 / n2
+    num = 0.0
+    if quant_bits:
+        qy = fake_quant_sym(y, quant_bits)[0] if quant_mode == "sym" else fake_quant_zp(y, quant_bits, clip_ratio)[0]
+        num = float(np.sum((y - qy) ** 2))
+    return float(pr.sum()), float(rho.sum()), num, float(np.sum(x[used] ** 2)), int(used.sum())
 
 
 def polar_svd(m):

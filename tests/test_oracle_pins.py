@@ -470,3 +470,47 @@ def test_zero_point_mode_statistics_and_shift_sensitivity():
     # scale invariance of the codes: a positive row scale changes nothing
     orc2 = O.OpuOracle(d, r, quant_bits=4, quant_mode="zp", clip_ratio=0.9).step(x * np.exp(rng.standard_normal((n, 1))))
     assert abs(orc2.J - orc.J) < 1e-12 and np.allclose(orc2.M, orc.M, atol=1e-13)
+
+
+# ---- diagnostics of Section 4 (participation ratio, dynamic-range ratio, relative quantisation error)
+
+def test_participation_ratio_and_dynamic_range_bounds_and_extremes():
+    d = 64
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((200, d)) * np.exp(rng.standard_normal((200, 1)))
+    spr, srho, num, den, n = O.token_diagnostics(x, np.eye(d))
+    assert n == 200 and num == 0.0 and abs(den - np.sum(x * x)) < 1e-9 * den
+    # per-row bounds 1/d <= PR/d <= 1, 1/d <= rho <= 1, and PR >= 1/rho (||y||_4^4 <= ||y||_inf^2 ||y||_2^2)
+    for row in x[:20]:
+        pr, rho, _, _, _ = O.token_diagnostics(row[None], np.eye(d))
+        assert 1 / d - 1e-12 <= pr <= 1 + 1e-12 and 1 / d - 1e-12 <= rho <= 1 + 1e-12 and pr * rho >= 1 / d - 1e-12
+    # extremes printed in the paper: one-sparse -> 1/d, equal magnitudes -> 1
+    one_hot = np.zeros((1, d)); one_hot[0, 5] = -3.0
+    corner = np.where(rng.random((1, d)) < 0.5, -1.0, 1.0) * 0.7
+    assert abs(O.token_diagnostics(one_hot, np.eye(d))[0] - 1 / d) < 1e-15 and abs(O.token_diagnostics(one_hot, np.eye(d))[1] - 1) < 1e-15
+    assert abs(O.token_diagnostics(corner, np.eye(d))[0] - 1) < 1e-12 and abs(O.token_diagnostics(corner, np.eye(d))[1] - 1 / d) < 1e-12
+    # a Hadamard rotation turns one-hot rows into corners (PR/d: 1/d -> 1)
+    h = I.hadamard_pm1(d) / np.sqrt(d)
+    assert abs(O.token_diagnostics(one_hot, h)[0] - 1) < 1e-12
+    # invariance to the row scale and to skipped rows
+    x2 = x * 7.0; x2[3] = 0.0
+    a = O.token_diagnostics(np.delete(x, 3, axis=0), np.eye(d)); b = O.token_diagnostics(x2, np.eye(d))
+    assert abs(a[0] - b[0]) < 1e-10 and abs(a[1] - b[1]) < 1e-10 and b[4] == 199
+
+
+@pytest.mark.parametrize("mode,clip", [("sym", 1.0), ("zp", 1.0), ("zp", 0.9)])
+def test_relative_quantisation_error_definition_and_bound(mode, clip):
+    d, n, bits = 32, 40, 4
+    rng = np.random.default_rng(22)
+    x = rng.standard_normal((n, d)) * np.exp(rng.standard_normal((n, 1)))
+    r = np.linalg.qr(rng.standard_normal((d, d)))[0]
+    spr, srho, num, den, used = O.token_diagnostics(x, r, bits, mode, clip)
+    y = x @ r
+    q = O.fake_quant_sym(y, bits)[0] if mode == "sym" else O.fake_quant_zp(y, bits, clip)[0]
+    assert abs(num - np.linalg.norm(y - q) ** 2) < 1e-12 * num and abs(den - np.linalg.norm(x) ** 2) < 1e-12 * den
+    if clip == 1.0:      # Appendix B: ||Q(y) - y||^2 <= d Delta^2 / 4 per row
+        delta = (np.abs(y).max(axis=1) / 7) if mode == "sym" else ((y.max(axis=1) - y.min(axis=1)) / 15)
+        assert num <= np.sum(d * delta ** 2 / 4) + 1e-12
+    # the error is relative: scaling the activations changes nothing
+    num2, den2 = O.token_diagnostics(3.0 * x, r, bits, mode, clip)[2:4]
+    assert abs(num2 / den2 - num / den) < 1e-12
