@@ -82,6 +82,8 @@ typedef struct {
                                CONQUR_QUANT_ZEROPOINT: Q_zp of Appendix B (delta = c (max y - min y) / (2^b - 1), integer
                                zero-point, codes clamped to 0..2^b-1), the quantiser the paper's evaluation uses */
   float    clip_ratio;      /* c in (0, 1] for the zero-point quantiser (Appendix C uses 0.9 for activations); 0 = 1 */
+  int32_t  diagnostics;     /* 1: every step also gathers the diagnostics of Section 4 (conqur_get_diagnostics); the step
+                               then forms the rotated rows in memory first (two passes) */
 } conqur_config;
 
 typedef struct {
@@ -166,6 +168,23 @@ int conqur_get_R(conqur_ctx* ctx, float* R_out_dev);
  * n_tokens[p] = rows used.  Host arrays of cfg.batch entries.  Synchronises.
  */
 int conqur_get_objective(conqur_ctx* ctx, double* J_sum, int64_t* n_tokens);
+
+/*
+ * Diagnostics of Section 4 over the rows used since the last update, at the R those steps used (cfg.diagnostics = 1):
+ *   sum_pr_over_d  sum_i PR(y_i)/d,  PR(y)/d = ||y||_2^4 / (d ||y||_4^4) in [1/d, 1]  (normalised participation ratio)
+ *   sum_rho        sum_i rho(y_i),   rho(y) = ||y||_inf^2 / ||y||_2^2 in [1/d, 1]     (dynamic-range ratio, Appendix B)
+ *   qerr_num/den   ||X R - Q(X R)||_F^2 and ||X||_F^2 on the un-normalised rows       (relative squared quantisation
+ *                  error; num = 0 when quant_bits == 0), Q the configured per-token fake-quantiser
+ * with y_i = x_i R.  out: host array of cfg.batch entries with struct_size set.  Synchronises.
+ * Not gathered by tensor-core contexts with batch > 1 (conqur_init rejects that combination).
+ */
+typedef struct {
+  uint32_t struct_size;     /* = sizeof(conqur_diagnostics) */
+  int32_t  reserved;
+  double   sum_pr_over_d, sum_rho, qerr_num, qerr_den;
+  int64_t  n_tokens;
+} conqur_diagnostics;
+int conqur_get_diagnostics(conqur_ctx* ctx, conqur_diagnostics* out);
 
 /* Cross-covariance accumulated since the last update, including the 1/sqrt(d):
  * device fp32 batch x d x d.  Synchronises. */

@@ -25,6 +25,7 @@ EXPORTS = [
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
+    "conqur_get_diagnostics",
     "conqur_strerror",
 ]
 
@@ -34,7 +35,7 @@ class conqur_config(C.Structure):
         ("struct_size", C.c_uint32), ("in_dtype", C.c_int32), ("mode", C.c_int32), ("quant_bits", C.c_int32),
         ("ns_steps", C.c_int32), ("ns_max_steps", C.c_int32), ("orth_tol", C.c_float), ("prior_rel", C.c_float),
         ("ns_sigma_min_rel", C.c_float), ("n_max", C.c_int64), ("batch", C.c_int32),
-        ("quant_mode", C.c_int32), ("clip_ratio", C.c_float),
+        ("quant_mode", C.c_int32), ("clip_ratio", C.c_float), ("diagnostics", C.c_int32),
     ]
 
 
@@ -43,6 +44,13 @@ class conqur_stats(C.Structure):
         ("struct_size", C.c_uint32), ("status", C.c_int32), ("ns_steps_used", C.c_int32), ("updates", C.c_int32),
         ("orth_err", C.c_float), ("orth_fro", C.c_float), ("scale", C.c_float), ("n_skipped", C.c_int64),
         ("last_J", C.c_double), ("last_N", C.c_int64),
+    ]
+
+
+class conqur_diagnostics(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("reserved", C.c_int32), ("sum_pr_over_d", C.c_double), ("sum_rho", C.c_double),
+        ("qerr_num", C.c_double), ("qerr_den", C.c_double), ("n_tokens", C.c_int64),
     ]
 
 
@@ -109,6 +117,8 @@ def load() -> C.CDLL:
     lib.conqur_objective_noalloc.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, vp]
     lib.conqur_debug_gemm.restype = C.c_int
     lib.conqur_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.conqur_get_diagnostics.restype = C.c_int
+    lib.conqur_get_diagnostics.argtypes = [vp, C.POINTER(conqur_diagnostics)]
     lib.conqur_debug_wait_timeout.restype = C.c_int
     lib.conqur_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.conqur_strerror.restype = C.c_char_p
@@ -123,9 +133,9 @@ def strerror(status: int) -> str:
 
 def make_config(*, in_dtype=CONQUR_BF16, mode=CONQUR_TC_BF16, quant_bits=0, ns_steps=0, ns_max_steps=0,
                 orth_tol=0.0, prior_rel=0.0, ns_sigma_min_rel=0.0, n_max=1, batch=1, quant_mode=CONQUR_QUANT_SYMMETRIC,
-                clip_ratio=0.0) -> conqur_config:
+                clip_ratio=0.0, diagnostics=0) -> conqur_config:
     return conqur_config(C.sizeof(conqur_config), in_dtype, mode, quant_bits, ns_steps, ns_max_steps, orth_tol,
-                         prior_rel, ns_sigma_min_rel, n_max, batch, quant_mode, clip_ratio)
+                         prior_rel, ns_sigma_min_rel, n_max, batch, quant_mode, clip_ratio, diagnostics)
 
 
 # ---- the C calls, one to one -------------------------------------------------------------------
@@ -246,7 +256,7 @@ class Context:
     """One calibration context on the current CUDA device / current torch stream."""
 
     def __init__(self, d: int, n_max: int, *, in_dtype="bf16", mode="tc", quant_bits=0, batch=1, prior_rel=0.0,
-                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None, quant_mode="sym", clip_ratio=0.0):
+                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None, quant_mode="sym", clip_ratio=0.0, diagnostics=False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("conqur needs a CUDA device (B200); there is no CPU path")
@@ -258,7 +268,7 @@ class Context:
                                ns_max_steps=ns_max_steps, orth_tol=orth_tol, prior_rel=prior_rel,
                                ns_sigma_min_rel=ns_sigma_min_rel, n_max=n_max, batch=batch,
                                quant_mode={"sym": CONQUR_QUANT_SYMMETRIC, "zp": CONQUR_QUANT_ZEROPOINT}[quant_mode],
-                               clip_ratio=clip_ratio)
+                               clip_ratio=clip_ratio, diagnostics=int(bool(diagnostics)))
         nbytes = conqur_workspace_bytes(self.d, self.cfg)
         if nbytes == 0:
             raise ConqurError(-1, "conqur_workspace_bytes")
@@ -316,6 +326,15 @@ class Context:
         if check:
             self._chk(rc, "conqur_get_objective")
         return (float(j[0]), int(n[0])) if self.batch == 1 else (j, n)
+
+    def get_diagnostics(self):
+        """Section-4 diagnostics since the last update: list of dicts (one per problem)."""
+        arr = (conqur_diagnostics * self.batch)()
+        for a in arr:
+            a.struct_size = C.sizeof(conqur_diagnostics)
+        self._chk(load().conqur_get_diagnostics(self.h, arr), "conqur_get_diagnostics")
+        return [dict(sum_pr_over_d=a.sum_pr_over_d, sum_rho=a.sum_rho, qerr_num=a.qerr_num, qerr_den=a.qerr_den,
+                     n_tokens=a.n_tokens) for a in arr]
 
     def debug_get_signs(self, n: int):
         out = self.torch.empty((n, self.d), dtype=self.torch.int8, device="cuda")

@@ -29,7 +29,7 @@ inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 inline int cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, flags_agg, R, M, rnorm, rowmax, part_d, part_f, sched;
+  size_t state, flags_agg, R, M, rnorm, rowmax, part_d, part_f, part_diag, sched;
   size_t C;                 // exact: fp32 C' / Y (P x n_max x d); TC quant mode: fp32 Y
   size_t Xa, Xb, E, B;      // Newton-Schulz fp32 matrices (P x d x d each)
   size_t splitk;            // exact accumulate split-K partials
@@ -42,6 +42,7 @@ struct Layout {
 struct Cfg {
   int d, P, in_dtype, mode, quant_bits, ns_max_steps;
   QuantSpec qs;
+  int diagnostics;
   int64_t n_max;
   float orth_tol, prior_rel, fro_tol, margin;
   bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode)
@@ -63,6 +64,8 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   if (c->quant_bits != 0 && (c->quant_bits < 2 || c->quant_bits > 8)) return false;
   if (c->quant_mode != CONQUR_QUANT_SYMMETRIC && c->quant_mode != CONQUR_QUANT_ZEROPOINT) return false;
   if (c->clip_ratio < 0.f || c->clip_ratio > 1.f) return false;
+  if (c->diagnostics != 0 && c->diagnostics != 1) return false;
+  if (c->diagnostics && c->mode == CONQUR_TC_BF16 && c->batch > 1) return false;   // the fused per-head kernel gathers none
   if (c->prior_rel < 0.f || c->orth_tol < 0.f || c->ns_sigma_min_rel < 0.f || c->ns_steps < 0 || c->ns_max_steps < 0)
     return false;
   if (c->mode == CONQUR_TC_BF16 && !tc_supported_shape(d, c->batch)) return false;
@@ -83,6 +86,7 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   L->max_partials = mp;
   L->part_d = take(sizeof(double) * mp * P);
   L->part_f = take(sizeof(float) * mp * P);
+  L->part_diag = c->diagnostics ? take(sizeof(double) * 4 * mp * P) : 0;
   L->sched = take(sizeof(SchedEntry) * NS_SCHED_MAX);
   L->acc_splits = 1;
   L->C = L->splitk = 0;
@@ -95,7 +99,7 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
     L->acc_splits = pick_acc_splits(d, (int)P, n);
     if (L->acc_splits > 1) L->splitk = take(sizeof(float) * dd * P * L->acc_splits);
   } else {
-    if (c->quant_bits && P == 1) L->C = take(sizeof(float) * (size_t)n * d);
+    if ((c->quant_bits || c->diagnostics) && P == 1) L->C = take(sizeof(float) * (size_t)n * d);
     tc_make_layout(d, (int)P, n, c->quant_bits, c->in_dtype, &L->tc, take);
   }
   L->total = off;
@@ -197,7 +201,8 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   CQ_LAUNCHED(c, K_ROWNORM);
   const dim3 grid1(cdiv(d, SG_BN), cdiv(n, SG_BM), P);
   int per_problem;
-  if (g.quant_bits == 0) {
+  double* pdiag = g.diagnostics ? c->at<double>(c->L.part_diag) : nullptr;
+  if (g.quant_bits == 0 && !g.diagnostics) {
     rotate_target_exact_kernel<TIn, false><<<grid1, SG_THREADS, 0, c->stream>>>(
         X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, nullptr, part);
     CQ_LAUNCHED(c, K_ROTATE);
@@ -211,11 +216,12 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
         X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, rowmin, part);
     CQ_LAUNCHED(c, K_ROTATE);
     quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, rowmin, g.qs,
-                                                                    part);
+                                                                    part, pdiag);
     CQ_LAUNCHED(c, K_OTHER);
     per_problem = cdiv(n, 8);
   }
-  finalize_step_kernel<<<P, 256, 0, c->stream>>>(st, part, per_problem, n, 1.0 / std::sqrt((double)d));
+  finalize_step_kernel<<<P, 256, 0, c->stream>>>(st, part, per_problem, n, 1.0 / std::sqrt((double)d), pdiag,
+                                                 pdiag ? cdiv(n, 8) : 0);
   CQ_LAUNCHED(c, K_OTHER);
   const int S = c->L.acc_splits;
   accumulate_exact_kernel<TIn><<<dim3(cdiv(d, SG_BN), cdiv(d, SG_BM), P * S), SG_THREADS, 0, c->stream>>>(
@@ -404,6 +410,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
   g.qs = QuantSpec{cfg->quant_bits, cfg->quant_mode, cfg->clip_ratio > 0.f ? cfg->clip_ratio : 1.0f};
+  g.diagnostics = cfg->diagnostics;
   g.simt_ns = (g.mode == CONQUR_EXACT_F32);
   g.ns_max_steps = cfg->ns_max_steps > 0 ? std::min(cfg->ns_max_steps, 120) : 0;   // 0: set from the schedule below
   g.orth_tol = cfg->orth_tol > 0.f ? cfg->orth_tol : 1e-4f;
@@ -440,7 +447,8 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
     int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
                      c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
                      c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
-                     cfg->quant_bits ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), g.qs, &c->prof);
+                     (cfg->quant_bits || cfg->diagnostics) ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), g.qs,
+                     g.diagnostics, g.diagnostics ? c->at<double>(L.part_diag) : nullptr, &c->prof);
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);
@@ -534,6 +542,21 @@ extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tok
   CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
   const int rc = sync_status(c);
   for (int p = 0; p < P; ++p) { J_sum[p] = h[p].J; n_tokens[p] = h[p].N; }
+  return rc;
+}
+
+extern "C" int conqur_get_diagnostics(conqur_ctx* c, conqur_diagnostics* out) {
+  if (!c || !out || !c->cfg.diagnostics) return CONQUR_ERR_INVALID_ARG;
+  const int P = c->cfg.P;
+  for (int p = 0; p < P; ++p)
+    if (out[p].struct_size != sizeof(conqur_diagnostics)) return CONQUR_ERR_INVALID_ARG;
+  std::vector<DevState> h(P);
+  CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
+  const int rc = sync_status(c);
+  for (int p = 0; p < P; ++p) {
+    out[p].sum_pr_over_d = h[p].diag_pr; out[p].sum_rho = h[p].diag_rho;
+    out[p].qerr_num = h[p].diag_qnum; out[p].qerr_den = h[p].diag_qden; out[p].n_tokens = h[p].N;
+  }
   return rc;
 }
 

@@ -305,37 +305,78 @@ __global__ void __launch_bounds__(SG_THREADS) rotate_target_exact_kernel(
 
 // Quant mode, second pass (Appendix B, per token).  One warp per row: k = clamp(rint(acc * inv), klo, khi),
 // C' = sgn(k) * rnorm, objective partial = rnorm * delta * sum_j |k_j|.  Works in place: Y and C' share the buffer.
+// Per-row quantities of the second pass, shared by both modes.  `y` is the row's un-normalised product, r = 1/||x||.
+//   k       code of the fake-quantiser (or y itself when bits == 0)
+//   returns the target sign; accumulates the objective term and, if asked, the Section-4 diagnostics
+struct RowDiag { float s2, s4, mx, qe; };       // sums over the row of yh^2, yh^4, max |yh|, (yh - Q(yh))^2 with yh = y r
+__device__ __forceinline__ float second_pass_elem(float y, float r, const QuantSpec qs, const RowQuant rq, float& qsum,
+                                                  bool diag, RowDiag& dg) {
+  float k, qv;
+  if (qs.bits == 0) { k = y; qv = y; }
+  else { k = fminf(fmaxf(rintf(y * rq.inv), rq.klo), rq.khi); qv = k * rq.delta; }
+  qsum += fabsf(k);
+  if (diag) {
+    const float yh = y * r, t2 = yh * yh, e = (y - qv) * r;
+    dg.s2 += t2; dg.s4 = fmaf(t2, t2, dg.s4); dg.mx = fmaxf(dg.mx, fabsf(yh)); dg.qe = fmaf(e, e, dg.qe);
+  }
+  return sgnf(k);
+}
+// warp-reduce a row's diagnostics and turn them into the four per-row terms (valid in lane 0)
+__device__ __forceinline__ void row_diag_terms(RowDiag dg, float r, int d, bool live, double (&out)[4]) {
+  dg.s2 = warp_sum(dg.s2); dg.s4 = warp_sum(dg.s4); dg.qe = warp_sum(dg.qe); dg.mx = warp_max(dg.mx);
+  out[0] = out[1] = out[2] = out[3] = 0.0;
+  if (live && dg.s4 > 0.f) {
+    out[0] = (double)dg.s2 * (double)dg.s2 / ((double)d * (double)dg.s4);     // PR / d
+    out[1] = (double)dg.mx * (double)dg.mx / (double)dg.s2;                    // rho
+    const double x2 = 1.0 / ((double)r * (double)r);                           // ||x||^2
+    out[2] = (double)dg.qe * x2;                                               // ||y - Q(y)||^2, un-normalised
+    out[3] = x2;
+  }
+}
+
+// Second pass of the two-pass step (exact mode; Appendix B per token).  One warp per row; works in place: Y and C'
+// share the buffer.  part_diag (optional): 4 arrays of per-block partial sums of the diagnostics.
 static __global__ void __launch_bounds__(256) quant_target_kernel(float* __restrict__ YC, int64_t n, int d,
                                                            int64_t c_pstride, const float* __restrict__ rnorm,
                                                            int64_t rnorm_pstride,
                                                            const unsigned int* __restrict__ rowmax_ord,
                                                            const unsigned int* __restrict__ rowmin_ord, QuantSpec qs,
-                                                           double* __restrict__ partials /* per block */) {
+                                                           double* __restrict__ partials /* per block */,
+                                                           double* __restrict__ part_diag) {
   const int p = blockIdx.y;
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  double contrib = 0.0;
+  const bool diag = part_diag != nullptr;
+  double contrib = 0.0, dterm[4] = {0.0, 0.0, 0.0, 0.0};
   if (row < n) {
     const float r = rnorm[(int64_t)p * rnorm_pstride + row];
-    const RowQuant rq = row_quant(qs, ord2f(rowmax_ord[(int64_t)p * rnorm_pstride + row]),
-                                  ord2f(rowmin_ord[(int64_t)p * rnorm_pstride + row]), r > 0.f);
+    RowQuant rq{0.f, 1.f, 0.f, 0.f};
+    if (qs.bits) rq = row_quant(qs, ord2f(rowmax_ord[(int64_t)p * rnorm_pstride + row]),
+                                ord2f(rowmin_ord[(int64_t)p * rnorm_pstride + row]), r > 0.f);
+    const bool live = qs.bits ? (rq.inv > 0.f) : (r > 0.f);
     float* y = YC + (int64_t)p * c_pstride + row * d;
     float qsum = 0.f;
+    RowDiag dg{0.f, 0.f, 0.f, 0.f};
     for (int j = lane; j < d; j += 32) {
-      const float k = fminf(fmaxf(rintf(y[j] * rq.inv), rq.klo), rq.khi);
-      qsum += fabsf(k);
-      y[j] = (rq.inv > 0.f) ? sgnf(k) * r : 0.f;
+      const float sg = second_pass_elem(y[j], r, qs, rq, qsum, diag && live, dg);
+      y[j] = live ? sg * r : 0.f;
     }
     qsum = warp_sum(qsum);
-    contrib = (double)(r * rq.delta) * (double)qsum;
+    if (live) contrib = (double)(r * rq.delta) * (double)qsum;
+    if (diag) row_diag_terms(dg, r, d, live, dterm);
   }
-  __shared__ double red[8];
-  if (lane == 0) red[threadIdx.x >> 5] = contrib;
+  __shared__ double red[8][5];
+  if (lane == 0) {
+    red[threadIdx.x >> 5][0] = contrib;
+    for (int k = 0; k < 4; ++k) red[threadIdx.x >> 5][1 + k] = dterm[k];
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < 5) {
     double t = 0.0;
-    for (int w = 0; w < 8; ++w) t += red[w];
-    partials[(int64_t)p * gridDim.x + blockIdx.x] = t;
+    for (int w = 0; w < 8; ++w) t += red[w][threadIdx.x];
+    const int64_t nb = gridDim.x;
+    if (threadIdx.x == 0) partials[(int64_t)p * nb + blockIdx.x] = t;
+    else if (diag) part_diag[((int64_t)p * 4 + (threadIdx.x - 1)) * nb + blockIdx.x] = t;
   }
 }
 
@@ -387,18 +428,27 @@ static __global__ void splitk_reduce_add_kernel(float* __restrict__ M, const flo
 
 // Adds the step's objective partials (fixed order) and token counts to the running sums.
 static __global__ void finalize_step_kernel(DevState* st, const double* __restrict__ partials, int per_problem, int64_t n,
-                                     double inv_sqrt_d) {
+                                     double inv_sqrt_d, const double* __restrict__ part_diag = nullptr, int diag_blocks = 0) {
   const int p = blockIdx.x;
   __shared__ double red[8];
   double v = 0.0;
   for (int i = threadIdx.x; i < per_problem; i += 256) v += partials[(int64_t)p * per_problem + i];
   const double tot = block_sum_d<256>(v, red);
+  double dsum[4] = {0.0, 0.0, 0.0, 0.0};
+  if (part_diag) {
+    for (int k = 0; k < 4; ++k) {
+      double w = 0.0;
+      for (int i = threadIdx.x; i < diag_blocks; i += 256) w += part_diag[((int64_t)p * 4 + k) * diag_blocks + i];
+      dsum[k] = block_sum_d<256>(w, red);
+    }
+  }
   if (threadIdx.x == 0) {
     DevState* s = st + p;
     s->J += tot * inv_sqrt_d;
     s->N += n - s->step_skipped;
     s->n_skipped += s->step_skipped;
     s->step_skipped = 0;
+    if (part_diag) { s->diag_pr += dsum[0]; s->diag_rho += dsum[1]; s->diag_qnum += dsum[2]; s->diag_qden += dsum[3]; }
   }
 }
 
@@ -637,6 +687,7 @@ static __global__ void ns_commit_state_kernel(DevState* st) {
     s->last_N = s->N;
     s->J = 0.0;
     s->N = 0;
+    s->diag_pr = s->diag_rho = s->diag_qnum = s->diag_qden = 0.0;
     s->updates += 1;
     s->last_orth = s->e_max;
     s->last_fro = s->e_fro;

@@ -830,48 +830,53 @@ __global__ void split_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* 
   }
 }
 
-// Quant mode, second pass for the tensor-core mode: Y (fp32, row-major) -> C' (bf16, row-major) + objective partials.
+// Second pass of the two-pass step in tensor-core mode (quant modes, or diagnostics): Y (fp32, row-major) ->
+// C' (bf16, row-major) + objective partials (+ diagnostics partials).
 __global__ void __launch_bounds__(256) quant_target_bf16_kernel(const float* __restrict__ Y, int64_t n, int d,
                                                                 const float* __restrict__ rnorm,
                                                                 const unsigned int* __restrict__ rowmax_ord,
                                                                 const unsigned int* __restrict__ rowmin_ord,
                                                                 QuantSpec qs, double* __restrict__ partials,
-                                                                __nv_bfloat16* __restrict__ Cp) {
+                                                                __nv_bfloat16* __restrict__ Cp, double* __restrict__ part_diag) {
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  double contrib = 0.0;
+  const bool diag = part_diag != nullptr;
+  double contrib = 0.0, dterm[4] = {0.0, 0.0, 0.0, 0.0};
   if (row < n) {
     const float r = rnorm[row];
-    const RowQuant rq = row_quant(qs, ord2f(rowmax_ord[row]), ord2f(rowmin_ord[row]), r > 0.f);
-    const bool live = rq.inv > 0.f;
+    RowQuant rq{0.f, 1.f, 0.f, 0.f};
+    if (qs.bits) rq = row_quant(qs, ord2f(rowmax_ord[row]), ord2f(rowmin_ord[row]), r > 0.f);
+    const bool live = qs.bits ? (rq.inv > 0.f) : (r > 0.f);
     const float* y = Y + row * (int64_t)d;
     __nv_bfloat16* c = Cp + row * (int64_t)d;
     float qsum = 0.f;
+    RowDiag dg{0.f, 0.f, 0.f, 0.f};
     for (int j = lane * 4; j < d; j += 128) {
       const float4 t = *reinterpret_cast<const float4*>(y + j);
       const float in[4] = {t.x, t.y, t.z, t.w};
-      uint32_t b[4];
+      float sg[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float k = fminf(fmaxf(rintf(in[e] * rq.inv), rq.klo), rq.khi);
-        qsum += fabsf(k);
-        b[e] = bf16_bits(live ? sgnf(k) * r : 0.f);
-      }
+      for (int e = 0; e < 4; ++e) sg[e] = live ? second_pass_elem(in[e], r, qs, rq, qsum, diag, dg) * r : 0.f;
       uint2 o;
-      o.x = b[0] | (b[1] << 16);
-      o.y = b[2] | (b[3] << 16);
+      o.x = bf16x2_pack(sg[0], sg[1]);
+      o.y = bf16x2_pack(sg[2], sg[3]);
       *reinterpret_cast<uint2*>(c + j) = o;
     }
     qsum = warp_sum(qsum);
-    contrib = (double)(r * rq.delta) * (double)qsum;
+    if (live) contrib = (double)(r * rq.delta) * (double)qsum;
+    if (diag) row_diag_terms(dg, r, d, live, dterm);
   }
-  __shared__ double red[8];
-  if (lane == 0) red[threadIdx.x >> 5] = contrib;
+  __shared__ double red[8][5];
+  if (lane == 0) {
+    red[threadIdx.x >> 5][0] = contrib;
+    for (int k = 0; k < 4; ++k) red[threadIdx.x >> 5][1 + k] = dterm[k];
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < 5) {
     double t = 0.0;
-    for (int w = 0; w < 8; ++w) t += red[w];
-    partials[blockIdx.x] = t;
+    for (int w = 0; w < 8; ++w) t += red[w][threadIdx.x];
+    if (threadIdx.x == 0) partials[blockIdx.x] = t;
+    else if (diag) part_diag[(int64_t)(threadIdx.x - 1) * gridDim.x + blockIdx.x] = t;
   }
 }
 
@@ -890,6 +895,8 @@ struct TcHost {
   float *R, *M, *Xa, *Xb, *E, *B, *rnorm, *Y;
   unsigned* rowmax;
   QuantSpec qs;
+  int diagnostics;                           // 1: every step takes the two-pass route and gathers the Section-4 diagnostics
+  double* part_diag;
   DevState* st;
   double* part_d;
   float* part_f;
@@ -1097,10 +1104,10 @@ inline int tc_query_pair_clusters() {
 
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
                    float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
-                   float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, Prof* prof) {
+                   float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, int diagnostics, double* part_diag, Prof* prof) {
   h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
   h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
-  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->qs = qs; h->prof = prof; h->ns_k = -1;
+  h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->qs = qs; h->diagnostics = diagnostics; h->part_diag = part_diag; h->prof = prof; h->ns_k = -1;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
   cudaDeviceProp prop;
@@ -1170,7 +1177,7 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
   TcGemmArgs g = tc_args(h, (int)n, d, d);
   g.rnorm = h.rnorm;
   int per_problem;
-  if (h.quant_bits == 0) {
+  if (h.quant_bits == 0 && !h.diagnostics) {
     g.outH = Cp; g.ldh = d;
     rc = tc_launch_n<false, true, TC_EPI_ROTATE>(h, s, tmXs_k, h.tmRb_mn, g);
     if (rc) return rc;
@@ -1182,12 +1189,13 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
     g.outF = h.Y; g.ldo = d; g.rowmax = h.rowmax; g.rowmin = rowmin;
     rc = tc_launch_n<false, true, TC_EPI_ROTATE_Q>(h, s, tmXs_k, h.tmRb_mn, g);
     if (rc) return rc;
-    quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, rowmin, h.qs, h.part_d, Cp);
+    quant_target_bf16_kernel<<<rb, 256, 0, s>>>(h.Y, n, d, h.rnorm, h.rowmax, rowmin, h.qs, h.part_d, Cp,
+                                                h.diagnostics ? h.part_diag : nullptr);
     if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
     if (h.prof) h.prof->count(K_OTHER);
     per_problem = rb;
   }
-  finalize_step_kernel<<<1, 256, 0, s>>>(h.st, h.part_d, per_problem, n, isd);
+  finalize_step_kernel<<<1, 256, 0, s>>>(h.st, h.part_d, per_problem, n, isd, h.diagnostics ? h.part_diag : nullptr, rb);
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_OTHER);
   TcGemmArgs a = tc_args(h, d, d, (int)n);

@@ -674,6 +674,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     if (threadIdx.x == 0) {
       if (converged) {
         s->last_J = s->J; s->last_N = s->N; s->J = 0.0; s->N = 0; s->updates += 1;
+        s->diag_pr = s->diag_rho = s->diag_qnum = s->diag_qden = 0.0;
         s->last_orth = s->e_max; s->last_fro = s->e_fro;
       } else {
         s->status_flags |= STATUS_FLAG_NS_FAILED;

@@ -245,3 +245,42 @@ def test_zero_point_quant_mode_int4(d, n, clip):
     assert rep["N_equal"] and rep["J_rel"] <= 1e-5, rep          # a tie in the zero-point moves a clamped code by one
     assert rep["M_rel_tie_aware"] <= T["M"] and rep["flips_outside_band"] == 0 and rep["flip_frac"] < 1e-3, rep
     _check_update(ctx, m, r)
+
+
+@pytest.mark.parametrize("mode", ["exact", "tc"])
+@pytest.mark.parametrize("quant", [(0, "sym", 1.0), (4, "sym", 1.0), (4, "zp", 0.9)])
+def test_section4_diagnostics(mode, quant):
+    """Participation ratio, dynamic-range ratio and relative quantisation error gathered by the step (two batches,
+    one skipped row) against the oracle's definition; reset by the update."""
+    from paper_2605_10793_b200 import binding as B
+    bits, qmode, clip = quant
+    d, n = 256, 700
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2)
+    r0 = I.initial_rotation(w)
+    ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode=mode, quant_bits=bits, quant_mode=qmode, clip_ratio=clip,
+                    diagnostics=True)
+    ctx.set_R(_dev(r0, "f32"))
+    ref = np.zeros(5)
+    orc = O.OpuOracle(d, r0.astype(np.float64), quant_bits=bits, quant_mode=qmode, clip_ratio=clip)
+    for b in range(2):
+        x = I.batch(w, b).copy()
+        if b == 1:
+            x[11] = 0.0
+        ctx.step(_dev(x, "bf16"))
+        ref += np.array(O.token_diagnostics(x, r0.astype(np.float64), bits, qmode, clip))
+        orc.step(x.astype(np.float64))
+    dg = ctx.get_diagnostics()[0]
+    j, nn = ctx.get_objective(check=False)
+    tol = 1e-5 if mode == "exact" else 2e-3
+    assert dg["n_tokens"] == ref[4] == nn
+    assert abs(j - orc.J) / orc.J <= (1e-5 if mode == "exact" else 1e-3)       # the two-pass route gives the same objective
+    assert abs(dg["sum_pr_over_d"] - ref[0]) / ref[0] <= tol, (dg, ref)
+    assert abs(dg["sum_rho"] - ref[1]) / ref[1] <= tol, (dg, ref)
+    assert abs(dg["qerr_den"] - ref[3]) / ref[3] <= tol
+    if bits:
+        assert abs(dg["qerr_num"] / dg["qerr_den"] - ref[2] / ref[3]) / (ref[2] / ref[3]) <= (1e-4 if mode == "exact" else 5e-3), (dg, ref)
+    else:
+        assert dg["qerr_num"] == 0.0
+    ctx.update()
+    dg = ctx.get_diagnostics()[0]
+    assert dg["sum_pr_over_d"] == 0.0 and dg["qerr_den"] == 0.0 and dg["n_tokens"] == 0
