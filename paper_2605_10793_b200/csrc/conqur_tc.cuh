@@ -887,6 +887,7 @@ struct TcLayout {
 
 struct TcHost {
   int d, P, quant_bits, num_sms;
+  int device;                                // CUDA device the context was created on
   int pair_clusters;                         // CTA pairs that can be co-resident (0: single-CTA kernels only)
   float e1_tau;                              // residual product runs one pass while mean sigma^2 of the iterate is below this
   int64_t n_max;
@@ -1026,11 +1027,11 @@ template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR, int NA = 1, int NB =
 inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
   using Cfg = TcCfg<BN, PAIR, NA, NB>;
   auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, PAIR, NA, NB>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int attr_dev_mask = 0;                    // the attribute is per device
+  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_set = true;
+    attr_dev_mask |= 1 << (h.device & 31);
   }
   const TcVariant v{PAIR, Cfg::TILE_M, BN};
   const int tiles = tc_tiles(v, g.M, g.N, g.sym);
@@ -1117,6 +1118,7 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
     return CONQUR_ERR_UNSUPPORTED;
   }
   h->num_sms = prop.multiProcessorCount;
+  h->device = dev;
   h->pair_clusters = tc_query_pair_clusters();
   h->e1_tau = 2e-3f;
   if (const char* env = std::getenv("CONQUR_NS_E1_TAU")) h->e1_tau = (float)std::atof(env);   // tuning knob
@@ -1287,6 +1289,7 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
   if (prop.major != 10) return CONQUR_ERR_UNSUPPORTED;
   h.num_sms = prop.multiProcessorCount;
+  h.device = dev;
   h.pair_clusters = tc_query_pair_clusters();
   const uint64_t mul = split ? 2 : 1;
   CUtensorMap ta, tb;

@@ -339,11 +339,11 @@ inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_
 
 // One streamed batch for all P problems.  X: device, bf16 or fp32 (fp32 is first rounded into the staging copy).
 inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int attr_dev_mask = 0;                    // the attribute is per device
+  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
     if (cudaFuncSetAttribute(tcb_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCB_SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_set = true;
+    attr_dev_mask |= 1 << (h.device & 31);
   }
   const void* src = X;
   int64_t src_ld = ld, src_ps = pstride;
@@ -696,11 +696,11 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
 }
 
 inline int tcb_update(TcHost& h, cudaStream_t s, const NsControlParams& ncp, float prior_rel, float margin) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int attr_dev_mask = 0;                    // the attribute is per device
+  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
     if (cudaFuncSetAttribute(tcb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCBU_SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_set = true;
+    attr_dev_mask |= 1 << (h.device & 31);
   }
   TcbUpdArgs g{};
   g.P = h.P; g.M = h.M; g.R = h.R; g.st = h.st; g.ncp = ncp; g.prior_rel = prior_rel; g.margin = margin;
