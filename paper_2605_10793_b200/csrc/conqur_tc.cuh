@@ -257,6 +257,8 @@ struct TcAux {
   float red_t[8];
 };
 
+static_assert(sizeof(TcAux) <= 1024, "TcCfg::AUX_BYTES");
+
 // Bounded wait.  Returns false when the wait was abandoned (timeout here, or another role aborted).
 __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                         long long limit = TC_WAIT_LIMIT) {

@@ -23,7 +23,8 @@ constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = tw
 constexpr int TCB_XSTAGES = 3;
 constexpr int TCB_THREADS = 320;                 // 2 + 8 warps
 constexpr int TCB_EPI_THREADS = 256;
-constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + 1024 + 1024;
+constexpr int TCB_AUX_BYTES = 4096;
+constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + TCB_AUX_BYTES + 1024;
 
 struct TcbAux {
   uint64_t rfull, rempty, mfull, mempty;
@@ -34,7 +35,10 @@ struct TcbAux {
   double red_d[8];
   int red_i[8];
   int red_f[8];
+  float ss_x[2][2][128];     // [tile parity][column half][row]: half-row sums of squares exchanged between the two warps of a row
 };
+
+static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
 
 struct TcbStepArgs {
   int n, P;
@@ -180,19 +184,24 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int yb = it & 1, xs = it % TCB_XSTAGES;
         const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
-        // a1: row norm from the tile in shared memory (both warps of a row form the full sum)
+        // a1: row norm from the tile in shared memory: each of the row's two warps sums its half of the columns and
+        // they swap the halves (named barriers 2..5, one per TMEM lane quarter; both warps have just passed the
+        // same wait, so both arrive).  The two halves are added in a fixed order.
         uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
-        float ss = 0.f;
+        float ssh = 0.f;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, c));
+        for (int c = 0; c < 8; ++c) {
+          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, half * 8 + c));
           const uint32_t u[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float a = __uint_as_float(u[e] << 16), b = __uint_as_float(u[e] & 0xffff0000u);
-            ss = fmaf(a, a, ss); ss = fmaf(b, b, ss);
+            ssh = fmaf(a, a, ssh); ssh = fmaf(b, b, ssh);
           }
         }
+        aux->ss_x[it & 1][half][r] = ssh;
+        asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
+        const float ss = aux->ss_x[it & 1][0][r] + aux->ss_x[it & 1][1][r];
         const bool valid = (t * 128 + r) < g.n;
         const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
         if (valid && !good) {
@@ -227,17 +236,28 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
           uint32_t w[16];
+          if (g.qs.bits > 0) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a = v[2 * i], b = v[2 * i + 1];
-            if (g.qs.bits > 0) {
-              a = fminf(fmaxf(rintf(a * rq.inv), rq.klo), rq.khi);
-              b = fminf(fmaxf(rintf(b * rq.inv), rq.klo), rq.khi);
+            for (int i = 0; i < 16; ++i) {
+              const float a = fminf(fmaxf(rintf(v[2 * i] * rq.inv), rq.klo), rq.khi);
+              const float b = fminf(fmaxf(rintf(v[2 * i + 1] * rq.inv), rq.klo), rq.khi);
+              acc_t += fabsf(a) + fabsf(b);
+              const uint32_t lo = (a == 0.f) ? 0u : (rn_bits | ((__float_as_uint(a) >> 16) & 0x8000u));
+              const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
+              w[i] = live ? (lo | (hi << 16)) : 0u;
             }
-            acc_t += fabsf(a) + fabsf(b);
-            const uint32_t lo = (a == 0.f) ? 0u : (rn_bits | ((__float_as_uint(a) >> 16) & 0x8000u));
-            const uint32_t hi = (b == 0.f) ? 0u : (rn_bits | ((__float_as_uint(b) >> 16) & 0x8000u));
-            w[i] = live ? (lo | (hi << 16)) : 0u;
+          } else {
+            // two elements per instruction: sign bits and a non-zero mask from the packed bf16 pair
+            const uint32_t rn2 = live ? (rn_bits | (rn_bits << 16)) : 0u;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float a = v[2 * i], b = v[2 * i + 1];
+              acc_t += fabsf(a) + fabsf(b);
+              const uint32_t pk = bf16x2_pack(a, b);
+              const uint32_t mag = pk & 0x7fff7fffu;
+              const uint32_t nz = (((mag + 0x7fff7fffu) >> 15) & 0x00010001u) * 0xffffu;     // 0xffff per non-zero half
+              w[i] = (rn2 | (pk & 0x80008000u)) & nz;
+            }
           }
 #pragma unroll
           for (int k = 0; k < 4; ++k)
@@ -409,6 +429,8 @@ struct TcbUpdAux {
   DevState state;                    // the problem's state while it is being iterated (written back once at the end)
   SchedEntry sched[NS_SCHED_MAX];    // the polynomial schedule (copied once per CTA)
 };
+
+static_assert(sizeof(TcbUpdAux) <= 4096, "the control block must fit its reserved shared memory");
 
 struct TcbUpdArgs {
   int P;
