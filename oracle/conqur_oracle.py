@@ -29,6 +29,16 @@ What each function follows:
                       quantisation error ||X R - Q(X R)||_F^2 / ||X||_F^2 (on un-normalised rows)
   polar_svd           Section 3.3, C = U Sigma V^T, R <- U V^T
   OpuOracle.update    Section 3.3 / Algorithm 1: R replaced, statistics reset
+  run_algorithm1      Algorithm 1: per mini-batch, the attention-input and MLP-input activations of
+                      every block accumulate into the shared R_1 problem, every head of every
+                      block's o_proj input is its own d_h x d_h problem updated at once, and R_1 is
+                      updated at the end of the mini-batch
+  fold_weight         Appendix A: X W^T = (X R)(W R)^T, so a layer reading rotated activations
+                      takes W R, and a layer writing into the rotated space takes R^T W
+                      (block-diagonal R for the per-head rotations)
+  hadamard_matrix / hadamard_rows
+                      the fixed online transforms R_3, R_4 of Appendix A: the Sylvester
+                      (Walsh-Hadamard) matrix H_d, applied as x H_d / sqrt(d)
 
 Readings where the paper is silent (kept identical in the CUDA library):
   * sign(0) = 0: a zero coordinate adds nothing to the target or objective.
@@ -261,3 +271,84 @@ def run_batched(d, xs, r0s, quant_bits=0, prior_rel=0.0):
         orc.update()
         out.append({"R": orc.R, "J": j, "N": n, "M": m})
     return out
+
+
+# ----------------------------------------------------------------------------- Algorithm 1, Appendix A
+def run_algorithm1(d, n_heads, d_head, n_layers, minibatches, r1_0, r2_0, quant_bits=0, prior_rel=0.0,
+                   quant_mode="sym", clip_ratio=1.0):
+    """Algorithm 1 on given activations.
+
+    minibatches: iterable; each item is a list over the L blocks of dicts with the activations collected at
+    the three calibration sites of the block: "attn" and "mlp" (n x d, inputs of the attention and MLP
+    sublayers) and "o" (n x n_heads*d_head, input of the attention output projection, head h in columns
+    h*d_head .. (h+1)*d_head).  r1_0: d x d; r2_0: L x n_heads x d_head x d_head.
+    Returns (R_1, R_2 as L x n_heads x d_head x d_head, log) where log holds, per mini-batch, the objective
+    and token count of the R_1 problem and of every head problem before its update.
+    """
+    o1 = OpuOracle(d, r1_0, quant_bits, prior_rel, quant_mode, clip_ratio)
+    r2 = np.array(r2_0, dtype=np.float64)
+    assert r2.shape == (n_layers, n_heads, d_head, d_head)
+    log = []
+    for sites in minibatches:
+        assert len(sites) == n_layers
+        rec = {"J2": np.zeros((n_layers, n_heads)), "N2": np.zeros((n_layers, n_heads), dtype=np.int64)}
+        for ell in range(n_layers):
+            o1.step(sites[ell]["attn"])                           # accumulate into X_1
+            o1.step(sites[ell]["mlp"])
+            xo = np.asarray(sites[ell]["o"], dtype=np.float64)
+            for h in range(n_heads):                              # R_{2,ell} is block diagonal: one problem per head
+                oh = OpuOracle(d_head, r2[ell, h], quant_bits, prior_rel, quant_mode, clip_ratio)
+                oh.step(xo[:, h * d_head:(h + 1) * d_head])
+                rec["J2"][ell, h], rec["N2"][ell, h] = oh.J, oh.N
+                oh.update()                                       # R_{2,ell} <- OPU(R_{2,ell}, X_o)
+                r2[ell, h] = oh.R
+        rec["J1"], rec["N1"] = o1.J, o1.N
+        o1.update()                                               # R_1 <- OPU(R_1, X_1)
+        log.append(rec)
+    return o1.R, r2, log
+
+
+def block_diag_rotation(blocks):
+    """Dense (k*b) x (k*b) matrix with the given b x b blocks on its diagonal."""
+    blocks = np.asarray(blocks, dtype=np.float64)
+    if blocks.ndim == 2:
+        return blocks
+    k, b, _ = blocks.shape
+    out = np.zeros((k * b, k * b))
+    for i in range(k):
+        out[i * b:(i + 1) * b, i * b:(i + 1) * b] = blocks[i]
+    return out
+
+
+def fold_weight(w, r_blocks, side):
+    """Appendix A.  w: d_out x d_in weight of a layer y = x W^T.
+
+    side "input":  the layer's input is rotated (x_hat = x R):              W' = W R
+    side "output": the layer's output lives in the rotated space (y R):     W' = R^T W
+    r_blocks: one square matrix, or a stack of blocks forming a block-diagonal R.
+    """
+    w = np.asarray(w, dtype=np.float64)
+    r = block_diag_rotation(r_blocks)
+    if side == "input":
+        return w @ r
+    if side == "output":
+        return r.T @ w
+    raise ValueError(side)
+
+
+def hadamard_matrix(d):
+    """Sylvester construction: H_1 = [1], H_2m = [[H_m, H_m], [H_m, -H_m]] (entries +-1, H H^T = d I)."""
+    d = int(d)
+    if d < 1 or d & (d - 1):
+        raise ValueError("d must be a power of two")
+    h = np.ones((1, 1))
+    while h.shape[0] < d:
+        h = np.block([[h, h], [h, -h]])
+    return h
+
+
+def hadamard_rows(x):
+    """Each row times the orthonormal Walsh-Hadamard matrix: x H_d / sqrt(d) (the online R_3 / R_4 transform)."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    return x @ hadamard_matrix(d) / np.sqrt(d)

@@ -195,3 +195,69 @@ def stream(w: Workload):
 
 def storage_bytes_per_element(w: Workload) -> int:
     return 2 if w.dtype == "bf16" else 4
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1: calibration sites of a synthetic transformer
+# ----------------------------------------------------------------------------
+
+
+@dataclass(frozen=True)
+class SiteModel:
+    """Shapes of a pre-norm transformer as Algorithm 1 sees it, and the recipes of its site activations.
+
+    Per mini-batch every block yields three activation matrices: the attention input and the MLP input
+    (n x d, residual-stream statistics: recipe ``resid``) and the input of the attention output projection
+    (n x n_heads*d_head, head h in columns h*d_head..(h+1)*d_head: recipe ``head`` per head).
+    """
+
+    name: str
+    index: int
+    d: int
+    n_heads: int
+    d_head: int
+    n_layers: int
+    n: int                 # tokens per mini-batch (sequences x sequence length)
+    n_minibatches: int
+    resid: Workload
+    head: Workload
+    d_ff: int = 0          # MLP width, for the weight-folding shapes
+
+
+def _site_model(name, index, d, n_heads, d_head, n_layers, n, n_minibatches, dtype, d_ff) -> SiteModel:
+    resid = Workload(name + "_resid", 20 + index, d, n, n_minibatches, 1, dtype, "student_t3", max(1, d // 256), 100.0,
+                     0.5, 1, 1000.0, "hadamard")
+    head = Workload(name + "_head", 40 + index, d_head, n, n_minibatches, 1, dtype, "student_t3", 2, 30.0, 0.5, 0, 1.0,
+                    "hadamard")
+    return SiteModel(name, index, d, n_heads, d_head, n_layers, n, n_minibatches, resid, head, d_ff)
+
+
+SITE_MODELS: Dict[str, SiteModel] = {
+    # a model the float64 oracle runs in seconds: 2 blocks, 2 heads of 128, residual width 256
+    "a1_small": _site_model("a1_small", 0, 256, 2, 128, 2, 640, 2, "bf16", 512),
+    # 8B-class shapes: 32 blocks, residual width 4096, 32 heads of 128, two 2048-token sequences per mini-batch
+    "a1_8b": _site_model("a1_8b", 1, 4096, 32, 128, 32, 4096, 1, "bf16", 14336),
+}
+
+
+def site_activations(a: SiteModel, minibatch: int, layer: int) -> Dict[str, np.ndarray]:
+    """The three activation matrices of block ``layer`` for one mini-batch (float32, exact in the storage type)."""
+    b_attn = (minibatch * a.n_layers + layer) * 2
+    attn = batch(a.resid, b_attn)
+    mlp = batch(a.resid, b_attn + 1)
+    heads = [batch(a.head, minibatch * a.n_layers + layer, problem=h) for h in range(a.n_heads)]
+    return {"attn": attn, "mlp": mlp, "o": np.concatenate(heads, axis=1)}
+
+
+def site_initial_rotations(a: SiteModel):
+    """(R_1 as d x d, R_2 as n_layers x n_heads x d_head x d_head), float32."""
+    r1 = initial_rotation(a.resid)
+    r2 = np.stack([np.stack([initial_rotation(a.head, problem=l * a.n_heads + h) for h in range(a.n_heads)])
+                   for l in range(a.n_layers)])
+    return r1, r2
+
+
+def random_weight(seed: int, rows: int, cols: int) -> np.ndarray:
+    """A linear layer's weight (rows = outputs, cols = inputs), float32, N(0, 1/cols) entries."""
+    rng = np.random.Generator(np.random.PCG64(9_000_000 + seed))
+    return (rng.standard_normal((rows, cols)) / np.sqrt(cols)).astype(np.float32)
