@@ -282,6 +282,50 @@ int conqur_debug_wait_timeout(void* scratch_dev, int64_t limit_cycles, void* cud
 int conqur_objective_noalloc(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ld,
                              const float* R_dev, double* J_out_dev, int64_t* N_out_dev, void* cuda_stream);
 
+/*
+ * Appendix A, rotation invariance: with activations rotated as X_hat = X R, a linear layer y = x W^T
+ * (W: rows = outputs, cols = inputs, row-major) keeps its function when the rotation is absorbed into W:
+ *   CONQUR_FOLD_INPUT   the layer READS rotated activations (q/k/v/up/gate projections for R_1; o_proj for R_2):
+ *                       W' = W R          since X W^T = (X R)(W R)^T
+ *   CONQUR_FOLD_OUTPUT  the layer WRITES into the rotated space (o_proj and down projection for R_1, whose outputs
+ *                       join the rotated residual stream; the value projection for R_2):
+ *                       W' = R^T W        since (X W^T) R = X (R^T W)^T
+ * R is block diagonal with square blocks of size `block` (one full rotation when block equals the folded
+ * dimension; block = d_h for the per-head rotations R_2): R_dev holds the blocks one after another, each
+ * block x block fp32 row-major.  The folded dimension (cols for INPUT, rows for OUTPUT) must be a multiple of
+ * block.
+ *   W_dev / out_dev   device fp32, rows x cols, row strides ldw / ldo elements (>= cols); out_dev must not
+ *                     overlap W_dev
+ *   mode              CONQUR_EXACT_F32: fp32 CUDA-core product.
+ *                     CONQUR_TC_BF16: for one full rotation (block == folded dimension, a multiple of 128;
+ *                     rows % 8 == 0 for INPUT, cols % 32 == 0 for OUTPUT; ldw, ldo multiples of 4; 16-byte
+ *                     aligned pointers) both operands are split into bf16 hi + lo and the product is taken
+ *                     in three tensor-core passes (hi hi, hi lo, lo hi) with fp32 accumulation, relative
+ *                     error about 2^-16; shapes outside these limits return CONQUR_ERR_UNSUPPORTED.
+ *                     Block-diagonal folds (block < folded dimension) use the fp32 product in either mode.
+ *   scratch_dev       device memory, 256-byte aligned, >= conqur_fold_scratch_bytes(...) bytes (returns -1 for
+ *                     invalid arguments); owned by the caller, free to reuse after the call returns
+ * Synchronises the stream and returns the status (CONQUR_ERR_TIMEOUT if a bounded device wait expired).
+ */
+enum { CONQUR_FOLD_INPUT = 0, CONQUR_FOLD_OUTPUT = 1 };
+int64_t conqur_fold_scratch_bytes(int32_t rows, int32_t cols, int32_t block, int32_t side, int32_t mode);
+int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows, int32_t cols, const float* R_dev,
+                       int32_t block, int32_t side, int32_t mode, float* out_dev, int64_t ldo, void* scratch_dev,
+                       int64_t scratch_bytes, void* cuda_stream);
+
+/*
+ * The fixed online rotations R_3 / R_4 of Appendix A: every row times the orthonormal Walsh-Hadamard matrix,
+ *   y = x H_d / sqrt(d),   H_d the Sylvester matrix, H[i][j] = (-1)^popcount(i & j),
+ * computed with log2(d) butterfly stages in fp32 (no matrix is formed).  d a power of two, 4 <= d <= 8192.
+ *   X_dev   device, n rows of d elements of in_dtype (CONQUR_F32 | CONQUR_BF16), row stride ldx elements
+ *   Y_dev   device, n rows of d elements of out_dtype, row stride ldy; may be X_dev itself (same type and
+ *           stride): every row is read completely before it is written
+ *   ldx, ldy multiples of 4; pointers aligned to 4 elements.
+ * Enqueued on the stream; not synchronised.  Invalid arguments return CONQUR_ERR_INVALID_ARG and do nothing.
+ */
+int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,
+                         int32_t out_dtype, int64_t ldy, void* cuda_stream);
+
 const char* conqur_strerror(int status);
 
 #ifdef __cplusplus

@@ -1,0 +1,95 @@
+"""Algorithm 1 (online calibration of the shared and the per-block rotations) as a sequence of library calls.
+
+One context holds the shared rotation R_1: the attention-input and MLP-input activations of every block are
+accumulated into it (`conqur_step`) and it is updated once per mini-batch (`conqur_update`).  Every block has
+one batched context for R_{2,l}: its n_heads diagonal blocks are independent d_head x d_head problems fed from
+the head-interleaved o_proj input in one `conqur_step_batched` call and updated right away.
+
+This file only sequences calls and moves pointers; all arithmetic runs in the library's kernels.  Weight
+folding (Appendix A) for one transformer block is at the end.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+from . import binding as B
+
+
+class Calibrator:
+    def __init__(self, d: int, n_heads: int, d_head: int, n_layers: int, n_max: int, *, in_dtype="bf16", mode="tc",
+                 quant_bits=0, quant_mode="sym", clip_ratio=0.0, prior_rel=0.0, record: Optional[str] = None):
+        """n_max: most tokens in one activation matrix.  record: None | "objective" | "full" (also keeps each
+        cross-covariance, read before its update; both synchronise and are meant for tests and logging)."""
+        kw = dict(in_dtype=in_dtype, mode=mode, quant_bits=quant_bits, quant_mode=quant_mode, clip_ratio=clip_ratio,
+                  prior_rel=prior_rel)
+        self.d, self.n_heads, self.d_head, self.n_layers = d, n_heads, d_head, n_layers
+        self.ctx1 = B.Context(d=d, n_max=n_max, **kw)
+        self.ctx2: List[B.Context] = [B.Context(d=d_head, n_max=n_max, batch=n_heads, **kw) for _ in range(n_layers)]
+        self.record = record
+        self.log: List[Dict] = []
+        self._cur: Dict = {}
+
+    def set_rotations(self, r1, r2):
+        """r1: (d, d); r2: (n_layers, n_heads, d_head, d_head); fp32 CUDA tensors."""
+        self.ctx1.set_R(r1.contiguous())
+        for l, c in enumerate(self.ctx2):
+            c.set_R(r2[l].contiguous())
+
+    def collect(self, layer: int, x_attn, x_mlp, x_o):
+        """The body of Algorithm 1's loop over blocks for block `layer`: both residual-stream sites go into the R_1
+        statistics; R_{2,layer} <- OPU(R_{2,layer}, X_o).  x_o: (n, n_heads*d_head), head h in columns h*d_head.."""
+        self.ctx1.step(x_attn)
+        self.ctx1.step(x_mlp)
+        c = self.ctx2[layer]
+        assert x_o.shape[1] == self.n_heads * self.d_head and x_o.stride(1) == 1
+        c.step_batched(x_o, x_o.shape[0], x_o.stride(0), self.d_head)
+        if self.record:
+            j, n = c.get_objective()
+            rec = self._cur.setdefault("heads", {})
+            rec[layer] = {"J": j.copy(), "N": n.copy()}
+            if self.record == "full":
+                rec[layer]["M"] = c.get_M().cpu().numpy()
+        c.update()
+
+    def end_minibatch(self):
+        """R_1 <- OPU(R_1, X_1) with everything accumulated since the last call."""
+        if self.record:
+            j, n = self.ctx1.get_objective()
+            self._cur["J1"], self._cur["N1"] = j, n
+            if self.record == "full":
+                self._cur["M1"] = self.ctx1.get_M().cpu().numpy()
+            self.log.append(self._cur)
+            self._cur = {}
+        self.ctx1.update()
+
+    def rotations(self):
+        """(R_1 (d, d), R_2 (n_layers, n_heads, d_head, d_head)) as fp32 CUDA tensors."""
+        import torch
+        return self.ctx1.get_R(), torch.stack([c.get_R().reshape(self.n_heads, self.d_head, self.d_head) for c in self.ctx2])
+
+    def close(self):
+        self.ctx1.close()
+        for c in self.ctx2:
+            c.close()
+
+
+# which side of which projection absorbs which rotation (Appendix A)
+FOLD_PLAN = {
+    "q": [("input", "r1")], "k": [("input", "r1")], "up": [("input", "r1")], "gate": [("input", "r1")],
+    "v": [("input", "r1"), ("output", "r2")],
+    "o": [("input", "r2"), ("output", "r1")],
+    "down": [("output", "r1")],
+}
+
+
+def fold_block(weights: Dict[str, "object"], r1, r2_layer, mode: str = "tc") -> Dict[str, "object"]:
+    """Fold R_1 and one block's R_2 into that block's projection weights.
+
+    weights: name -> fp32 CUDA tensor (out_features, in_features) for any of q, k, v, o, up, gate, down (the RMSNorm
+    scales already merged into the projections that follow them).  r2_layer: (n_heads, d_head, d_head)."""
+    out = {}
+    for name, w in weights.items():
+        for side, which in FOLD_PLAN[name]:
+            w = B.conqur_fold_weight(w, r1 if which == "r1" else r2_layer, side, mode)
+        out[name] = w
+    return out

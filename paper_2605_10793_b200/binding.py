@@ -19,13 +19,14 @@ _lib = None
 CONQUR_F32, CONQUR_BF16 = 0, 1
 CONQUR_EXACT_F32, CONQUR_TC_BF16 = 0, 1
 CONQUR_QUANT_SYMMETRIC, CONQUR_QUANT_ZEROPOINT = 0, 1
+CONQUR_FOLD_INPUT, CONQUR_FOLD_OUTPUT = 0, 1
 
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
-    "conqur_get_diagnostics",
+    "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows",
     "conqur_strerror",
 ]
 
@@ -121,6 +122,12 @@ def load() -> C.CDLL:
     lib.conqur_get_diagnostics.argtypes = [vp, C.POINTER(conqur_diagnostics)]
     lib.conqur_debug_wait_timeout.restype = C.c_int
     lib.conqur_debug_wait_timeout.argtypes = [vp, i64, vp]
+    lib.conqur_fold_scratch_bytes.restype = i64
+    lib.conqur_fold_scratch_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.conqur_fold_weight.restype = C.c_int
+    lib.conqur_fold_weight.argtypes = [vp, i64, i32, i32, vp, i32, i32, i32, vp, i64, vp, i64, vp]
+    lib.conqur_hadamard_rows.restype = C.c_int
+    lib.conqur_hadamard_rows.argtypes = [vp, i32, i64, i32, i64, vp, i32, i64, vp]
     lib.conqur_strerror.restype = C.c_char_p
     lib.conqur_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -247,6 +254,49 @@ def conqur_debug_gemm(a, b, m: int, n: int, k: int, a_mn: bool, b_mn: bool, spli
                                   int(split), scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
     if rc != 0:
         raise ConqurError(rc, "conqur_debug_gemm")
+    return out
+
+
+def conqur_fold_scratch_bytes(rows: int, cols: int, block: int, side: int, mode: int) -> int:
+    return int(load().conqur_fold_scratch_bytes(rows, cols, block, side, mode))
+
+
+def conqur_fold_weight(w, r, side: str, mode: str = "tc"):
+    """Appendix A: W' = W R (side "input") or R^T W (side "output"); see include/conqur.h.
+
+    w: fp32 CUDA tensor (rows, cols), unit column stride.  r: fp32 CUDA tensor, one (b, b) rotation or a stack
+    (k, b, b) of diagonal blocks.  Returns a new fp32 tensor (rows, cols)."""
+    import torch
+    assert w.is_cuda and w.dtype == torch.float32 and w.dim() == 2 and w.stride(1) == 1
+    assert r.is_cuda and r.dtype == torch.float32 and r.is_contiguous() and r.shape[-1] == r.shape[-2]
+    side_c = {"input": CONQUR_FOLD_INPUT, "output": CONQUR_FOLD_OUTPUT}[side]
+    mode_c = {"exact": CONQUR_EXACT_F32, "tc": CONQUR_TC_BF16}[mode]
+    rows, cols, block = int(w.shape[0]), int(w.shape[1]), int(r.shape[-1])
+    nbytes = conqur_fold_scratch_bytes(rows, cols, block, side_c, mode_c)
+    if nbytes < 0:
+        raise ConqurError(-1, "conqur_fold_scratch_bytes")
+    scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    sp = (scratch.data_ptr() + 255) // 256 * 256
+    out = torch.empty((rows, cols), dtype=torch.float32, device="cuda")
+    rc = load().conqur_fold_weight(w.data_ptr(), w.stride(0), rows, cols, r.data_ptr(), block, side_c, mode_c,
+                                   out.data_ptr(), out.stride(0), sp, nbytes, torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise ConqurError(rc, "conqur_fold_weight")
+    return out
+
+
+def conqur_hadamard_rows(x, out_dtype=None, out=None):
+    """y = x H_d / sqrt(d) for every row of a 2-D fp32 / bf16 CUDA tensor (see include/conqur.h)."""
+    import torch
+    code = {torch.float32: CONQUR_F32, torch.bfloat16: CONQUR_BF16}
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1 and x.dtype in code
+    if out is None:
+        out = torch.empty(x.shape, dtype=out_dtype or x.dtype, device="cuda")
+    assert out.is_cuda and out.shape == x.shape and out.stride(1) == 1 and out.dtype in code
+    rc = load().conqur_hadamard_rows(x.data_ptr(), code[x.dtype], x.shape[0], x.shape[1], x.stride(0), out.data_ptr(),
+                                     code[out.dtype], out.stride(0), torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise ConqurError(rc, "conqur_hadamard_rows")
     return out
 
 

@@ -18,6 +18,7 @@
 #include "conqur_simt.cuh"
 #include "conqur_tc.cuh"
 #include "conqur_tc_batched.cuh"
+#include "conqur_aux.cuh"
 #include "ns_schedule.h"
 
 using namespace conqur;
@@ -691,6 +692,103 @@ extern "C" int conqur_debug_wait_timeout(void* scratch_dev, int64_t limit_cycles
   CQ_CUDA(cudaMemcpyAsync(&h, scratch_dev, sizeof(DevState), cudaMemcpyDeviceToHost, s));
   CQ_CUDA(cudaStreamSynchronize(s));
   return flags_to_status(h.status_flags);
+}
+
+// ---------------------------------------------------------------- Appendix A: weight folding, online Hadamard
+namespace {
+bool fold_args_ok(int64_t ldw, int32_t rows, int32_t cols, int32_t block, int32_t side, int64_t ldo) {
+  if (rows < 1 || cols < 1 || block < 1 || ldw < cols || ldo < cols) return false;
+  if (side == CONQUR_FOLD_INPUT) return cols % block == 0;
+  if (side == CONQUR_FOLD_OUTPUT) return rows % block == 0;
+  return false;
+}
+// the tensor-core route: one full rotation, sizes the stand-alone product accepts
+bool fold_tc_shape(int32_t rows, int32_t cols, int32_t block, int32_t side) {
+  const int d = block;
+  if (d % 128) return false;
+  return side == CONQUR_FOLD_INPUT ? (cols == d && rows % 8 == 0) : (rows == d && cols % 32 == 0);
+}
+}  // namespace
+
+extern "C" int64_t conqur_fold_scratch_bytes(int32_t rows, int32_t cols, int32_t block, int32_t side, int32_t mode) {
+  if (!fold_args_ok(cols, rows, cols, block, side, cols)) return -1;
+  if (mode == CONQUR_EXACT_F32) return 512;
+  if (mode != CONQUR_TC_BF16) return -1;
+  if (!fold_tc_shape(rows, cols, block, side)) return 512;          // block-diagonal folds run on the fp32 kernel
+  return (int64_t)(512 + align_up((size_t)rows * cols * 4) + align_up((size_t)block * block * 4));
+}
+
+extern "C" int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows, int32_t cols, const float* R_dev,
+                                  int32_t block, int32_t side, int32_t mode, float* out_dev, int64_t ldo,
+                                  void* scratch_dev, int64_t scratch_bytes, void* cuda_stream) {
+  if (!W_dev || !R_dev || !out_dev || !scratch_dev || W_dev == out_dev) return CONQUR_ERR_INVALID_ARG;
+  if (!fold_args_ok(ldw, rows, cols, block, side, ldo)) return CONQUR_ERR_INVALID_ARG;
+  if (mode != CONQUR_EXACT_F32 && mode != CONQUR_TC_BF16) return CONQUR_ERR_INVALID_ARG;
+  const int64_t need = conqur_fold_scratch_bytes(rows, cols, block, side, mode);
+  if (need < 0) return CONQUR_ERR_INVALID_ARG;
+  if (scratch_bytes < need) return CONQUR_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int nblk = (side == CONQUR_FOLD_INPUT ? cols : rows) / block;
+  if (mode == CONQUR_TC_BF16 && nblk == 1) {
+    if (!fold_tc_shape(rows, cols, block, side)) return CONQUR_ERR_UNSUPPORTED;
+    if ((ldw % 4) || (ldo % 4) || (reinterpret_cast<uintptr_t>(W_dev) & 15) || (reinterpret_cast<uintptr_t>(out_dev) & 15) ||
+        (reinterpret_cast<uintptr_t>(R_dev) & 15) || (reinterpret_cast<uintptr_t>(scratch_dev) & 255))
+      return CONQUR_ERR_INVALID_ARG;
+    const int d = block;
+    uint8_t* base = static_cast<uint8_t*>(scratch_dev);
+    DevState* st = reinterpret_cast<DevState*>(base);
+    __nv_bfloat16* Ws = reinterpret_cast<__nv_bfloat16*>(base + 512);
+    __nv_bfloat16* Rs = reinterpret_cast<__nv_bfloat16*>(base + 512 + align_up((size_t)rows * cols * 4));
+    CQ_CUDA(cudaMemsetAsync(st, 0, sizeof(DevState), s));
+    split_bf16_2d_kernel<<<ew_blocks((int64_t)rows * cols / 4), 256, 0, s>>>(W_dev, ldw, rows, cols, Ws);
+    CQ_LAUNCH_CHECK();
+    split_bf16_2d_kernel<<<ew_blocks((int64_t)d * d / 4), 256, 0, s>>>(R_dev, d, d, d, Rs);
+    CQ_LAUNCH_CHECK();
+    int rc;
+    if (side == CONQUR_FOLD_INPUT)     // out (rows x d) = W R: A = W, K-major; B(n, k) = R[k][n], MN-major
+      rc = tc_debug_gemm(Ws, Rs, out_dev, rows, d, d, 0, 1, 1, st, s, ldo);
+    else                               // out (d x cols) = R^T W: A(m, k) = R[k][m] and B(n, k) = W[k][n], both MN-major
+      rc = tc_debug_gemm(Rs, Ws, out_dev, d, cols, d, 1, 1, 1, st, s, ldo);
+    if (rc) return rc;
+    DevState h;
+    CQ_CUDA(cudaMemcpyAsync(&h, st, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+    CQ_CUDA(cudaStreamSynchronize(s));
+    return flags_to_status(h.status_flags);
+  }
+  if (side == CONQUR_FOLD_INPUT) {
+    const dim3 grid(cdiv(block, SG_BN), cdiv(rows, SG_BM), nblk);
+    fold_exact_kernel<0><<<grid, SG_THREADS, 0, s>>>(W_dev, ldw, R_dev, block, rows, cols, out_dev, ldo);
+  } else {
+    const dim3 grid(cdiv(cols, SG_BN), cdiv(block, SG_BM), nblk);
+    fold_exact_kernel<1><<<grid, SG_THREADS, 0, s>>>(W_dev, ldw, R_dev, block, rows, cols, out_dev, ldo);
+  }
+  CQ_LAUNCH_CHECK();
+  CQ_CUDA(cudaStreamSynchronize(s));
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,
+                                    int32_t out_dtype, int64_t ldy, void* cuda_stream) {
+  if (n < 0 || d < 4 || d > 8192 || (d & (d - 1)) || ldx < d || ldy < d) return CONQUR_ERR_INVALID_ARG;
+  if (n > 0 && (!X_dev || !Y_dev)) return CONQUR_ERR_INVALID_ARG;
+  if ((in_dtype != CONQUR_F32 && in_dtype != CONQUR_BF16) || (out_dtype != CONQUR_F32 && out_dtype != CONQUR_BF16))
+    return CONQUR_ERR_INVALID_ARG;
+  // 4-element vector accesses
+  const uintptr_t am = (in_dtype == CONQUR_F32) ? 15 : 7, bm = (out_dtype == CONQUR_F32) ? 15 : 7;
+  if ((ldx % 4) || (ldy % 4) || (reinterpret_cast<uintptr_t>(X_dev) & am) || (reinterpret_cast<uintptr_t>(Y_dev) & bm))
+    return CONQUR_ERR_INVALID_ARG;
+  if (n == 0) return CONQUR_OK;
+  int logd = 0;
+  while ((1 << logd) < d) ++logd;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  using bf = __nv_bfloat16;
+  if (in_dtype == CONQUR_F32 && out_dtype == CONQUR_F32)
+    return hadamard_launch(static_cast<const float*>(X_dev), ldx, static_cast<float*>(Y_dev), ldy, n, logd, s);
+  if (in_dtype == CONQUR_F32)
+    return hadamard_launch(static_cast<const float*>(X_dev), ldx, static_cast<bf*>(Y_dev), ldy, n, logd, s);
+  if (out_dtype == CONQUR_F32)
+    return hadamard_launch(static_cast<const bf*>(X_dev), ldx, static_cast<float*>(Y_dev), ldy, n, logd, s);
+  return hadamard_launch(static_cast<const bf*>(X_dev), ldx, static_cast<bf*>(Y_dev), ldy, n, logd, s);
 }
 
 extern "C" const char* conqur_strerror(int s) {

@@ -1278,12 +1278,14 @@ inline int tc_ns_commit(TcHost& h, cudaStream_t s) {
 
 inline const __nv_bfloat16* tc_cp_ptr(const TcHost& h) { return reinterpret_cast<const __nv_bfloat16*>(h.ws + h.L.Cp); }
 
-// Stand-alone product for tests: D (fp32, M x N) = A * B^T-style contraction with the given orientations.
-// a_mn / b_mn: 0 = K-major ([M|N rows][K cols]), 1 = MN-major ([K rows][M|N cols]).  split: operands are stacked
-// [hi; lo] pairs (3 products).  All device pointers; bf16 operands; caller guarantees the shapes below.
+// Stand-alone product (tests, weight folding): D (fp32, M x N, row stride ldo; 0 = N) = A * B^T-style contraction with
+// the given orientations.  a_mn / b_mn: 0 = K-major ([M|N rows][K cols]), 1 = MN-major ([K rows][M|N cols]).  split:
+// operands are stacked [hi; lo] pairs (3 products).  All device pointers; bf16 operands; shapes as checked below.
 inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* D, int M, int N, int K, int a_mn,
-                         int b_mn, int split, DevState* st, cudaStream_t s) {
+                         int b_mn, int split, DevState* st, cudaStream_t s, long long ldo = 0) {
   if (M < 1 || N < 32 || (N % 32) || K < 1 || (K % 8) || (M % 8)) return CONQUR_ERR_INVALID_ARG;
+  if (ldo == 0) ldo = N;
+  if (ldo < N || (ldo % 4)) return CONQUR_ERR_INVALID_ARG;
   TcHost h{};
   h.prof = nullptr; h.ns_k = -1;
   int dev = 0;
@@ -1305,7 +1307,7 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   TcGemmArgs g{};
   g.M = M; g.N = N; g.K = K; g.nseg = split ? 3 : 1; g.st = st;
   g.a_off[2] = a_mn ? K : M; g.b_off[1] = b_mn ? K : N;
-  g.outF = D; g.ldo = N;
+  g.outF = D; g.ldo = ldo;
   if (!a_mn && !b_mn) return tc_launch_n<false, false, TC_EPI_PLAIN>(h, s, ta, tb, g);
   if (!a_mn && b_mn) return tc_launch_n<false, true, TC_EPI_PLAIN>(h, s, ta, tb, g);
   if (a_mn && !b_mn) return tc_launch_n<true, false, TC_EPI_PLAIN>(h, s, ta, tb, g);

@@ -42,6 +42,8 @@ static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block mus
 
 struct TcbStepArgs {
   int n, P;
+  int xp_outer_tokens;        // 1: the input map's dimensions are (column, problem, token) -- head-interleaved rows --
+                              //    instead of (column, token, problem)
   QuantSpec qs;               // bits == 0: corner target of the rotated row; else per-token fake-quantisation first
   float* M;                   // P x 128 x 128 fp32 (without the 1/sqrt(d))
   double* part_d;             // P objective partials (sum |y| * rnorm, or the quantised equivalent)
@@ -109,8 +111,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (!tc_wait(&aux->xempty[xs], xph ^ 1u, abort_flag)) { ok = false; timeout_site = 12; break; }
           uint8_t* dst = sX + xs * TCB_TILE_BYTES;
           ptx::mbar_expect_tx(&aux->xfull[xs], TCB_TILE_BYTES);
-          tma_load_3d(dst, &tmX, &aux->xfull[xs], 0, t * 128, p);
-          tma_load_3d(dst + 16384, &tmX, &aux->xfull[xs], 64, t * 128, p);
+          const int c1 = g.xp_outer_tokens ? p : t * 128, c2 = g.xp_outer_tokens ? t * 128 : p;
+          tma_load_3d(dst, &tmX, &aux->xfull[xs], 0, c1, c2);
+          tma_load_3d(dst + 16384, &tmX, &aux->xfull[xs], 64, c1, c2);
           ++issued;
           if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
         }
@@ -340,12 +343,21 @@ __global__ void tcb_stage_f32_kernel(const float* __restrict__ X, int64_t n, int
 }
 
 // 3-D view of a batched bf16 input: (128 features, n rows with stride ld, P problems with stride pstride); box 64 x 128 x 1.
-inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_t ld, uint64_t pstride, uint64_t P) {
+// Dimensions are ordered by stride: (column, token, problem) when a problem's rows lie together, (column, problem,
+// token) when the problems' columns are interleaved inside one row (problem stride < row stride).  Either way a box
+// is 128 tokens x 64 columns of one problem and lands in shared memory row by row.
+inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_t ld, uint64_t pstride, uint64_t P,
+                           int* outer_tokens) {
   PFN_encodeTiled fn = tc_encode_fn();
   if (!fn) return CONQUR_ERR_CUDA;
-  const cuuint64_t dims[3] = {TCB_D, n, P};
-  const cuuint64_t strides[2] = {ld * 2, (P > 1 ? pstride : ld * n) * 2};
-  const cuuint32_t box[3] = {64, 128, 1};
+  const uint64_t ps = P > 1 ? pstride : ld * n;
+  *outer_tokens = ps < ld ? 1 : 0;
+  const cuuint64_t dims_tp[3] = {TCB_D, n, P}, dims_pt[3] = {TCB_D, P, n};
+  const cuuint64_t strides_tp[2] = {ld * 2, ps * 2}, strides_pt[2] = {ps * 2, ld * 2};
+  const cuuint32_t box_tp[3] = {64, 128, 1}, box_pt[3] = {64, 1, 128};
+  const cuuint64_t* dims = *outer_tokens ? dims_pt : dims_tp;
+  const cuuint64_t* strides = *outer_tokens ? strides_pt : strides_tp;
+  const cuuint32_t* box = *outer_tokens ? box_pt : box_tp;
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -378,10 +390,11 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
     return CONQUR_ERR_INVALID_ARG;            // TMA needs 16-byte aligned rows and problem bases
   }
   CUtensorMap tmX;
-  int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)h.P);
+  int outer_tokens = 0;
+  int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)h.P, &outer_tokens);
   if (rc) return rc;
   TcbStepArgs g{};
-  g.n = (int)n; g.P = h.P; g.qs = h.qs;
+  g.n = (int)n; g.P = h.P; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
   g.M = h.M; g.part_d = h.part_d; g.st = h.st;
   const int grid = h.P < h.num_sms ? h.P : h.num_sms;
   Prof::Rec rec{};

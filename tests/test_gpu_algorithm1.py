@@ -1,0 +1,95 @@
+"""GPU parity of Algorithm 1's site scheduling: the shared R_1 context fed by every block's two residual-stream
+sites, one batched per-head context per block fed from head-interleaved o_proj inputs, against the oracle's
+Algorithm-1 composition.  Teacher-forced per mini-batch: the oracle starts each mini-batch from the library's
+current rotations, so differences are that mini-batch's own arithmetic."""
+import numpy as np
+import pytest
+
+from oracle import conqur_oracle as O
+from paper_2605_10793_b200 import inputs as I
+from tests.parity_util import TOL, update_parity
+
+pytestmark = pytest.mark.gpu
+
+# raw cross-covariance difference: sign decisions of near-zero products differ between fp32 / bf16 and float64
+M_RAW = {"exact": 2e-3, "tc": 3e-2}
+
+
+def _torch():
+    import torch
+    return torch
+
+
+@pytest.mark.parametrize("mode,quant", [("exact", (0, "sym", 1.0)), ("tc", (0, "sym", 1.0)), ("tc", (4, "zp", 0.9))])
+def test_algorithm1_small_model_against_the_oracle(mode, quant):
+    torch = _torch()
+    from paper_2605_10793_b200 import algorithm1 as A1
+    a = I.SITE_MODELS["a1_small"]
+    T = TOL[mode]
+    bits, qmode, clip = quant
+    cal = A1.Calibrator(a.d, a.n_heads, a.d_head, a.n_layers, a.n, in_dtype="bf16", mode=mode, quant_bits=bits,
+                        quant_mode=qmode, clip_ratio=clip, record="full")
+    r1, r2 = I.site_initial_rotations(a)
+    cal.set_rotations(torch.from_numpy(r1).cuda(), torch.from_numpy(r2).cuda())
+    for mb in range(a.n_minibatches):
+        g1, g2 = cal.rotations()
+        g1, g2 = g1.cpu().numpy().astype(np.float64), g2.cpu().numpy().astype(np.float64)
+        sites = [I.site_activations(a, mb, l) for l in range(a.n_layers)]
+        for l, s in enumerate(sites):
+            dev = {k: torch.from_numpy(v).cuda().to(torch.bfloat16) for k, v in s.items()}
+            cal.collect(l, dev["attn"], dev["mlp"], dev["o"])
+        cal.end_minibatch()
+        assert cal.ctx1.get_stats().status == 0
+        sites64 = [{k: v.astype(np.float64) for k, v in s.items()} for s in sites]
+        _, _, log = O.run_algorithm1(a.d, a.n_heads, a.d_head, a.n_layers, [sites64], g1, g2, quant_bits=bits,
+                                     quant_mode=qmode, clip_ratio=clip)
+        ref, got = log[0], cal.log[mb]
+        # the shared rotation's problem: all 2L sites pooled
+        assert got["N1"] == ref["N1"] == 2 * a.n_layers * a.n
+        assert abs(got["J1"] - ref["J1"]) / ref["J1"] <= T["J"]
+        m1_ref = np.zeros((a.d, a.d))
+        orc = O.OpuOracle(a.d, g1, bits, 0.0, qmode, clip)
+        for s in sites64:
+            orc.step(s["attn"]).step(s["mlp"])
+        m1 = got["M1"].astype(np.float64)
+        assert np.linalg.norm(m1 - orc.M) / np.linalg.norm(orc.M) <= M_RAW[mode]
+        n1, n2 = cal.rotations()
+        n1, n2 = n1.cpu().numpy().astype(np.float64), n2.cpu().numpy().astype(np.float64)
+        rep = update_parity(m1, n1)
+        assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], rep
+        # every head of every block: its own problem, updated inside the loop over blocks
+        for l in range(a.n_layers):
+            for h in range(a.n_heads):
+                assert got["heads"][l]["N"][h] == ref["N2"][l, h] == a.n
+                assert abs(got["heads"][l]["J"][h] - ref["J2"][l, h]) / ref["J2"][l, h] <= T["J"], (l, h)
+                oh = O.OpuOracle(a.d_head, g2[l, h], bits, 0.0, qmode, clip)
+                oh.step(sites64[l]["o"][:, h * a.d_head:(h + 1) * a.d_head])
+                mh = got["heads"][l]["M"][h].astype(np.float64)
+                assert np.linalg.norm(mh - oh.M) / np.linalg.norm(oh.M) <= M_RAW[mode], (l, h)
+                rep = update_parity(mh, n2[l, h])
+                assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], (l, h, rep)
+    cal.close()
+
+
+def test_algorithm1_free_running_matches_the_oracle_chain():
+    """No teacher forcing: both sides run both mini-batches from the same initial rotations (exact mode); the final
+    rotations agree to the accuracy the conditioning of the polar factor allows."""
+    torch = _torch()
+    from paper_2605_10793_b200 import algorithm1 as A1
+    a = I.SITE_MODELS["a1_small"]
+    cal = A1.Calibrator(a.d, a.n_heads, a.d_head, a.n_layers, a.n, in_dtype="bf16", mode="exact")
+    r1, r2 = I.site_initial_rotations(a)
+    cal.set_rotations(torch.from_numpy(r1).cuda(), torch.from_numpy(r2).cuda())
+    mbs = []
+    for mb in range(a.n_minibatches):
+        sites = [I.site_activations(a, mb, l) for l in range(a.n_layers)]
+        mbs.append([{k: v.astype(np.float64) for k, v in s.items()} for s in sites])
+        for l, s in enumerate(sites):
+            cal.collect(l, *(torch.from_numpy(s[k]).cuda().to(torch.bfloat16) for k in ("attn", "mlp", "o")))
+        cal.end_minibatch()
+    o1, o2, _ = O.run_algorithm1(a.d, a.n_heads, a.d_head, a.n_layers, mbs, r1.astype(np.float64), r2.astype(np.float64))
+    g1, g2 = cal.rotations()
+    g1, g2 = g1.cpu().numpy().astype(np.float64), g2.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(g1 - o1) / np.sqrt(a.d) <= 5e-3
+    assert np.linalg.norm(g2 - o2) / np.sqrt(g2.size / a.d_head) <= 5e-3
+    cal.close()
