@@ -14,7 +14,7 @@
  * including the workspace.  The library allocates no device memory.  Pointers
  * without that suffix are HOST memory.  All matrices are dense row-major.
  *
- * Ordering: conqur_step / conqur_step_batched / conqur_update only ENQUEUE work on
+ * Ordering: conqur_step / conqur_step_batched(_range) / conqur_update only ENQUEUE work on
  * the context's stream and return; X must stay valid until that work has run.
  * The conqur_get_* calls synchronise the stream.  A context is not thread-safe.
  *
@@ -147,6 +147,19 @@ int conqur_step(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld);
  */
 int conqur_step_batched(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld,
                         int64_t problem_stride);
+
+/*
+ * The same for a contiguous range of the context's problems: problems first_problem ..
+ * first_problem + n_problems - 1 each take one batch (problem first_problem + q reads its rows at
+ * X_dev + q*problem_stride + i*ld); the others are untouched.  This is how Algorithm 1's per-block
+ * rotations R_{2,l} share one context of L*n_heads problems: block l feeds problems l*n_heads ..
+ * (l+1)*n_heads - 1 when its o_proj input arrives, and one conqur_update at the end of the mini-batch
+ * updates all of them (the problems are independent, so this equals updating each block inside the
+ * loop).  conqur_update returns CONQUR_ERR_EMPTY_UPDATE while any problem of the context has
+ * received no rows since the last update.
+ */
+int conqur_step_batched_range(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld, int64_t problem_stride,
+                              int32_t first_problem, int32_t n_problems);
 
 /*
  * R <- polar(M_eff) = U V^T of the SVD M_eff = U S V^T (Section 3.3), computed by

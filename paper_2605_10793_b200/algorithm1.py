@@ -1,9 +1,12 @@
 """Algorithm 1 (online calibration of the shared and the per-block rotations) as a sequence of library calls.
 
 One context holds the shared rotation R_1: the attention-input and MLP-input activations of every block are
-accumulated into it (`conqur_step`) and it is updated once per mini-batch (`conqur_update`).  Every block has
-one batched context for R_{2,l}: its n_heads diagonal blocks are independent d_head x d_head problems fed from
-the head-interleaved o_proj input in one `conqur_step_batched` call and updated right away.
+accumulated into it (`conqur_step`) and it is updated once per mini-batch (`conqur_update`).  One batched
+context holds all L * n_heads diagonal blocks of the R_{2,l}: they are independent d_head x d_head problems; block l
+feeds its n_heads problems from the head-interleaved o_proj input in one `conqur_step_batched_range` call.
+Algorithm 1 updates R_{2,l} inside the loop over blocks; since R_{2,l} is not used again before the next
+mini-batch and the problems are independent, all of them are updated here by ONE batched `conqur_update` at the
+end of the mini-batch, which gives the same rotations with 1 instead of L latency-bound launches.
 
 This file only sequences calls and moves pointers; all arithmetic runs in the library's kernels.  Weight
 folding (Appendix A) for one transformer block is at the end.
@@ -24,7 +27,7 @@ class Calibrator:
                   prior_rel=prior_rel)
         self.d, self.n_heads, self.d_head, self.n_layers = d, n_heads, d_head, n_layers
         self.ctx1 = B.Context(d=d, n_max=n_max, **kw)
-        self.ctx2: List[B.Context] = [B.Context(d=d_head, n_max=n_max, batch=n_heads, **kw) for _ in range(n_layers)]
+        self.ctx2 = B.Context(d=d_head, n_max=n_max, batch=n_layers * n_heads, **kw)
         self.record = record
         self.log: List[Dict] = []
         self._cur: Dict = {}
@@ -32,45 +35,40 @@ class Calibrator:
     def set_rotations(self, r1, r2):
         """r1: (d, d); r2: (n_layers, n_heads, d_head, d_head); fp32 CUDA tensors."""
         self.ctx1.set_R(r1.contiguous())
-        for l, c in enumerate(self.ctx2):
-            c.set_R(r2[l].contiguous())
+        self.ctx2.set_R(r2.reshape(self.n_layers * self.n_heads, self.d_head, self.d_head).contiguous())
 
     def collect(self, layer: int, x_attn, x_mlp, x_o):
         """The body of Algorithm 1's loop over blocks for block `layer`: both residual-stream sites go into the R_1
-        statistics; R_{2,layer} <- OPU(R_{2,layer}, X_o).  x_o: (n, n_heads*d_head), head h in columns h*d_head.."""
+        statistics, the o_proj input into the statistics of the block's n_heads problems.
+        x_o: (n, n_heads*d_head), head h in columns h*d_head.."""
         self.ctx1.step(x_attn)
         self.ctx1.step(x_mlp)
-        c = self.ctx2[layer]
         assert x_o.shape[1] == self.n_heads * self.d_head and x_o.stride(1) == 1
-        c.step_batched(x_o, x_o.shape[0], x_o.stride(0), self.d_head)
-        if self.record:
-            j, n = c.get_objective()
-            rec = self._cur.setdefault("heads", {})
-            rec[layer] = {"J": j.copy(), "N": n.copy()}
-            if self.record == "full":
-                rec[layer]["M"] = c.get_M().cpu().numpy()
-        c.update()
+        self.ctx2.step_batched_range(x_o, x_o.shape[0], x_o.stride(0), self.d_head, layer * self.n_heads, self.n_heads)
 
     def end_minibatch(self):
-        """R_1 <- OPU(R_1, X_1) with everything accumulated since the last call."""
+        """R_{2,l} <- OPU(R_{2,l}, X_o^(l)) for every block, and R_1 <- OPU(R_1, X_1), with everything accumulated
+        since the last call."""
         if self.record:
+            L, H, dh = self.n_layers, self.n_heads, self.d_head
             j, n = self.ctx1.get_objective()
-            self._cur["J1"], self._cur["N1"] = j, n
+            j2, n2 = self.ctx2.get_objective()
+            self._cur = {"J1": j, "N1": n, "J2": j2.reshape(L, H).copy(), "N2": n2.reshape(L, H).copy()}
             if self.record == "full":
                 self._cur["M1"] = self.ctx1.get_M().cpu().numpy()
+                self._cur["M2"] = self.ctx2.get_M().cpu().numpy().reshape(L, H, dh, dh)
             self.log.append(self._cur)
             self._cur = {}
+        self.ctx2.update()
         self.ctx1.update()
 
     def rotations(self):
         """(R_1 (d, d), R_2 (n_layers, n_heads, d_head, d_head)) as fp32 CUDA tensors."""
-        import torch
-        return self.ctx1.get_R(), torch.stack([c.get_R().reshape(self.n_heads, self.d_head, self.d_head) for c in self.ctx2])
+        return self.ctx1.get_R(), self.ctx2.get_R().reshape(self.n_layers, self.n_heads, self.d_head, self.d_head)
 
     def close(self):
         self.ctx1.close()
-        for c in self.ctx2:
-            c.close()
+        self.ctx2.close()
 
 
 # which side of which projection absorbs which rotation (Appendix A)

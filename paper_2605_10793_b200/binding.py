@@ -23,7 +23,7 @@ CONQUR_FOLD_INPUT, CONQUR_FOLD_OUTPUT = 0, 1
 
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
-    "conqur_step_batched", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
+    "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
     "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows",
@@ -94,6 +94,8 @@ def load() -> C.CDLL:
     lib.conqur_step.argtypes = [vp, vp, i64, i64]
     lib.conqur_step_batched.restype = C.c_int
     lib.conqur_step_batched.argtypes = [vp, vp, i64, i64, i64]
+    lib.conqur_step_batched_range.restype = C.c_int
+    lib.conqur_step_batched_range.argtypes = [vp, vp, i64, i64, i64, i32, i32]
     lib.conqur_update.restype = C.c_int
     lib.conqur_update.argtypes = [vp]
     lib.conqur_get_R.restype = C.c_int
@@ -173,6 +175,10 @@ def conqur_step(h: int, x_ptr: int, n: int, ld: int) -> int:
 
 def conqur_step_batched(h: int, x_ptr: int, n: int, ld: int, problem_stride: int) -> int:
     return load().conqur_step_batched(h, x_ptr, n, ld, problem_stride)
+
+
+def conqur_step_batched_range(h: int, x_ptr: int, n: int, ld: int, problem_stride: int, first: int, count: int) -> int:
+    return load().conqur_step_batched_range(h, x_ptr, n, ld, problem_stride, first, count)
 
 
 def conqur_update(h: int) -> int:
@@ -347,6 +353,11 @@ class Context:
     def step_batched(self, x, n: int, ld: int, problem_stride: int):
         assert x.is_cuda and x.dtype == self._x_dtype()
         self._chk(conqur_step_batched(self.h, x.data_ptr(), n, ld, problem_stride), "conqur_step_batched")
+
+    def step_batched_range(self, x, n: int, ld: int, problem_stride: int, first: int, count: int):
+        assert x.is_cuda and x.dtype == self._x_dtype()
+        self._chk(conqur_step_batched_range(self.h, x.data_ptr(), n, ld, problem_stride, first, count),
+                  "conqur_step_batched_range")
 
     def update(self):
         self._chk(conqur_update(self.h), "conqur_update")

@@ -114,7 +114,7 @@ struct conqur_ctx {
   Layout L;
   char* ws;
   cudaStream_t stream;
-  int64_t tokens_since_update;
+  std::vector<int64_t> tokens;   // per problem: rows enqueued since the last update
   int64_t last_n;            // rows of the last step (for debug_get_signs)
   int n_sched, first_endgame, reenter_idx;
   std::vector<NsStep> sched;
@@ -190,10 +190,13 @@ int ew_blocks(int64_t count) { return (int)std::min<int64_t>(148 * 8, (count + 2
 
 // ---------------------------------------------------------------- exact-mode step
 template <typename TIn>
-int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstride) {
+int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstride, int p0, int np) {
+  // problems [p0, p0 + np): state, R and M are theirs; the per-step scratch (row norms, targets, partials) is used
+  // from its start
   const Cfg& g = c->cfg;
-  const int d = g.d, P = g.P;
-  DevState* st = c->state();
+  const int d = g.d, P = np;
+  const int64_t pdd = (int64_t)p0 * d * d;
+  DevState* st = c->state() + p0;
   float* rnorm = c->at<float>(c->L.rnorm);
   float* C = c->at<float>(c->L.C);
   double* part = c->at<double>(c->L.part_d);
@@ -205,16 +208,16 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   double* pdiag = g.diagnostics ? c->at<double>(c->L.part_diag) : nullptr;
   if (g.quant_bits == 0 && !g.diagnostics) {
     rotate_target_exact_kernel<TIn, false><<<grid1, SG_THREADS, 0, c->stream>>>(
-        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, nullptr, part);
+        X, ld, pstride, c->at<float>(c->L.R) + pdd, (int)n, d, rnorm, g.n_max, C, c_ps, nullptr, nullptr, part);
     CQ_LAUNCHED(c, K_ROTATE);
     per_problem = grid1.x * grid1.y;
   } else {
     unsigned* rowmax = c->at<unsigned>(c->L.rowmax);
-    unsigned* rowmin = rowmax + g.n_max * P;
+    unsigned* rowmin = rowmax + g.n_max * g.P;
     CQ_CUDA(cudaMemsetAsync(rowmax, 0, sizeof(unsigned) * g.n_max * P, c->stream));
     CQ_CUDA(cudaMemsetAsync(rowmin, 0xff, sizeof(unsigned) * g.n_max * P, c->stream));
     rotate_target_exact_kernel<TIn, true><<<grid1, SG_THREADS, 0, c->stream>>>(
-        X, ld, pstride, c->at<float>(c->L.R), (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, rowmin, part);
+        X, ld, pstride, c->at<float>(c->L.R) + pdd, (int)n, d, rnorm, g.n_max, C, c_ps, rowmax, rowmin, part);
     CQ_LAUNCHED(c, K_ROTATE);
     quant_target_kernel<<<dim3(cdiv(n, 8), P), 256, 0, c->stream>>>(C, n, d, c_ps, rnorm, g.n_max, rowmax, rowmin, g.qs,
                                                                     part, pdiag);
@@ -226,12 +229,12 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   CQ_LAUNCHED(c, K_OTHER);
   const int S = c->L.acc_splits;
   accumulate_exact_kernel<TIn><<<dim3(cdiv(d, SG_BN), cdiv(d, SG_BM), P * S), SG_THREADS, 0, c->stream>>>(
-      X, ld, pstride, C, c_ps, rnorm, g.n_max, (int)n, d, S, c->at<float>(c->L.M),
+      X, ld, pstride, C, c_ps, rnorm, g.n_max, (int)n, d, S, c->at<float>(c->L.M) + pdd,
       S > 1 ? c->at<float>(c->L.splitk) : nullptr);
   CQ_LAUNCHED(c, K_ACCUM);
   if (S > 1) {
     splitk_reduce_add_kernel<<<dim3(ew_blocks((int64_t)d * d), P), 256, 0, c->stream>>>(
-        c->at<float>(c->L.M), c->at<float>(c->L.splitk), (int64_t)d * d, S);
+        c->at<float>(c->L.M) + pdd, c->at<float>(c->L.splitk), (int64_t)d * d, S);
     CQ_LAUNCHED(c, K_OTHER);
   }
   return CONQUR_OK;
@@ -405,7 +408,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   c->L = L;
   c->ws = static_cast<char*>(workspace_dev);
   c->stream = static_cast<cudaStream_t>(cuda_stream);
-  c->tokens_since_update = 0;
+  c->tokens.assign(cfg->batch, 0);
   c->last_n = 0;
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
@@ -493,39 +496,51 @@ extern "C" int conqur_set_R(conqur_ctx* c, const float* R_dev) {
   return CONQUR_OK;
 }
 
-static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int64_t pstride) {
+static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int64_t pstride, int p0, int np) {
   if (!c || !X) return CONQUR_ERR_INVALID_ARG;
   const Cfg& g = c->cfg;
-  if (n < 0 || n > g.n_max || ld < g.d || pstride < 0 || (g.P > 1 && pstride == 0)) return CONQUR_ERR_INVALID_ARG;
+  if (n < 0 || n > g.n_max || ld < g.d || pstride < 0 || (np > 1 && pstride == 0)) return CONQUR_ERR_INVALID_ARG;
+  if (p0 < 0 || np < 1 || p0 + np > g.P) return CONQUR_ERR_INVALID_ARG;
   if (n == 0) return CONQUR_OK;
   int rc;
   if (g.mode == CONQUR_EXACT_F32) {
-    rc = (g.in_dtype == CONQUR_F32) ? step_exact<float>(c, static_cast<const float*>(X), n, ld, pstride)
-                                    : step_exact<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(X), n, ld, pstride);
+    rc = (g.in_dtype == CONQUR_F32)
+             ? step_exact<float>(c, static_cast<const float*>(X), n, ld, pstride, p0, np)
+             : step_exact<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(X), n, ld, pstride, p0, np);
   } else {
-    rc = g.P > 1 ? tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride)
+    rc = g.P > 1 ? tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride, p0, np)
                  : tc_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride);
   }
-  if (rc == CONQUR_OK) { c->tokens_since_update += n; c->last_n = n; }
+  if (rc == CONQUR_OK) {
+    for (int p = p0; p < p0 + np; ++p) c->tokens[p] += n;
+    c->last_n = n;
+  }
   return rc;
 }
 
 extern "C" int conqur_step(conqur_ctx* c, const void* X_dev, int64_t n, int64_t ld) {
   if (!c || c->cfg.P != 1) return CONQUR_ERR_INVALID_ARG;
-  return step_common(c, X_dev, n, ld, 0);
+  return step_common(c, X_dev, n, ld, 0, 0, 1);
 }
 
 extern "C" int conqur_step_batched(conqur_ctx* c, const void* X_dev, int64_t n, int64_t ld, int64_t problem_stride) {
   if (!c) return CONQUR_ERR_INVALID_ARG;
-  return step_common(c, X_dev, n, ld, problem_stride);
+  return step_common(c, X_dev, n, ld, problem_stride, 0, c->cfg.P);
+}
+
+extern "C" int conqur_step_batched_range(conqur_ctx* c, const void* X_dev, int64_t n, int64_t ld, int64_t problem_stride,
+                                         int32_t first_problem, int32_t n_problems) {
+  if (!c) return CONQUR_ERR_INVALID_ARG;
+  return step_common(c, X_dev, n, ld, problem_stride, first_problem, n_problems);
 }
 
 extern "C" int conqur_update(conqur_ctx* c) {
   if (!c) return CONQUR_ERR_INVALID_ARG;
-  if (c->tokens_since_update == 0) return CONQUR_ERR_EMPTY_UPDATE;
-  if (c->tokens_since_update < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
+  const int64_t fewest = *std::min_element(c->tokens.begin(), c->tokens.end());     // every problem is updated
+  if (fewest == 0) return CONQUR_ERR_EMPTY_UPDATE;
+  if (fewest < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
   const int rc = update_enqueue(c);
-  if (rc == CONQUR_OK) c->tokens_since_update = 0;
+  if (rc == CONQUR_OK) std::fill(c->tokens.begin(), c->tokens.end(), 0);
   return rc;
 }
 
@@ -586,9 +601,7 @@ extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_s
   set_sums_kernel<<<1, 256, 0, c->stream>>>(c->state(), dJ, dN, P);
   CQ_LAUNCHED(c, K_OTHER);
   CQ_CUDA(cudaStreamSynchronize(c->stream));
-  int64_t tot = 0;
-  for (int p = 0; p < P; ++p) tot = std::max<int64_t>(tot, n_tokens[p]);
-  c->tokens_since_update = tot;
+  for (int p = 0; p < P; ++p) c->tokens[p] = n_tokens[p];
   return CONQUR_OK;
 }
 

@@ -41,7 +41,8 @@ struct TcbAux {
 static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
 
 struct TcbStepArgs {
-  int n, P;
+  int n, P;                   // P problems; M, part_d, st point at the first of them
+  int p0;                     // its index in the context (row block of the rotation map)
   int xp_outer_tokens;        // 1: the input map's dimensions are (column, problem, token) -- head-interleaved rows --
                               //    instead of (column, token, problem)
   QuantSpec qs;               // bits == 0: corner target of the rotated row; else per-token fake-quantisation first
@@ -105,8 +106,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
         if (!tc_wait(&aux->rempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 11; break; }
         ptx::mbar_expect_tx(&aux->rfull, TCB_TILE_BYTES);
-        ptx::tma_load_2d(sR, &tmR, &aux->rfull, 0, p * TCB_D);
-        ptx::tma_load_2d(sR + 16384, &tmR, &aux->rfull, 64, p * TCB_D);
+        ptx::tma_load_2d(sR, &tmR, &aux->rfull, 0, (g.p0 + p) * TCB_D);
+        ptx::tma_load_2d(sR + 16384, &tmR, &aux->rfull, 64, (g.p0 + p) * TCB_D);
         for (int t = 0; t < T; ++t) {
           if (!tc_wait(&aux->xempty[xs], xph ^ 1u, abort_flag)) { ok = false; timeout_site = 12; break; }
           uint8_t* dst = sX + xs * TCB_TILE_BYTES;
@@ -370,7 +371,9 @@ inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_
 }
 
 // One streamed batch for all P problems.  X: device, bf16 or fp32 (fp32 is first rounded into the staging copy).
-inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride) {
+// Problems [p0, p0 + np) of the context; X holds those np problems.
+inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride, int p0,
+                    int np) {
   static int attr_dev_mask = 0;                    // the attribute is per device
   if (!(attr_dev_mask & (1 << (h.device & 31)))) {
     if (cudaFuncSetAttribute(tcb_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCB_SMEM_BYTES) != cudaSuccess)
@@ -381,8 +384,8 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   int64_t src_ld = ld, src_ps = pstride;
   if (in_dtype == CONQUR_F32) {
     __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xs);
-    tcb_stage_f32_kernel<<<tc_ew_blocks((int64_t)h.P * n * (TCB_D / 4)), 256, 0, s>>>(static_cast<const float*>(X), n, ld,
-                                                                                     pstride, h.P, Xs);
+    tcb_stage_f32_kernel<<<tc_ew_blocks((int64_t)np * n * (TCB_D / 4)), 256, 0, s>>>(static_cast<const float*>(X), n, ld,
+                                                                                    pstride, np, Xs);
     if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
     if (h.prof) h.prof->count(K_ROWNORM);
     src = Xs; src_ld = TCB_D; src_ps = n * TCB_D;
@@ -391,16 +394,16 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   }
   CUtensorMap tmX;
   int outer_tokens = 0;
-  int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)h.P, &outer_tokens);
+  int rc = tcb_make_x_tmap(&tmX, src, (uint64_t)n, (uint64_t)src_ld, (uint64_t)src_ps, (uint64_t)np, &outer_tokens);
   if (rc) return rc;
   TcbStepArgs g{};
-  g.n = (int)n; g.P = h.P; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
-  g.M = h.M; g.part_d = h.part_d; g.st = h.st;
-  const int grid = h.P < h.num_sms ? h.P : h.num_sms;
+  g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
+  g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0;
+  const int grid = np < h.num_sms ? np : h.num_sms;
   Prof::Rec rec{};
   const bool timed = h.prof && h.prof->enabled;
   if (timed) {
-    rec.cls = K_ROTATE; rec.flops = 4.0 * (double)h.P * (double)n * TCB_D * TCB_D; rec.ns_k = -1; rec.nseg = 1;
+    rec.cls = K_ROTATE; rec.flops = 4.0 * (double)np * (double)n * TCB_D * TCB_D; rec.ns_k = -1; rec.nseg = 1;
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
@@ -408,7 +411,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_ROTATE);
-  finalize_step_kernel<<<h.P, 256, 0, s>>>(h.st, h.part_d, 1, n, 1.0 / std::sqrt((double)TCB_D));
+  finalize_step_kernel<<<np, 256, 0, s>>>(g.st, h.part_d, 1, n, 1.0 / std::sqrt((double)TCB_D));
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_OTHER);
   return CONQUR_OK;

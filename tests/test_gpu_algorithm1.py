@@ -1,6 +1,7 @@
 """GPU parity of Algorithm 1's site scheduling: the shared R_1 context fed by every block's two residual-stream
-sites, one batched per-head context per block fed from head-interleaved o_proj inputs, against the oracle's
-Algorithm-1 composition.  Teacher-forced per mini-batch: the oracle starts each mini-batch from the library's
+sites, one batched context of all per-head problems fed block by block from head-interleaved o_proj inputs and
+updated once per mini-batch, against the oracle's Algorithm-1 composition (which updates each block's heads
+inside the loop over blocks, as the paper writes it).  Teacher-forced per mini-batch: the oracle starts each mini-batch from the library's
 current rotations, so differences are that mini-batch's own arithmetic."""
 import numpy as np
 import pytest
@@ -60,11 +61,11 @@ def test_algorithm1_small_model_against_the_oracle(mode, quant):
         # every head of every block: its own problem, updated inside the loop over blocks
         for l in range(a.n_layers):
             for h in range(a.n_heads):
-                assert got["heads"][l]["N"][h] == ref["N2"][l, h] == a.n
-                assert abs(got["heads"][l]["J"][h] - ref["J2"][l, h]) / ref["J2"][l, h] <= T["J"], (l, h)
+                assert got["N2"][l, h] == ref["N2"][l, h] == a.n
+                assert abs(got["J2"][l, h] - ref["J2"][l, h]) / ref["J2"][l, h] <= T["J"], (l, h)
                 oh = O.OpuOracle(a.d_head, g2[l, h], bits, 0.0, qmode, clip)
                 oh.step(sites64[l]["o"][:, h * a.d_head:(h + 1) * a.d_head])
-                mh = got["heads"][l]["M"][h].astype(np.float64)
+                mh = got["M2"][l, h].astype(np.float64)
                 assert np.linalg.norm(mh - oh.M) / np.linalg.norm(oh.M) <= M_RAW[mode], (l, h)
                 rep = update_parity(mh, n2[l, h])
                 assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], (l, h, rep)
@@ -93,3 +94,39 @@ def test_algorithm1_free_running_matches_the_oracle_chain():
     assert np.linalg.norm(g1 - o1) / np.sqrt(a.d) <= 5e-3
     assert np.linalg.norm(g2 - o2) / np.sqrt(g2.size / a.d_head) <= 5e-3
     cal.close()
+
+
+@pytest.mark.parametrize("mode", ["exact", "tc"])
+def test_problem_ranges_of_a_batched_context(mode):
+    """conqur_step_batched_range: feeding a context's problems range by range (in any order, ranges of different
+    sizes, stacked and head-interleaved inputs) gives bit for bit what one conqur_step_batched over all problems
+    gives; an update with an unfed problem is refused."""
+    torch = _torch()
+    from paper_2605_10793_b200 import binding as B
+    w = I.scaled(I.WORKLOADS["c4b"], n=300, problems=7)
+    P, d, n = 7, w.d, w.n
+    xs = [I.batch(w, 0, problem=p) for p in range(P)]
+    r0 = torch.from_numpy(np.stack([I.initial_rotation(w, p) for p in range(P)])).cuda()
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
+    whole = B.Context(d=d, n_max=n, in_dtype="bf16", mode=mode, batch=P)
+    whole.set_R(r0)
+    whole.step_batched(dev(np.concatenate(xs, axis=1)), n, P * d, d)
+    jw, nw = whole.get_objective()
+    mw = whole.get_M().cpu().numpy()
+    parts = B.Context(d=d, n_max=n, in_dtype="bf16", mode=mode, batch=P)
+    parts.set_R(r0)
+    parts.step_batched_range(dev(np.concatenate(xs[4:7], axis=1)), n, 3 * d, d, 4, 3)       # interleaved, last three
+    assert B.conqur_update(parts.h) == -4                                                   # problems 0..3 have no rows yet
+    parts.step_batched_range(dev(np.concatenate(xs[0:3], axis=0)), n, d, n * d, 0, 3)       # stacked, first three
+    parts.step_batched_range(dev(xs[3]), n, d, 0, 3, 1)                                     # a single problem
+    jp, npp = parts.get_objective()
+    assert np.array_equal(nw, npp) and np.array_equal(jw, jp)
+    assert np.array_equal(mw, parts.get_M().cpu().numpy())
+    whole.update()
+    parts.update()
+    assert np.array_equal(whole.get_R().cpu().numpy(), parts.get_R().cpu().numpy())
+    lib = B.load()
+    x = dev(xs[0])
+    assert lib.conqur_step_batched_range(parts.h, x.data_ptr(), n, d, n * d, 6, 2) == -1    # past the last problem
+    assert lib.conqur_step_batched_range(parts.h, x.data_ptr(), n, d, n * d, -1, 1) == -1
+    assert lib.conqur_step_batched_range(parts.h, x.data_ptr(), n, d, n * d, 0, 0) == -1
