@@ -301,6 +301,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
     torch.cuda.set_device(g.local_rank)
     B.load()
+    if args.workload not in I.WORKLOADS:
+        from paper_2605_10793_b200 import bench_extra as X      # Algorithm-1 mini-batch, Hadamard transform, weight folding
+        return X.RUNNERS[args.workload](args, g, ClockSampler, _peaks())
     w = I.WORKLOADS[args.workload]
     if w.problems > 1:
         return run_batched(args, g, w)

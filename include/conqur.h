@@ -335,9 +335,16 @@ int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows, int32_t co
  *           stride): every row is read completely before it is written
  *   ldx, ldy multiples of 4; pointers aligned to 4 elements.
  * Enqueued on the stream; not synchronised.  Invalid arguments return CONQUR_ERR_INVALID_ARG and do nothing.
+ * Rows that start on 16-byte boundaries (X_dev and ldx * element size multiples of 16, d * element size too) are
+ * staged through shared memory by bulk asynchronous copies; other layouts take a plain-load kernel.
+ *
+ * conqur_hadamard_status: synchronises the stream and returns CONQUR_ERR_TIMEOUT if, since the last call on
+ * this device, a transform kernel abandoned a bounded wait for one of its bulk copies (its output is then
+ * incomplete), CONQUR_OK otherwise; clears the latch.
  */
 int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,
                          int32_t out_dtype, int64_t ldy, void* cuda_stream);
+int conqur_hadamard_status(void* cuda_stream);
 
 const char* conqur_strerror(int status);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
-    "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows",
+    "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows", "conqur_hadamard_status",
     "conqur_strerror",
 ]
 
@@ -130,6 +130,8 @@ def load() -> C.CDLL:
     lib.conqur_fold_weight.argtypes = [vp, i64, i32, i32, vp, i32, i32, i32, vp, i64, vp, i64, vp]
     lib.conqur_hadamard_rows.restype = C.c_int
     lib.conqur_hadamard_rows.argtypes = [vp, i32, i64, i32, i64, vp, i32, i64, vp]
+    lib.conqur_hadamard_status.restype = C.c_int
+    lib.conqur_hadamard_status.argtypes = [vp]
     lib.conqur_strerror.restype = C.c_char_p
     lib.conqur_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -304,6 +306,12 @@ def conqur_hadamard_rows(x, out_dtype=None, out=None):
     if rc != 0:
         raise ConqurError(rc, "conqur_hadamard_rows")
     return out
+
+
+def conqur_hadamard_status() -> int:
+    """Synchronise the current stream; status of the transform kernels run since the last call (0 = ok)."""
+    import torch
+    return int(load().conqur_hadamard_status(torch.cuda.current_stream().cuda_stream))
 
 
 # ---- convenience wrapper: owns the workspace tensor, checks status codes ------------------------

@@ -804,6 +804,17 @@ extern "C" int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t
   return hadamard_launch(static_cast<const bf*>(X_dev), ldx, static_cast<bf*>(Y_dev), ldy, n, logd, s);
 }
 
+extern "C" int conqur_hadamard_status(void* cuda_stream) {
+  CQ_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+  int f = 0;
+  CQ_CUDA(cudaMemcpyFromSymbol(&f, g_aux_status_flags, sizeof(int)));
+  if (f) {
+    const int zero = 0;
+    CQ_CUDA(cudaMemcpyToSymbol(g_aux_status_flags, &zero, sizeof(int)));
+  }
+  return flags_to_status(f);
+}
+
 extern "C" const char* conqur_strerror(int s) {
   switch (s) {
     case CONQUR_OK: return "ok";

@@ -2,6 +2,7 @@
 // fixed online Walsh-Hadamard transform (the R_3 / R_4 rotations).
 #pragma once
 #include "conqur_simt.cuh"
+#include "conqur_tc.cuh"
 
 namespace conqur {
 
@@ -66,76 +67,77 @@ static __global__ void split_bf16_2d_kernel(const float* __restrict__ src, int64
 // ------------------------------------------------------------------ Walsh-Hadamard transform of rows
 // y = x H_d / sqrt(d), H_d the Sylvester matrix (H[i][j] = (-1)^popcount(i & j)), d = 2^logd, 4 <= d <= 256 E.
 //
-// A CTA of 256 threads transforms a block of 256 E consecutive elements (one row, or several whole rows when d is
-// smaller).  The transform is a butterfly over each of the logd index bits, in any order:
-//   load     thread t reads the 16-byte pieces t, t+256, ... (coalesced); element index = 4 (t + 256 j) + e, so
-//            bits 0-1 (e) and bits 10.. (j) of the index are in the thread's own registers: those butterflies run
-//            right away, and the values go to shared memory;
-//   passes   bits 2..9 in one or two passes through shared memory: a thread gathers the 2^B elements that differ
-//            only in the pass's B bits, transforms them in registers and puts them back (in place, disjoint groups);
-//   store    pieces are read back in the load order, scaled by 1/sqrt(d) and written out (coalesced).
-// Shared-memory index swizzle: bits 2-4 ^= bits 6-8, which keeps 16-byte pieces whole and spreads both the
-// stride-4 groups of the first pass and the stride-64 groups of the second over the banks.
+// A CTA of 256 threads transforms blocks of 256 E consecutive elements (one row, or several whole rows when d is
+// smaller).  The transform is a butterfly over each of the logd index bits, in any order; the bits are handled in
+// up to three groups, each while the thread that owns an element also owns its partners:
+//   first    thread t takes the 16-byte pieces t, t+256, ... of the block (coalesced; element index =
+//            4 (t + 256 j) + e): index bits 0-1 (e) and 10.. (j) are inside the thread, their butterflies run in
+//            registers, and the values go to a work buffer in shared memory;
+//   middle   bits 2-5: a thread gathers the 16 elements that differ only in these bits (stride 4), transforms them
+//            in registers and puts them back in place;
+//   last     bits 6-9: the same with stride 64;
+//   store    pieces are read back in the first group's layout, scaled by 1/sqrt(d), converted and written out
+//            (coalesced 16- or 8-byte pieces; storing straight from the last group's registers, 2 or 4 bytes per
+//            lane, measured 1.5x slower).
+// Work-buffer layout: 4 floats of padding after every 64, i.e. position i lives at i + 4 (i >> 6): every
+// access pattern above is free of bank conflicts and every offset inside a group is a compile-time constant.
+//
+// The input is staged by bulk asynchronous copies (the TMA engine's 1-D form): a persistent CTA walks its blocks
+// with a ring of S raw-input stages in shared memory, each filled by `cp.async.bulk` (one copy per block when the
+// rows are contiguous, else one per row) that signals an mbarrier; the copy of block i+S is issued as soon as every
+// thread has taken block i out of its stage.  The data in flight lives in shared memory rather than in registers:
+// S stages x the resident CTAs hold > 100 KB in flight per SM.  Needs 16-byte aligned rows (base and row stride);
+// other layouts take the plain-load kernel below (one block per CTA).  Every wait is bounded; a wait that gives up
+// latches the TIMEOUT flag in g_aux_status_flags, lets the copies in flight land, and the CTA ends.
 constexpr int HAD_THREADS = 256;
+static __device__ int g_aux_status_flags;
 
-__device__ __forceinline__ int had_swz(int i) { return i ^ (((i >> 6) & 7) << 2); }
+namespace ptx {
+__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+}  // namespace ptx
 
-template <int B>
-__device__ __forceinline__ void had_pass(float* sm, int s, int groups) {
-  for (int q = 0; q < groups; ++q) {
-    const int u = threadIdx.x + HAD_THREADS * q;
-    const int base = ((u >> s) << (s + B)) | (u & ((1 << s) - 1));
-    float w[1 << B];
+__device__ __forceinline__ int had_pad(int i) { return i + ((i >> 6) << 2); }
+template <int E> struct HadWork { static constexpr int FLOATS = HAD_THREADS * E + HAD_THREADS * E / 16; };
+
+template <int N>
+__device__ __forceinline__ void had_butterflies(float (&w)[N], int nbits) {
 #pragma unroll
-    for (int k = 0; k < (1 << B); ++k) w[k] = sm[had_swz(base | (k << s))];
+  for (int m = 0; (1 << m) < N; ++m)
+    if (m < nbits) {
 #pragma unroll
-    for (int m = 0; m < B; ++m)
-#pragma unroll
-      for (int k = 0; k < (1 << B); ++k)
+      for (int k = 0; k < N; ++k)
         if (!(k & (1 << m))) {
           const float a = w[k], c = w[k | (1 << m)];
           w[k] = a + c; w[k | (1 << m)] = a - c;
         }
-#pragma unroll
-    for (int k = 0; k < (1 << B); ++k) sm[had_swz(base | (k << s))] = w[k];
-  }
-}
-
-__device__ __forceinline__ void had_pass_n(float* sm, int s, int b, int E) {
-  switch (b) {
-    case 1: had_pass<1>(sm, s, E >> 1); break;
-    case 2: had_pass<2>(sm, s, E >> 2); break;
-    case 3: had_pass<3>(sm, s, E >> 3); break;
-    case 4: had_pass<4>(sm, s, E >> 4); break;
-    default: break;
-  }
+    }
 }
 
 __device__ __forceinline__ void st4_from_float(float* p, const float4 v) { *reinterpret_cast<float4*>(p) = v; }
 __device__ __forceinline__ void st4_from_float(__nv_bfloat16* p, const float4 v) {
-  const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
   uint2 o;
-  o.x = *reinterpret_cast<const uint32_t*>(&a);
-  o.y = *reinterpret_cast<const uint32_t*>(&b);
+  o.x = bf16x2_pack(v.x, v.y);
+  o.y = bf16x2_pack(v.z, v.w);
   *reinterpret_cast<uint2*>(p) = o;
 }
+__device__ __forceinline__ void st1_from_float(float* p, float v) { *p = v; }
+__device__ __forceinline__ void st1_from_float(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
-template <typename TIn, typename TOut, int E>
-__global__ void __launch_bounds__(HAD_THREADS) hadamard_rows_kernel(const TIn* X, int64_t ldx,
-                                                                     TOut* Y, int64_t ldy, int64_t n, int logd,
-                                                                     float scale) {
-  __shared__ __align__(16) float sm[HAD_THREADS * E];
-  const int d = 1 << logd;
+// First group for one block: `src` is the block's raw input (global memory, or a stage in shared memory) addressed
+// through row(i) -> pointer; the values land in the work buffer.
+template <typename TIn, int E, typename RowPtr>
+__device__ __forceinline__ void had_first(float* sm, int logd, int64_t rows_left, RowPtr&& elem_ptr) {
   const int t = threadIdx.x;
-  const int64_t row0 = (int64_t)blockIdx.x * ((HAD_THREADS * E) >> logd);
   float v[E];
 #pragma unroll
   for (int j = 0; j < E / 4; ++j) {
     const int i = 4 * (t + HAD_THREADS * j);
-    const int64_t row = row0 + (i >> logd);
     float x[4] = {0.f, 0.f, 0.f, 0.f};
-    if (row < n) ld4_as_float(X + row * ldx + (i & (d - 1)), x);
-    // bits 0 and 1
+    if ((i >> logd) < rows_left) ld4_as_float(elem_ptr(i), x);
     const float s0 = x[0] + x[1], d0 = x[0] - x[1], s1 = x[2] + x[3], d1 = x[2] - x[3];
     v[4 * j + 0] = s0 + s1; v[4 * j + 1] = d0 + d1; v[4 * j + 2] = s0 - s1; v[4 * j + 3] = d0 - d1;
   }
@@ -152,32 +154,185 @@ __global__ void __launch_bounds__(HAD_THREADS) hadamard_rows_kernel(const TIn* X
     }
 #pragma unroll
   for (int j = 0; j < E / 4; ++j)
-    *reinterpret_cast<float4*>(&sm[had_swz(4 * (t + HAD_THREADS * j))]) =
+    *reinterpret_cast<float4*>(&sm[had_pad(4 * (t + HAD_THREADS * j))]) =
         make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-  const int r = (logd < 10 ? logd : 10) - 2;          // index bits 2 .. 2+r-1 go through shared memory
-  if (r > 0) {
-    __syncthreads();
-    had_pass_n(sm, 2, r < 4 ? r : 4, E);
-    if (r > 4) {
-      __syncthreads();
-      had_pass_n(sm, 6, r - 4, E);
-    }
+}
+
+// Middle group (bits 2-5, `nbits` of them), in place.
+template <int E>
+__device__ __forceinline__ void had_middle(float* sm, int nbits) {
+#pragma unroll
+  for (int q = 0; q < E / 16; ++q) {
+    const int u = threadIdx.x + HAD_THREADS * q;
+    float* p = sm + had_pad(((u >> 2) << 6) | (u & 3));
+    float w[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) w[k] = p[4 * k];
+    had_butterflies(w, nbits);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) p[4 * k] = w[k];
   }
-  __syncthreads();
+}
+
+// Last group (bits 6-9, `nbits` of them), in place.
+template <int E>
+__device__ __forceinline__ void had_last(float* sm, int nbits) {
+#pragma unroll
+  for (int q = 0; q < E / 16; ++q) {
+    const int u = threadIdx.x + HAD_THREADS * q;
+    float* p = sm + had_pad(((u >> 6) << 10) | (u & 63));
+    float w[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) w[k] = p[68 * k];
+    had_butterflies(w, nbits);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) p[68 * k] = w[k];
+  }
+}
+
+// Out of the work buffer in the first group's layout: scaled, converted, 16-byte (fp32) / 8-byte (bf16) pieces.
+template <typename TOut, int E>
+__device__ __forceinline__ void had_plain_store(const float* sm, int logd, int64_t rows_left, float scale, TOut* Yblk, int64_t ldy) {
+  const int d = 1 << logd;
 #pragma unroll
   for (int j = 0; j < E / 4; ++j) {
-    const int i = 4 * (t + HAD_THREADS * j);
-    const int64_t row = row0 + (i >> logd);
-    if (row >= n) continue;
-    float4 o = *reinterpret_cast<const float4*>(&sm[had_swz(i)]);
+    const int i = 4 * (threadIdx.x + HAD_THREADS * j);
+    if ((i >> logd) >= rows_left) continue;
+    float4 o = *reinterpret_cast<const float4*>(&sm[had_pad(i)]);
     o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
-    st4_from_float(Y + row * ldy + (i & (d - 1)), o);
+    st4_from_float(Yblk + (int64_t)(i >> logd) * ldy + (i & (d - 1)), o);
   }
+}
+
+// Everything after the first group for one block (the work buffer is filled; ends with the block stored).
+template <typename TOut, int E>
+__device__ __forceinline__ void had_finish(float* sm, int logd, int64_t rows_left, float scale, TOut* Yblk, int64_t ldy) {
+  const int r = (logd < 10 ? logd : 10) - 2;                // index bits 2 .. 2+r-1 go through the work buffer
+  if (r > 0) had_middle<E>(sm, r < 4 ? r : 4);
+  if (r > 4) {
+    __syncthreads();
+    had_last<E>(sm, r - 4);
+  }
+  __syncthreads();
+  had_plain_store<TOut, E>(sm, logd, rows_left, scale, Yblk, ldy);
+}
+
+template <typename TIn, typename TOut, int E>
+__global__ void __launch_bounds__(HAD_THREADS) hadamard_rows_kernel(const TIn* X, int64_t ldx, TOut* Y, int64_t ldy, int64_t n,
+                                                                     int logd, float scale) {
+  __shared__ __align__(16) float sm[HadWork<E>::FLOATS];
+  const int d = 1 << logd;
+  const int64_t row0 = (int64_t)blockIdx.x * ((HAD_THREADS * E) >> logd);
+  const TIn* Xblk = X + row0 * ldx;
+  had_first<TIn, E>(sm, logd, n - row0, [&](int i) { return Xblk + (int64_t)(i >> logd) * ldx + (i & (d - 1)); });
+  __syncthreads();
+  had_finish<TOut, E>(sm, logd, n - row0, scale, Y + row0 * ldy, ldy);
+}
+
+template <typename TIn, int E, int S>
+constexpr int had_bulk_smem_bytes() { return HadWork<E>::FLOATS * 4 + S * HAD_THREADS * E * (int)sizeof(TIn) + 128; }
+
+template <typename TIn, typename TOut, int E, int S>
+__global__ void __launch_bounds__(HAD_THREADS, E == 16 ? 4 : 2) hadamard_rows_bulk_kernel(const TIn* X, int64_t ldx, TOut* Y,
+                                                                                           int64_t ldy, int64_t n, int logd,
+                                                                                           float scale, int64_t nblocks) {
+  extern __shared__ __align__(128) uint8_t had_smem[];
+  constexpr int NB = HAD_THREADS * E;                       // elements per block
+  constexpr int WORK_BYTES = HadWork<E>::FLOATS * 4;
+  float* sm = reinterpret_cast<float*>(had_smem);
+  TIn* stage = reinterpret_cast<TIn*>(had_smem + WORK_BYTES);
+  uint64_t* full = reinterpret_cast<uint64_t*>(had_smem + WORK_BYTES + S * NB * sizeof(TIn));
+  __shared__ int abort_flag;
+  const int d = 1 << logd;
+  const int rows_per_block = NB >> logd;
+  const int t = threadIdx.x;
+
+  auto issue = [&](int64_t blk, int s) {                    // one thread
+    const int64_t row0 = blk * rows_per_block;
+    const int rows = (int)((n - row0 < rows_per_block) ? (n - row0) : rows_per_block);
+    const uint32_t row_bytes = (uint32_t)d * sizeof(TIn);
+    ptx::mbar_expect_tx(&full[s], (uint32_t)rows * row_bytes);
+    TIn* dst = stage + (size_t)s * NB;
+    if (ldx == d) {
+      ptx::bulk_load_1d(dst, X + row0 * ldx, (uint32_t)rows * row_bytes, &full[s]);
+    } else {
+      for (int r = 0; r < rows; ++r) ptx::bulk_load_1d(dst + (size_t)r * d, X + (row0 + r) * ldx, row_bytes, &full[s]);
+    }
+  };
+
+  if (t == 0) {
+    for (int s = 0; s < S; ++s) ptx::mbar_init(&full[s], 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  __syncthreads();
+  int issued = 0;
+  if (t == 0)
+    for (int s = 0; s < S; ++s) {
+      const int64_t blk = (int64_t)blockIdx.x + (int64_t)s * gridDim.x;
+      if (blk < nblocks) { issue(blk, s); ++issued; }
+    }
+  int s = 0;
+  uint32_t parity = 0;
+  bool bad = false;
+  for (int64_t blk = blockIdx.x; blk < nblocks; blk += gridDim.x) {
+    const bool ok = tc_wait(&full[s], parity, &abort_flag);
+    const int64_t row0 = blk * rows_per_block;
+    const TIn* src = stage + (size_t)s * NB;
+    // (the work buffer is free: the previous block's last group ended with a barrier)
+    had_first<TIn, E>(sm, logd, ok ? n - row0 : 0, [&](int i) { return src + i; });
+    // everyone has taken this block out of its stage (and knows whether a wait gave up)
+    if (__syncthreads_or(!ok)) { bad = true; break; }
+    if (t == 0) {
+      const int64_t nxt = blk + (int64_t)S * gridDim.x;
+      if (nxt < nblocks) { issue(nxt, s); ++issued; }
+    }
+    had_finish<TOut, E>(sm, logd, n - row0, scale, Y + row0 * ldy, ldy);
+    __syncthreads();
+    if (++s == S) { s = 0; parity ^= 1u; }
+  }
+  if (bad && t == 0) {
+    atomicOr(&g_aux_status_flags, STATUS_FLAG_TIMEOUT);
+    if (issued > 0) {                                       // let the copies in flight land before the CTA's shared memory goes
+      const long long t0 = clock64();
+      while (clock64() - t0 < 4000000ll) {}
+    }
+  }
+}
+
+template <typename TIn, typename TOut, int E, int S>
+inline int hadamard_launch_bulk(const TIn* X, int64_t ldx, TOut* Y, int64_t ldy, int64_t n, int logd, float scale,
+                                cudaStream_t s) {
+  constexpr int smem = had_bulk_smem_bytes<TIn, E, S>();
+  auto kern = hadamard_rows_bulk_kernel<TIn, TOut, E, S>;
+  static int attr_dev_mask = 0, ctas_per_sm = 0, sms = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (!(attr_dev_mask & (1 << (dev & 31)))) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas_per_sm, kern, HAD_THREADS, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (ctas_per_sm < 1) return CONQUR_ERR_UNSUPPORTED;
+    attr_dev_mask |= 1 << (dev & 31);
+  }
+  const int64_t rows_per_block = (HAD_THREADS * E) >> logd;
+  const int64_t nblocks = (n + rows_per_block - 1) / rows_per_block;
+  const int64_t grid = nblocks < (int64_t)sms * ctas_per_sm ? nblocks : (int64_t)sms * ctas_per_sm;
+  kern<<<(unsigned)grid, HAD_THREADS, smem, s>>>(X, ldx, Y, ldy, n, logd, scale, nblocks);
+  return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
 
 template <typename TIn, typename TOut>
 inline int hadamard_launch(const TIn* X, int64_t ldx, TOut* Y, int64_t ldy, int64_t n, int logd, cudaStream_t s) {
   const float scale = (float)(1.0 / sqrt((double)(1 << logd)));
+  const int d = 1 << logd;
+  // bulk copies need 16-byte aligned rows of a multiple of 16 bytes
+  const bool bulk = ((reinterpret_cast<uintptr_t>(X) & 15) == 0) && ((ldx * sizeof(TIn)) % 16 == 0) && ((d * sizeof(TIn)) % 16 == 0);
+  if (bulk) {
+    if (logd <= 12) return hadamard_launch_bulk<TIn, TOut, 16, sizeof(TIn) == 2 ? 4 : 3>(X, ldx, Y, ldy, n, logd, scale, s);
+    return hadamard_launch_bulk<TIn, TOut, 32, 2>(X, ldx, Y, ldy, n, logd, scale, s);
+  }
   if (logd <= 12) {
     const int64_t rows_per_block = (HAD_THREADS * 16) >> logd;
     const int64_t blocks = (n + rows_per_block - 1) / rows_per_block;

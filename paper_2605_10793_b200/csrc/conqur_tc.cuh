@@ -1288,13 +1288,23 @@ inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   if (ldo < N || (ldo % 4)) return CONQUR_ERR_INVALID_ARG;
   TcHost h{};
   h.prof = nullptr; h.ns_k = -1;
+  // device facts, looked up once per device (the queries cost milliseconds)
+  struct DevFacts { int known, major, sms, pair_clusters; };
+  static DevFacts facts[64] = {};
   int dev = 0;
-  cudaDeviceProp prop;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
-  if (prop.major != 10) return CONQUR_ERR_UNSUPPORTED;
-  h.num_sms = prop.multiProcessorCount;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONQUR_ERR_CUDA;
+  DevFacts& f = facts[dev];
+  if (!f.known) {
+    if (cudaDeviceGetAttribute(&f.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return CONQUR_ERR_CUDA;
+    f.pair_clusters = f.major == 10 ? tc_query_pair_clusters() : 0;
+    f.known = 1;
+  }
+  if (f.major != 10) return CONQUR_ERR_UNSUPPORTED;
+  h.num_sms = f.sms;
   h.device = dev;
-  h.pair_clusters = tc_query_pair_clusters();
+  h.pair_clusters = f.pair_clusters;
   const uint64_t mul = split ? 2 : 1;
   CUtensorMap ta, tb;
   int rc;

@@ -46,6 +46,31 @@ def test_hadamard_rows_match_the_matrix_definition(d, io):
     if io[1] == "bf16":
         bound = bound + 2.0 ** -8 * np.abs(ref)
     assert (np.abs(got - ref) <= bound + 1e-30).all(), float(np.max(np.abs(got - ref) / (bound + 1e-30)))
+    assert _B().conqur_hadamard_status() == 0
+
+
+@pytest.mark.parametrize("d,n", [(128, 40000), (4096, 3000), (8192, 700)])
+def test_hadamard_many_blocks_per_cta(d, n):
+    """More blocks than resident CTAs, so every CTA walks several blocks through its ring of stages; rows with an odd
+    16-byte-unaligned stride take the plain-load kernel and must agree bit for bit."""
+    torch = _torch()
+    B = _B()
+    x = torch.randn(n, d, device="cuda")
+    y = B.conqur_hadamard_rows(x)
+    assert B.conqur_hadamard_status() == 0
+    sel = np.random.default_rng(0).choice(n, size=64, replace=False)
+    ref = O.hadamard_rows(x[sel].cpu().numpy().astype(np.float64))
+    bound = np.log2(d) * 2.0 ** -24 * np.linalg.norm(x[sel].cpu().numpy().astype(np.float64), axis=1, keepdims=True)
+    assert (np.abs(y[sel].cpu().numpy() - ref) <= bound).all()
+    # involution over the whole array (every block of every CTA)
+    z = B.conqur_hadamard_rows(y)
+    assert torch.allclose(z, x, atol=1e-4)
+    xb = x.to(torch.bfloat16)
+    view = torch.zeros(n, d + 8, dtype=torch.bfloat16, device="cuda")
+    v4 = view[:, 4:4 + d]                                        # bf16 rows 8 bytes off a 16-byte boundary: plain-load kernel
+    v4.copy_(xb)
+    assert v4.data_ptr() % 16 == 8
+    assert torch.equal(B.conqur_hadamard_rows(v4, out_dtype=torch.float32), B.conqur_hadamard_rows(xb, out_dtype=torch.float32))
 
 
 def test_hadamard_strides_in_place_empty_and_argument_errors():
