@@ -32,7 +32,7 @@ from paper_2605_10793_b200 import inputs as I        # noqa: E402
 
 METRIC = "calibration tokens/sec at d=4096 (whole path incl. polar update every 8 batches)"
 # DRAM bytes per launch at d = 4096, n = 2048 from the ncu capture summarised under profiles/ (same kernels)
-NCU_DRAM_BYTES_PER_LAUNCH = {"rotate_target": 53.0e6, "accumulate": 114.8e6, "ns_poly": 78.4e6, "ns_next": 384.9e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"rotate_target": 53.6e6, "accumulate": 113.0e6, "ns_residual": 36.4e6, "ns_poly": 36.0e6, "ns_next": 235.6e6}
 WORKLOAD = "c2"
 
 
