@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libconqur.so")
 SOURCES = ["conqur.cu", "conqur_noalloc.cu"]
-HEADERS = ["conqur_internal.h", "conqur_simt.cuh", "conqur_tc.cuh", "conqur_tc_batched.cuh", "conqur_aux.cuh", "ns_schedule.h",
+HEADERS = ["conqur_internal.h", "conqur_simt.cuh", "conqur_tc.cuh", "conqur_tc_batched.cuh", "conqur_aux.cuh", "conqur_hadamard_tc.cuh", "ns_schedule.h",
            os.path.join("..", "..", "include", "conqur.h")]
 
 

@@ -19,6 +19,7 @@
 #include "conqur_tc.cuh"
 #include "conqur_tc_batched.cuh"
 #include "conqur_aux.cuh"
+#include "conqur_hadamard_tc.cuh"
 #include "ns_schedule.h"
 
 using namespace conqur;
@@ -795,6 +796,15 @@ extern "C" int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t
   while ((1 << logd) < d) ++logd;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   using bf = __nv_bfloat16;
+  // bf16 rows that lie back to back: the 128-point sub-transforms run on the tensor cores
+  const char* env = std::getenv("CONQUR_HADAMARD_SIMT");            // "1": CUDA-core kernels only (tests compare the two)
+  const bool simt_only = env && env[0] == '1';
+  if (!simt_only && in_dtype == CONQUR_BF16 && ldx == d && ldy == d && (reinterpret_cast<uintptr_t>(X_dev) & 15) == 0 &&
+      (reinterpret_cast<uintptr_t>(Y_dev) & 15) == 0 && (n * d) % 128 == 0) {
+    const int rc = (out_dtype == CONQUR_F32) ? hadamard_tc_launch(static_cast<const bf*>(X_dev), static_cast<float*>(Y_dev), n, logd, s)
+                                             : hadamard_tc_launch(static_cast<const bf*>(X_dev), static_cast<bf*>(Y_dev), n, logd, s);
+    if (rc != CONQUR_ERR_UNSUPPORTED) return rc;
+  }
   if (in_dtype == CONQUR_F32 && out_dtype == CONQUR_F32)
     return hadamard_launch(static_cast<const float*>(X_dev), ldx, static_cast<float*>(Y_dev), ldy, n, logd, s);
   if (in_dtype == CONQUR_F32)

@@ -70,7 +70,17 @@ def test_hadamard_many_blocks_per_cta(d, n):
     v4 = view[:, 4:4 + d]                                        # bf16 rows 8 bytes off a 16-byte boundary: plain-load kernel
     v4.copy_(xb)
     assert v4.data_ptr() % 16 == 8
-    assert torch.equal(B.conqur_hadamard_rows(v4, out_dtype=torch.float32), B.conqur_hadamard_rows(xb, out_dtype=torch.float32))
+    import os
+    y_tc = B.conqur_hadamard_rows(xb, out_dtype=torch.float32)           # contiguous bf16: tensor-core kernel
+    os.environ["CONQUR_HADAMARD_SIMT"] = "1"
+    try:
+        y_bulk = B.conqur_hadamard_rows(xb, out_dtype=torch.float32)     # the same rows through the bulk-copy CUDA-core kernel
+    finally:
+        del os.environ["CONQUR_HADAMARD_SIMT"]
+    assert torch.equal(B.conqur_hadamard_rows(v4, out_dtype=torch.float32), y_bulk)
+    assert B.conqur_hadamard_status() == 0
+    tol = float(np.log2(d)) * 2.0 ** -23 * torch.linalg.norm(xb.float(), dim=1, keepdim=True)
+    assert ((y_tc - y_bulk).abs() <= tol).all()
 
 
 def test_hadamard_strides_in_place_empty_and_argument_errors():
