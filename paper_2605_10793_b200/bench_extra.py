@@ -208,14 +208,14 @@ def run_hadamard(args, g, ClockSampler, peaks):
         print(json.dumps({
             "metric": "rows/sec of the online Walsh-Hadamard transform at d=4096", "value": g.world * n / (ms * 1e-3), "unit": "rows/s",
             "n_gpus": g.world, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"hadamard: {n} x {d} bf16 in, bf16 out", "l2": "256 MB in + 256 MB out per launch, larger than L2"},
             "clocks": clocks,
             "e2e": {"value": g.world * n / (ms_e2e * 1e-3), "unit": "rows/s", "h2d_bytes_per_step": int(nbytes / 2),
                     "d2h_bytes_per_step": int(nbytes / 2), "ms_per_step": ms_e2e},
             "gpu_launches": K,
             "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                         "traffic": None, "kernel": "hadamard_rows_kernel<bf16, bf16, 16>", "avg_launch_ms": ms,
+                         "traffic": None, "kernel": "hadamard_tc_kernel<bf16>", "avg_launch_ms": ms,
                          "bytes_per_launch": nbytes, "peak_source": peaks["source"]},
             "cpu_baseline": None}))
     D.finish(g)
