@@ -47,7 +47,9 @@ struct TcbStepArgs {
                               //    instead of (column, token, problem)
   QuantSpec qs;               // bits == 0: corner target of the rotated row; else per-token fake-quantisation first
   float* M;                   // P x 128 x 128 fp32 (without the 1/sqrt(d))
-  double* part_d;             // P objective partials (sum |y| * rnorm, or the quantised equivalent)
+  int S;                      // token splits per problem: work item i = (problem i / S, tiles [T (i % S) / S, T (i % S + 1) / S))
+  float* Mpart;               // S > 1: P * S partial cross-covariances (item order), summed into M by tcb_finish_kernel
+  double* part_d;             // P * S objective partials (sum |y| * rnorm, or the quantised equivalent), item order
   DevState* st;               // P
 };
 
@@ -103,12 +105,14 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int lp = 0;
       bool ok = true;
       int issued = 0;
-      for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+      for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
+        const int p = item / g.S, sp = item - p * g.S;
+        const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
         if (!tc_wait(&aux->rempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 11; break; }
         ptx::mbar_expect_tx(&aux->rfull, TCB_TILE_BYTES);
         ptx::tma_load_2d(sR, &tmR, &aux->rfull, 0, (g.p0 + p) * TCB_D);
         ptx::tma_load_2d(sR + 16384, &tmR, &aux->rfull, 64, (g.p0 + p) * TCB_D);
-        for (int t = 0; t < T; ++t) {
+        for (int t = t_begin; t < t_end; ++t) {
           if (!tc_wait(&aux->xempty[xs], xph ^ 1u, abort_flag)) { ok = false; timeout_site = 12; break; }
           uint8_t* dst = sX + xs * TCB_TILE_BYTES;
           ptx::mbar_expect_tx(&aux->xfull[xs], TCB_TILE_BYTES);
@@ -151,10 +155,12 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ++it2;
         return true;
       };
-      for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+      for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
+        const int sp = item % g.S;
+        const int T_item = (int)((long long)T * (sp + 1) / g.S) - (int)((long long)T * sp / g.S);
         if (!tc_wait(&aux->rfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 20; break; }
         if (!tc_wait(&aux->mempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 21; break; }
-        for (int t = 0; t < T && ok; ++t) {
+        for (int t = 0; t < T_item && ok; ++t) {
           const int yb = it & 1;
           if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 22; break; }
           if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
@@ -165,12 +171,12 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             ptx::umma_bf16(tmem_base + yb * 128, tc_smem_desc(xa + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024),
                            tc_smem_desc(sR_a + j * 2048, 16384, 1024), idesc1, j > 0 ? 1u : 0u);
           ptx::umma_commit(&aux->yfull[yb]);
-          if (t == T - 1) ptx::umma_commit(&aux->rempty);     // R may be replaced once every first product has run
+          if (t == T_item - 1) ptx::umma_commit(&aux->rempty);     // R may be replaced once every first product has run
           if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
           ++it;
           if (t > 0) ok = second_product(t == 1);
         }
-        if (ok) ok = second_product(T == 1);
+        if (ok) ok = second_product(T_item == 1);
         if (ok) ptx::umma_commit(&aux->mfull);
       }
     }
@@ -181,10 +187,12 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int r = q * 32 + lane;                   // token inside the tile; later: row of M
     int it = 0, lp = 0;
     bool ok = true;
-    for (int p = blockIdx.x; p < g.P && ok; p += gridDim.x, ++lp) {
+    for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
+      const int p = item / g.S, sp = item - p * g.S;
+      const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
       double acc = 0.0;
       int skipped = 0, nonfinite = 0;
-      for (int t = 0; t < T && ok; ++t, ++it) {
+      for (int t = t_begin; t < t_end && ok; ++t, ++it) {
         const int yb = it & 1, xs = it % TCB_XSTAGES;
         const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
@@ -280,18 +288,24 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       ptx::tc_fence_after();
       {
         const uint32_t t_addr = tmem_base + 256u + ((uint32_t)(q * 32) << 16);
-        float* dst = g.M + ((long long)p * TCB_D + r) * TCB_D;
+        // one item per problem: straight into M; several: into the item's partial (summed in item order afterwards)
+        float* dst = (g.S == 1) ? g.M + ((long long)p * TCB_D + r) * TCB_D : g.Mpart + ((long long)item * TCB_D + r) * TCB_D;
 #pragma unroll 1
         for (int cc = 0; cc < 2; ++cc) {
           const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
           float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
+          if (g.S == 1) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float4 o = d4[i];
-            o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
-            d4[i] = o;
+            for (int i = 0; i < 8; ++i) {
+              float4 o = d4[i];
+              o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
+              d4[i] = o;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
           }
         }
       }
@@ -308,8 +322,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         double tot = 0.0;
         int sk = 0, nf = 0;
         for (int i = 0; i < 8; ++i) { tot += aux->red_d[i]; sk += aux->red_i[i]; nf |= aux->red_f[i]; }
-        g.part_d[p] = tot;
-        if (sk) g.st[p].step_skipped += sk;                      // this CTA is the only writer of problem p's state
+        g.part_d[item] = tot;
+        if (sk) atomicAdd(reinterpret_cast<unsigned long long*>(&g.st[p].step_skipped), (unsigned long long)sk);
         if (nf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -326,6 +340,18 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
+}
+
+// M[p] += partial[p * S + 0] + ... + partial[p * S + S - 1], in that order.  grid (16, problems), 256 threads.
+static __global__ void tcb_sum_partials_kernel(float* __restrict__ M, const float* __restrict__ part, int S) {
+  const int p = blockIdx.y;
+  const int i = (blockIdx.x * 256 + threadIdx.x) * 4;
+  float4 m = *reinterpret_cast<const float4*>(M + (size_t)p * TCB_D * TCB_D + i);
+  for (int sp = 0; sp < S; ++sp) {
+    const float4 v = *reinterpret_cast<const float4*>(part + ((size_t)p * S + sp) * TCB_D * TCB_D + i);
+    m.x += v.x; m.y += v.y; m.z += v.z; m.w += v.w;
+  }
+  *reinterpret_cast<float4*>(M + (size_t)p * TCB_D * TCB_D + i) = m;
 }
 
 // fp32 -> bf16 staging of a batched input (problem p, row i at X + p*pstride + i*ld) into a dense P x n x 128 copy
@@ -399,7 +425,14 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   TcbStepArgs g{};
   g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
   g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0;
-  const int grid = np < h.num_sms ? np : h.num_sms;
+  // few problems: split each problem's tokens over several CTAs (partials land in the idle Newton-Schulz buffers,
+  // 4 P matrices of 128 x 128 starting at Xa, and are summed in a fixed order)
+  const int T = (int)((n + 127) / 128);
+  int S = 1;
+  if (np < h.num_sms) S = std::max(1, std::min(std::min(h.num_sms / np, T), 4 * h.P / np));
+  g.S = S; g.Mpart = h.Xa;
+  const int items = np * S;
+  const int grid = items < h.num_sms ? items : h.num_sms;
   Prof::Rec rec{};
   const bool timed = h.prof && h.prof->enabled;
   if (timed) {
@@ -411,7 +444,12 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_ROTATE);
-  finalize_step_kernel<<<np, 256, 0, s>>>(g.st, h.part_d, 1, n, 1.0 / std::sqrt((double)TCB_D));
+  if (S > 1) {
+    tcb_sum_partials_kernel<<<dim3(16, np), 256, 0, s>>>(g.M, g.Mpart, S);
+    if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+    if (h.prof) h.prof->count(K_OTHER);
+  }
+  finalize_step_kernel<<<np, 256, 0, s>>>(g.st, h.part_d, S, n, 1.0 / std::sqrt((double)TCB_D));
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_OTHER);
   return CONQUR_OK;
