@@ -56,7 +56,7 @@ hadamard_tc_kernel(const __grid_constant__ CUtensorMap tmX, TOut* Y, long long N
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < HTC_STAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->dfull[b], 1); ptx::mbar_init(&aux->dempty[b], 32 * HTC_EPI_WARPS); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->dfull[b], 1); ptx::mbar_init(&aux->dempty[b], HTC_EPI_WARPS); }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmX);
@@ -177,7 +177,8 @@ hadamard_tc_kernel(const __grid_constant__ CUtensorMap tmX, TOut* Y, long long N
         }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&aux->dempty[buf]);
+      __syncwarp();                                // one arrival per warp
+      if (lane == 0) ptx::mbar_arrive(&aux->dempty[buf]);
     }
   }
 

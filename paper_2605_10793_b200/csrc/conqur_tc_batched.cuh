@@ -23,6 +23,7 @@ constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = tw
 constexpr int TCB_XSTAGES = 3;
 constexpr int TCB_THREADS = 320;                 // 2 + 8 warps
 constexpr int TCB_EPI_THREADS = 256;
+constexpr int TCB_EPI_WARPS = TCB_EPI_THREADS / 32;
 constexpr int TCB_AUX_BYTES = 4096;
 constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + TCB_AUX_BYTES + 1024;
 
@@ -80,11 +81,11 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
-    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, TCB_EPI_THREADS);
+    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, TCB_EPI_WARPS);
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
     for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_THREADS);
-      ptx::mbar_init(&aux->cready[b], TCB_EPI_THREADS); ptx::mbar_init(&aux->cfree[b], 1);
+      ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
+      ptx::mbar_init(&aux->cready[b], TCB_EPI_WARPS); ptx::mbar_init(&aux->cfree[b], 1);
     }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
@@ -259,15 +260,16 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               w[i] = live ? (lo | (hi << 16)) : 0u;
             }
           } else {
-            // two elements per instruction: sign bits and a non-zero mask from the packed bf16 pair
+            // two elements per instruction: sign bits and a non-zero mask from the packed bf16 pair.  mag + 0x7fff sets
+            // bit 15 of a half exactly when the half is non-zero; the byte permute spreads that bit over the half.
             const uint32_t rn2 = live ? (rn_bits | (rn_bits << 16)) : 0u;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const float a = v[2 * i], b = v[2 * i + 1];
               acc_t += fabsf(a) + fabsf(b);
               const uint32_t pk = bf16x2_pack(a, b);
-              const uint32_t mag = pk & 0x7fff7fffu;
-              const uint32_t nz = (((mag + 0x7fff7fffu) >> 15) & 0x00010001u) * 0xffffu;     // 0xffff per non-zero half
+              uint32_t nz;                                    // 0xffff per non-zero half (prmt: selector msb = replicate the byte's sign)
+              asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(nz) : "r"((pk & 0x7fff7fffu) + 0x7fff7fffu));
               w[i] = (rn2 | (pk & 0x80008000u)) & nz;
             }
           }
@@ -279,8 +281,11 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
         ptx::tc_fence_before();
         ptx::fence_proxy_async();
-        ptx::mbar_arrive(&aux->cready[yb]);
-        ptx::mbar_arrive(&aux->yempty[yb]);
+        __syncwarp();                              // one arrival per warp: every lane's fences precede it
+        if (lane == 0) {
+          ptx::mbar_arrive(&aux->cready[yb]);
+          ptx::mbar_arrive(&aux->yempty[yb]);
+        }
       }
       if (!ok) break;
       // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T)
@@ -310,7 +315,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&aux->mempty);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&aux->mempty);
       // per-problem reductions in a fixed order (named barrier 1: the eight epilogue warps only)
       const double wsum = warp_sum_d(acc);
       int wsk = skipped, wnf = nonfinite;
