@@ -687,7 +687,7 @@ extern "C" int conqur_debug_gemm(const void* A_dev, const void* B_dev, float* D_
   if (!A_dev || !B_dev || !D_dev || !scratch_dev) return CONQUR_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   CQ_CUDA(cudaMemsetAsync(scratch_dev, 0, sizeof(DevState), s));
-  int rc = tc_debug_gemm(static_cast<const __nv_bfloat16*>(A_dev), static_cast<const __nv_bfloat16*>(B_dev), D_dev, M,
+  int rc = tc_plain_gemm(static_cast<const __nv_bfloat16*>(A_dev), static_cast<const __nv_bfloat16*>(B_dev), D_dev, M,
                          N, K, a_mn_major, b_mn_major, split, static_cast<DevState*>(scratch_dev), s);
   if (rc) return rc;
   DevState h;
@@ -760,9 +760,9 @@ extern "C" int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows,
     CQ_LAUNCH_CHECK();
     int rc;
     if (side == CONQUR_FOLD_INPUT)     // out (rows x d) = W R: A = W, K-major; B(n, k) = R[k][n], MN-major
-      rc = tc_debug_gemm(Ws, Rs, out_dev, rows, d, d, 0, 1, 1, st, s, ldo);
+      rc = tc_plain_gemm(Ws, Rs, out_dev, rows, d, d, 0, 1, 1, st, s, ldo);
     else                               // out (d x cols) = R^T W: A(m, k) = R[k][m] and B(n, k) = W[k][n], both MN-major
-      rc = tc_debug_gemm(Rs, Ws, out_dev, d, cols, d, 1, 1, 1, st, s, ldo);
+      rc = tc_plain_gemm(Rs, Ws, out_dev, d, cols, d, 1, 1, 1, st, s, ldo);
     if (rc) return rc;
     DevState h;
     CQ_CUDA(cudaMemcpyAsync(&h, st, sizeof(DevState), cudaMemcpyDeviceToHost, s));

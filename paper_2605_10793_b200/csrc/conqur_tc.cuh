@@ -1281,7 +1281,7 @@ inline const __nv_bfloat16* tc_cp_ptr(const TcHost& h) { return reinterpret_cast
 // Stand-alone product (tests, weight folding): D (fp32, M x N, row stride ldo; 0 = N) = A * B^T-style contraction with
 // the given orientations.  a_mn / b_mn: 0 = K-major ([M|N rows][K cols]), 1 = MN-major ([K rows][M|N cols]).  split:
 // operands are stacked [hi; lo] pairs (3 products).  All device pointers; bf16 operands; shapes as checked below.
-inline int tc_debug_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* D, int M, int N, int K, int a_mn,
+inline int tc_plain_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* D, int M, int N, int K, int a_mn,
                          int b_mn, int split, DevState* st, cudaStream_t s, long long ldo = 0) {
   if (M < 1 || N < 32 || (N % 32) || K < 1 || (K % 8) || (M % 8)) return CONQUR_ERR_INVALID_ARG;
   if (ldo == 0) ldo = N;
