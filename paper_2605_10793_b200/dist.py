@@ -83,3 +83,43 @@ def finish(g: Group) -> None:
     if g.active:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+class TokenSharded:
+    """One rotation calibrated on token shards: every rank holds the same R and streams its own rows through its own
+    context; at update time the statistics of the Procrustes problem -- the cross-covariance M (d x d) and the
+    objective sums J, N, all plain sums over tokens (Sections 3.3-3.4) -- are summed over the ranks with one
+    all-reduce each, after which every rank runs the same update on the same M and ends with the same R.
+
+    `ctx` is a single-problem calibration context (step / get_M / set_M / get_objective / update / get_R, as
+    binding.Context); with NCCL the all-reduce runs on the context's device tensors.  The sum enters the context
+    through conqur_get_M / conqur_set_M, i.e. two extra d x d copies per update.
+    Not run on more than one GPU so far (single-GPU runs only); the exchange logic is covered by a two-rank gloo test
+    with a CPU stand-in for the context.
+    """
+
+    def __init__(self, ctx, g: Group):
+        self.ctx, self.g = ctx, g
+
+    def step(self, x_local):
+        self.ctx.step(x_local)
+
+    def reduce_statistics(self):
+        """All-reduce (sum) M, J, N over the ranks; returns the global (J, N)."""
+        j, n = self.ctx.get_objective()
+        if not self.g.active:
+            return j, n
+        import torch
+        import torch.distributed as dist
+        m = self.ctx.get_M()
+        jn = torch.tensor([float(j), float(n)], dtype=torch.float64, device=m.device)
+        dist.all_reduce(m, op=dist.ReduceOp.SUM)
+        dist.all_reduce(jn, op=dist.ReduceOp.SUM)
+        j_tot, n_tot = float(jn[0].item()), int(round(float(jn[1].item())))
+        self.ctx.set_M(m, [j_tot], [n_tot])
+        return j_tot, n_tot
+
+    def update(self):
+        jn = self.reduce_statistics()
+        self.ctx.update()
+        return jn
