@@ -31,12 +31,12 @@ struct TcbAux {
   uint64_t rfull, rempty, mfull, mempty;
   uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
   uint64_t yfull[2], yempty[2], cready[2], cfree[2];
-  uint64_t gfull, gempty;
   uint32_t tmem_base;
   int abort_flag;
   double red_d[8];
   int red_i[8];
   int red_f[8];
+  float ss_x[2][2][128];     // [tile parity][column half][row]: half-row sums of squares exchanged between the two warps of a row
 };
 
 static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
@@ -82,7 +82,6 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
     ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, TCB_EPI_WARPS);
-    ptx::mbar_init(&aux->gfull, 1); ptx::mbar_init(&aux->gempty, TCB_EPI_WARPS);
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
@@ -98,8 +97,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
-  const uint32_t tmem_base = aux->tmem_base;     // columns [0,128) and [128,256): Y buffers; [256,384): M accumulator;
-                                                 // [384,512): Gram matrix of the tile (its diagonal = the rows' sums of squares)
+  const uint32_t tmem_base = aux->tmem_base;     // columns [0,128) and [128,256): Y buffers; [256,384): M accumulator
   int timeout_site = 0;
 
   if (warp == 0) {
@@ -166,19 +164,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         for (int t = 0; t < T_item && ok; ++t) {
           const int yb = it & 1;
           if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 22; break; }
-          const uint32_t xa = sX_a + xs * TCB_TILE_BYTES;
-          // a1 on the tensor cores: G = X_tile X_tile^T (both operands the K-major tile, exact bf16 products, fp32 sums);
-          // the epilogue takes the diagonal as the rows' sums of squares
-          if (!tc_wait(&aux->gempty, ((uint32_t)it & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 25; break; }
-          ptx::tc_fence_after();
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint64_t xd = tc_smem_desc(xa + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024);
-            ptx::umma_bf16(tmem_base + 384u, xd, xd, idesc_base, j > 0 ? 1u : 0u);
-          }
-          ptx::umma_commit(&aux->gfull);
           if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
           ptx::tc_fence_after();
+          const uint32_t xa = sX_a + xs * TCB_TILE_BYTES;
 #pragma unroll
           for (int j = 0; j < 8; ++j)        // 16 features per instruction: chunk j/4, 32 bytes per step inside the swizzled row
             ptx::umma_bf16(tmem_base + yb * 128, tc_smem_desc(xa + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024),
@@ -209,22 +197,24 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int yb = it & 1, xs = it % TCB_XSTAGES;
         const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
-        // a1: the row's sum of squares is element (r, r) of the tile's Gram matrix in TMEM: this warp's lane quarter and
-        // the matching 32 columns hold the diagonal block, lane l takes column l
+        // a1: row norm from the tile in shared memory: each of the row's two warps sums its half of the columns and
+        // they swap the halves (named barriers 2..5, one per TMEM lane quarter; both warps have just passed the
+        // same wait, so both arrive).  The two halves are added in a fixed order.
         uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
-        if (!tc_wait(&aux->gfull, (uint32_t)it & 1u, abort_flag)) { ok = false; timeout_site = 34; break; }
-        ptx::tc_fence_after();
-        float ss;
-        {
-          float gv[32];
-          ptx::tmem_ld32(tmem_base + 384u + (uint32_t)(q * 32) + ((uint32_t)(q * 32) << 16), gv);
-          ss = gv[0];
+        float ssh = 0.f;
 #pragma unroll
-          for (int k = 1; k < 32; ++k) ss = (lane == k) ? gv[k] : ss;
+        for (int c = 0; c < 8; ++c) {
+          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, half * 8 + c));
+          const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float a = __uint_as_float(u[e] << 16), b = __uint_as_float(u[e] & 0xffff0000u);
+            ssh = fmaf(a, a, ssh); ssh = fmaf(b, b, ssh);
+          }
         }
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&aux->gempty);
+        aux->ss_x[it & 1][half][r] = ssh;
+        asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
+        const float ss = aux->ss_x[it & 1][0][r] + aux->ss_x[it & 1][1][r];
         const bool valid = (t * 128 + r) < g.n;
         const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
         if (valid && !good) {
