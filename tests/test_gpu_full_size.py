@@ -189,3 +189,62 @@ def test_c4b_1024_heads_sampled_problems():
         assert rep["orth"] <= T["orth"] and rep["gap"] <= T["gap"], (p, rep)
     # identical problems give bit-identical results wherever they ran
     assert np.array_equal(ms[5], ms[64 + 5]) and np.array_equal(rs[5], rs[64 * 7 + 5])
+
+
+def test_fold_hadamard_and_algorithm1_legs_at_bench_sizes():
+    """The three extra bench legs at the sizes bench.py times them, on outputs the oracle can afford:
+    weight folding R^T W with W 4096 x 14336 (tensor-core mode) on sampled output columns; the Walsh-Hadamard
+    transform of 32768 x 4096 bf16 rows on sampled rows; block 0 of the 8B-class Algorithm-1 mini-batch (4096 tokens:
+    two residual-stream steps at d = 4096 and the 32 head problems) on objective, token counts and sampled heads."""
+    torch = _torch()
+    from paper_2605_10793_b200 import algorithm1 as A1
+    from paper_2605_10793_b200 import binding as B
+    rng = np.random.default_rng(11)
+    # --- fold
+    d, cols = 4096, 14336
+    w = I.random_weight(1, d, cols)
+    q, _ = np.linalg.qr(np.random.default_rng(2).standard_normal((d, d)))
+    r = q.astype(np.float32)
+    out = B.conqur_fold_weight(torch.from_numpy(w).cuda(), torch.from_numpy(r).cuda(), "output", "tc").cpu().numpy()
+    sel = rng.choice(cols, size=48, replace=False)
+    ref = r.astype(np.float64).T @ w[:, sel].astype(np.float64)
+    assert np.linalg.norm(out[:, sel] - ref) / np.linalg.norm(ref) <= 2e-5
+    mag = np.abs(r.astype(np.float64)).T @ np.abs(w[:, sel].astype(np.float64))
+    assert np.max(np.abs(out[:, sel] - ref) / mag) <= 8e-5
+    del out
+    # --- Hadamard
+    n = 32768
+    x = torch.randn(n, d, device="cuda").to(torch.bfloat16)
+    y = B.conqur_hadamard_rows(x)
+    assert B.conqur_hadamard_status() == 0
+    rows = rng.choice(n, size=32, replace=False)
+    xs = x[rows].float().cpu().numpy().astype(np.float64)
+    ref = O.hadamard_rows(xs)
+    got = y[rows].float().cpu().numpy().astype(np.float64)
+    bound = np.log2(d) * 2.0 ** -24 * np.linalg.norm(xs, axis=1, keepdims=True) + 2.0 ** -8 * np.abs(ref)
+    assert (np.abs(got - ref) <= bound).all()
+    del x, y
+    # --- Algorithm 1, block 0 of a mini-batch
+    a = I.SITE_MODELS["a1_8b"]
+    cal = A1.Calibrator(a.d, a.n_heads, a.d_head, a.n_layers, a.n, in_dtype="bf16", mode="tc")
+    r1, r2 = I.site_initial_rotations(a)
+    cal.set_rotations(torch.from_numpy(r1).cuda(), torch.from_numpy(r2).cuda())
+    s = I.site_activations(a, 0, 0)
+    dev = {k: torch.from_numpy(v).cuda().to(torch.bfloat16) for k, v in s.items()}
+    cal.collect(0, dev["attn"], dev["mlp"], dev["o"])
+    j1, n1 = cal.ctx1.get_objective()
+    j_ref = 0.0
+    for k in ("attn", "mlp"):
+        xt, used = O.normalise_rows(s[k].astype(np.float64))
+        j_ref += np.abs(xt @ r1.astype(np.float64)).sum() / np.sqrt(a.d)
+        assert used.all()
+    assert n1 == 2 * a.n and abs(j1 - j_ref) / j_ref <= T["J"]
+    j2, n2 = cal.ctx2.get_objective()
+    m2 = cal.ctx2.get_M().cpu().numpy().astype(np.float64)
+    assert (n2[:a.n_heads] == a.n).all() and not n2[a.n_heads:].any()          # only block 0's problems were fed
+    for h in (0, 13, 31):
+        oh = O.OpuOracle(a.d_head, r2[0, h].astype(np.float64)).step(s["o"][:, h * a.d_head:(h + 1) * a.d_head].astype(np.float64))
+        assert abs(j2[h] - oh.J) / oh.J <= T["J"], h
+        assert np.linalg.norm(m2[h] - oh.M) / np.linalg.norm(oh.M) <= 3e-2, h
+    assert B.conqur_update(cal.ctx2.h) == -4                                    # the other blocks' problems have no rows yet
+    cal.close()
