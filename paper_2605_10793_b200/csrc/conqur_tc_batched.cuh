@@ -546,8 +546,10 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
   // descriptor of k-step j (16 of the 128 contraction indices) of a 128 x 128 tile held as two swizzled 64-column chunks
   auto desc_k = [](uint32_t base, int j) { return tc_smem_desc(base + (j >> 2) * 16384 + (j & 3) * 32, 16, 1024); };   // contraction along columns
   auto desc_mn = [](uint32_t base, int j) { return tc_smem_desc(base + j * 2048, 16384, 1024); };                        // contraction along rows
-  // all threads: make shared-memory writes visible to the tensor cores, then thread 0 issues `issue` and everyone waits
-  auto run_products = [&](auto issue) -> bool {
+  // all threads: make shared-memory writes visible to the tensor cores, then thread 0 issues `issue`; the block barrier
+  // inside also publishes whatever the threads wrote to the control block before the call.  wait_products: everyone
+  // waits for the products issued last.  Work placed between the two overlaps the products.
+  auto issue_products = [&](auto issue) {
     ptx::fence_proxy_async();
     ptx::tc_fence_before();
     __syncthreads();
@@ -556,10 +558,20 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       issue();
       ptx::umma_commit(&aux->mbar);
     }
+  };
+  auto wait_products = [&]() -> bool {
     const bool okw = tc_wait(&aux->mbar, mph, abort_flag);
     mph ^= 1u;
     ptx::tc_fence_after();
     return okw;
+  };
+  auto issue_gram = [&] {                          // G = X^T X (hi hi + hi lo + lo hi)
+    const uint32_t aa[3] = {aXh, aXh, aXl}, bb[3] = {aXh, aXl, aXh};
+#pragma unroll
+    for (int seg = 0; seg < 3; ++seg)
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        ptx::umma_bf16(tmem_base, desc_mn(aa[seg], j), desc_mn(bb[seg], j), idesc_mm, (seg > 0 || j > 0) ? 1u : 0u);
   };
 
   for (int p = blockIdx.x; p < g.P && !timed_out; p += gridDim.x) {
@@ -610,16 +622,12 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         *reinterpret_cast<uint4*>(sXh + tcb_piece(r, c16)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
         *reinterpret_cast<uint4*>(sXl + tcb_piece(r, c16)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
       }
+      issue_products(issue_gram);
+      bool gram_in_flight = true;
       for (int k = 0; k <= ncp.max_steps; ++k) {
-        // ---- G = X^T X
-        if (!run_products([&] {
-              const uint32_t aa[3] = {aXh, aXh, aXl}, bb[3] = {aXh, aXl, aXh};
-#pragma unroll
-              for (int seg = 0; seg < 3; ++seg)
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  ptx::umma_bf16(tmem_base, desc_mn(aa[seg], j), desc_mn(bb[seg], j), idesc_mm, (seg > 0 || j > 0) ? 1u : 0u);
-            })) { timed_out = true; break; }
+        // ---- G = X^T X (issued before the loop / at the end of the previous step)
+        gram_in_flight = false;
+        if (!wait_products()) { timed_out = true; break; }
         // ---- statistics of G - I; E = G - tau I
         const float tau = aux->tau;
         float mx = 0.f, tr = 0.f;
@@ -649,27 +657,28 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           const double wsq = warp_sum_d(sq), wtr = warp_sum_d((double)tr);
           const float wmx = warp_max(mx);
           if (lane == 0) { aux->red_d[warp] = wsq; aux->red_t[warp] = wtr; aux->red_f[warp] = wmx; }
-          __syncthreads();
-          if (threadIdx.x == 0) {
-            double tsq = 0.0, ttr = 0.0;
-            float tmx = 0.f;
-            for (int i = 0; i < 8; ++i) { tsq += aux->red_d[i]; ttr += aux->red_t[i]; tmx = fmaxf(tmx, aux->red_f[i]); }
-            ns_control_decide(s, tmx, tsq, ttr, k, 0, ncp);
-            aux->done = s->ns_done;
-            aux->coef[0] = s->coef[0]; aux->coef[1] = s->coef[1]; aux->coef[2] = s->coef[2]; aux->coef[3] = s->coef[3];
-            aux->seg_x = s->seg_x;
-          }
-          __syncthreads();
         }
+        // ---- E E, which does not depend on the control decision: issued first, the decision is taken while it runs
+        // (a step that turns out to be the last one throws the product away)
+        issue_products([&] {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            ptx::umma_bf16(tmem_base + 128, desc_k(aEB, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
+        });
+        if (threadIdx.x == 0) {
+          double tsq = 0.0, ttr = 0.0;
+          float tmx = 0.f;
+          for (int i = 0; i < 8; ++i) { tsq += aux->red_d[i]; ttr += aux->red_t[i]; tmx = fmaxf(tmx, aux->red_f[i]); }
+          ns_control_decide(s, tmx, tsq, ttr, k, 0, ncp);
+          aux->done = s->ns_done;
+          aux->coef[0] = s->coef[0]; aux->coef[1] = s->coef[1]; aux->coef[2] = s->coef[2]; aux->coef[3] = s->coef[3];
+          aux->seg_x = s->seg_x;
+        }
+        __syncthreads();
+        if (!wait_products()) { timed_out = true; break; }
         if (aux->done) break;
         const float cg = aux->coef[0], cb1 = aux->coef[1], cb2 = aux->coef[2], ck = aux->coef[3];
         const int seg_x = aux->seg_x;
-        // ---- E E
-        if (!run_products([&] {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                ptx::umma_bf16(tmem_base + 128, desc_k(aEB, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
-            })) { timed_out = true; break; }
         // ---- B = beta2 E E + beta1 E - kappa I (over E: the product that read it has finished)
 #pragma unroll 1
         for (int c = half * 2; c < half * 2 + 2; ++c) {
@@ -692,14 +701,15 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
             *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
         }
         // ---- X B
-        if (!run_products([&] {
+        issue_products([&] {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXh, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
-              if (seg_x > 1) {
+          for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXh, j), desc_mn(aEB, j), idesc_km, j > 0 ? 1u : 0u);
+          if (seg_x > 1) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXl, j), desc_mn(aEB, j), idesc_km, 1u);
-              }
-            })) { timed_out = true; break; }
+            for (int j = 0; j < 8; ++j) ptx::umma_bf16(tmem_base, desc_k(aXl, j), desc_mn(aEB, j), idesc_km, 1u);
+          }
+        });
+        if (!wait_products()) { timed_out = true; break; }
         // ---- X <- (gamma + kappa) X + X B; tau of the next step
         double x2 = 0.0;
 #pragma unroll 1
@@ -726,9 +736,21 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           }
           x2 += (double)x2f;
         }
-        const double tx2 = tcbu_block_sum(x2, aux->red_d, warp, lane);
-        if (threadIdx.x == 0) { s->tau = (float)(tx2 / (double)TCB_D); aux->tau = s->tau; }
+        {
+          const double wx2 = warp_sum_d(x2);
+          if (lane == 0) aux->red_d[warp] = wx2;
+        }
+        // ---- the next step's G needs the new iterate but not its tau: issued now, tau is summed while it runs
+        if (k < ncp.max_steps) { issue_products(issue_gram); gram_in_flight = true; } else { __syncthreads(); }
+        if (threadIdx.x == 0) {
+          const double tx2 = ((aux->red_d[0] + aux->red_d[1]) + (aux->red_d[2] + aux->red_d[3])) +
+                             ((aux->red_d[4] + aux->red_d[5]) + (aux->red_d[6] + aux->red_d[7]));
+          s->tau = (float)(tx2 / (double)TCB_D); aux->tau = s->tau;
+        }
         __syncthreads();
+      }
+      if (gram_in_flight && !timed_out) {          // nothing may be in flight when the tiles are reused
+        if (!wait_products()) timed_out = true;
       }
     }
     if (timed_out) break;
