@@ -215,7 +215,10 @@ def run_hadamard(args, g, ClockSampler, peaks):
                     "d2h_bytes_per_step": int(nbytes / 2), "ms_per_step": ms_e2e},
             "gpu_launches": K,
             "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                         "traffic": None, "kernel": "hadamard_tc_kernel<bf16>", "avg_launch_ms": ms,
+                         "traffic": 218.1e6 * n / 16384, "kernel": "hadamard_tc_kernel<bf16>", "avg_launch_ms": ms,
+                         "traffic_note": "dram read+write of an ncu capture at 16384 rows (134.3 MB read = the input once, 83.8 MB "
+                                         "written by the end of the launch, the rest of the output still in L2; "
+                                         "profiles/hadamard_kernels_d4096_n16384_ncu.md), scaled by the rows processed",
                          "bytes_per_launch": nbytes, "peak_source": peaks["source"]},
             "cpu_baseline": None}))
     D.finish(g)
