@@ -328,18 +328,24 @@ int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows, int32_t co
 
 /*
  * The fixed online rotations R_3 / R_4 of Appendix A: every row times the orthonormal Walsh-Hadamard matrix,
- *   y = x H_d / sqrt(d),   H_d the Sylvester matrix, H[i][j] = (-1)^popcount(i & j),
- * computed with log2(d) butterfly stages in fp32 (no matrix is formed).  d a power of two, 4 <= d <= 8192.
+ *   y = x H_d / sqrt(d),   H_d the Sylvester matrix, H[i][j] = (-1)^popcount(i & j).
+ * d a power of two, 4 <= d <= 8192.
  *   X_dev   device, n rows of d elements of in_dtype (CONQUR_F32 | CONQUR_BF16), row stride ldx elements
  *   Y_dev   device, n rows of d elements of out_dtype, row stride ldy; may be X_dev itself (same type and
  *           stride): every row is read completely before it is written
  *   ldx, ldy multiples of 4; pointers aligned to 4 elements.
  * Enqueued on the stream; not synchronised.  Invalid arguments return CONQUR_ERR_INVALID_ARG and do nothing.
- * Rows that start on 16-byte boundaries (X_dev and ldx * element size multiples of 16, d * element size too) are
- * staged through shared memory by bulk asynchronous copies; other layouts take a plain-load kernel.
+ * Arithmetic: fp32 throughout, error per element <= log2(d) 2^-24 ||x||_2 (plus the rounding of a bf16 output).
+ *   - bf16 rows lying back to back (ldx == ldy == d, 16-byte aligned pointers, n*d a multiple of 128): H_d is
+ *     taken as H_{d/128} (x) H_128; the 128-point transforms of all 128-element chunks run as one tensor-core
+ *     product per tile with exact operands (the bf16 input and a +-1 matrix, fp32 accumulation), the remaining
+ *     log2(d/128) butterfly levels in registers.  No d x d matrix is formed.
+ *   - every other layout (fp32 input, strided or unaligned rows): log2(d) butterfly levels on the CUDA cores; rows
+ *     that start on 16-byte boundaries are staged through shared memory by bulk asynchronous copies, others by
+ *     plain loads.
  *
  * conqur_hadamard_status: synchronises the stream and returns CONQUR_ERR_TIMEOUT if, since the last call on
- * this device, a transform kernel abandoned a bounded wait for one of its bulk copies (its output is then
+ * this device, a transform kernel abandoned a bounded wait for one of its copies or products (its output is then
  * incomplete), CONQUR_OK otherwise; clears the latch.
  */
 int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,

@@ -101,6 +101,11 @@ def test_hadamard_strides_in_place_empty_and_argument_errors():
     assert np.allclose(z.cpu().numpy(), ref, atol=2e-5)
     B.conqur_hadamard_rows(z, out=z)
     assert torch.allclose(z, z0, atol=2e-5)
+    # in place on contiguous bf16 rows (the tensor-core kernel): same result as out of place
+    zb = torch.randn(3000, 1024, device="cuda").to(torch.bfloat16)
+    want = B.conqur_hadamard_rows(zb)
+    B.conqur_hadamard_rows(zb, out=zb)
+    assert torch.equal(zb, want) and B.conqur_hadamard_status() == 0
     # empty input is a no-op; bad sizes are refused
     e = torch.empty(0, d, device="cuda")
     assert B.conqur_hadamard_rows(e).shape == (0, d)
