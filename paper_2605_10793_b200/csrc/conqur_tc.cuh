@@ -773,6 +773,39 @@ __global__ void __launch_bounds__(256) rownorm_stage_kernel(const TIn* __restric
   const int lane = threadIdx.x & 31;
   if (row >= n) return;
   const TIn* x = X + row * ld;
+  __nv_bfloat16* dst = Xs + row * (int64_t)d;
+  if (sizeof(TIn) == 2 && d <= 4096 && (d & 255) == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+    // bf16 rows of up to 4096 elements: the whole row sits in the warp's registers (16-byte pieces, all loads in
+    // flight at once), is read from memory once and written out from the registers
+    const int nchunk = d >> 8;                          // 256 elements = 32 lanes x 16 bytes
+    uint4 buf[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      buf[c] = (c < nchunk) ? __ldg(reinterpret_cast<const uint4*>(x + c * 256 + lane * 8)) : make_uint4(0u, 0u, 0u, 0u);
+    float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const uint32_t u[4] = {buf[c].x, buf[c].y, buf[c].z, buf[c].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float a = __uint_as_float(u[e] << 16), b = __uint_as_float(u[e] & 0xffff0000u);
+        s4[e] = fmaf(a, a, s4[e]); s4[e] = fmaf(b, b, s4[e]);
+      }
+    }
+    const float ssr = warp_sum((s4[0] + s4[1]) + (s4[2] + s4[3]));
+    const bool goodr = (ssr > 0.f) && (ssr <= 3.0e38f);
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      if (c < nchunk) *reinterpret_cast<uint4*>(dst + c * 256 + lane * 8) = goodr ? buf[c] : make_uint4(0u, 0u, 0u, 0u);
+    if (lane == 0) {
+      if (!goodr) {
+        atomicAdd(reinterpret_cast<unsigned long long*>(&st->step_skipped), 1ull);
+        if (!(ssr == 0.f)) atomicOr(&st->status_flags, STATUS_FLAG_NONFINITE);
+      }
+      rnorm[row] = goodr ? 1.0f / sqrtf(ssr) : 0.f;
+    }
+    return;
+  }
   const bool vec = (reinterpret_cast<uintptr_t>(x) & (sizeof(TIn) * 4 - 1)) == 0;    // d is a multiple of 128
   float ss = 0.f;
   for (int k = lane * 4; k < d; k += 128) {
@@ -793,7 +826,6 @@ __global__ void __launch_bounds__(256) rownorm_stage_kernel(const TIn* __restric
   }
   ss = warp_sum(ss);
   const bool good = (ss > 0.f) && (ss <= 3.0e38f);
-  __nv_bfloat16* dst = Xs + row * (int64_t)d;
   for (int k = lane * 4; k < d; k += 128) {
     float v[4] = {0.f, 0.f, 0.f, 0.f};
     if (good) {
