@@ -13,7 +13,7 @@ import numpy as np
 
 from oracle import conqur_oracle as O
 
-# tolerances (benchmark spec): exact fp32 mode / bf16 tensor-core mode
+# tolerances: exact fp32 mode / bf16 tensor-core mode (M and J: stated requirements of the path; orth, gap: derived from the arithmetic)
 TOL = {
     "exact": {"M": 1e-5, "J": 1e-6, "orth": 1e-4, "gap": 2e-5},
     "tc": {"M": 1e-2, "J": 1e-3, "orth": 1e-4, "gap": 1e-3},
