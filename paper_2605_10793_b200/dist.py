@@ -1,8 +1,10 @@
 """Process-group plumbing for multi-GPU runs (one process per GPU, launched by torchrun).
 
-The calibration path of one rotation does not shard in this build (one context = one GPU), so N > 1
-means N independent replicas: no data-path collective.  The only communication is the barrier around
-the timed region and a max-reduction of the measured time.  Works with NCCL (GPU) and gloo (CPU tests).
+By default N > 1 means N independent replicas (one context = one GPU, no data-path collective): the only
+communication is the barrier around a timed region and a max-reduction of the measured time; independent problems
+(the per-head variant) are split over the ranks without any exchange.  `TokenSharded` is the one place with a
+data-path collective: one rotation calibrated on token shards, its statistics summed over the ranks before the
+update.  Works with NCCL (GPU) and gloo (CPU tests).
 """
 from __future__ import annotations
 
@@ -94,8 +96,7 @@ class TokenSharded:
     `ctx` is a single-problem calibration context (step / get_M / set_M / get_objective / update / get_R, as
     binding.Context); with NCCL the all-reduce runs on the context's device tensors.  The sum enters the context
     through conqur_get_M / conqur_set_M, i.e. two extra d x d copies per update.
-    Not run on more than one GPU so far (single-GPU runs only); the exchange logic is covered by a two-rank gloo test
-    with a CPU stand-in for the context.
+    The exchange logic is covered by a two-rank gloo test with a CPU stand-in for the context.
     """
 
     def __init__(self, ctx, g: Group):
