@@ -885,16 +885,26 @@ __global__ void __launch_bounds__(256) quant_target_bf16_kernel(const float* __r
     __nv_bfloat16* c = Cp + row * (int64_t)d;
     float qsum = 0.f;
     RowDiag dg{0.f, 0.f, 0.f, 0.f};
-    for (int j = lane * 4; j < d; j += 128) {
-      const float4 t = *reinterpret_cast<const float4*>(y + j);
-      const float in[4] = {t.x, t.y, t.z, t.w};
-      float sg[4];
+    for (int j0 = lane * 4; j0 < d; j0 += 1024) {              // eight 16-byte loads in flight per lane (Y is read once)
+      float4 t8[8];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) sg[e] = live ? second_pass_elem(in[e], r, qs, rq, qsum, diag, dg) * r : 0.f;
-      uint2 o;
-      o.x = bf16x2_pack(sg[0], sg[1]);
-      o.y = bf16x2_pack(sg[2], sg[3]);
-      *reinterpret_cast<uint2*>(c + j) = o;
+      for (int u = 0; u < 8; ++u) {
+        const int j = j0 + 128 * u;
+        t8[u] = (j < d) ? __ldcs(reinterpret_cast<const float4*>(y + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int j = j0 + 128 * u;
+        if (j >= d) break;
+        const float in[4] = {t8[u].x, t8[u].y, t8[u].z, t8[u].w};
+        float sg[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sg[e] = live ? second_pass_elem(in[e], r, qs, rq, qsum, diag, dg) * r : 0.f;
+        uint2 o;
+        o.x = bf16x2_pack(sg[0], sg[1]);
+        o.y = bf16x2_pack(sg[2], sg[3]);
+        *reinterpret_cast<uint2*>(c + j) = o;
+      }
     }
     qsum = warp_sum(qsum);
     if (live) contrib = (double)(r * rq.delta) * (double)qsum;
