@@ -293,9 +293,13 @@ int update_impl(conqur_ctx* c) {
   }
   ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau);
   CQ_LAUNCHED(c, K_OTHER);
-  ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
-  CQ_LAUNCHED(c, K_OTHER);
-  if (!g.simt_ns) { int rc = tc_ns_begin(c->tc, c->stream); if (rc) return rc; }
+  if (g.simt_ns) {
+    ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
+    CQ_LAUNCHED(c, K_OTHER);
+  } else {
+    int rc = tc_ns_begin(c->tc, c->stream);      // the same X0, written as the bf16 pair the products read
+    if (rc) return rc;
+  }
 
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);

@@ -1249,10 +1249,22 @@ inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64
   return tc_launch_n<true, true, TC_EPI_ACCUM>(h, s, tmXs_mn, tmCp_mn, a);
 }
 
-// X0 (fp32, in Xa) -> stacked bf16 split in Xh[0]
+// X0 = (M_raw + lam R) * x0_scale, written straight as the stacked bf16 split [hi; lo] (no fp32 copy of X0)
+static __global__ void tc_x0_split_kernel(const float* __restrict__ M, const float* __restrict__ R,
+                                          __nv_bfloat16* __restrict__ dst, int64_t dd, const DevState* st) {
+  const float lam = st->lam, sc = st->x0_scale;
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < dd; i += (int64_t)gridDim.x * blockDim.x * 4) {
+    const float4 m = *reinterpret_cast<const float4*>(M + i), r = *reinterpret_cast<const float4*>(R + i);
+    uint2 o, l;
+    bf16x2_split(fmaf(lam, r.x, m.x) * sc, fmaf(lam, r.y, m.y) * sc, o.x, l.x);
+    bf16x2_split(fmaf(lam, r.z, m.z) * sc, fmaf(lam, r.w, m.w) * sc, o.y, l.y);
+    *reinterpret_cast<uint2*>(dst + i) = o;
+    *reinterpret_cast<uint2*>(dst + dd + i) = l;
+  }
+}
 inline int tc_ns_begin(TcHost& h, cudaStream_t s) {
   const int64_t dd = (int64_t)h.d * h.d;
-  split_bf16_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.Xa, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[0]), dd, dd);
+  tc_x0_split_kernel<<<tc_ew_blocks(dd / 4), 256, 0, s>>>(h.M, h.R, reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xh[0]), dd, h.st);
   if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }
