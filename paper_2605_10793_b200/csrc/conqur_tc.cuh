@@ -2,7 +2,10 @@
 // shared memory ring -> tcgen05.mma with fp32 accumulators in TMEM -> tcgen05.ld epilogue) with the
 // path's steps fused into its epilogues, plus the small element-wise kernels around it.
 //
-//   D[m][n] = sum_k A(m,k) * B(n,k),  tile 128 x BN, BK = 64, bf16 operands, fp32 accumulation.
+//   D[m][n] = sum_k A(m,k) * B(n,k),  BK = 64, bf16 operands, fp32 accumulation.  Default variant: clusters of two
+//   CTAs work on one 256 x 256 tile with cta_group::2 instructions (each CTA loads half of the operands, CTA 0 issues
+//   the products for both, each CTA's epilogue warps read their own 128 rows of the accumulator); a single-CTA
+//   128 x BN variant remains for devices where such clusters cannot be resident.
 //
 // Each operand is a row-major bf16 matrix read in place in either orientation:
 //   K-major : rows are m (or n), k contiguous      -> TMA box 64(k) x 128|BN rows
@@ -12,7 +15,8 @@
 // Split precision: an operand may be a stacked pair [hi; lo] of bf16 matrices (value = hi + lo).  With
 // nseg = 3 the k loop runs three times over (hi,hi), (hi,lo), (lo,hi), accumulating into the same TMEM tile.
 //
-// No cluster launch and no multicast copies are used anywhere.  Every mbarrier wait is bounded: on expiry
+// Copies are never multicast (every CTA fetches its own operand tiles; the only cluster-wide signal is the commit
+// that releases a stage in both CTAs of a pair).  Every mbarrier wait is bounded: on expiry
 // the CTA raises a shared abort flag, latches STATUS_FLAG_TIMEOUT in the device state, drains its own
 // copies with a bounded wait, frees its TMEM and returns.
 #pragma once
