@@ -57,8 +57,9 @@ enum { CONQUR_QUANT_SYMMETRIC = 0, CONQUR_QUANT_ZEROPOINT = 1 };   /* fake-quant
  * mode CONQUR_EXACT_F32: fp32 CUDA-core contractions throughout (parity anchor).
  * mode CONQUR_TC_BF16:   bf16 operands, fp32 accumulation on the tcgen05 tensor
  *                        cores; fp32 X is rounded to bf16 on the way in; the
- *                        Newton-Schulz products use a two-term bf16 split of each
- *                        operand (three tensor-core products per matrix product).
+ *                        Newton-Schulz iterate is held as a two-term bf16 split hi + lo
+ *                        and each of its products takes one to three bf16 passes
+ *                        (hi hi, hi lo, lo hi), chosen per step on the device.
  */
 typedef struct {
   uint32_t struct_size;     /* = sizeof(conqur_config) */
@@ -75,7 +76,7 @@ typedef struct {
   float    prior_rel;       /* lam_rel >= 0: update is polar(M + lam R_prev),
                                lam = lam_rel * ||M||_F / sqrt(d); 0 = the paper's update */
   float    ns_sigma_min_rel;/* assumed lower bound on sigma_min(M)/||M||_F used to plan the
-                               polynomial schedule; 0 = default 1e-7 */
+                               polynomial schedule; 0 = default 1e-9 */
   int64_t  n_max;           /* largest n of any step call (sizes the workspace) */
   int32_t  batch;           /* P >= 1 independent problems of size d */
   int32_t  quant_mode;      /* CONQUR_QUANT_SYMMETRIC: Q_sym of Appendix B (delta = max|y| / (2^(b-1)-1));
@@ -84,7 +85,27 @@ typedef struct {
   float    clip_ratio;      /* c in (0, 1] for the zero-point quantiser (Appendix C uses 0.9 for activations); 0 = 1 */
   int32_t  diagnostics;     /* 1: every step also gathers the diagnostics of Section 4 (conqur_get_diagnostics); the step
                                then forms the rotated rows in memory first (two passes) */
+  int32_t  defer_batches;   /* tensor-core contexts with batch == 1: conqur_step only normalises and keeps a bf16 copy of
+                               its rows; the two products run once over all queued rows when this many batches are
+                               queued, and at the next conqur_update / conqur_get_* / conqur_set_* call (Section 3.4:
+                               the cross-covariance is accumulated with R fixed, so the grouping changes no result
+                               beyond fp32 summation order).  Use the update cadence; the workspace grows by
+                               4*d*n_max bytes per deferred batch.  0 or 1: every step runs its products at once */
+  float    ns_gram_single_pass_tau;  /* tensor-core mode tuning: the Gram product of a Newton-Schulz step runs one bf16
+                               pass instead of three while the iterate's mean squared singular value is below this;
+                               0 = default */
+  float    ns_lo_gap_budget;/* tensor-core mode tuning: bound on the Procrustes gap given up by dropping the low bf16
+                               half of the iterate in the next-iterate product of late steps; 0 = default 1e-4 */
+  int32_t  debug_flags;     /* test hooks, 0 in production: CONQUR_DEBUG_CANARIES | CONQUR_DEBUG_SINGLE_CTA |
+                               CONQUR_DEBUG_NO_GRAPH */
 } conqur_config;
+
+/* debug_flags bits.  CANARIES: every region of the workspace is followed by a 256-byte guard band with a fixed
+ * pattern, checked by conqur_debug_check_canaries (a stand-in for a memory checker).  SINGLE_CTA: the tensor-core
+ * products never use CTA pairs (exercises the single-CTA kernels on a device that would use pairs).  NO_GRAPH: the
+ * update's launch sequence is enqueued directly every time instead of being replayed from a captured graph (so that a
+ * profiler's launch list shows its kernels). */
+enum { CONQUR_DEBUG_CANARIES = 1, CONQUR_DEBUG_SINGLE_CTA = 2, CONQUR_DEBUG_NO_GRAPH = 4 };
 
 typedef struct {
   uint32_t struct_size;     /* = sizeof(conqur_stats) */
@@ -207,9 +228,27 @@ int conqur_get_M(conqur_ctx* ctx, float* M_out_dev);
  * resume / teacher forcing.  J_sum, n_tokens: host arrays of cfg.batch entries. */
 int conqur_set_M(conqur_ctx* ctx, const float* M_dev, const double* J_sum, const int64_t* n_tokens);
 
-/* Sign decisions of the last conqur_step: device int8, n x d row-major, values -1/0/+1
- * (0 also for skipped rows).  Single-problem contexts.  Synchronises. */
-int conqur_debug_get_signs(conqur_ctx* ctx, int8_t* S_out_dev);
+/* Sign decisions of the last step call (tie-aware parity, Eq. 2: which corner each row was sent to): device int8,
+ * values -1/0/+1 (0 also for skipped rows), for every problem q the call covered its n x d matrix, row-major, problem
+ * after problem ((q*n + i)*d + j).  A context with defer_batches > 1 reports the rows its products last ran over
+ * instead: all batches queued since the run before, in order (n = their total).  capacity_rows: rows S_out_dev has
+ * room for; fewer than problems * n returns CONQUR_ERR_INVALID_ARG and writes nothing.  Exact-mode contexts and single-problem tensor-core contexts (they keep
+ * the targets of the last step in the workspace); CONQUR_ERR_UNSUPPORTED for tensor-core contexts with batch > 1,
+ * see conqur_debug_capture_signs.  Synchronises. */
+int conqur_debug_get_signs(conqur_ctx* ctx, int8_t* S_out_dev, int64_t capacity_rows);
+
+/* The same read-out for tensor-core contexts with batch > 1, whose fused per-head kernel keeps the targets in shared
+ * memory only (Section 3.4, a Procrustes problem per head): after this call every conqur_step_batched(_range) also
+ * writes the decisions it takes to S_dev, laid out as above with q counted from the call's first problem; a call with
+ * problems * n > capacity_rows then returns CONQUR_ERR_INVALID_ARG and enqueues nothing.  S_dev: device, 16-byte
+ * aligned, owned by the caller, valid until replaced; NULL switches the capture off.  Synchronises. */
+int conqur_debug_capture_signs(conqur_ctx* ctx, int8_t* S_dev, int64_t capacity_rows);
+
+/* Test hook (no counterpart in the paper): with CONQUR_DEBUG_CANARIES set, counts the guard bands behind the
+ * workspace regions whose pattern has been overwritten (0 = all intact; a kernel of this library wrote past a region
+ * otherwise).  Returns that count, or a negative status (CONQUR_ERR_INVALID_ARG when the context was created without
+ * the flag).  Synchronises. */
+int conqur_debug_check_canaries(conqur_ctx* ctx);
 
 /* Counters of the last update and the latched device status (cleared).  Synchronises. */
 int conqur_get_stats(conqur_ctx* ctx, conqur_stats* out);
@@ -220,7 +259,9 @@ int conqur_get_stats(conqur_ctx* ctx, conqur_stats* out);
  * (residual X^T X - I, polynomial, next iterate), 6 everything else (reductions, element-wise).
  * Launch counts are always kept.  With profiling enabled each contraction launch is bracketed by
  * CUDA events on the context's stream and conqur_update synchronises at its end (so enable it only
- * in a measurement pass); flops are the algorithmic 2*M*N*K of launches that did not early-exit.
+ * in a measurement pass); flops are those of the tiles a launch computes (2 * 128|256 * tile width * K per tile
+ * and bf16 pass: a symmetric product counts its upper-triangle tiles only, a split product every pass it
+ * takes), for launches that did not early-exit.
  */
 #define CONQUR_KERNEL_CLASSES 8
 typedef struct {
@@ -348,8 +389,9 @@ int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows, int32_t co
  * this device, a transform kernel abandoned a bounded wait for one of its copies or products (its output is then
  * incomplete), CONQUR_OK otherwise; clears the latch.
  */
+enum { CONQUR_HADAMARD_CUDA_CORES_ONLY = 1 };   /* flags: never take the tensor-core kernel (tests compare the two) */
 int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,
-                         int32_t out_dtype, int64_t ldy, void* cuda_stream);
+                         int32_t out_dtype, int64_t ldy, int32_t flags, void* cuda_stream);
 int conqur_hadamard_status(void* cuda_stream);
 
 const char* conqur_strerror(int status);

@@ -28,6 +28,7 @@ What each function follows:
                       rho(y) = ||y||_inf^2 / ||y||_2^2 (Appendix B), and the relative squared
                       quantisation error ||X R - Q(X R)||_F^2 / ||X||_F^2 (on un-normalised rows)
   polar_svd           Section 3.3, C = U Sigma V^T, R <- U V^T
+  procrustes_optimum  Section 3.3, the value tr(R^T C) = sum of singular values the update attains
   OpuOracle.update    Section 3.3 / Algorithm 1: R replaced, statistics reset
   run_algorithm1      Algorithm 1: per mini-batch, the attention-input and MLP-input activations of
                       every block accumulate into the shared R_1 problem, every head of every
@@ -148,6 +149,14 @@ def polar_svd(m):
     """Orthogonal polar factor of m via the SVD: m = U S V^T -> U V^T (Section 3.3)."""
     u, s, vt = np.linalg.svd(np.asarray(m, dtype=np.float64))
     return u @ vt, s
+
+
+def procrustes_optimum(m):
+    """The value tr(R^T m) reaches at R = U V^T: the sum of the singular values of m (Section 3.3; for a full-rank m the
+    maximiser is unique and no orthogonal R gives more).  Singular values only -- at d = 8192 the full factorisation
+    of polar_svd takes minutes, this a fraction of that -- so an updated rotation can be judged by how much of the
+    optimum it reaches."""
+    return float(np.sum(np.linalg.svd(np.asarray(m, dtype=np.float64), compute_uv=False)))
 
 
 class OpuOracle:

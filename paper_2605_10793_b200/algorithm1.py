@@ -22,7 +22,8 @@ class Calibrator:
     def __init__(self, d: int, n_heads: int, d_head: int, n_layers: int, n_max: int, *, in_dtype="bf16", mode="tc",
                  quant_bits=0, quant_mode="sym", clip_ratio=0.0, prior_rel=0.0, record: Optional[str] = None):
         """n_max: most tokens in one activation matrix.  record: None | "objective" | "full" (also keeps each
-        cross-covariance, read before its update; both synchronise and are meant for tests and logging)."""
+        cross-covariance, read before its update, and the sign decisions of every step; both synchronise and are
+        meant for tests and logging)."""
         kw = dict(in_dtype=in_dtype, mode=mode, quant_bits=quant_bits, quant_mode=quant_mode, clip_ratio=clip_ratio,
                   prior_rel=prior_rel)
         self.d, self.n_heads, self.d_head, self.n_layers = d, n_heads, d_head, n_layers
@@ -31,6 +32,13 @@ class Calibrator:
         self.record = record
         self.log: List[Dict] = []
         self._cur: Dict = {}
+        self._signs: Dict = {}
+        self._capture = None
+        if record == "full" and mode == "tc":
+            # the fused per-head kernel keeps nothing of a step in memory: its sign decisions are captured as it runs
+            import torch
+            self._capture = torch.zeros((n_heads * n_max, d_head), dtype=torch.int8, device="cuda")
+            self.ctx2.debug_capture_signs(self._capture)
 
     def set_rotations(self, r1, r2):
         """r1: (d, d); r2: (n_layers, n_heads, d_head, d_head); fp32 CUDA tensors."""
@@ -41,10 +49,23 @@ class Calibrator:
         """The body of Algorithm 1's loop over blocks for block `layer`: both residual-stream sites go into the R_1
         statistics, the o_proj input into the statistics of the block's n_heads problems.
         x_o: (n, n_heads*d_head), head h in columns h*d_head.."""
+        full = self.record == "full"
         self.ctx1.step(x_attn)
+        if full:
+            self._signs[("attn", layer)] = self.ctx1.debug_get_signs(x_attn.shape[0]).cpu().numpy()
         self.ctx1.step(x_mlp)
+        if full:
+            self._signs[("mlp", layer)] = self.ctx1.debug_get_signs(x_mlp.shape[0]).cpu().numpy()
         assert x_o.shape[1] == self.n_heads * self.d_head and x_o.stride(1) == 1
-        self.ctx2.step_batched_range(x_o, x_o.shape[0], x_o.stride(0), self.d_head, layer * self.n_heads, self.n_heads)
+        n = x_o.shape[0]
+        self.ctx2.step_batched_range(x_o, n, x_o.stride(0), self.d_head, layer * self.n_heads, self.n_heads)
+        if full:
+            if self._capture is not None:
+                self.ctx2.stream.synchronize()
+                s2 = self._capture[: self.n_heads * n].reshape(self.n_heads, n, self.d_head).cpu().numpy()
+            else:
+                s2 = self.ctx2.debug_get_signs(n, problems=self.n_heads).cpu().numpy()
+            self._signs[("o", layer)] = s2
 
     def end_minibatch(self):
         """R_{2,l} <- OPU(R_{2,l}, X_o^(l)) for every block, and R_1 <- OPU(R_1, X_1), with everything accumulated
@@ -57,6 +78,8 @@ class Calibrator:
             if self.record == "full":
                 self._cur["M1"] = self.ctx1.get_M().cpu().numpy()
                 self._cur["M2"] = self.ctx2.get_M().cpu().numpy().reshape(L, H, dh, dh)
+                self._cur["signs"] = self._signs
+                self._signs = {}
             self.log.append(self._cur)
             self._cur = {}
         self.ctx2.update()

@@ -20,11 +20,19 @@ CONQUR_F32, CONQUR_BF16 = 0, 1
 CONQUR_EXACT_F32, CONQUR_TC_BF16 = 0, 1
 CONQUR_QUANT_SYMMETRIC, CONQUR_QUANT_ZEROPOINT = 0, 1
 CONQUR_FOLD_INPUT, CONQUR_FOLD_OUTPUT = 0, 1
+CONQUR_DEBUG_CANARIES, CONQUR_DEBUG_SINGLE_CTA, CONQUR_DEBUG_NO_GRAPH = 1, 2, 4
+CONQUR_HADAMARD_CUDA_CORES_ONLY = 1
+
+# Test support: when set, every Context is created with guard bands around its workspace regions, registers itself
+# here, and has them checked when it is closed; damaged bands are collected in CANARY_FAILURES.
+DEBUG_CANARIES = False
+CANARY_FAILURES: list = []
+_live_contexts = None
 
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
-    "conqur_set_M", "conqur_debug_get_signs", "conqur_get_stats", "conqur_plan_schedule", "conqur_debug_gemm",
+    "conqur_set_M", "conqur_debug_get_signs", "conqur_debug_capture_signs", "conqur_get_stats", "conqur_debug_check_canaries", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
     "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows", "conqur_hadamard_status",
     "conqur_strerror",
@@ -37,6 +45,8 @@ class conqur_config(C.Structure):
         ("ns_steps", C.c_int32), ("ns_max_steps", C.c_int32), ("orth_tol", C.c_float), ("prior_rel", C.c_float),
         ("ns_sigma_min_rel", C.c_float), ("n_max", C.c_int64), ("batch", C.c_int32),
         ("quant_mode", C.c_int32), ("clip_ratio", C.c_float), ("diagnostics", C.c_int32),
+        ("defer_batches", C.c_int32), ("ns_gram_single_pass_tau", C.c_float), ("ns_lo_gap_budget", C.c_float),
+        ("debug_flags", C.c_int32),
     ]
 
 
@@ -107,7 +117,11 @@ def load() -> C.CDLL:
     lib.conqur_set_M.restype = C.c_int
     lib.conqur_set_M.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.conqur_debug_get_signs.restype = C.c_int
-    lib.conqur_debug_get_signs.argtypes = [vp, vp]
+    lib.conqur_debug_get_signs.argtypes = [vp, vp, i64]
+    lib.conqur_debug_capture_signs.restype = C.c_int
+    lib.conqur_debug_capture_signs.argtypes = [vp, vp, i64]
+    lib.conqur_debug_check_canaries.restype = C.c_int
+    lib.conqur_debug_check_canaries.argtypes = [vp]
     lib.conqur_get_stats.restype = C.c_int
     lib.conqur_get_stats.argtypes = [vp, C.POINTER(conqur_stats)]
     lib.conqur_plan_schedule.restype = C.c_int
@@ -129,7 +143,7 @@ def load() -> C.CDLL:
     lib.conqur_fold_weight.restype = C.c_int
     lib.conqur_fold_weight.argtypes = [vp, i64, i32, i32, vp, i32, i32, i32, vp, i64, vp, i64, vp]
     lib.conqur_hadamard_rows.restype = C.c_int
-    lib.conqur_hadamard_rows.argtypes = [vp, i32, i64, i32, i64, vp, i32, i64, vp]
+    lib.conqur_hadamard_rows.argtypes = [vp, i32, i64, i32, i64, vp, i32, i64, i32, vp]
     lib.conqur_hadamard_status.restype = C.c_int
     lib.conqur_hadamard_status.argtypes = [vp]
     lib.conqur_strerror.restype = C.c_char_p
@@ -144,9 +158,11 @@ def strerror(status: int) -> str:
 
 def make_config(*, in_dtype=CONQUR_BF16, mode=CONQUR_TC_BF16, quant_bits=0, ns_steps=0, ns_max_steps=0,
                 orth_tol=0.0, prior_rel=0.0, ns_sigma_min_rel=0.0, n_max=1, batch=1, quant_mode=CONQUR_QUANT_SYMMETRIC,
-                clip_ratio=0.0, diagnostics=0) -> conqur_config:
+                clip_ratio=0.0, diagnostics=0, defer_batches=0, ns_gram_single_pass_tau=0.0, ns_lo_gap_budget=0.0,
+                debug_flags=0) -> conqur_config:
     return conqur_config(C.sizeof(conqur_config), in_dtype, mode, quant_bits, ns_steps, ns_max_steps, orth_tol,
-                         prior_rel, ns_sigma_min_rel, n_max, batch, quant_mode, clip_ratio, diagnostics)
+                         prior_rel, ns_sigma_min_rel, n_max, batch, quant_mode, clip_ratio, diagnostics,
+                         defer_batches, ns_gram_single_pass_tau, ns_lo_gap_budget, debug_flags)
 
 
 # ---- the C calls, one to one -------------------------------------------------------------------
@@ -210,8 +226,12 @@ def conqur_set_M(h: int, m_ptr: int, j_sum, n_tokens) -> int:
     return load().conqur_set_M(h, m_ptr, j, n)
 
 
-def conqur_debug_get_signs(h: int, out_ptr: int) -> int:
-    return load().conqur_debug_get_signs(h, out_ptr)
+def conqur_debug_get_signs(h: int, out_ptr: int, capacity_rows: int) -> int:
+    return load().conqur_debug_get_signs(h, out_ptr, capacity_rows)
+
+
+def conqur_debug_capture_signs(h: int, buf_ptr: int, capacity_rows: int) -> int:
+    return load().conqur_debug_capture_signs(h, buf_ptr, capacity_rows)
 
 
 def conqur_get_stats(h: int) -> Tuple[int, conqur_stats]:
@@ -293,7 +313,7 @@ def conqur_fold_weight(w, r, side: str, mode: str = "tc"):
     return out
 
 
-def conqur_hadamard_rows(x, out_dtype=None, out=None):
+def conqur_hadamard_rows(x, out_dtype=None, out=None, cuda_cores_only=False):
     """y = x H_d / sqrt(d) for every row of a 2-D fp32 / bf16 CUDA tensor (see include/conqur.h)."""
     import torch
     code = {torch.float32: CONQUR_F32, torch.bfloat16: CONQUR_BF16}
@@ -302,7 +322,9 @@ def conqur_hadamard_rows(x, out_dtype=None, out=None):
         out = torch.empty(x.shape, dtype=out_dtype or x.dtype, device="cuda")
     assert out.is_cuda and out.shape == x.shape and out.stride(1) == 1 and out.dtype in code
     rc = load().conqur_hadamard_rows(x.data_ptr(), code[x.dtype], x.shape[0], x.shape[1], x.stride(0), out.data_ptr(),
-                                     code[out.dtype], out.stride(0), torch.cuda.current_stream().cuda_stream)
+                                     code[out.dtype], out.stride(0),
+                                     CONQUR_HADAMARD_CUDA_CORES_ONLY if cuda_cores_only else 0,
+                                     torch.cuda.current_stream().cuda_stream)
     if rc != 0:
         raise ConqurError(rc, "conqur_hadamard_rows")
     return out
@@ -320,7 +342,8 @@ class Context:
     """One calibration context on the current CUDA device / current torch stream."""
 
     def __init__(self, d: int, n_max: int, *, in_dtype="bf16", mode="tc", quant_bits=0, batch=1, prior_rel=0.0,
-                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None, quant_mode="sym", clip_ratio=0.0, diagnostics=False):
+                 ns_steps=0, ns_max_steps=0, orth_tol=0.0, ns_sigma_min_rel=0.0, stream=None, quant_mode="sym", clip_ratio=0.0,
+                 diagnostics=False, defer_batches=0, ns_gram_single_pass_tau=0.0, ns_lo_gap_budget=0.0, debug_flags=0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("conqur needs a CUDA device (B200); there is no CPU path")
@@ -332,7 +355,9 @@ class Context:
                                ns_max_steps=ns_max_steps, orth_tol=orth_tol, prior_rel=prior_rel,
                                ns_sigma_min_rel=ns_sigma_min_rel, n_max=n_max, batch=batch,
                                quant_mode={"sym": CONQUR_QUANT_SYMMETRIC, "zp": CONQUR_QUANT_ZEROPOINT}[quant_mode],
-                               clip_ratio=clip_ratio, diagnostics=int(bool(diagnostics)))
+                               clip_ratio=clip_ratio, diagnostics=int(bool(diagnostics)), defer_batches=defer_batches,
+                               ns_gram_single_pass_tau=ns_gram_single_pass_tau, ns_lo_gap_budget=ns_lo_gap_budget,
+                               debug_flags=debug_flags | (CONQUR_DEBUG_CANARIES if DEBUG_CANARIES else 0))
         nbytes = conqur_workspace_bytes(self.d, self.cfg)
         if nbytes == 0:
             raise ConqurError(-1, "conqur_workspace_bytes")
@@ -341,6 +366,12 @@ class Context:
         self._ws_ptr = (base + 255) // 256 * 256
         self.stream = stream if stream is not None else torch.cuda.current_stream()
         self.h = conqur_init(self.d, self.cfg, self._ws_ptr, nbytes, self.stream.cuda_stream)
+        if DEBUG_CANARIES:
+            global _live_contexts
+            if _live_contexts is None:
+                import weakref
+                _live_contexts = weakref.WeakSet()
+            _live_contexts.add(self)
 
     def _chk(self, rc: int, where: str):
         if rc != 0:
@@ -405,10 +436,23 @@ class Context:
         return [dict(sum_pr_over_d=a.sum_pr_over_d, sum_rho=a.sum_rho, qerr_num=a.qerr_num, qerr_den=a.qerr_den,
                      n_tokens=a.n_tokens) for a in arr]
 
-    def debug_get_signs(self, n: int):
-        out = self.torch.empty((n, self.d), dtype=self.torch.int8, device="cuda")
-        self._chk(conqur_debug_get_signs(self.h, out.data_ptr()), "conqur_debug_get_signs")
+    def debug_get_signs(self, n: int, problems: int = 1):
+        """Sign decisions of the last step call: (n, d) int8, or (problems, n, d) for a batched call."""
+        shape = (n, self.d) if problems == 1 else (problems, n, self.d)
+        out = self.torch.empty(shape, dtype=self.torch.int8, device="cuda")
+        self._chk(conqur_debug_get_signs(self.h, out.data_ptr(), n * problems), "conqur_debug_get_signs")
         return out
+
+    def debug_capture_signs(self, buf):
+        """Tensor-core contexts with batch > 1: let the following batched steps write their sign decisions to `buf`
+        (int8 CUDA tensor, rows x d; None stops it).  The tensor must stay alive while the capture is on."""
+        if buf is None:
+            self._sign_buf = None
+            self._chk(conqur_debug_capture_signs(self.h, 0, 0), "conqur_debug_capture_signs")
+            return
+        assert buf.is_cuda and buf.dtype == self.torch.int8 and buf.is_contiguous()
+        self._sign_buf = buf
+        self._chk(conqur_debug_capture_signs(self.h, buf.data_ptr(), buf.numel() // self.d), "conqur_debug_capture_signs")
 
     def get_stats(self) -> conqur_stats:
         rc, st = conqur_get_stats(self.h)
@@ -427,8 +471,19 @@ class Context:
                          "flops": float(pr.flops[i]), "ms": float(pr.ms[i])}
         return out
 
+    def check_canaries(self) -> int:
+        """Guard bands of the workspace that were overwritten (0 = intact); needs CONQUR_DEBUG_CANARIES."""
+        rc = load().conqur_debug_check_canaries(self.h)
+        if rc < 0:
+            raise ConqurError(rc, "conqur_debug_check_canaries")
+        return rc
+
     def close(self):
         if getattr(self, "h", None):
+            if self.cfg.debug_flags & CONQUR_DEBUG_CANARIES:
+                bad = load().conqur_debug_check_canaries(self.h)
+                if bad != 0:
+                    CANARY_FAILURES.append((self.d, self.batch, self.mode, bad))
             conqur_destroy(self.h)
             self.h = None
 

@@ -39,10 +39,15 @@ struct Layout {
   size_t total;
   int64_t max_partials;
   int acc_splits;
+  int64_t n_rows;           // rows the per-step buffers hold: n_max, times the deferred batches of a tensor-core context
+  int n_guards;             // CONQUR_DEBUG_CANARIES: guard bands behind the regions, at guard[i]
+  size_t guard[48];
 };
+constexpr size_t GUARD_BYTES = 256;
+constexpr unsigned char GUARD_PATTERN = 0xC5;
 
 struct Cfg {
-  int d, P, in_dtype, mode, quant_bits, ns_max_steps;
+  int d, P, in_dtype, mode, quant_bits, ns_max_steps, defer, debug_flags;
   QuantSpec qs;
   int diagnostics;
   int64_t n_max;
@@ -71,10 +76,25 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   if (c->prior_rel < 0.f || c->orth_tol < 0.f || c->ns_sigma_min_rel < 0.f || c->ns_steps < 0 || c->ns_max_steps < 0)
     return false;
   if (c->mode == CONQUR_TC_BF16 && !tc_supported_shape(d, c->batch)) return false;
-  const int64_t P = c->batch, n = c->n_max;
+  if (c->defer_batches < 0 || c->defer_batches > 64) return false;
+  if (c->defer_batches > 1 && (c->mode != CONQUR_TC_BF16 || c->batch != 1)) return false;
+  if (c->ns_gram_single_pass_tau < 0.f || c->ns_lo_gap_budget < 0.f) return false;
+  if (c->debug_flags & ~(CONQUR_DEBUG_CANARIES | CONQUR_DEBUG_SINGLE_CTA | CONQUR_DEBUG_NO_GRAPH)) return false;
+  const int64_t P = c->batch;
+  // a deferring context keeps the rows of up to defer_batches steps: every per-row buffer is that much longer
+  const int64_t n = c->n_max * std::max(1, c->defer_batches);
+  if (n > (int64_t)1 << 30) return false;
+  L->n_rows = n;
   const size_t dd = (size_t)d * d;
   size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  const bool guards = (c->debug_flags & CONQUR_DEBUG_CANARIES) != 0;
+  L->n_guards = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes);
+    if (guards && L->n_guards < 48) { L->guard[L->n_guards++] = off; off += GUARD_BYTES; }
+    return o;
+  };
   L->state = take(sizeof(DevState) * P);
   L->flags_agg = take(sizeof(int) * 4);
   L->R = take(sizeof(float) * dd * P);
@@ -116,7 +136,12 @@ struct conqur_ctx {
   char* ws;
   cudaStream_t stream;
   std::vector<int64_t> tokens;   // per problem: rows enqueued since the last update
-  int64_t last_n;            // rows of the last step (for debug_get_signs)
+  int64_t last_n;            // rows per problem of the last step (for debug_get_signs)
+  int last_np;               // problems the last step call covered
+  int64_t pending_rows = 0;  // deferring context: rows staged but not yet run through the two products
+  int pending_batches = 0;
+  int8_t* sign_capture = nullptr;   // conqur_debug_capture_signs: where the fused per-head kernel writes its decisions
+  int64_t sign_capture_rows = 0;
   int n_sched, first_endgame, reenter_idx;
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
@@ -241,6 +266,28 @@ int step_exact(conqur_ctx* c, const TIn* X, int64_t n, int64_t ld, int64_t pstri
   return CONQUR_OK;
 }
 
+// A deferring context (cfg.defer_batches > 1) queues the staged rows of its steps; this runs the two products over
+// everything queued.  Called when the queue is full and before anything reads or replaces the statistics or R.
+int flush_pending(conqur_ctx* c) {
+  if (c->pending_rows == 0) return CONQUR_OK;
+  const int rc = tc_process(c->tc, c->stream, c->pending_rows);
+  c->last_n = c->pending_rows;                 // what debug_get_signs reports: the rows this run covered
+  c->pending_rows = 0;
+  c->pending_batches = 0;
+  return rc;
+}
+
+// CONQUR_DEBUG_CANARIES: one block per guard band; counts the bands that no longer hold the pattern.
+struct GuardList { int n; unsigned long long off[48]; };
+__global__ void check_guards_kernel(const unsigned char* ws, const GuardList gl, int* bad) {
+  __shared__ int hit;
+  if (threadIdx.x == 0) hit = 0;
+  __syncthreads();
+  if (ws[gl.off[blockIdx.x] + threadIdx.x] != GUARD_PATTERN) hit = 1;
+  __syncthreads();
+  if (threadIdx.x == 0 && hit) atomicAdd(bad, 1);
+}
+
 // ---------------------------------------------------------------- update (both modes share the control flow)
 // residual check of the fp32 matrix X (P x d x d) into E; fills the partials.
 int launch_residual(conqur_ctx* c, const float* X, int buf) {
@@ -347,7 +394,7 @@ int update_impl(conqur_ctx* c) {
 
 // Enqueue one update: directly the first time (kernel attributes get set), then through a captured graph.
 int update_enqueue(conqur_ctx* c) {
-  static const bool no_graph = [] { const char* e = std::getenv("CONQUR_NO_GRAPH"); return e && e[0] == '1'; }();
+  const bool no_graph = (c->cfg.debug_flags & CONQUR_DEBUG_NO_GRAPH) != 0;
   const bool eligible = !no_graph && c->cfg.mode == CONQUR_TC_BF16 && c->cfg.P == 1 && !c->prof.enabled;
   if (!eligible || c->updates_enqueued++ == 0) return update_impl(c);
   if (!c->upd_graph) {
@@ -415,9 +462,12 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->tokens.assign(cfg->batch, 0);
   c->last_n = 0;
+  c->last_np = 0;
   Cfg& g = c->cfg;
   g.d = d; g.P = cfg->batch; g.in_dtype = cfg->in_dtype; g.mode = cfg->mode; g.quant_bits = cfg->quant_bits;
   g.n_max = cfg->n_max;
+  g.defer = (g.mode == CONQUR_TC_BF16 && g.P == 1) ? std::max(1, cfg->defer_batches) : 1;
+  g.debug_flags = cfg->debug_flags;
   g.qs = QuantSpec{cfg->quant_bits, cfg->quant_mode, cfg->clip_ratio > 0.f ? cfg->clip_ratio : 1.0f};
   g.diagnostics = cfg->diagnostics;
   g.simt_ns = (g.mode == CONQUR_EXACT_F32);
@@ -432,6 +482,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   pp.margin = g.margin;
   pp.d = g.simt_ns ? 0 : d;
   pp.max_len = NS_SCHED_MAX;
+  if (cfg->ns_lo_gap_budget > 0.f) pp.gap_budget = cfg->ns_lo_gap_budget;
   c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(std::min(cfg->ns_steps, NS_SCHED_MAX), pp, &c->first_endgame)
                                : plan_schedule(pp, &c->first_endgame);
   c->n_sched = (int)c->sched.size();
@@ -444,7 +495,10 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
     coef[i] = SchedEntry{(float)s.a, (float)s.b, (float)s.c, (float)s.l, s.lift, s.seg_x};
   }
   auto fail = [&](int rc) { delete c; return rc; };
-  if (cudaMemsetAsync(c->ws, 0, L.R, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);   // state + flags
+  for (int i = 0; i < L.n_guards; ++i)
+    if (cudaMemsetAsync(c->ws + L.guard[i], GUARD_PATTERN, GUARD_BYTES, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);
+  if (cudaMemsetAsync(c->ws, 0, sizeof(DevState) * g.P, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);
+  if (cudaMemsetAsync(c->ws + L.flags_agg, 0, sizeof(int) * 4, c->stream) != cudaSuccess) return fail(CONQUR_ERR_CUDA);
   if (cudaMemsetAsync(c->ws + L.M, 0, sizeof(float) * (size_t)d * d * g.P, c->stream) != cudaSuccess)
     return fail(CONQUR_ERR_CUDA);
   if (cudaMemcpyAsync(c->ws + L.sched, coef.data(), sizeof(SchedEntry) * NS_SCHED_MAX, cudaMemcpyHostToDevice,
@@ -453,11 +507,12 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   set_identity_kernel<<<ew_blocks((int64_t)d * d * g.P), 256, 0, c->stream>>>(c->at<float>(L.R), d, g.P);
   if (cudaGetLastError() != cudaSuccess) return fail(CONQUR_ERR_CUDA);
   if (g.mode == CONQUR_TC_BF16) {
-    int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, g.n_max, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
+    int rc = tc_init(&c->tc, c->ws, L.tc, d, g.P, L.n_rows, g.quant_bits, c->at<float>(L.R), c->at<float>(L.M),
                      c->at<float>(L.Xa), c->at<float>(L.Xb), c->at<float>(L.E), c->at<float>(L.B),
                      c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
                      (cfg->quant_bits || cfg->diagnostics) ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), g.qs,
-                     g.diagnostics, g.diagnostics ? c->at<double>(L.part_diag) : nullptr, &c->prof);
+                     g.diagnostics, g.diagnostics ? c->at<double>(L.part_diag) : nullptr, &c->prof,
+                     (g.debug_flags & CONQUR_DEBUG_SINGLE_CTA) != 0, cfg->ns_gram_single_pass_tau);
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);
@@ -480,6 +535,7 @@ extern "C" int conqur_set_R(conqur_ctx* c, const float* R_dev) {
   if (!c || !R_dev) return CONQUR_ERR_INVALID_ARG;
   const Cfg& g = c->cfg;
   const int64_t dd = (int64_t)g.d * g.d;
+  { const int frc = flush_pending(c); if (frc) return frc; }      // queued rows belong to the rotation being replaced
   // check orthogonality with the exact fp32 residual product, whatever the mode
   float* Xa = c->at<float>(c->L.Xa);
   CQ_CUDA(cudaMemcpyAsync(Xa, R_dev, sizeof(float) * dd * g.P, cudaMemcpyDeviceToDevice, c->stream));
@@ -513,12 +569,23 @@ static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int6
              ? step_exact<float>(c, static_cast<const float*>(X), n, ld, pstride, p0, np)
              : step_exact<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(X), n, ld, pstride, p0, np);
   } else {
-    rc = g.P > 1 ? tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride, p0, np)
-                 : tc_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride);
+    if (g.P > 1 && c->sign_capture && (int64_t)np * n > c->sign_capture_rows) return CONQUR_ERR_INVALID_ARG;
+    if (g.P > 1) {
+      rc = tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride, p0, np, c->sign_capture);
+    } else {
+      // stage the rows behind those already queued; run the products when the queue is full (at once if not deferring)
+      if (c->pending_rows + n > c->L.n_rows) { rc = flush_pending(c); if (rc) return rc; }
+      rc = tc_stage(c->tc, c->stream, X, g.in_dtype, n, ld, c->pending_rows);
+      if (rc == CONQUR_OK) {
+        c->pending_rows += n;
+        if (++c->pending_batches >= g.defer) rc = flush_pending(c);
+      }
+    }
   }
   if (rc == CONQUR_OK) {
     for (int p = p0; p < p0 + np; ++p) c->tokens[p] += n;
-    c->last_n = n;
+    if (!(g.mode == CONQUR_TC_BF16 && g.P == 1)) c->last_n = n;      // (set by flush_pending for queueing contexts)
+    c->last_np = np;
   }
   return rc;
 }
@@ -544,6 +611,7 @@ extern "C" int conqur_update(conqur_ctx* c) {
   const int64_t fewest = *std::min_element(c->tokens.begin(), c->tokens.end());     // every problem is updated
   if (fewest == 0) return CONQUR_ERR_EMPTY_UPDATE;
   if (fewest < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int rc = update_enqueue(c);
   if (rc == CONQUR_OK) std::fill(c->tokens.begin(), c->tokens.end(), 0);
   return rc;
@@ -551,6 +619,7 @@ extern "C" int conqur_update(conqur_ctx* c) {
 
 extern "C" int conqur_get_R(conqur_ctx* c, float* R_out_dev) {
   if (!c || !R_out_dev) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const size_t bytes = sizeof(float) * (size_t)c->cfg.d * c->cfg.d * c->cfg.P;
   CQ_CUDA(cudaMemcpyAsync(R_out_dev, c->at<float>(c->L.R), bytes, cudaMemcpyDeviceToDevice, c->stream));
   return sync_status(c);
@@ -558,6 +627,7 @@ extern "C" int conqur_get_R(conqur_ctx* c, float* R_out_dev) {
 
 extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tokens) {
   if (!c || !J_sum || !n_tokens) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int P = c->cfg.P;
   std::vector<DevState> h(P);
   CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
@@ -568,6 +638,7 @@ extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tok
 
 extern "C" int conqur_get_diagnostics(conqur_ctx* c, conqur_diagnostics* out) {
   if (!c || !out || !c->cfg.diagnostics) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int P = c->cfg.P;
   for (int p = 0; p < P; ++p)
     if (out[p].struct_size != sizeof(conqur_diagnostics)) return CONQUR_ERR_INVALID_ARG;
@@ -583,6 +654,7 @@ extern "C" int conqur_get_diagnostics(conqur_ctx* c, conqur_diagnostics* out) {
 
 extern "C" int conqur_get_M(conqur_ctx* c, float* M_out_dev) {
   if (!c || !M_out_dev) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int64_t count = (int64_t)c->cfg.d * c->cfg.d * c->cfg.P;
   scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(c->at<float>(c->L.M), M_out_dev, count,
                                                              (float)(1.0 / std::sqrt((double)c->cfg.d)));
@@ -592,6 +664,7 @@ extern "C" int conqur_get_M(conqur_ctx* c, float* M_out_dev) {
 
 extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_sum, const int64_t* n_tokens) {
   if (!c || !M_dev || !J_sum || !n_tokens) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int P = c->cfg.P;
   const int64_t count = (int64_t)c->cfg.d * c->cfg.d * P;
   scale_copy_kernel<<<ew_blocks(count), 256, 0, c->stream>>>(M_dev, c->at<float>(c->L.M), count,
@@ -610,23 +683,53 @@ extern "C" int conqur_set_M(conqur_ctx* c, const float* M_dev, const double* J_s
   return CONQUR_OK;
 }
 
-extern "C" int conqur_debug_get_signs(conqur_ctx* c, int8_t* S_out_dev) {
-  if (!c || !S_out_dev || c->cfg.P != 1) return CONQUR_ERR_INVALID_ARG;
-  if (c->last_n == 0) return CONQUR_ERR_INVALID_ARG;
-  const int64_t total = c->last_n * c->cfg.d;
-  if (c->cfg.mode == CONQUR_EXACT_F32) {
-    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(c->at<float>(c->L.C), nullptr, c->last_n, c->cfg.d,
-                                                                 S_out_dev);
+extern "C" int conqur_debug_get_signs(conqur_ctx* c, int8_t* S_out_dev, int64_t capacity_rows) {
+  if (!c || !S_out_dev) return CONQUR_ERR_INVALID_ARG;
+  const Cfg& g = c->cfg;
+  if (g.mode == CONQUR_TC_BF16 && g.P > 1) return CONQUR_ERR_UNSUPPORTED;     // nothing of a fused step stays in memory
+  { const int frc = flush_pending(c); if (frc) return frc; }
+  if (c->last_n == 0 || c->last_np == 0) return CONQUR_ERR_INVALID_ARG;
+  if (capacity_rows < c->last_n * c->last_np) return CONQUR_ERR_INVALID_ARG;
+  const int64_t total = c->last_n * g.d;
+  const dim3 grid(ew_blocks(total), c->last_np);
+  if (g.mode == CONQUR_EXACT_F32) {
+    signs_from_c_kernel<<<grid, 256, 0, c->stream>>>(c->at<float>(c->L.C), nullptr, c->last_n, g.d, (int64_t)g.n_max * g.d,
+                                                     S_out_dev);
   } else {
-    signs_from_c_kernel<<<ew_blocks(total), 256, 0, c->stream>>>(nullptr, tc_cp_ptr(c->tc), c->last_n, c->cfg.d,
-                                                                 S_out_dev);
+    signs_from_c_kernel<<<grid, 256, 0, c->stream>>>(nullptr, tc_cp_ptr(c->tc), c->last_n, g.d, 0, S_out_dev);
   }
   CQ_LAUNCHED(c, K_OTHER);
   return sync_status(c);
 }
 
+extern "C" int conqur_debug_capture_signs(conqur_ctx* c, int8_t* S_dev, int64_t capacity_rows) {
+  if (!c || capacity_rows < 0 || (S_dev && capacity_rows == 0)) return CONQUR_ERR_INVALID_ARG;
+  if (c->cfg.mode != CONQUR_TC_BF16 || c->cfg.P == 1) return CONQUR_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(S_dev) & 15) return CONQUR_ERR_INVALID_ARG;
+  CQ_CUDA(cudaStreamSynchronize(c->stream));           // no step in flight still writes to the previous buffer
+  c->sign_capture = S_dev;
+  c->sign_capture_rows = S_dev ? capacity_rows : 0;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_debug_check_canaries(conqur_ctx* c) {
+  if (!c || !(c->cfg.debug_flags & CONQUR_DEBUG_CANARIES) || c->L.n_guards == 0) return CONQUR_ERR_INVALID_ARG;
+  GuardList gl;
+  gl.n = c->L.n_guards;
+  for (int i = 0; i < gl.n; ++i) gl.off[i] = c->L.guard[i];
+  int* bad = c->at<int>(c->L.flags_agg) + 1;
+  CQ_CUDA(cudaMemsetAsync(bad, 0, sizeof(int), c->stream));
+  check_guards_kernel<<<gl.n, (int)GUARD_BYTES, 0, c->stream>>>(reinterpret_cast<const unsigned char*>(c->ws), gl, bad);
+  CQ_LAUNCHED(c, K_OTHER);
+  int h = 0;
+  CQ_CUDA(cudaMemcpyAsync(&h, bad, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  return h;
+}
+
 extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
   if (!c || !out || out->struct_size != sizeof(conqur_stats)) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
   const int P = c->cfg.P;
   std::vector<DevState> h(P);
   CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
@@ -786,7 +889,8 @@ extern "C" int conqur_fold_weight(const float* W_dev, int64_t ldw, int32_t rows,
 }
 
 extern "C" int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t n, int32_t d, int64_t ldx, void* Y_dev,
-                                    int32_t out_dtype, int64_t ldy, void* cuda_stream) {
+                                    int32_t out_dtype, int64_t ldy, int32_t flags, void* cuda_stream) {
+  if (flags & ~CONQUR_HADAMARD_CUDA_CORES_ONLY) return CONQUR_ERR_INVALID_ARG;
   if (n < 0 || d < 4 || d > 8192 || (d & (d - 1)) || ldx < d || ldy < d) return CONQUR_ERR_INVALID_ARG;
   if (n > 0 && (!X_dev || !Y_dev)) return CONQUR_ERR_INVALID_ARG;
   if ((in_dtype != CONQUR_F32 && in_dtype != CONQUR_BF16) || (out_dtype != CONQUR_F32 && out_dtype != CONQUR_BF16))
@@ -801,8 +905,7 @@ extern "C" int conqur_hadamard_rows(const void* X_dev, int32_t in_dtype, int64_t
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   using bf = __nv_bfloat16;
   // bf16 rows that lie back to back: the 128-point sub-transforms run on the tensor cores
-  const char* env = std::getenv("CONQUR_HADAMARD_SIMT");            // "1": CUDA-core kernels only (tests compare the two)
-  const bool simt_only = env && env[0] == '1';
+  const bool simt_only = (flags & CONQUR_HADAMARD_CUDA_CORES_ONLY) != 0;
   if (!simt_only && in_dtype == CONQUR_BF16 && ldx == d && ldy == d && (reinterpret_cast<uintptr_t>(X_dev) & 15) == 0 &&
       (reinterpret_cast<uintptr_t>(Y_dev) & 15) == 0 && (n * d) % 128 == 0) {
     const int rc = (out_dtype == CONQUR_F32) ? hadamard_tc_launch(static_cast<const bf*>(X_dev), static_cast<float*>(Y_dev), n, logd, s)

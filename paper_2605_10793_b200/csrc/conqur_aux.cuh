@@ -306,15 +306,24 @@ inline int hadamard_launch_bulk(const TIn* X, int64_t ldx, TOut* Y, int64_t ldy,
                                 cudaStream_t s) {
   constexpr int smem = had_bulk_smem_bytes<TIn, E, S>();
   auto kern = hadamard_rows_bulk_kernel<TIn, TOut, E, S>;
-  static int attr_dev_mask = 0, ctas_per_sm = 0, sms = 0;
+  // per device: the shared-memory attribute, and how many CTAs fit (looked up once, under a lock)
+  struct Facts { int known, ctas_per_sm, sms; };
+  static std::mutex mu;
+  static Facts facts[64] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
-  if (!(attr_dev_mask & (1 << (dev & 31)))) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas_per_sm, kern, HAD_THREADS, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
-    if (ctas_per_sm < 1) return CONQUR_ERR_UNSUPPORTED;
-    attr_dev_mask |= 1 << (dev & 31);
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONQUR_ERR_CUDA;
+  int ctas_per_sm = 0, sms = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    Facts& f = facts[dev];
+    if (!f.known) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&f.ctas_per_sm, kern, HAD_THREADS, smem) != cudaSuccess) return CONQUR_ERR_CUDA;
+      if (cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+      if (f.ctas_per_sm < 1) return CONQUR_ERR_UNSUPPORTED;
+      f.known = 1;
+    }
+    ctas_per_sm = f.ctas_per_sm; sms = f.sms;
   }
   const int64_t rows_per_block = (HAD_THREADS * E) >> logd;
   const int64_t nblocks = (n + rows_per_block - 1) / rows_per_block;

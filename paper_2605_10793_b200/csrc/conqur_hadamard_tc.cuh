@@ -194,23 +194,17 @@ hadamard_tc_kernel(const __grid_constant__ CUtensorMap tmX, TOut* Y, long long N
 // n rows of d bf16 elements, contiguous (row stride d), 16-byte aligned base, n * d a multiple of 128.
 template <typename TOut>
 inline int hadamard_tc_launch(const __nv_bfloat16* X, TOut* Y, int64_t n, int logd, cudaStream_t s) {
-  struct DevFacts { int known, major, sms; };
-  static DevFacts facts[64] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONQUR_ERR_CUDA;
-  DevFacts& f = facts[dev];
+  if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  TcDevFacts f;
+  if (tc_device_facts(dev, &f) != CONQUR_OK) return CONQUR_ERR_CUDA;
   auto kern = hadamard_tc_kernel<TOut>;
-  if (!f.known) {
-    if (cudaDeviceGetAttribute(&f.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return CONQUR_ERR_CUDA;
-    f.known = 1;
-  }
   if (f.major != 10) return CONQUR_ERR_UNSUPPORTED;
-  static int attr_dev_mask = 0;
-  if (!(attr_dev_mask & (1 << (dev & 31)))) {
+  static std::atomic<unsigned long long> attr_dev_mask{0};      // the attribute is per device
+  const unsigned long long dev_bit = 1ull << (dev & 63);
+  if (!(attr_dev_mask.load(std::memory_order_acquire) & dev_bit)) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HTC_SMEM_BYTES) != cudaSuccess) return CONQUR_ERR_CUDA;
-    attr_dev_mask |= 1 << (dev & 31);
+    attr_dev_mask.fetch_or(dev_bit, std::memory_order_release);
   }
   const long long NC = (long long)n * (1ll << logd) / 128;
   if (NC < 1 || NC > 0x7fffff00ll) return CONQUR_ERR_INVALID_ARG;

@@ -708,13 +708,16 @@ static __global__ void set_identity_kernel(float* __restrict__ R, int d, int P) 
     R[i] = ((e / d) == (e % d)) ? 1.f : 0.f;
   }
 }
-// sign matrix of the last step from C' (n x d, row-major) held as fp32 (exact mode) or bf16 (tensor-core mode)
+// sign matrices of the last step from C' (per problem n x d, row-major, problems src_ps elements apart) held as fp32
+// (exact mode) or bf16 (tensor-core mode); written densely, problem after problem.  grid.y = problems.
 static __global__ void signs_from_c_kernel(const float* __restrict__ C, const __nv_bfloat16* __restrict__ Cb, int64_t n,
-                                    int d, int8_t* __restrict__ S) {
+                                    int d, int64_t src_ps, int8_t* __restrict__ S) {
   const int64_t total = n * d;
+  const int64_t src0 = (int64_t)blockIdx.y * src_ps;
+  int8_t* out = S + (int64_t)blockIdx.y * total;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const float v = C ? C[i] : __bfloat162float(Cb[i]);
-    S[i] = (v > 0.f) ? 1 : ((v < 0.f) ? -1 : 0);
+    const float v = C ? C[src0 + i] : __bfloat162float(Cb[src0 + i]);
+    out[i] = (v > 0.f) ? 1 : ((v < 0.f) ? -1 : 0);
   }
 }
 

@@ -25,8 +25,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 
 #include "../../include/conqur.h"
 #include "conqur_internal.h"
@@ -1075,11 +1077,13 @@ template <int BN, bool A_MN, bool B_MN, int EPI, bool PAIR, int NA = 1, int NB =
 inline int tc_launch(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const TcGemmArgs& g) {
   using Cfg = TcCfg<BN, PAIR, NA, NB>;
   auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, PAIR, NA, NB>;
-  static int attr_dev_mask = 0;                    // the attribute is per device
-  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
+  // the attribute is per device; setting it twice from two threads is harmless, so an atomic mask is enough
+  static std::atomic<unsigned long long> attr_dev_mask{0};
+  const unsigned long long dev_bit = 1ull << (h.device & 63);
+  if (!(attr_dev_mask.load(std::memory_order_acquire) & dev_bit)) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_dev_mask |= 1 << (h.device & 31);
+    attr_dev_mask.fetch_or(dev_bit, std::memory_order_release);
   }
   const TcVariant v{PAIR, Cfg::TILE_M, BN};
   const int tiles = tc_tiles(v, g.M, g.N, g.sym);
@@ -1133,10 +1137,8 @@ inline int tc_launch_n(TcHost& h, cudaStream_t s, const CUtensorMap& a, const CU
   return tc_launch<128, A_MN, B_MN, EPI, false>(h, s, a, b, g);
 }
 
-// How many CTA pairs of the 256 x 256 kernel can be resident at once (0: use single CTAs).
+// How many CTA pairs of the 256 x 256 kernel can be resident at once on the current device (0: use single CTAs).
 inline int tc_query_pair_clusters() {
-  const char* env = std::getenv("CONQUR_TC_SINGLE_CTA");
-  if (env && env[0] == '1') return 0;
   using Cfg = TcCfg<256, true>;
   auto kern = tc_gemm_kernel<256, false, true, TC_EPI_PLAIN, true>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess) return 0;
@@ -1151,25 +1153,44 @@ inline int tc_query_pair_clusters() {
   return n > 0 ? n : 0;
 }
 
+// Facts about a device, looked up once per device under a lock (the queries cost milliseconds).
+struct TcDevFacts { int known, major, sms, pair_clusters; };
+inline int tc_device_facts(int dev, TcDevFacts* out) {
+  static std::mutex mu;
+  static TcDevFacts facts[64] = {};
+  if (dev < 0 || dev >= 64) return CONQUR_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  TcDevFacts& f = facts[dev];
+  if (!f.known) {
+    if (cudaDeviceGetAttribute(&f.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return CONQUR_ERR_CUDA;
+    f.pair_clusters = f.major == 10 ? tc_query_pair_clusters() : 0;
+    f.known = 1;
+  }
+  *out = f;
+  return CONQUR_OK;
+}
+
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
                    float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
-                   float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, int diagnostics, double* part_diag, Prof* prof) {
+                   float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, int diagnostics, double* part_diag, Prof* prof,
+                   int single_cta, float gram_single_pass_tau) {
   h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
   h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
   h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->qs = qs; h->diagnostics = diagnostics; h->part_diag = part_diag; h->prof = prof; h->ns_k = -1;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CONQUR_ERR_CUDA;
-  if (prop.major != 10) {
-    std::fprintf(stderr, "conqur: the tensor-core mode needs an sm_100 device (found sm_%d%d)\n", prop.major, prop.minor);
+  TcDevFacts f;
+  if (tc_device_facts(dev, &f) != CONQUR_OK) return CONQUR_ERR_CUDA;
+  if (f.major != 10) {
+    std::fprintf(stderr, "conqur: the tensor-core mode needs an sm_100 device (found compute capability %d.x)\n", f.major);
     return CONQUR_ERR_UNSUPPORTED;
   }
-  h->num_sms = prop.multiProcessorCount;
+  h->num_sms = f.sms;
   h->device = dev;
-  h->pair_clusters = tc_query_pair_clusters();
-  h->e1_tau = 2e-3f;
-  if (const char* env = std::getenv("CONQUR_NS_E1_TAU")) h->e1_tau = (float)std::atof(env);   // tuning knob
+  h->pair_clusters = single_cta ? 0 : f.pair_clusters;
+  h->e1_tau = gram_single_pass_tau > 0.f ? gram_single_pass_tau : 2e-3f;
   const uint64_t D = (uint64_t)d;
   int rc = 0;
   if (P > 1) {
@@ -1206,17 +1227,28 @@ inline TcGemmArgs tc_args(const TcHost& h, int M, int N, int K) {
   return g;
 }
 
-inline int tc_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t) {
+// a1 of one streamed batch: row norms and the sanitised bf16 copy, written at rows [row0, row0 + n) of the per-step
+// buffers (row0 > 0 only in a context that queues several batches before running the products).
+inline int tc_stage(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t row0) {
+  const int d = h.d;
+  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xs) + row0 * d;
+  const int rb = (int)((n + 7) / 8);
+  if (in_dtype == CONQUR_F32)
+    rownorm_stage_kernel<float><<<rb, 256, 0, s>>>(static_cast<const float*>(X), n, d, ld, h.rnorm + row0, Xs, h.st);
+  else
+    rownorm_stage_kernel<__nv_bfloat16><<<rb, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(X), n, d, ld, h.rnorm + row0, Xs, h.st);
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_ROWNORM);
+  return CONQUR_OK;
+}
+
+// a2-a5 over the first n staged rows: rotate + target (+ the second pass of the fake-quant / diagnostics route),
+// objective, accumulate.
+inline int tc_process(TcHost& h, cudaStream_t s, int64_t n) {
   const int d = h.d;
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Xs);
   __nv_bfloat16* Cp = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Cp);
   const int rb = (int)((n + 7) / 8);
-  if (in_dtype == CONQUR_F32)
-    rownorm_stage_kernel<float><<<rb, 256, 0, s>>>(static_cast<const float*>(X), n, d, ld, h.rnorm, Xs, h.st);
-  else
-    rownorm_stage_kernel<__nv_bfloat16><<<rb, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(X), n, d, ld, h.rnorm, Xs, h.st);
-  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
-  if (h.prof) h.prof->count(K_ROWNORM);
   // per-call maps over the first n rows: rows past n read as zeros
   CUtensorMap tmXs_k, tmXs_mn, tmCp_mn;
   int rc = tc_make_tmap(&tmXs_k, Xs, (uint64_t)n, (uint64_t)d, (uint64_t)d, 128);
@@ -1346,19 +1378,10 @@ inline int tc_plain_gemm(const __nv_bfloat16* A, const __nv_bfloat16* B, float* 
   if (ldo < N || (ldo % 4)) return CONQUR_ERR_INVALID_ARG;
   TcHost h{};
   h.prof = nullptr; h.ns_k = -1;
-  // device facts, looked up once per device (the queries cost milliseconds)
-  struct DevFacts { int known, major, sms, pair_clusters; };
-  static DevFacts facts[64] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONQUR_ERR_CUDA;
-  DevFacts& f = facts[dev];
-  if (!f.known) {
-    if (cudaDeviceGetAttribute(&f.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return CONQUR_ERR_CUDA;
-    f.pair_clusters = f.major == 10 ? tc_query_pair_clusters() : 0;
-    f.known = 1;
-  }
+  if (cudaGetDevice(&dev) != cudaSuccess) return CONQUR_ERR_CUDA;
+  TcDevFacts f;
+  if (tc_device_facts(dev, &f) != CONQUR_OK) return CONQUR_ERR_CUDA;
   if (f.major != 10) return CONQUR_ERR_UNSUPPORTED;
   h.num_sms = f.sms;
   h.device = dev;

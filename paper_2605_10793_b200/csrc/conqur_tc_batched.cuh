@@ -52,6 +52,7 @@ struct TcbStepArgs {
   float* Mpart;               // S > 1: P * S partial cross-covariances (item order), summed into M by tcb_finish_kernel
   double* part_d;             // P * S objective partials (sum |y| * rnorm, or the quantised equivalent), item order
   DevState* st;               // P
+  int8_t* signs;              // test hook: when set, the sign decisions (-1/0/+1) of this call, (P * n) x 128 row-major
 };
 
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int x, int y, int z) {
@@ -276,6 +277,25 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             *reinterpret_cast<uint4*>(crow + tcb_piece(r, c * 4 + k)) = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+          if (g.signs != nullptr && valid) {
+            // the decisions exactly as they enter the second product: sign bit and non-zero test of each bf16 half of C'
+            uint32_t sb[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              uint32_t o = 0;
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const uint32_t pr = w[2 * k + e];
+                const uint32_t lo = pr & 0xffffu, hi = pr >> 16;
+                o |= ((lo & 0x7fffu) ? ((lo & 0x8000u) ? 0xffu : 1u) : 0u) << (16 * e);
+                o |= ((hi & 0x7fffu) ? ((hi & 0x8000u) ? 0xffu : 1u) : 0u) << (16 * e + 8);
+              }
+              sb[k] = o;
+            }
+            uint4* so = reinterpret_cast<uint4*>(g.signs + ((long long)p * g.n + (long long)t * 128 + r) * TCB_D + c * 32);
+            so[0] = make_uint4(sb[0], sb[1], sb[2], sb[3]);
+            so[1] = make_uint4(sb[4], sb[5], sb[6], sb[7]);
+          }
         }
         if (live) acc += (g.qs.bits > 0) ? (double)(rn * rq.delta) * (double)acc_t : (double)(acc_t * rn);
         // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
@@ -405,12 +425,13 @@ inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_
 // One streamed batch for all P problems.  X: device, bf16 or fp32 (fp32 is first rounded into the staging copy).
 // Problems [p0, p0 + np) of the context; X holds those np problems.
 inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride, int p0,
-                    int np) {
-  static int attr_dev_mask = 0;                    // the attribute is per device
-  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
+                    int np, int8_t* signs_out = nullptr) {
+  static std::atomic<unsigned long long> attr_dev_mask{0};      // the attribute is per device
+  const unsigned long long dev_bit = 1ull << (h.device & 63);
+  if (!(attr_dev_mask.load(std::memory_order_acquire) & dev_bit)) {
     if (cudaFuncSetAttribute(tcb_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCB_SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_dev_mask |= 1 << (h.device & 31);
+    attr_dev_mask.fetch_or(dev_bit, std::memory_order_release);
   }
   const void* src = X;
   int64_t src_ld = ld, src_ps = pstride;
@@ -430,7 +451,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   if (rc) return rc;
   TcbStepArgs g{};
   g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
-  g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0;
+  g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0; g.signs = signs_out;
   // few problems: split each problem's tokens over several CTAs (partials land in the idle Newton-Schulz buffers,
   // 4 P matrices of 128 x 128 starting at Xa, and are summed in a fixed order)
   const int T = (int)((n + 127) / 128);
@@ -800,11 +821,12 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
 }
 
 inline int tcb_update(TcHost& h, cudaStream_t s, const NsControlParams& ncp, float prior_rel, float margin) {
-  static int attr_dev_mask = 0;                    // the attribute is per device
-  if (!(attr_dev_mask & (1 << (h.device & 31)))) {
+  static std::atomic<unsigned long long> attr_dev_mask{0};      // the attribute is per device
+  const unsigned long long dev_bit = 1ull << (h.device & 63);
+  if (!(attr_dev_mask.load(std::memory_order_acquire) & dev_bit)) {
     if (cudaFuncSetAttribute(tcb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TCBU_SMEM_BYTES) != cudaSuccess)
       return CONQUR_ERR_CUDA;
-    attr_dev_mask |= 1 << (h.device & 31);
+    attr_dev_mask.fetch_or(dev_bit, std::memory_order_release);
   }
   TcbUpdArgs g{};
   g.P = h.P; g.M = h.M; g.R = h.R; g.st = h.st; g.ncp = ncp; g.prior_rel = prior_rel; g.margin = margin;

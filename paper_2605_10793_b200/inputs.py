@@ -76,6 +76,7 @@ class Workload:
     same_batch: bool = False   # every step sees batch 0 (alternation on a fixed batch)
     quant_mode: str = "sym"    # "sym": symmetric per-token quantiser; "zp": zero-point quantiser
     clip_ratio: float = 1.0    # range clipping ratio of the zero-point quantiser
+    ns_steps: int = 0          # Newton-Schulz steps the polar update plans for (0 = the library's default plan)
 
 
 WORKLOADS: Dict[str, Workload] = {
@@ -93,7 +94,7 @@ WORKLOADS: Dict[str, Workload] = {
                    "hadamard"),
     # 70B-class residual width
     "c3": Workload("c3", 3, 8192, 4096, 64, 16, "bf16", "student_t3", 32, 100.0, 0.5, 4, 1000.0,
-                   "hadamard"),
+                   "hadamard", ns_steps=8),
     # c2 with per-token symmetric INT4 fake-quantisation of the rotated rows
     "c4a": Workload("c4a", 4, 4096, 2048, 128, 8, "bf16", "student_t3", 16, 100.0, 0.5, 4, 1000.0,
                     "hadamard", quant_bits=4),

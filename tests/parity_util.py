@@ -20,6 +20,32 @@ TOL = {
 }
 
 
+# figures measured by the GPU tests of this session (written out by --parity-report)
+REPORT: list = []
+
+
+def log_parity(config: str, mode: str, what: str, rep: dict, **extra) -> None:
+    """Record the numbers of one comparison (config = workload name, what = which step / update of it)."""
+    keep = ("J_rel", "M_rel_tie_aware", "M_rel_raw", "flip_frac", "flips_outside_band", "orth", "gap", "R_dist", "cond")
+    row = {"config": config, "mode": mode, "what": what}
+    row.update({k: (float(rep[k]) if not isinstance(rep[k], int) else rep[k]) for k in keep if k in rep})
+    row.update(extra)
+    REPORT.append(row)
+
+
+def assert_step(rep: dict, mode: str, flip_max: float) -> None:
+    """The step assertions shared by every parity test: token count, objective, tie-aware cross-covariance, every
+    differing sign inside the rounding band; and the raw cross-covariance too whenever no sign differs."""
+    t = TOL[mode]
+    assert rep["N_equal"], rep
+    assert rep["J_rel"] <= t["J"], rep
+    assert rep["M_rel_tie_aware"] <= t["M"], rep
+    assert rep["flips_outside_band"] == 0, rep
+    assert rep["flip_frac"] < flip_max, rep
+    if rep["flip_frac"] == 0.0:
+        assert rep["M_rel_raw"] <= t["M"], rep
+
+
 def unit_roundoff(mode: str, d: int) -> float:
     """Relative size of the rounding band around a sign decision."""
     if mode == "exact":

@@ -47,6 +47,18 @@ def test_workspace_bytes_and_argument_checks(B):
     # tensor-core mode wants d to be a multiple of 128
     tc = B.make_config(in_dtype=B.CONQUR_BF16, mode=B.CONQUR_TC_BF16, n_max=256)
     assert B.conqur_workspace_bytes(100, tc) == 0
+    # deferring batches: tensor-core single-problem contexts only; every per-row buffer grows with the queue
+    plain = B.conqur_workspace_bytes(256, tc)
+    queued = B.conqur_workspace_bytes(256, B.make_config(in_dtype=B.CONQUR_BF16, mode=B.CONQUR_TC_BF16, n_max=256, defer_batches=8))
+    assert queued >= plain + 7 * 4 * 256 * 256
+    assert B.conqur_workspace_bytes(128, B.make_config(in_dtype=B.CONQUR_BF16, mode=B.CONQUR_TC_BF16, n_max=256, batch=4,
+                                                       defer_batches=8)) == 0
+    assert B.conqur_workspace_bytes(64, B.make_config(in_dtype=B.CONQUR_F32, mode=B.CONQUR_EXACT_F32, n_max=16, defer_batches=2)) == 0
+    assert B.conqur_workspace_bytes(64, B.make_config(in_dtype=B.CONQUR_F32, mode=B.CONQUR_EXACT_F32, n_max=16, debug_flags=64)) == 0
+    # guard bands (test hook) cost 256 bytes per workspace region
+    guarded = B.conqur_workspace_bytes(128, B.make_config(in_dtype=B.CONQUR_F32, mode=B.CONQUR_EXACT_F32, n_max=2048,
+                                                          debug_flags=B.CONQUR_DEBUG_CANARIES))
+    assert small < guarded <= small + 48 * 256
 
 
 def test_init_rejects_bad_arguments_without_a_device(B):

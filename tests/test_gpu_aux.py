@@ -70,13 +70,8 @@ def test_hadamard_many_blocks_per_cta(d, n):
     v4 = view[:, 4:4 + d]                                        # bf16 rows 8 bytes off a 16-byte boundary: plain-load kernel
     v4.copy_(xb)
     assert v4.data_ptr() % 16 == 8
-    import os
     y_tc = B.conqur_hadamard_rows(xb, out_dtype=torch.float32)           # contiguous bf16: tensor-core kernel
-    os.environ["CONQUR_HADAMARD_SIMT"] = "1"
-    try:
-        y_bulk = B.conqur_hadamard_rows(xb, out_dtype=torch.float32)     # the same rows through the bulk-copy CUDA-core kernel
-    finally:
-        del os.environ["CONQUR_HADAMARD_SIMT"]
+    y_bulk = B.conqur_hadamard_rows(xb, out_dtype=torch.float32, cuda_cores_only=True)   # ... and the bulk-copy CUDA-core kernel
     assert torch.equal(B.conqur_hadamard_rows(v4, out_dtype=torch.float32), y_bulk)
     assert B.conqur_hadamard_status() == 0
     tol = float(np.log2(d)) * 2.0 ** -23 * torch.linalg.norm(xb.float(), dim=1, keepdim=True)
@@ -112,11 +107,11 @@ def test_hadamard_strides_in_place_empty_and_argument_errors():
     lib = B.load()
     s = torch.cuda.current_stream().cuda_stream
     good = torch.zeros(4, 96, device="cuda")
-    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 96, 96, good.data_ptr(), 0, 96, s) == -1    # not a power of two
-    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 16384, 16384, good.data_ptr(), 0, 16384, s) == -1
-    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 64, 32, good.data_ptr(), 0, 64, s) == -1    # stride < d
-    assert lib.conqur_hadamard_rows(good.data_ptr() + 4, 0, 4, 64, 96, good.data_ptr(), 0, 96, s) == -1  # misaligned
-    assert lib.conqur_hadamard_rows(good.data_ptr(), 7, 4, 64, 96, good.data_ptr(), 0, 96, s) == -1
+    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 96, 96, good.data_ptr(), 0, 96, 0, s) == -1    # not a power of two
+    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 16384, 16384, good.data_ptr(), 0, 16384, 0, s) == -1
+    assert lib.conqur_hadamard_rows(good.data_ptr(), 0, 4, 64, 32, good.data_ptr(), 0, 64, 0, s) == -1    # stride < d
+    assert lib.conqur_hadamard_rows(good.data_ptr() + 4, 0, 4, 64, 96, good.data_ptr(), 0, 96, 0, s) == -1  # misaligned
+    assert lib.conqur_hadamard_rows(good.data_ptr(), 7, 4, 64, 96, good.data_ptr(), 0, 96, 0, s) == -1
     assert not good.any().item()
 
 

@@ -1,0 +1,291 @@
+"""GPU parity on the stated workloads at their full sizes and at their cadence, both arithmetic modes, through the
+C ABI: exact mode (fp32 CUDA-core products) at the widths 3072 / 4096 / 8192, the d = 8192 stream as it runs
+(16 batches per update, no proximal term), a cycle after the first update (where R is a Newton-Schulz output and
+the rotated rows sit near corners), and the fake-quantised cycle with its update.
+
+Where a float64 step or factorisation is too slow for a whole stream a stated subset is checked in full and the rest
+on the objective (one float64 product per batch).  Every comparison is teacher-forced (tests/parity_util.py) and
+its figures go to the parity report (pytest --parity-report FILE)."""
+import numpy as np
+import pytest
+
+from oracle import conqur_oracle as O
+from paper_2605_10793_b200 import inputs as I
+from tests.parity_util import TOL, assert_step, effective_m, log_parity, step_parity, unit_roundoff, update_parity
+
+pytestmark = pytest.mark.gpu
+
+FLIP_MAX = {"exact": 1e-3, "tc": 2e-2}
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ctx(w, mode, **kw):
+    from paper_2605_10793_b200 import binding as B
+    args = dict(d=w.d, n_max=w.n, in_dtype="bf16", mode=mode, quant_bits=w.quant_bits, prior_rel=w.prior_rel,
+                quant_mode=w.quant_mode, clip_ratio=w.clip_ratio)
+    if mode == "tc" and w.problems == 1:
+        args["defer_batches"] = w.update_every         # the configuration bench.py runs
+    args.update(kw)
+    return B.Context(**args)
+
+
+def _dev_bf16(x):
+    torch = _torch()
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda().to(torch.bfloat16)
+
+
+def _f64(t):
+    return t.cpu().numpy().astype(np.float64)
+
+
+def _full_step(ctx, w, x, before, mode, what):
+    """One library step compared in full with the oracle (objective, tie-aware cross-covariance, sign band)."""
+    r = _f64(ctx.get_R())
+    ctx.step(_dev_bf16(x))
+    j, n = ctx.get_objective()
+    m = _f64(ctx.get_M())
+    s = ctx.debug_get_signs(x.shape[0]).cpu().numpy()
+    mb, jb, nb = before if before is not None else (None, 0.0, 0)
+    rep = step_parity(x.astype(np.float64), r, s, m, j, n, mode, w.quant_bits, mb, jb, nb, w.quant_mode, w.clip_ratio)
+    log_parity(w.name, mode, what, rep)
+    assert_step(rep, mode, FLIP_MAX[mode])
+    return (m, j, n), r
+
+
+def _objective_only_step(ctx, w, x, r64, before, mode):
+    """A step checked on its objective and token count: one float64 product for the plain corner target, an oracle step
+    where the fake-quantiser sits in between."""
+    ctx.step(_dev_bf16(x))
+    j, n = ctx.get_objective()
+    if w.quant_bits == 0:
+        xt, used = O.normalise_rows(x)
+        j_ref, n_ref = np.abs(xt @ r64).sum() / np.sqrt(w.d), int(used.sum())
+    else:
+        ref = O.OpuOracle(w.d, r64, quant_bits=w.quant_bits, quant_mode=w.quant_mode, clip_ratio=w.clip_ratio)
+        ref.step(x.astype(np.float64))
+        j_ref, n_ref = ref.J, ref.N
+    jb, nb = (before[1], before[2]) if before is not None else (0.0, 0)
+    assert n == nb + n_ref
+    assert abs((j - jb) - j_ref) / j_ref <= TOL[mode]["J"], (j - jb, j_ref)
+    return (None, j, n)
+
+
+def _update_check(ctx, w, m64, r_prev64, mode, what, max_steps=None):
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, (st.status, st.ns_steps_used)
+    if max_steps is not None:
+        assert st.ns_steps_used <= max_steps, st.ns_steps_used
+    r_new = _f64(ctx.get_R())
+    m_eff = effective_m(m64, r_prev64, w.prior_rel)
+    rep = update_parity(m_eff, r_new)
+    log_parity(w.name, mode, what, rep, ns_steps_used=int(st.ns_steps_used))
+    assert rep["orth"] <= TOL[mode]["orth"], rep
+    assert rep["gap"] <= TOL[mode]["gap"], rep
+    j, n = ctx.get_objective()
+    assert j == 0.0 and n == 0
+    return r_new, st
+
+
+def _cycle(ctx, w, mode, first_batch, label):
+    """One update cycle of the workload: first and last step in full, the steps between on the objective, then the
+    update against the SVD polar factor of the library's own cross-covariance."""
+    before, r = None, None
+    for k in range(w.update_every):
+        x = I.batch(w, first_batch + k)
+        if k in (0, w.update_every - 1):
+            if before is not None and before[0] is None:
+                before = (_f64(ctx.get_M()), before[1], before[2])
+            before, r = _full_step(ctx, w, x, before, mode, f"{label} step {k + 1}/{w.update_every}")
+        else:
+            before = _objective_only_step(ctx, w, x, r, before, mode)
+    m, j, n = before
+    assert n == w.update_every * w.n
+    r_new, st = _update_check(ctx, w, m, r, mode, f"{label} update")
+    if w.prior_rel == 0.0 and w.quant_bits == 0:
+        assert np.sum(r_new * m) >= j * (1.0 - 1e-3)          # ascent on the statistics the update was computed from
+    return st
+
+
+# ------------------------------------------------------------------ exact mode at the full widths
+
+def test_c1_exact_step_and_proximal_update_at_d3072():
+    w = I.WORKLOADS["c1"]
+    ctx = _ctx(w, "exact")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _cycle(ctx, w, "exact", 0, "cycle 1")
+
+
+def test_c2_exact_first_cycle_at_d4096():
+    w = I.WORKLOADS["c2"]
+    ctx = _ctx(w, "exact")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _cycle(ctx, w, "exact", 0, "cycle 1")
+
+
+@pytest.mark.parametrize("name", ["c4a", "c4a_zp"])
+def test_c4a_exact_fake_quant_step_at_d4096(name):
+    w = I.WORKLOADS[name]
+    ctx = _ctx(w, "exact")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _full_step(ctx, w, I.batch(w, 0), None, "exact", "cycle 1 step 1/8")
+
+
+def _sampled_column_step(ctx, w, x, mode, what, n_cols=24):
+    """d = 8192: a float64 step takes tens of seconds, so one step is checked on its objective (one float64 product)
+    and on sampled columns of the cross-covariance (tie-aware, every differing sign inside the band)."""
+    d = w.d
+    r64 = _f64(ctx.get_R())
+    ctx.step(_dev_bf16(x))
+    j, nn = ctx.get_objective()
+    m = _f64(ctx.get_M())
+    s_gpu = ctx.debug_get_signs(x.shape[0]).cpu().numpy()
+    xt, used = O.normalise_rows(x)
+    y = xt @ r64
+    j_ref = np.abs(y).sum() / np.sqrt(d)
+    cols = np.random.default_rng(3).choice(d, size=n_cols, replace=False)
+    s_ref = O.sgn(y[:, cols])
+    diff = s_gpu[:, cols].astype(np.float64) != s_ref
+    band = 6.0 * unit_roundoff(mode, d) * np.sqrt((xt * xt) @ (r64[:, cols] ** 2))
+    m_ta = xt.T @ (s_gpu[:, cols].astype(np.float64) / np.sqrt(d))
+    m_ref = xt.T @ (s_ref / np.sqrt(d))
+    rep = {"J_rel": abs(j - j_ref) / j_ref, "N_equal": nn == int(used.sum()),
+           "M_rel_tie_aware": float(np.linalg.norm(m[:, cols] - m_ta) / np.linalg.norm(m_ta)),
+           "M_rel_raw": float(np.linalg.norm(m[:, cols] - m_ref) / np.linalg.norm(m_ref)),
+           "flip_frac": float(diff.mean()), "flips_outside_band": int((diff & (np.abs(y[:, cols]) > band)).sum())}
+    log_parity(w.name, mode, what + f" ({n_cols} sampled columns)", rep)
+    assert_step(rep, mode, FLIP_MAX[mode])
+    return r64, (m, j, nn)
+
+
+def test_c3_exact_step_sampled_columns_at_d8192():
+    w = I.WORKLOADS["c3"]
+    ctx = _ctx(w, "exact")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _sampled_column_step(ctx, w, I.batch(w, 0), "exact", "cycle 1 step 1/16")
+
+
+def test_c4b_exact_sampled_heads():
+    """The 1024 per-head problems in exact mode (64 distinct seeded problems repeated 16 times, as in the tensor-core
+    test): sampled problems in full against independent oracle runs."""
+    w = I.WORKLOADS["c4b"]
+    torch = _torch()
+    P, distinct = w.problems, 64
+    xs = [I.batch(w, 0, problem=p) for p in range(distinct)]
+    r0s = [I.initial_rotation(w, p) for p in range(distinct)]
+    x_all = _dev_bf16(np.concatenate(xs, axis=0)).repeat(P // distinct, 1)
+    r_all = torch.from_numpy(np.stack(r0s)).cuda().repeat(P // distinct, 1, 1).contiguous()
+    ctx = _ctx(w, "exact", batch=P)
+    ctx.set_R(r_all)
+    ctx.step_batched(x_all, w.n, w.d, w.n * w.d)
+    js, ns = ctx.get_objective()
+    ms = _f64(ctx.get_M())
+    signs = ctx.debug_get_signs(w.n, problems=P)
+    ctx.update()
+    assert ctx.get_stats().status == 0
+    rs = _f64(ctx.get_R())
+    for p in (0, 63, 64 + 17, 1023):
+        q = p % distinct
+        rep = step_parity(xs[q].astype(np.float64), r0s[q].astype(np.float64), signs[p].cpu().numpy(), ms[p], js[p], ns[p],
+                          "exact")
+        log_parity(w.name, "exact", f"problem {p} step", rep)
+        assert_step(rep, "exact", FLIP_MAX["exact"])
+        urep = update_parity(ms[p], rs[p])
+        log_parity(w.name, "exact", f"problem {p} update", urep)
+        assert urep["orth"] <= TOL["exact"]["orth"] and urep["gap"] <= TOL["exact"]["gap"], (p, urep)
+
+
+# ------------------------------------------------------------------ tensor-core mode, the workloads as they run
+
+def test_c3_tc_sixteen_batches_then_the_plain_update_at_d8192():
+    """The d = 8192 stream as the workload runs it: 16 batches of 4096 tokens queued with R fixed and run through the
+    two products in one go, then the update with no proximal term and a planned budget of 8 Newton-Schulz steps.
+    Objective and token count of all 65536 rows against float64 products (one per batch); the cross-covariance on
+    sampled columns, tie-aware over all rows with every differing sign inside the band; the update by the
+    orthogonality of the new rotation in float64 and by how much of the optimum sum of singular values of the
+    library's own cross-covariance it reaches.  The steps the iteration really took are recorded."""
+    w = I.WORKLOADS["c3"]
+    d = w.d
+    ctx = _ctx(w, "tc", ns_steps=w.ns_steps, defer_batches=w.update_every)
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    r64 = _f64(ctx.get_R())
+    cols = np.random.default_rng(3).choice(d, size=24, replace=False)
+    band_scale = 6.0 * unit_roundoff("tc", d)
+    j_ref, n_ref, kept = 0.0, 0, []
+    for k in range(w.update_every):
+        x = I.batch(w, k)
+        ctx.step(_dev_bf16(x))
+        xt, used = O.normalise_rows(x)
+        y = xt @ r64
+        j_ref += np.abs(y).sum() / np.sqrt(d)
+        n_ref += int(used.sum())
+        kept.append((xt[:, :].astype(np.float32), y[:, cols].copy(), np.sqrt((xt * xt) @ (r64[:, cols] ** 2))))
+        del xt, y
+    j, n = ctx.get_objective()
+    assert n == n_ref == w.update_every * w.n
+    m = _f64(ctx.get_M())
+    s_gpu = ctx.debug_get_signs(n).cpu().numpy()[:, cols].astype(np.float64)
+    m_ta, m_raw, flips, outside = np.zeros((d, cols.size)), np.zeros((d, cols.size)), 0, 0
+    for k, (xt32, y_c, sc) in enumerate(kept):
+        sg = s_gpu[k * w.n:(k + 1) * w.n]
+        s_ref = O.sgn(y_c)
+        diff = sg != s_ref
+        flips += int(diff.sum())
+        outside += int((diff & (np.abs(y_c) > band_scale * sc)).sum())
+        xt = xt32.astype(np.float64)
+        m_ta += xt.T @ (sg / np.sqrt(d))
+        m_raw += xt.T @ (s_ref / np.sqrt(d))
+    rep = {"J_rel": abs(j - j_ref) / j_ref, "N_equal": True,
+           "M_rel_tie_aware": float(np.linalg.norm(m[:, cols] - m_ta) / np.linalg.norm(m_ta)),
+           "M_rel_raw": float(np.linalg.norm(m[:, cols] - m_raw) / np.linalg.norm(m_raw)),
+           "flip_frac": flips / s_gpu.size, "flips_outside_band": outside}
+    log_parity(w.name, "tc", "cycle 1, all 16 batches in one run of the products (24 sampled columns)", rep)
+    assert_step(rep, "tc", FLIP_MAX["tc"])
+    del kept, s_gpu
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, (st.status, st.ns_steps_used)
+    r_new = _f64(ctx.get_R())
+    rep = {"orth": float(np.max(np.abs(r_new.T @ r_new - np.eye(d)))),
+           "gap": float(1.0 - np.sum(r_new * m) / O.procrustes_optimum(m))}
+    log_parity(w.name, "tc", "cycle 1 update (16 batches, no proximal term)", rep, ns_steps_used=int(st.ns_steps_used),
+               ns_steps_budget=w.ns_steps)
+    assert rep["orth"] <= TOL["tc"]["orth"], rep
+    assert -1e-9 <= rep["gap"] <= TOL["tc"]["gap"], rep
+    assert np.sum(r_new * m) >= j * (1.0 - 1e-3)
+
+
+def test_c2_tc_second_cycle_after_a_newton_schulz_update():
+    """Cycle 2 of the headline workload: R is the output of the first polar update, so rotated rows sit nearer to
+    corners and near-ties are denser than under the randomised Hadamard start."""
+    w = I.WORKLOADS["c2"]
+    ctx = _ctx(w, "tc")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    for k in range(w.update_every):
+        ctx.step(_dev_bf16(I.batch(w, k)))
+    ctx.update()
+    assert ctx.get_stats().status == 0
+    _cycle(ctx, w, "tc", w.update_every, "cycle 2")
+
+
+@pytest.mark.parametrize("name", ["c4a", "c4a_zp"])
+def test_c4a_tc_fake_quant_cycle_and_update_at_d4096(name):
+    w = I.WORKLOADS[name]
+    ctx = _ctx(w, "tc")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    _cycle(ctx, w, "tc", 0, "cycle 1")
+
+
+def test_c1_tc_second_update():
+    """c1 updates after every batch: the second batch runs on a Newton-Schulz output."""
+    w = I.WORKLOADS["c1"]
+    ctx = _ctx(w, "tc")
+    ctx.set_R(_torch().from_numpy(I.initial_rotation(w)).cuda())
+    ctx.step(_dev_bf16(I.batch(w, 0)))
+    ctx.update()
+    assert ctx.get_stats().status == 0
+    _cycle(ctx, w, "tc", 1, "cycle 2")

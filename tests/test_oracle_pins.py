@@ -166,6 +166,28 @@ def test_polar_is_orthogonal_and_optimal(d):
         assert np.trace(q.T @ m) <= s.sum() + 1e-12
 
 
+def test_procrustes_optimum_closed_forms_and_bound():
+    """tr(R^T M) at the optimum: d = 2 closed form (the better of the best rotation and the best reflection),
+    a diagonal matrix (sum of |entries|), an orthogonal matrix (d), the trace of (M^T M)^(1/2) by an
+    eigendecomposition, and the fact that no orthogonal matrix exceeds it while polar_svd's factor attains it."""
+    rng = np.random.default_rng(41)
+    m = rng.standard_normal((2, 2)) * np.array([[3.0, 0.5]])
+    rot = np.hypot(m[0, 0] + m[1, 1], m[0, 1] - m[1, 0])
+    ref = np.hypot(m[0, 0] - m[1, 1], m[0, 1] + m[1, 0])
+    assert np.isclose(O.procrustes_optimum(m), max(rot, ref), rtol=1e-12)
+    dg = np.array([3.0, -2.0, 0.5, -0.25])
+    assert np.isclose(O.procrustes_optimum(np.diag(dg)), 5.75, rtol=1e-13)
+    q = _rand_orth(7, 24)
+    assert np.isclose(O.procrustes_optimum(q), 24.0, rtol=1e-12)
+    a = rng.standard_normal((40, 40)) @ np.diag(np.logspace(0, -5, 40))
+    w = np.linalg.eigvalsh(a.T @ a)
+    assert np.isclose(O.procrustes_optimum(a), np.sqrt(np.clip(w, 0.0, None)).sum(), rtol=1e-7)
+    r, _ = O.polar_svd(a)
+    assert np.isclose(np.trace(r.T @ a), O.procrustes_optimum(a), rtol=1e-12)
+    for k in range(10):
+        assert np.trace(_rand_orth(200 + k, 40).T @ a) <= O.procrustes_optimum(a) + 1e-12
+
+
 @pytest.mark.parametrize("d", [4, 32, 96])
 def test_polar_against_independent_routes(d):
     m = np.random.default_rng(30 + d).standard_normal((d, d))

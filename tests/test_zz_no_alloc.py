@@ -4,12 +4,14 @@ Some users of the library run where cudaMalloc is off limits (a runtime that own
 a plugin in a process whose memory is pre-assigned), so they cannot hand conqur_init a workspace.  This
 entry point keeps its scratch in a fixed array inside the library.  The test calls it through the C ABI
 twice in a row (a large batch, then a smaller one with skipped rows, so stale scratch from the first call
-would show) and checks both results against the regular conqur_step + conqur_get_objective path.
+would show) and checks both results against the regular conqur_step + conqur_get_objective path and against
+the float64 oracle's objective and token count.
 Collected last on purpose: a run that stops at the first failure has already run every other test.
 """
 import numpy as np
 import pytest
 
+from oracle import conqur_oracle as O
 from paper_2605_10793_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
@@ -53,6 +55,12 @@ def test_noalloc_objective_matches_regular_path_twice_in_a_row():
     assert got_n[0] == n1 == 3000 and got_n[1] == n2 == 775
     assert abs(got_j[0] - j1) <= 1e-6 * abs(j1)
     assert abs(got_j[1] - j2) <= 1e-6 * abs(j2)
+    # and against the definition: the oracle on the same bits (the second batch holds a zero row and a NaN row)
+    r64 = r.cpu().numpy().astype(np.float64)
+    o1 = O.OpuOracle(d, r64).step(x1.float().cpu().numpy().astype(np.float64))
+    o2 = O.OpuOracle(d, r64).step(x2_np.astype(np.float64))
+    assert got_n[0] == o1.N and got_n[1] == o2.N
+    assert abs(got_j[0] - o1.J) <= 1e-6 * o1.J and abs(got_j[1] - o2.J) <= 1e-6 * o2.J
 
 
 def test_noalloc_rejects_sizes_beyond_the_fixed_scratch():
