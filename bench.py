@@ -7,6 +7,8 @@ path (row norms, rotate + corner target, cross-covariance accumulate, Newton-Sch
 its orthogonality check).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --workload c1|c3|c4a|c4a_zp|c4b|a1_8b|fold|hadamard      other workloads, same line layout
+  python bench.py --profile-case path|heads|hadamard [--d ..] [--n ..]     a small bounded run for profiler captures
 
 N > 1 (torchrun): N independent replicas, one per GPU, no data-path collective ("weak" scaling).
 --impl reference: times the float64 CPU oracle, as it stands, on the host cores.
@@ -31,9 +33,22 @@ from paper_2605_10793_b200 import dist as D          # noqa: E402
 from paper_2605_10793_b200 import inputs as I        # noqa: E402
 
 METRIC = "calibration tokens/sec at d=4096 (whole path incl. polar update every 8 batches)"
-# DRAM bytes per launch at d = 4096, n = 2048 from the ncu capture summarised under profiles/ (same kernels)
-NCU_DRAM_BYTES_PER_LAUNCH = {"rotate_target": 53.6e6, "accumulate": 113.0e6, "ns_residual": 36.4e6, "ns_poly": 36.0e6, "ns_next": 235.6e6}
 WORKLOAD = "c2"
+NOMINAL_BF16_TFLOPS = 2250.0          # B200 dense bf16 datasheet figure (context next to the measured peaks)
+
+
+def ncu_traffic(tag: str):
+    """DRAM bytes per launch of a kernel, as counted by a profiler capture: every summary under profiles/ carries
+    lines `traffic <tag> <bytes>`; None when there is no capture of that kernel."""
+    import glob
+    import re
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        with open(path) as fh:
+            for line in fh:
+                m = re.match(r"\s*traffic\s+(\S+)\s+([0-9.eE+]+)\s*$", line)
+                if m and m.group(1) == tag:
+                    return float(m.group(2)), os.path.relpath(path, ROOT)
+    return None, None
 
 
 def _peaks():
@@ -63,22 +78,28 @@ def generate_batches(name: str, count: int, replica: int, workers: int):
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks / throttle reasons sampled every 50 ms while the timed region runs."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
+        # name the device by its UUID: under CUDA_VISIBLE_DEVICES the CUDA ordinal is not nvidia-smi's index
+        self.gpu = str(gpu_index)
+        try:
+            import torch
+            self.gpu = "GPU-" + str(torch.cuda.get_device_properties(gpu_index).uuid)
+        except Exception:
+            pass
         self.proc = None
         self.lines = []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                ["nvidia-smi", "-i", self.gpu, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except Exception:
@@ -116,8 +137,10 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def cpu_oracle_sample(w, cycles: int = 1):
-    """Time the float64 oracle, as it stands, on one update cycle of the workload (steps + one SVD update)."""
+def cpu_oracle_sample(w, cycles: int = 1, keep=None):
+    """Time the float64 oracle, as it stands, on one update cycle of the workload (steps + one SVD update).
+    keep: a dict that receives the first cycle's sign matrices, cross-covariance and objective (copied outside the
+    timed sections) for the parity figures of the bench line."""
     from oracle import conqur_oracle as O
     try:
         from threadpoolctl import threadpool_info
@@ -133,6 +156,10 @@ def cpu_oracle_sample(w, cycles: int = 1):
             t0 = time.perf_counter()
             orc.step(x)
             t_step += time.perf_counter() - t0
+            if keep is not None and c == 0:
+                keep.setdefault("signs", []).append(orc.last_S.astype(np.int8))
+        if keep is not None and c == 0:
+            keep.update(M=orc.M.copy(), J=orc.J, N=orc.N)
         t0 = time.perf_counter()
         orc.update()
         t_upd += time.perf_counter() - t0
@@ -281,6 +308,123 @@ def _workload_desc(w):
             f"R0=randomised Hadamard, polar update every {w.update_every} batches")
 
 
+def parity_sample(ctx, w, r0, dev, keep):
+    """The first cycle of the stream through the library once more, compared with what the oracle's timed sample of
+    the same cycle left behind: fraction of sign decisions that differ, raw cross-covariance and objective error."""
+    import torch
+    cyc = w.update_every
+    ctx.set_R(r0)
+    for b in range(cyc):
+        ctx.step(dev[b])
+    j, n = ctx.get_objective()
+    m = ctx.get_M().cpu().numpy().astype(np.float64)
+    s_gpu = ctx.debug_get_signs(cyc * w.n).cpu().numpy()
+    s_ref = np.concatenate(keep["signs"], axis=0)
+    ctx.update()
+    torch.cuda.synchronize()
+    return {"what": f"cycle 1 ({cyc} batches from R0) against the float64 oracle",
+            "sign_flip_fraction": float((s_gpu != s_ref).mean()),
+            "M_rel_raw": float(np.linalg.norm(m - keep["M"]) / np.linalg.norm(keep["M"])),
+            "J_rel": float(abs(j - keep["J"]) / keep["J"]), "N_equal": bool(n == keep["N"])}
+
+
+def heads_entry(peaks, K: int = 10, W: int = 3):
+    """The per-head workload (1024 problems of d = 128, 4096 tokens each) inside the headline run: one batched step and
+    one batched update, device-timed.  64 distinct seeded problems, stored 16 times at distinct addresses (every byte
+    is still read from HBM once per step)."""
+    import torch
+    from paper_2605_10793_b200 import binding as B
+    w = I.WORKLOADS["c4b"]
+    P, n, d, distinct = w.problems, w.n, w.d, 64
+    gen = [_gen_problem((w.name, p)) for p in range(distinct)]
+    x = torch.from_numpy(np.concatenate([b for b, _ in gen], axis=0).view(np.int16)).cuda().view(torch.bfloat16)
+    x = x.repeat(P // distinct, 1).contiguous()
+    r0 = torch.from_numpy(np.stack([r for _, r in gen])).cuda().repeat(P // distinct, 1, 1).contiguous()
+    ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", batch=P)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    for k in range(W + K):
+        ctx.set_R(r0)
+        e = ev[max(0, k - W)]
+        e[0].record()
+        ctx.step_batched(x, n, d, n * d)
+        e[1].record()
+        ctx.update()
+        e[2].record()
+    torch.cuda.synchronize()
+    st = ctx.get_stats()
+    step_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    upd_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    gbs = 2.0 * P * n * d / (step_ms * 1e-3) / 1e9
+    ctx.close()
+    return {"workload": f"c4b: {P} problems x ({n} x {d}) bf16", "step_ms": step_ms, "polar_update_ms": upd_ms,
+            "tokens_per_s": P * n / ((step_ms + upd_ms) * 1e-3), "step_hbm_gbs": gbs, "step_frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+            "ns_steps_used": int(st.ns_steps_used), "status": int(st.status)}
+
+
+def hadamard_entry(peaks, K: int = 20, W: int = 3):
+    """conqur_hadamard_rows on 32768 x 4096 bf16 -> bf16 inside the headline run, device-timed."""
+    import torch
+    from paper_2605_10793_b200 import binding as B
+    n, d = 32768, 4096
+    x = torch.randn(n, d, device="cuda").to(torch.bfloat16)
+    y = torch.empty_like(x)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for k in range(W + K):
+        if k == W:
+            e0.record()
+        B.conqur_hadamard_rows(x, out=y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K
+    gbs = 4.0 * n * d / (ms * 1e-3) / 1e9
+    return {"workload": f"hadamard: {n} x {d} bf16 in, bf16 out", "ms": ms, "hbm_gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+            "status": int(B.conqur_hadamard_status())}
+
+
+def profile_case(args):
+    """A small, bounded invocation for profiler captures: a few dozen launches, well under a few GB on the device.
+    Prints what it ran so that a plain run can be checked before a capture.
+      path      --batches B batches of --n tokens at width --d through conqur_step (queued, one run of the two
+                products) and one conqur_update
+      heads     the per-head kernels: --problems problems of d = 128, --n tokens each, two (step, update) rounds
+      hadamard  conqur_hadamard_rows on --n x --d bf16, three launches"""
+    import torch
+    from paper_2605_10793_b200 import binding as B
+    if args.profile_case == "hadamard":
+        x = torch.randn(args.n, args.d, device="cuda").to(torch.bfloat16)
+        y = torch.empty_like(x)
+        for _ in range(3):
+            B.conqur_hadamard_rows(x, out=y)
+        rc = B.conqur_hadamard_status()
+        print(f"profile-case hadamard n={args.n} d={args.d} bf16: status={rc} |y|max={y.float().abs().max().item():.3f}")
+        return 0 if rc == 0 else 1
+    if args.profile_case == "heads":
+        P, n, d = args.problems, args.n, 128
+        x = (torch.randn(P * n, d, device="cuda") * (1.0 + 20.0 * (torch.arange(d, device="cuda") < 2))).to(torch.bfloat16)
+        ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", batch=P)
+        for _ in range(2):
+            ctx.step_batched(x, n, d, n * d)
+            ctx.update()
+        st = ctx.get_stats()
+        print(f"profile-case heads P={P} n={n}: ns_steps={st.ns_steps_used} orth={st.orth_err:.2e} status={st.status}")
+        return 0 if st.status == 0 else 1
+    d, n, nb = args.d, args.n, max(1, args.batches)
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, r0="hadamard" if d & (d - 1) == 0 else "qr")
+    ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", defer_batches=nb,
+                    prior_rel=0.0 if nb * n >= 2 * d else 1e-2, debug_flags=B.CONQUR_DEBUG_NO_GRAPH)
+    ctx.set_R(torch.from_numpy(I.initial_rotation(w)).cuda())
+    xs = [torch.from_numpy(I.batch(w, b)).cuda().to(torch.bfloat16) for b in range(nb)]
+    torch.cuda.synchronize()
+    for x in xs:
+        ctx.step(x)
+    j, cnt = ctx.get_objective()
+    ctx.update()
+    st = ctx.get_stats()
+    print(f"profile-case path d={d} n={n} batches={nb}: J/N={j / cnt:.5f} ns_steps={st.ns_steps_used} "
+          f"orth={st.orth_err:.2e} status={st.status} launches={ctx.get_profile()['total_launches']}")
+    return 0 if st.status == 0 else 1
+
+
 # ------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -292,9 +436,19 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--distinct-cycles", type=int, default=0, help="cycles of distinct batches kept resident (0=all)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the per-head and Walsh-Hadamard entries of the line")
+    ap.add_argument("--profile-case", default=None, choices=["path", "heads", "hadamard"],
+                    help="run a small bounded case (for profiler captures) instead of the benchmark")
+    ap.add_argument("--d", type=int, default=4096)
+    ap.add_argument("--n", type=int, default=2048)
+    ap.add_argument("--problems", type=int, default=592)
+    ap.add_argument("--batches", type=int, default=1, help="--profile-case path: batches queued before the products run")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue the update's launches directly (profiler launch lists)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.profile_case:
+        return profile_case(args)
 
     import torch
     from paper_2605_10793_b200 import binding as B
@@ -304,7 +458,7 @@ def main():
     torch.cuda.set_device(g.local_rank)
     B.load()
     if args.workload not in I.WORKLOADS:
-        from paper_2605_10793_b200 import bench_extra as X      # Algorithm-1 mini-batch, Hadamard transform, weight folding
+        import bench_extra as X      # Algorithm-1 mini-batch, Hadamard transform, weight folding
         return X.RUNNERS[args.workload](args, g, ClockSampler, _peaks())
     w = I.WORKLOADS[args.workload]
     if w.problems > 1:
@@ -326,8 +480,10 @@ def main():
     resident_bytes = sum(t.numel() * 2 for t in dev)
     r0 = torch.from_numpy(I.initial_rotation(w)).cuda()
 
+    # the products of a cycle run once over all its batches (conqur_config.defer_batches = the update cadence)
     ctx = B.Context(d=w.d, n_max=w.n, in_dtype="bf16", mode="tc", quant_bits=w.quant_bits, prior_rel=w.prior_rel,
-                    quant_mode=w.quant_mode, clip_ratio=w.clip_ratio)
+                    quant_mode=w.quant_mode, clip_ratio=w.clip_ratio, defer_batches=cyc, ns_steps=w.ns_steps,
+                    debug_flags=B.CONQUR_DEBUG_NO_GRAPH if args.no_graph else 0)
     ctx.set_R(r0)
 
     def cycle_resident(c):
@@ -450,25 +606,32 @@ def main():
     tot_fl = sum(prof[k]["flops"] for k in gemm_classes)
     tot_ms = sum(prof[k]["ms"] for k in gemm_classes)
     tot_n = sum(prof[k]["timed"] for k in gemm_classes)
-    peak = peaks["bf16_tflops_sustained"]
+    # every launch is timed alone between its own events and the SM clock stays near its maximum over the short
+    # timed region, so the burst figure is the denominator (the sustained one is given beside it)
+    peak = peaks["bf16_tflops"]
     detail = {k: {"launches": prof[k]["timed"], "avg_ms": prof[k]["ms"] / max(1, prof[k]["timed"]),
                   "tflops": (prof[k]["flops"] / (prof[k]["ms"] * 1e-3) / 1e12) if prof[k]["ms"] > 0 else 0.0}
               for k in gemm_classes}
+    for k in gemm_classes:
+        detail[k]["frac_of_measured_burst"] = detail[k]["tflops"] / peaks["bf16_tflops"]
+        detail[k]["frac_of_nominal_2250"] = detail[k]["tflops"] / NOMINAL_BF16_TFLOPS
     # the dominant kernel: the instantiation of tc_gemm_kernel with the largest share of device time
     dom = max(gemm_classes, key=lambda k: prof[k]["ms"])
     dom_fl, dom_ms, dom_n = prof[dom]["flops"], prof[dom]["ms"], max(1, prof[dom]["timed"])
     achieved = dom_fl / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
     all_tf = tot_fl / (tot_ms * 1e-3) / 1e12 if tot_ms > 0 else 0.0
+    traffic, traffic_src = ncu_traffic(f"{w.name}.{dom}")
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom) if w.name in ("c2", "c4a") else None,
+                "traffic": traffic,
                 "kernel": f"tc_gemm_kernel, {dom} epilogue (largest share of device time)", "launches": dom_n,
                 "flops_per_launch": dom_fl / dom_n, "avg_launch_ms": dom_ms / dom_n,
                 "flops_note": "flops of the tiles computed (a symmetric product counts its upper-triangle tiles, a split "
                               "product each pass), summed over the launches and divided by their summed event time",
-                "traffic_note": "dram__bytes_read+write per launch, ncu capture summarised in "
-                                "profiles/tc_gemm_kernel_d4096_n2048_ncu_full.md",
-                "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
-                "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+                "traffic_note": (f"dram__bytes_read+write per launch, ncu capture summarised in {traffic_src}"
+                                 if traffic_src else "no profiler capture of this kernel at this size"),
+                "peak_source": f"{peaks['source']} burst bf16 (sustained {peaks['bf16_tflops_sustained']})",
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                 "all_contractions": {"achieved": all_tf, "frac": all_tf / peak, "launches": tot_n,
                                      "share_of_cycle": tot_ms / max(1, min(K, 4)) / (ms / K)},
                 "per_epilogue": detail}
@@ -477,22 +640,28 @@ def main():
         D.finish(g)
         return 0
 
-    cpu_base = None
+    cpu_base, parity = None, None
     if not args.no_cpu_baseline and g.world == 1:
-        cpu_base = cpu_oracle_sample(w, 1)
+        keep = {}
+        cpu_base = cpu_oracle_sample(w, 1, keep)
         cpu_base = {k: cpu_base[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        parity = parity_sample(ctx, w, r0, dev, keep)
+    extra = None
+    if not args.no_extra and g.world == 1 and w.name == WORKLOAD:
+        extra = {"c4b": heads_entry(peaks), "hadamard": hadamard_entry(peaks)}
 
     out = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": g.world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": _workload_desc(w), "tokens_per_step": cyc * w.n, "mode": "tc (bf16 operands, fp32 accumulate; "
-                   "Newton-Schulz: residual product as 3-term bf16 split on symmetric tiles, polynomial product 1 term, "
-                   "iterate product 2 terms then 1)", "l2": f"inputs larger than L2: {resident_bytes / 1e6:.0f} MB "
+                   "the two step products run once per cycle over its 8 queued batches; Newton-Schulz: residual product "
+                   "as 1- or 3-term bf16 split on symmetric tiles, polynomial product 1 term, iterate product 2 terms "
+                   "then 1)", "l2": f"inputs larger than L2: {resident_bytes / 1e6:.0f} MB "
                    f"of distinct batches resident, each read once per cycle", "replicas": g.world,
                    "input_gen_s": round(t_gen, 1)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu_base,
+        "roofline": roofline, "cpu_baseline": cpu_base, "parity_sample": parity, "extra": extra,
         "polar_update_ms": float(np.mean(upd_ms)) if upd_ms else None,
         "polar_update_ms_min": float(np.min(upd_ms)) if upd_ms else None,
         "ns_steps_used": int(st2.ns_steps_used), "orth_err": float(st2.orth_err),

@@ -17,8 +17,8 @@ import time
 
 import numpy as np
 
-from . import dist as D
-from . import inputs as I
+from paper_2605_10793_b200 import dist as D
+from paper_2605_10793_b200 import inputs as I
 
 
 def _gen_site(args):
@@ -40,7 +40,7 @@ def _pool_map(fn, jobs, world):
 
 def run_algorithm1(args, g, ClockSampler, peaks):
     import torch
-    from . import algorithm1 as A1
+    from paper_2605_10793_b200 import algorithm1 as A1
     a = I.SITE_MODELS["a1_8b"]
     K, W = args.steps, max(args.warmup, 3)
     L, n = a.n_layers, a.n
@@ -169,7 +169,7 @@ def run_algorithm1(args, g, ClockSampler, peaks):
 
 def run_hadamard(args, g, ClockSampler, peaks):
     import torch
-    from . import binding as B
+    from paper_2605_10793_b200 import binding as B
     K, W = args.steps, max(args.warmup, 3)
     n, d = 32768, 4096
     x = torch.randn(n, d, device="cuda").to(torch.bfloat16)
@@ -227,7 +227,7 @@ def run_hadamard(args, g, ClockSampler, peaks):
 
 def run_fold(args, g, ClockSampler, peaks):
     import torch
-    from . import binding as B
+    from paper_2605_10793_b200 import binding as B
     K, W = args.steps, max(args.warmup, 3)
     d, cols = 4096, 14336
     w = torch.from_numpy(I.random_weight(1, d, cols)).cuda()

@@ -51,7 +51,7 @@ struct Cfg {
   QuantSpec qs;
   int diagnostics;
   int64_t n_max;
-  float orth_tol, prior_rel, fro_tol, margin;
+  float orth_tol, prior_rel, fro_tol, margin, lo_budget;
   bool simt_ns;             // the Newton-Schulz products run on the fp32 CUDA-core kernels (exact mode)
 };
 
@@ -112,10 +112,12 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   L->sched = take(sizeof(SchedEntry) * NS_SCHED_MAX);
   L->acc_splits = 1;
   L->C = L->splitk = 0;
-  L->Xa = take(sizeof(float) * dd * P);
-  L->Xb = take(sizeof(float) * dd * P);
-  L->E = take(sizeof(float) * dd * P);
-  L->B = take(sizeof(float) * dd * P);
+  // the four Newton-Schulz matrices form ONE region: a token-split per-head step borrows all of it as scratch
+  const size_t ns_one = align_up(sizeof(float) * dd * P);
+  L->Xa = take(4 * ns_one);
+  L->Xb = L->Xa + ns_one;
+  L->E = L->Xb + ns_one;
+  L->B = L->E + ns_one;
   if (c->mode == CONQUR_EXACT_F32) {
     L->C = take(sizeof(float) * (size_t)n * d * P);
     L->acc_splits = pick_acc_splits(d, (int)P, n);
@@ -142,7 +144,7 @@ struct conqur_ctx {
   int pending_batches = 0;
   int8_t* sign_capture = nullptr;   // conqur_debug_capture_signs: where the fused per-head kernel writes its decisions
   int64_t sign_capture_rows = 0;
-  int n_sched, first_endgame, reenter_idx;
+  int n_sched, n_lift_init;   // device schedule: entry 0 = lifting quintic, 1 .. n_sched-1 = endgame; planned lifting steps
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
   Prof prof;
@@ -325,20 +327,20 @@ int update_impl(conqur_ctx* c) {
   const float isd = (float)(1.0 / std::sqrt((double)d));
   if (g.mode == CONQUR_TC_BF16 && P > 1) {
     // many small problems: the whole iteration of a problem runs inside one CTA
-    const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->first_endgame, c->reenter_idx, g.ns_max_steps, d, 1,
-                              g.orth_tol, g.fro_tol};
+    const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, d, 1,
+                              g.orth_tol, g.fro_tol, g.margin, g.lo_budget};
     return tcb_update(c->tc, c->stream, ncp, g.prior_rel, g.margin);
   }
 
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
   CQ_LAUNCHED(c, K_OTHER);
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau, c->n_lift_init);
   CQ_LAUNCHED(c, K_OTHER);
   if (g.prior_rel > 0.f) {
     sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 1, pd);
     CQ_LAUNCHED(c, K_OTHER);
   }
-  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau);
+  ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau, c->n_lift_init);
   CQ_LAUNCHED(c, K_OTHER);
   if (g.simt_ns) {
     ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
@@ -350,7 +352,8 @@ int update_impl(conqur_ctx* c) {
 
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);
-  const NsControlParams ncp{sched, c->n_sched, c->first_endgame, c->reenter_idx, g.ns_max_steps, d, use_shift, g.orth_tol, g.fro_tol};
+  const NsControlParams ncp{sched, c->n_sched, c->n_lift_init, g.ns_max_steps, d, use_shift, g.orth_tol, g.fro_tol, g.margin,
+                            g.lo_budget};
   for (int k = 0; k <= g.ns_max_steps; ++k) {
     const int cur = k & 1;
     float* X = cur ? Xb : Xa;
@@ -379,7 +382,7 @@ int update_impl(conqur_ctx* c) {
     if (rc) return rc;
   }
   if (g.mode == CONQUR_TC_BF16) { int rc = tc_refresh_R(c->tc, c->stream, /*only_if_converged=*/1); if (rc) return rc; }
-  ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st);
+  ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st, c->n_sched - 1);
   CQ_LAUNCHED(c, K_OTHER);
   c->tc.ns_k = -1;
   if (c->prof.enabled) {
@@ -483,12 +486,12 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   pp.d = g.simt_ns ? 0 : d;
   pp.max_len = NS_SCHED_MAX;
   if (cfg->ns_lo_gap_budget > 0.f) pp.gap_budget = cfg->ns_lo_gap_budget;
-  c->sched = cfg->ns_steps > 0 ? plan_schedule_for_steps(std::min(cfg->ns_steps, NS_SCHED_MAX), pp, &c->first_endgame)
-                               : plan_schedule(pp, &c->first_endgame);
+  g.lo_budget = (float)pp.gap_budget;
+  c->sched = plan_device_schedule(pp, &c->n_lift_init);
   c->n_sched = (int)c->sched.size();
-  if (g.ns_max_steps == 0) g.ns_max_steps = std::min(120, c->n_sched + 12);
-  // if the schedule runs out (sigma_min below the assumed bound): two more lifting steps, then the endgame again
-  c->reenter_idx = std::max(0, c->first_endgame - 2);
+  // ns_steps > 0: the caller's budget of steps; the lifting count starts from what the budget leaves after the endgame
+  if (cfg->ns_steps > 0) c->n_lift_init = std::max(0, std::min(cfg->ns_steps, NS_SCHED_MAX) - (c->n_sched - 1));
+  if (g.ns_max_steps == 0) g.ns_max_steps = std::min(120, c->n_lift_init + c->n_sched - 1 + 12);
   std::vector<SchedEntry> coef(NS_SCHED_MAX);
   for (int i = 0; i < NS_SCHED_MAX; ++i) {
     const NsStep& s = c->sched[std::min(i, c->n_sched - 1)];

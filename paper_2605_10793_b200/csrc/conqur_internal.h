@@ -37,6 +37,11 @@ struct DevState {
   int ns_idx;               // next entry of the polynomial schedule
   int seg_x;                // tensor-core mode: passes of the next-iterate product of the step in flight (1 or 2)
   int seg_e;                // tensor-core mode: passes of the next residual product (1 while the iterate is tiny, else 3)
+  // How many lifting steps an update starts with is learnt per problem from the updates before it (bisection between
+  // the largest count that fell short and the smallest that sufficed); see ns_adapt_lift_plan.
+  int lift_init, lift_plan, lift_lo, lift_hi;
+  int lift_left;            // lifting steps still to run in the update in flight
+  float growth;             // cumulative growth of the smallest singular values in the update in flight
   double diag_pr, diag_rho, diag_qnum, diag_qden;   // Section-4 diagnostics accumulated since the last update
   unsigned char seg_log[128];   // seg_x | seg_e << 4 of each step of the last update (launch accounting)
 };

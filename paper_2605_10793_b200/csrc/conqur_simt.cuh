@@ -534,8 +534,39 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
 
 // phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
 // phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
+// Arm the lifting phase of an update: the count learnt so far, or the planned one on a problem's first update.
+__device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
+  if (!s->lift_init) { s->lift_plan = n_lift_init; s->lift_lo = -1; s->lift_hi = 127; s->lift_init = 1; }
+  s->lift_left = s->lift_plan;
+  s->ns_idx = 1;                       // first endgame entry of the device schedule (entry 0 is the lifting quintic)
+  s->growth = 1.0f;
+}
+
+// After an update has converged in `steps_used` steps: learn how many lifting steps the next one should start with.
+// The plan was lift_plan lifting + n_endgame endgame steps.  Converging within it proves lift_plan sufficient; needing
+// more proves it short (the extra steps were the slower continuation of the endgame, so nothing is lost but time).
+// Bisection between the largest count known short and the smallest known sufficient; when conditions change and a
+// count that used to suffice falls short, the bracket reopens upwards.
+__device__ __forceinline__ void ns_adapt_lift_plan(DevState* s, int n_endgame, int converged) {
+  const int plan = s->lift_plan;
+  if (!converged) { s->lift_plan = min(plan + 2, 60); s->lift_lo = plan; s->lift_hi = 127; return; }
+  const int extra = s->ns_steps_used - (plan + n_endgame);
+  if (extra <= 0) {
+    s->lift_hi = min(s->lift_hi, plan);
+  } else {
+    s->lift_lo = max(s->lift_lo, plan);
+    if (s->lift_hi <= s->lift_lo) s->lift_hi = 127;
+  }
+  int next;
+  if (s->lift_hi == 127) next = plan + max(1, (extra + 1) / 2);
+  else if (s->lift_hi - s->lift_lo > 1) next = (s->lift_lo + s->lift_hi) / 2;
+  else next = s->lift_hi;
+  s->lift_plan = min(max(next, 0), 60);
+}
+
 static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
-                                float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift, float e1_tau) {
+                                float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift, float e1_tau,
+                                int n_lift_init) {
   const int p = blockIdx.x;
   __shared__ double red[8];
   double v = 0.0;
@@ -553,7 +584,7 @@ static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ 
       s->ns_done = ok ? 0 : NS_DONE_FAILED;
       s->ns_steps_used = 0;
       s->ns_final_buf = 0;
-      s->ns_idx = 0;
+      ns_arm_lifting(s, n_lift_init);
       s->seg_x = 2;
       // ||X_0||_F = 1/(1+margin): mean sigma^2 of the first iterate (the tensor-core mode shifts by it)
       s->tau = use_shift ? 1.0f / ((1.0f + margin) * (1.0f + margin) * (float)d) : 1.0f;
@@ -572,19 +603,27 @@ static __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __
 }
 
 // After the residual product of step k: reduce the per-tile partials (max|G - I|, sum (G - I)^2, trace G with
-// G = X^T X), decide convergence, and pick the quintic of this step from the schedule:
-//   * normally the next entry;
+// G = X^T X), decide convergence, and pick the quintic of this step from the device schedule (entry 0 = the lifting
+// quintic p_f, entries 1 .. n_sched-1 = the endgame for a spectrum in [floor of p_f, 1]):
+//   * while lifting steps are left (the count is learnt per problem, see ns_adapt_lift_plan): p_f;
+//   * then the endgame entries in order;
 //   * once ||G - I||_F < 0.7 every singular value is known to lie above sqrt(1 - ||G - I||_F), so the schedule
-//     jumps ahead to the last endgame entry fitted for an interval that still contains the spectrum;
-//   * if the schedule ran out without convergence (sigma_min was below the assumed bound) it re-enters at
-//     `reenter_idx` (lifting steps are safe to repeat: they never push a singular value below their floor).
+//     jumps to the last endgame entry fitted for an interval that still contains the spectrum;
+//   * if the endgame ran out without convergence (the lifting phase was too short for the smallest singular value):
+//     the last, order-3 convergent entry again while only a little is missing (||G - I||_F < 0.97: whatever lags has
+//     sigma^2 > 0.03 and doubles per step), otherwise two more lifting steps (safe to repeat: they never push a
+//     singular value below their floor) and the endgame again.
+// The very first step also rescales: ||G_0||_F^(1/2) = (sum sigma^4)^(1/4) bounds the largest singular value of X_0
+// from above, far more tightly than the Frobenius norm X_0 was scaled by, and dividing X_0 by it is the same as
+// applying p(x / s): a / s, b / s^3, c / s^5.
 // The step is handed to the product kernels in shifted residual form (see ns_schedule.h): coef = (gamma + kappa,
 // beta1, beta2, kappa) where kappa = mean diagonal of beta1 E + beta2 E^2 is moved from the matrix that gets
 // rounded to bf16 into the scalar multiple of X.  use_shift == 0 (exact mode): tau = 1, kappa = 0.
 struct NsControlParams {
   const SchedEntry* sched;
-  int n_sched, first_endgame, reenter_idx, max_steps, d, use_shift;
-  float tol, fro_tol;
+  int n_sched, n_lift_init, max_steps, d, use_shift;
+  float tol, fro_tol, margin;
+  float lo_budget;          // tensor-core mode: the iterate enters the last product as hi + lo while d 2^-8 / growth exceeds this
 };
 
 // The decision itself (one thread): tmx = max|G - I|, tsq = ||G - I||_F^2, ttr = tr G of step k.
@@ -602,14 +641,30 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
     s->ns_done = NS_DONE_FAILED;
   } else {
     int idx = s->ns_idx;
+    bool lifting = false;
     if (fro < 0.7f) {
+      s->lift_left = 0;                                            // nothing is small any more
       const float lb = sqrtf(1.0f - fro);
-      for (int j = c.n_sched - 1; j >= c.first_endgame && j > idx; --j)
-        if (c.sched[j].l <= lb) { idx = j; break; }
+      for (int j = c.n_sched - 1; j >= 1; --j)
+        if (c.sched[j].l <= lb) { if (j > idx || idx >= c.n_sched) idx = j; break; }
     }
-    if (idx >= c.n_sched) idx = c.reenter_idx;
-    const SchedEntry e = c.sched[idx];
-    const double a = e.a, b = e.b, cc = e.c;
+    if (s->lift_left > 0) {
+      lifting = true;
+      s->lift_left -= 1;
+    } else if (idx >= c.n_sched) {
+      if (fro < 0.97f) { idx = c.n_sched - 1; }
+      else { lifting = true; s->lift_left = 1; idx = 1; }
+    }
+    const SchedEntry e = c.sched[lifting ? 0 : idx];
+    if (!lifting) idx += 1;
+    double a = e.a, b = e.b, cc = e.c;
+    if (k == 0 && c.use_shift) {
+      const double g2 = tsq + 2.0 * ttr - (double)c.d;            // ||G||_F^2 = ||G - I||_F^2 + 2 tr G - d
+      if (g2 > 0.0) {
+        const double sm = sqrt(sqrt(g2)) * (1.0 + (double)c.margin);
+        if (sm < 1.0) { const double s2 = sm * sm; a /= sm; b /= sm * s2; cc /= sm * s2 * s2; }
+      }
+    }
     const double tau = c.use_shift ? (double)s->tau : 1.0;
     const double b1 = b + 2.0 * cc * tau;
     double kappa = 0.0;
@@ -623,9 +678,13 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
     s->coef[1] = (float)b1;
     s->coef[2] = (float)cc;
     s->coef[3] = (float)kappa;
-    s->seg_x = e.seg_x;
-    if (k < 128) s->seg_log[k] = (unsigned char)(e.seg_x | (s->seg_e << 4));   // seg_e: what this step's residual product used
-    s->ns_idx = idx + 1;
+    // bf16 rounding of X adds noise of spectral size about 2^-8; after a cumulative growth G of the small singular
+    // values the directions it can scramble had sigma_0 <= 2^-8 / G, at most d of them: Procrustes gap <= d 2^-8 / G
+    const int seg_x = (!c.use_shift || (float)c.d * (1.0f / 256.0f) / s->growth > c.lo_budget) ? 2 : 1;
+    s->growth *= (float)a;
+    s->seg_x = seg_x;
+    if (k < 128) s->seg_log[k] = (unsigned char)(seg_x | (s->seg_e << 4));   // seg_e: what this step's residual product used
+    s->ns_idx = idx;
     s->ns_steps_used = k + 1;
   }
 }
@@ -679,9 +738,10 @@ static __global__ void ns_commit_kernel(DevState* st, const float* __restrict__ 
     M[p * dd + i] = 0.f;
   }
 }
-static __global__ void ns_commit_state_kernel(DevState* st) {
+static __global__ void ns_commit_state_kernel(DevState* st, int n_endgame) {
   DevState* s = st + blockIdx.x;
   if (threadIdx.x != 0) return;
+  ns_adapt_lift_plan(s, n_endgame, s->ns_done == NS_DONE_CONVERGED);
   if (s->ns_done == NS_DONE_CONVERGED) {
     s->last_J = s->J;
     s->last_N = s->N;

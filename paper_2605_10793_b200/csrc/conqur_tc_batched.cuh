@@ -625,7 +625,8 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       s->lam = lam; s->scale = fro;
       s->x0_scale = ok ? 1.0f / (fro * (1.0f + g.margin)) : 0.f;
       s->ns_done = ok ? 0 : NS_DONE_FAILED;
-      s->ns_steps_used = 0; s->ns_final_buf = 0; s->ns_idx = 0; s->seg_x = 2;
+      s->ns_steps_used = 0; s->ns_final_buf = 0; s->seg_x = 2;
+      ns_arm_lifting(s, g.ncp.n_lift_init);
       s->tau = 1.0f / ((1.0f + g.margin) * (1.0f + g.margin) * (float)TCB_D);
       aux->done = s->ns_done; aux->tau = s->tau; aux->x0s = s->x0_scale; aux->lam = lam;
     }
@@ -797,6 +798,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       }
     }
     if (threadIdx.x == 0) {
+      ns_adapt_lift_plan(s, ncp.n_sched - 1, converged ? 1 : 0);
       if (converged) {
         s->last_J = s->J; s->last_N = s->N; s->J = 0.0; s->N = 0; s->updates += 1;
         s->diag_pr = s->diag_rho = s->diag_qnum = s->diag_qden = 0.0;

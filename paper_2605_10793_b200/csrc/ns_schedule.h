@@ -181,6 +181,30 @@ inline std::vector<NsStep> plan_schedule(const NsPlanParams& p, int* first_endga
   return out;
 }
 
+// The schedule the device runs: entry 0 is the lifting quintic p_f, entries 1.. are the endgame for a spectrum in
+// [floor, 1], floor being the lower end of p_f's range on [l_f, 1].  How many times p_f is applied is decided per
+// update on the device; *n_lift receives the count that carries the assumed bound l0 above the floor.
+inline std::vector<NsStep> plan_device_schedule(const NsPlanParams& p, int* n_lift) {
+  NsStep f;
+  const double floor = ns_make_step(p.l_lift, p.margin, &f);
+  f.lift = 1;
+  std::vector<NsStep> out;
+  out.push_back(f);
+  NsPlanParams q = p;
+  q.l0 = floor;
+  q.max_len = p.max_len - 1;
+  for (const NsStep& s : plan_schedule(q)) out.push_back(s);
+  double l = std::min(std::max(p.l0, 1e-12), 1.0);
+  int n = 0;
+  while (l < floor && n < 60) {
+    const double l2 = l * l;
+    l = l * (f.a + l2 * (f.b + l2 * f.c));
+    ++n;
+  }
+  if (n_lift) *n_lift = n;
+  return out;
+}
+
 // The most conservative schedule (smallest l0) that still has at most `steps` entries.
 inline std::vector<NsStep> plan_schedule_for_steps(int steps, NsPlanParams p, int* first_endgame = nullptr) {
   double lo = std::log(1e-12), hi = std::log(0.9);

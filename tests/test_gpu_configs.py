@@ -255,7 +255,8 @@ def test_c3_tc_sixteen_batches_then_the_plain_update_at_d8192():
     log_parity(w.name, "tc", "cycle 1 update (16 batches, no proximal term)", rep, ns_steps_used=int(st.ns_steps_used),
                ns_steps_budget=w.ns_steps)
     assert rep["orth"] <= TOL["tc"]["orth"], rep
-    assert -1e-9 <= rep["gap"] <= TOL["tc"]["gap"], rep
+    # (a rotation that is orthogonal only to `orth` can exceed the optimum by about that much)
+    assert -2.0 * rep["orth"] <= rep["gap"] <= TOL["tc"]["gap"], rep
     assert np.sum(r_new * m) >= j * (1.0 - 1e-3)
 
 
