@@ -95,7 +95,8 @@ typedef struct {
                                pass instead of three while the iterate's mean squared singular value is below this;
                                0 = default */
   float    ns_lo_gap_budget;/* tensor-core mode tuning: bound on the Procrustes gap given up by dropping the low bf16
-                               half of the iterate in the next-iterate product of late steps; 0 = default 1e-4 */
+                               half of the iterate in the products of late steps (a worst-case bound: d directions at the
+                               noise floor under one dominant one; measured gaps are 20-50x smaller); 0 = default 5e-4 */
   int32_t  debug_flags;     /* test hooks, 0 in production: CONQUR_DEBUG_CANARIES | CONQUR_DEBUG_SINGLE_CTA |
                                CONQUR_DEBUG_NO_GRAPH */
 } conqur_config;
@@ -189,7 +190,9 @@ int conqur_step_batched_range(conqur_ctx* ctx, const void* X_dev, int64_t n, int
  * Host errors: CONQUR_ERR_EMPTY_UPDATE (no step since the last update),
  * CONQUR_ERR_RANK_DEFICIENT (tokens enqueued < d and prior_rel == 0).
  * If the iteration does not converge within ns_max_steps the old R and M are kept
- * and CONQUR_ERR_NS_NOT_CONVERGED is latched.
+ * and CONQUR_ERR_NS_NOT_CONVERGED is latched; read it with conqur_get_stats (which also puts the
+ * host-side row counts back, so that a later conqur_update sees the statistics that were kept)
+ * before the next conqur_update.  The rank check counts rows enqueued, skipped rows included.
  */
 int conqur_update(conqur_ctx* ctx);
 

@@ -138,6 +138,7 @@ struct conqur_ctx {
   char* ws;
   cudaStream_t stream;
   std::vector<int64_t> tokens;   // per problem: rows enqueued since the last update
+  std::vector<int64_t> tokens_at_update;   // ... as they stood when the last update was enqueued (restored if it is rejected)
   int64_t last_n;            // rows per problem of the last step (for debug_get_signs)
   int last_np;               // problems the last step call covered
   int64_t pending_rows = 0;  // deferring context: rows staged but not yet run through the two products
@@ -153,7 +154,10 @@ struct conqur_ctx {
   cudaStream_t cap_stream = nullptr;       // side stream used only to capture
   cudaGraphExec_t upd_graph = nullptr;
   int updates_enqueued = 0;
-  long long graph_launches[K_COUNT] = {0};
+  long long graph_launches[K_COUNT] = {0};     // launches of one graph replay (outside its loop, if it has one)
+  long long loop_body_launches[K_COUNT] = {0}; // launches of one pass of the looped graph's body
+  bool looped = false;                         // the graph holds a device-side loop
+  long long loop_passes_seen = 0;              // passes already folded into the launch counts
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   DevState* state() const { return at<DevState>(L.state); }
@@ -308,30 +312,19 @@ int ns_parts(const conqur_ctx* c) {
   return tc_ns_parts(c->tc);
 }
 
-int update_impl(conqur_ctx* c) {
+// The update in three parts, so that it can be enqueued unrolled (every step a fixed set of launches that early-exit once
+// the iteration has finished) or as a captured graph whose middle part is a device-side loop.
+int update_prologue(conqur_ctx* c) {
   const Cfg& g = c->cfg;
   const int d = g.d, P = g.P;
   const int64_t dd = (int64_t)d * d;
   DevState* st = c->state();
   float* M = c->at<float>(c->L.M);
   float* R = c->at<float>(c->L.R);
-  float* Xa = c->at<float>(c->L.Xa);
-  float* Xb = c->at<float>(c->L.Xb);
-  float* E = c->at<float>(c->L.E);
-  float* B = c->at<float>(c->L.B);
   double* pd = c->at<double>(c->L.part_d);
-  float* pf = c->at<float>(c->L.part_f);
-  const SchedEntry* sched = c->at<SchedEntry>(c->L.sched);
   const int use_shift = g.simt_ns ? 0 : 1;
   const int nb = (int)std::min<int64_t>(1024, (dd + 1023) / 1024);
   const float isd = (float)(1.0 / std::sqrt((double)d));
-  if (g.mode == CONQUR_TC_BF16 && P > 1) {
-    // many small problems: the whole iteration of a problem runs inside one CTA
-    const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, d, 1,
-                              g.orth_tol, g.fro_tol, g.margin, g.lo_budget};
-    return tcb_update(c->tc, c->stream, ncp, g.prior_rel, g.margin);
-  }
-
   sumsq_kernel<<<dim3(nb, P), 256, 0, c->stream>>>(M, R, dd, st, 0, pd);
   CQ_LAUNCHED(c, K_OTHER);
   ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 0, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau, c->n_lift_init);
@@ -343,56 +336,171 @@ int update_impl(conqur_ctx* c) {
   ns_setup_kernel<<<P, 256, 0, c->stream>>>(st, pd, nb, 1, g.prior_rel, isd, g.margin, d, use_shift, c->tc.e1_tau, c->n_lift_init);
   CQ_LAUNCHED(c, K_OTHER);
   if (g.simt_ns) {
-    ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, Xa, dd, st);
+    ns_x0_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(M, R, c->at<float>(c->L.Xa), dd, st);
     CQ_LAUNCHED(c, K_OTHER);
-  } else {
-    int rc = tc_ns_begin(c->tc, c->stream);      // the same X0, written as the bf16 pair the products read
-    if (rc) return rc;
+    return CONQUR_OK;
   }
+  return tc_ns_begin(c->tc, c->stream);          // the same X0, written as the bf16 pair the products read
+}
 
+// One Newton-Schulz step on the iterate in buffer `cur`: residual product, control decision, and (unless `last`)
+// the polynomial and next-iterate products.  k: the step's index, or -1 to take it from the device state.
+int update_step(conqur_ctx* c, int k, int cur, bool last) {
+  const Cfg& g = c->cfg;
+  const int d = g.d, P = g.P;
+  DevState* st = c->state();
+  float* Xa = c->at<float>(c->L.Xa);
+  float* Xb = c->at<float>(c->L.Xb);
+  float* E = c->at<float>(c->L.E);
+  float* B = c->at<float>(c->L.B);
+  double* pd = c->at<double>(c->L.part_d);
+  float* pf = c->at<float>(c->L.part_f);
+  const int use_shift = g.simt_ns ? 0 : 1;
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);
-  const NsControlParams ncp{sched, c->n_sched, c->n_lift_init, g.ns_max_steps, d, use_shift, g.orth_tol, g.fro_tol, g.margin,
-                            g.lo_budget};
-  for (int k = 0; k <= g.ns_max_steps; ++k) {
-    const int cur = k & 1;
-    float* X = cur ? Xb : Xa;
-    float* Xn = cur ? Xa : Xb;
-    c->tc.ns_k = k;
-    int rc = launch_residual(c, X, cur);
-    if (rc) return rc;
-    ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, use_shift ? pd + parts : nullptr, parts, k, cur, ncp);
-    CQ_LAUNCHED(c, K_OTHER);
-    if (k == g.ns_max_steps) break;
-    if (g.simt_ns) {
-      ns_gemm_exact_kernel<EPI_POLY><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(E, E, E, B, d, st, nullptr, nullptr);
-      CQ_LAUNCHED(c, K_NS_POLY);
-      ns_gemm_exact_kernel<EPI_NEXT><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(X, B, X, Xn, d, st, nullptr, nullptr);
-      CQ_LAUNCHED(c, K_NS_NEXT);
-    } else {
-      rc = tc_ns_poly_next(c->tc, c->stream, cur);
-      if (rc) return rc;
-    }
-  }
+  const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, d, use_shift, g.orth_tol,
+                            g.fro_tol, g.margin, g.lo_budget};
+  float* X = cur ? Xb : Xa;
+  float* Xn = cur ? Xa : Xb;
+  c->tc.ns_k = k;
+  int rc = launch_residual(c, X, cur);
+  if (rc) return rc;
+  ns_control_kernel<<<P, 256, 0, c->stream>>>(st, pf, pd, use_shift ? pd + parts : nullptr, parts, k, cur, ncp);
+  CQ_LAUNCHED(c, K_OTHER);
+  if (last) return CONQUR_OK;
   if (g.simt_ns) {
-    ns_commit_kernel<<<dim3(ew_blocks(dd), P), 256, 0, c->stream>>>(st, Xa, Xb, R, M, dd);
+    ns_gemm_exact_kernel<EPI_POLY><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(E, E, E, B, d, st, nullptr, nullptr);
+    CQ_LAUNCHED(c, K_NS_POLY);
+    ns_gemm_exact_kernel<EPI_NEXT><<<dim3(T, T, P), SG_THREADS, 0, c->stream>>>(X, B, X, Xn, d, st, nullptr, nullptr);
+    CQ_LAUNCHED(c, K_NS_NEXT);
+    return CONQUR_OK;
+  }
+  return tc_ns_poly_next(c->tc, c->stream, cur);
+}
+
+int update_epilogue(conqur_ctx* c) {
+  const Cfg& g = c->cfg;
+  const int64_t dd = (int64_t)g.d * g.d;
+  DevState* st = c->state();
+  if (g.simt_ns) {
+    ns_commit_kernel<<<dim3(ew_blocks(dd), g.P), 256, 0, c->stream>>>(st, c->at<float>(c->L.Xa), c->at<float>(c->L.Xb),
+                                                                     c->at<float>(c->L.R), c->at<float>(c->L.M), dd);
     CQ_LAUNCHED(c, K_OTHER);
   } else {
     int rc = tc_ns_commit(c->tc, c->stream);
     if (rc) return rc;
   }
   if (g.mode == CONQUR_TC_BF16) { int rc = tc_refresh_R(c->tc, c->stream, /*only_if_converged=*/1); if (rc) return rc; }
-  ns_commit_state_kernel<<<P, 32, 0, c->stream>>>(st, c->n_sched - 1);
+  ns_commit_state_kernel<<<g.P, 32, 0, c->stream>>>(st, c->n_sched - 1);
   CQ_LAUNCHED(c, K_OTHER);
   c->tc.ns_k = -1;
+  return CONQUR_OK;
+}
+
+int update_impl(conqur_ctx* c) {
+  const Cfg& g = c->cfg;
+  if (g.mode == CONQUR_TC_BF16 && g.P > 1) {
+    // many small problems: the whole iteration of a problem runs inside one CTA
+    const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, g.d, 1,
+                              g.orth_tol, g.fro_tol, g.margin, g.lo_budget};
+    return tcb_update(c->tc, c->stream, ncp, g.prior_rel, g.margin);
+  }
+  int rc = update_prologue(c);
+  if (rc) return rc;
+  for (int k = 0; k <= g.ns_max_steps; ++k) {
+    rc = update_step(c, k, k & 1, k == g.ns_max_steps);
+    if (rc) return rc;
+  }
+  rc = update_epilogue(c);
+  if (rc) return rc;
   if (c->prof.enabled) {
     // profiling pass only: find out how many of the enqueued steps actually ran
     DevState h0;
-    CQ_CUDA(cudaMemcpyAsync(&h0, st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CQ_CUDA(cudaMemcpyAsync(&h0, c->state(), sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
     CQ_CUDA(cudaStreamSynchronize(c->stream));
     c->prof.fold(h0.ns_steps_used, h0.seg_log);
   }
   return CONQUR_OK;
+}
+
+// Ends one pass of the graph's loop body (two Newton-Schulz steps): go round again while the iteration is running.
+// The pass counter bounds the loop whatever the data (the control kernel ends the iteration at ns_max_steps anyway).
+__global__ void ns_loop_condition_kernel(DevState* st, cudaGraphConditionalHandle handle, int max_passes) {
+  const int passes = ++st->loop_passes;
+  st->loop_passes_total += 1;
+  cudaGraphSetConditional(handle, (st->ns_done == 0 && passes < max_passes) ? 1u : 0u);
+}
+
+// The update as a graph: prologue, a WHILE node whose body is two steps (the iterate ping-pongs between two buffers,
+// and the tensor maps of a launch are fixed) and the loop condition, epilogue.  Steps that the iteration does not
+// need are then never launched.  Returns false if the driver cannot build it (the caller falls back to an unrolled capture).
+bool build_looped_update_graph(conqur_ctx* c) {
+  cudaGraph_t graph = nullptr;
+  if (cudaGraphCreate(&graph, 0) != cudaSuccess) { cudaGetLastError(); return false; }
+  cudaStream_t body_stream = nullptr;
+  bool ok = false, capturing = false, capturing_body = false;
+  cudaStream_t user = c->stream;
+  long long before[K_COUNT], total_before = c->prof.total;
+  for (int i = 0; i < K_COUNT; ++i) before[i] = c->prof.launches[i];
+  do {
+    cudaGraphConditionalHandle handle;
+    if (cudaGraphConditionalHandleCreate(&handle, graph, 1, cudaGraphCondAssignDefault) != cudaSuccess) break;
+    if (cudaStreamCreateWithFlags(&body_stream, cudaStreamNonBlocking) != cudaSuccess) break;
+    if (cudaStreamBeginCaptureToGraph(c->cap_stream, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) != cudaSuccess) break;
+    capturing = true;
+    c->stream = c->cap_stream;
+    if (update_prologue(c) != CONQUR_OK) break;
+    cudaStreamCaptureStatus status;
+    const cudaGraphNode_t* deps = nullptr;
+    size_t n_deps = 0;
+    if (cudaStreamGetCaptureInfo_v2(c->cap_stream, &status, nullptr, nullptr, &deps, &n_deps) != cudaSuccess) break;
+    cudaGraphNodeParams np = {};
+    np.type = cudaGraphNodeTypeConditional;
+    np.conditional.handle = handle;
+    np.conditional.type = cudaGraphCondTypeWhile;
+    np.conditional.size = 1;
+    cudaGraphNode_t loop_node;
+    if (cudaGraphAddNode(&loop_node, graph, deps, n_deps, &np) != cudaSuccess) break;
+    cudaGraph_t body = np.conditional.phGraph_out[0];
+    // ---- the loop body, captured on a stream of its own into the node's graph
+    for (int i = 0; i < K_COUNT; ++i) c->loop_body_launches[i] = -c->prof.launches[i];
+    if (cudaStreamBeginCaptureToGraph(body_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) != cudaSuccess) break;
+    capturing_body = true;
+    c->stream = body_stream;
+    if (update_step(c, -1, 0, false) != CONQUR_OK || update_step(c, -1, 1, false) != CONQUR_OK) break;
+    ns_loop_condition_kernel<<<1, 1, 0, body_stream>>>(c->state(), handle, c->cfg.ns_max_steps / 2 + 2);
+    if (cudaGetLastError() != cudaSuccess) break;
+    c->prof.count(K_OTHER);
+    cudaGraph_t body_out = nullptr;
+    capturing_body = false;
+    if (cudaStreamEndCapture(body_stream, &body_out) != cudaSuccess) break;
+    for (int i = 0; i < K_COUNT; ++i) c->loop_body_launches[i] += c->prof.launches[i];
+    // ---- what follows the loop
+    c->stream = c->cap_stream;
+    if (cudaStreamUpdateCaptureDependencies(c->cap_stream, &loop_node, 1, cudaStreamSetCaptureDependencies) != cudaSuccess) break;
+    if (update_epilogue(c) != CONQUR_OK) break;
+    cudaGraph_t out = nullptr;
+    capturing = false;
+    if (cudaStreamEndCapture(c->cap_stream, &out) != cudaSuccess) break;
+    if (cudaGraphInstantiate(&c->upd_graph, graph, 0) != cudaSuccess) { c->upd_graph = nullptr; break; }
+    ok = true;
+  } while (false);
+  c->stream = user;
+  c->tc.ns_k = -1;
+  cudaGraph_t junk = nullptr;
+  if (capturing_body) cudaStreamEndCapture(body_stream, &junk);
+  if (capturing) cudaStreamEndCapture(c->cap_stream, &junk);
+  if (body_stream) cudaStreamDestroy(body_stream);
+  cudaGraphDestroy(graph);
+  cudaGetLastError();
+  // launches of one replay outside the loop (the loop body's are added from the device's pass counter)
+  for (int i = 0; i < K_COUNT; ++i) {
+    c->graph_launches[i] = ok ? c->prof.launches[i] - before[i] - c->loop_body_launches[i] : 0;
+    c->prof.launches[i] = before[i];
+  }
+  c->prof.total = total_before;
+  c->looped = ok;
+  return ok;
 }
 
 // Enqueue one update: directly the first time (kernel attributes get set), then through a captured graph.
@@ -405,30 +513,33 @@ int update_enqueue(conqur_ctx* c) {
       cudaGetLastError();
       return update_impl(c);
     }
-    long long before[K_COUNT];
-    for (int i = 0; i < K_COUNT; ++i) before[i] = c->prof.launches[i];
-    const long long total_before = c->prof.total;
-    if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-      cudaGetLastError();
-      return update_impl(c);
+    if (!build_looped_update_graph(c)) {
+      // no conditional nodes: capture the unrolled sequence instead
+      long long before[K_COUNT];
+      for (int i = 0; i < K_COUNT; ++i) before[i] = c->prof.launches[i];
+      const long long total_before = c->prof.total;
+      if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        return update_impl(c);
+      }
+      cudaStream_t user = c->stream;
+      c->stream = c->cap_stream;
+      const int rc = update_impl(c);
+      c->stream = user;
+      cudaGraph_t graph = nullptr;
+      const cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
+      for (int i = 0; i < K_COUNT; ++i) { c->graph_launches[i] = c->prof.launches[i] - before[i]; c->prof.launches[i] = before[i]; }
+      c->prof.total = total_before;
+      if (rc != CONQUR_OK || e != cudaSuccess || !graph ||
+          cudaGraphInstantiate(&c->upd_graph, graph, 0) != cudaSuccess) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        c->upd_graph = nullptr;
+        c->updates_enqueued = -(1 << 30);          // stay on direct launches
+        return update_impl(c);
+      }
+      cudaGraphDestroy(graph);
     }
-    cudaStream_t user = c->stream;
-    c->stream = c->cap_stream;
-    const int rc = update_impl(c);
-    c->stream = user;
-    cudaGraph_t graph = nullptr;
-    const cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
-    for (int i = 0; i < K_COUNT; ++i) { c->graph_launches[i] = c->prof.launches[i] - before[i]; c->prof.launches[i] = before[i]; }
-    c->prof.total = total_before;
-    if (rc != CONQUR_OK || e != cudaSuccess || !graph ||
-        cudaGraphInstantiate(&c->upd_graph, graph, 0) != cudaSuccess) {
-      if (graph) cudaGraphDestroy(graph);
-      cudaGetLastError();
-      c->upd_graph = nullptr;
-      c->updates_enqueued = -(1 << 30);          // stay on direct launches
-      return update_impl(c);
-    }
-    cudaGraphDestroy(graph);
   }
   CQ_CUDA(cudaGraphLaunch(c->upd_graph, c->stream));
   for (int i = 0; i < K_COUNT; ++i) { c->prof.launches[i] += c->graph_launches[i]; c->prof.total += c->graph_launches[i]; }
@@ -515,7 +626,7 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
                      c->at<float>(L.rnorm), c->state(), c->at<double>(L.part_d), c->at<float>(L.part_f),
                      (cfg->quant_bits || cfg->diagnostics) ? c->at<float>(L.C) : nullptr, c->at<unsigned>(L.rowmax), g.qs,
                      g.diagnostics, g.diagnostics ? c->at<double>(L.part_diag) : nullptr, &c->prof,
-                     (g.debug_flags & CONQUR_DEBUG_SINGLE_CTA) != 0, cfg->ns_gram_single_pass_tau);
+                     (g.debug_flags & CONQUR_DEBUG_SINGLE_CTA) != 0, cfg->ns_gram_single_pass_tau, g.lo_budget);
     if (rc) return fail(rc);
     rc = tc_refresh_R(c->tc, c->stream, 0);
     if (rc) return fail(rc);
@@ -616,7 +727,10 @@ extern "C" int conqur_update(conqur_ctx* c) {
   if (fewest < c->cfg.d && c->cfg.prior_rel == 0.f) return CONQUR_ERR_RANK_DEFICIENT;
   { const int frc = flush_pending(c); if (frc) return frc; }
   const int rc = update_enqueue(c);
-  if (rc == CONQUR_OK) std::fill(c->tokens.begin(), c->tokens.end(), 0);
+  if (rc == CONQUR_OK) {
+    c->tokens_at_update = c->tokens;
+    std::fill(c->tokens.begin(), c->tokens.end(), 0);
+  }
   return rc;
 }
 
@@ -738,6 +852,11 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
   CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
   const int rc = sync_status(c);
   if (rc == CONQUR_ERR_CUDA) return rc;
+  if (rc == CONQUR_ERR_NS_NOT_CONVERGED && !c->tokens_at_update.empty()) {
+    // the device kept M, J and N of the rejected update: the host's row counts go back to match
+    for (size_t p = 0; p < c->tokens.size(); ++p) c->tokens[p] += c->tokens_at_update[p];
+    c->tokens_at_update.clear();
+  }
   clear_flags_kernel<<<1, 256, 0, c->stream>>>(c->state(), P, c->at<int>(c->L.flags_agg));
   CQ_LAUNCHED(c, K_OTHER);
   CQ_CUDA(cudaStreamSynchronize(c->stream));
@@ -757,9 +876,21 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
   return CONQUR_OK;
 }
 
+// The launches inside the update graph's loop: passes counted on the device x launches per pass (after a synchronise).
+static int fold_loop_launches(conqur_ctx* c) {
+  if (!c->looped) return CONQUR_OK;
+  DevState h0;
+  CQ_CUDA(cudaMemcpy(&h0, c->state(), sizeof(DevState), cudaMemcpyDeviceToHost));
+  const long long fresh = h0.loop_passes_total - c->loop_passes_seen;
+  c->loop_passes_seen = h0.loop_passes_total;
+  for (int i = 0; i < K_COUNT; ++i) { c->prof.launches[i] += fresh * c->loop_body_launches[i]; c->prof.total += fresh * c->loop_body_launches[i]; }
+  return CONQUR_OK;
+}
+
 extern "C" int conqur_set_profiling(conqur_ctx* c, int32_t enabled) {
   if (!c) return CONQUR_ERR_INVALID_ARG;
   CQ_CUDA(cudaStreamSynchronize(c->stream));
+  { const int lrc = fold_loop_launches(c); if (lrc) return lrc; }
   c->prof.fold(1 << 30);
   c->prof.reset();
   c->prof.enabled = enabled != 0;
@@ -770,6 +901,7 @@ extern "C" int conqur_get_profile(conqur_ctx* c, conqur_profile* out) {
   if (!c || !out || out->struct_size != sizeof(conqur_profile)) return CONQUR_ERR_INVALID_ARG;
   CQ_CUDA(cudaStreamSynchronize(c->stream));
   c->prof.fold(1 << 30);
+  { const int lrc = fold_loop_launches(c); if (lrc) return lrc; }
   for (int i = 0; i < CONQUR_KERNEL_CLASSES; ++i) {
     out->launches[i] = c->prof.launches[i];
     out->timed_launches[i] = c->prof.timed[i];

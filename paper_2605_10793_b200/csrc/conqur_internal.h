@@ -40,6 +40,8 @@ struct DevState {
   // How many lifting steps an update starts with is learnt per problem from the updates before it (bisection between
   // the largest count that fell short and the smallest that sufficed); see ns_adapt_lift_plan.
   int lift_init, lift_plan, lift_lo, lift_hi;
+  int loop_passes;          // passes of the update graph's loop body in the update in flight
+  long long loop_passes_total;   // ... since init (launch accounting)
   int lift_left;            // lifting steps still to run in the update in flight
   float growth;             // cumulative growth of the smallest singular values in the update in flight
   double diag_pr, diag_rho, diag_qnum, diag_qden;   // Section-4 diagnostics accumulated since the last update

@@ -532,12 +532,11 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
   if (threadIdx.x == 0) partials[(int64_t)p * gridDim.x + blockIdx.x] = tot;
 }
 
-// phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
-// phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
 // Arm the lifting phase of an update: the count learnt so far, or the planned one on a problem's first update.
 __device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
   if (!s->lift_init) { s->lift_plan = n_lift_init; s->lift_lo = -1; s->lift_hi = 127; s->lift_init = 1; }
   s->lift_left = s->lift_plan;
+  s->loop_passes = 0;
   s->ns_idx = 1;                       // first endgame entry of the device schedule (entry 0 is the lifting quintic)
   s->growth = 1.0f;
 }
@@ -545,8 +544,8 @@ __device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
 // After an update has converged in `steps_used` steps: learn how many lifting steps the next one should start with.
 // The plan was lift_plan lifting + n_endgame endgame steps.  Converging within it proves lift_plan sufficient; needing
 // more proves it short (the extra steps were the slower continuation of the endgame, so nothing is lost but time).
-// Bisection between the largest count known short and the smallest known sufficient; when conditions change and a
-// count that used to suffice falls short, the bracket reopens upwards.
+// The count moves inside the bracket between the largest count known short and the smallest known sufficient; when
+// conditions change and a count that used to suffice falls short, the bracket reopens upwards.
 __device__ __forceinline__ void ns_adapt_lift_plan(DevState* s, int n_endgame, int converged) {
   const int plan = s->lift_plan;
   if (!converged) { s->lift_plan = min(plan + 2, 60); s->lift_lo = plan; s->lift_hi = 127; return; }
@@ -557,13 +556,17 @@ __device__ __forceinline__ void ns_adapt_lift_plan(DevState* s, int n_endgame, i
     s->lift_lo = max(s->lift_lo, plan);
     if (s->lift_hi <= s->lift_lo) s->lift_hi = 127;
   }
+  // falling short costs about three steps per missing lifting step, one lifting step too many costs one: descend in
+  // thirds of the bracket, climb at once
   int next;
   if (s->lift_hi == 127) next = plan + max(1, (extra + 1) / 2);
-  else if (s->lift_hi - s->lift_lo > 1) next = (s->lift_lo + s->lift_hi) / 2;
+  else if (s->lift_hi - s->lift_lo > 1) next = s->lift_hi - max(1, (s->lift_hi - s->lift_lo - 1) / 3);
   else next = s->lift_hi;
   s->lift_plan = min(max(next, 0), 60);
 }
 
+// phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
+// phase 1: scale = ||M_raw + lam R||_F ; arms the iteration
 static __global__ void ns_setup_kernel(DevState* st, const double* __restrict__ partials, int nblocks, int phase,
                                 float prior_rel, float inv_sqrt_d, float margin, int d, int use_shift, float e1_tau,
                                 int n_lift_init) {
@@ -695,6 +698,7 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
   const int p = blockIdx.x;
   DevState* s = st + p;
   if (s->ns_done) return;
+  if (k < 0) k = s->ns_steps_used;           // inside the update graph's loop: the step's index lives on the device
   __shared__ double redd[8];
   __shared__ float redf[8];
   double sq = 0.0, tr = 0.0;
@@ -710,10 +714,16 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
   if (threadIdx.x == 0) ns_control_decide(s, tmx, tsq, ttr, k, cur_buf, c);
 }
 
-// tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode).
-// While the iterate is tiny (tau below e1_tau) the lo part cannot matter to G = X^T X: dropping it changes G by
-// about 4.4e-3 sqrt(tau) sigma_max, so the next residual product runs one bf16 pass instead of three.
-static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ part_x2, int nparts, int d, float e1_tau) {
+// tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode), and how
+// many bf16 passes that product takes.  Dropping the iterate's lo part changes G = X^T X by about
+// 4.4e-3 sqrt(tau) sigma_max (a symmetric perturbation).  One pass is enough
+//   * while the iterate is tiny (tau below e1_tau): the perturbation is small in absolute terms;
+//   * for a late lifting step, once the small singular values have grown so far (same bound as for the iterate's
+//     lo part in the last product: d 2^-8 / growth <= lo_budget) that the directions such noise can still scramble
+//     carry no weight.  Endgame steps and the acceptance check always take three passes: there a perturbation of
+//     G by a few 1e-3 costs a whole extra step.
+static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ part_x2, int nparts, int d, float e1_tau,
+                                     float lo_budget) {
   DevState* s = st + blockIdx.x;
   if (s->ns_done) return;
   __shared__ double redd[8];
@@ -722,7 +732,9 @@ static __global__ void ns_tau_kernel(DevState* st, const double* __restrict__ pa
   const double tot = block_sum_d<256>(v, redd);
   if (threadIdx.x == 0) {
     s->tau = (float)(tot / (double)d);
-    s->seg_e = (s->tau < e1_tau) ? 1 : 3;
+    const bool grown = (float)d * (1.0f / 256.0f) / s->growth <= lo_budget;
+    const bool next_is_lifting = s->lift_left > 0 && s->e_fro >= 0.7f;     // (control drops the rest of the lifting below 0.7)
+    s->seg_e = (s->tau < e1_tau || (grown && next_is_lifting)) ? 1 : 3;
   }
 }
 

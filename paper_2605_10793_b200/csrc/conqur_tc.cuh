@@ -940,6 +940,7 @@ struct TcHost {
   int device;                                // CUDA device the context was created on
   int pair_clusters;                         // CTA pairs that can be co-resident (0: single-CTA kernels only)
   float e1_tau;                              // residual product runs one pass while mean sigma^2 of the iterate is below this
+  float lo_budget;                           // ... and in mid-iteration, see ns_tau_kernel
   int64_t n_max;
   char* ws;
   TcLayout L;
@@ -1175,7 +1176,7 @@ inline int tc_device_facts(int dev, TcDevFacts* out) {
 inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t n_max, int quant_bits, float* R,
                    float* M, float* Xa, float* Xb, float* E, float* B, float* rnorm, DevState* st, double* part_d,
                    float* part_f, float* Y, unsigned* rowmax, QuantSpec qs, int diagnostics, double* part_diag, Prof* prof,
-                   int single_cta, float gram_single_pass_tau) {
+                   int single_cta, float gram_single_pass_tau, float lo_budget) {
   h->d = d; h->P = P; h->n_max = n_max; h->quant_bits = quant_bits; h->ws = ws; h->L = L;
   h->R = R; h->M = M; h->Xa = Xa; h->Xb = Xb; h->E = E; h->B = B; h->rnorm = rnorm; h->st = st;
   h->part_d = part_d; h->part_f = part_f; h->Y = Y; h->rowmax = rowmax; h->qs = qs; h->diagnostics = diagnostics; h->part_diag = part_diag; h->prof = prof; h->ns_k = -1;
@@ -1191,6 +1192,7 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
   h->device = dev;
   h->pair_clusters = single_cta ? 0 : f.pair_clusters;
   h->e1_tau = gram_single_pass_tau > 0.f ? gram_single_pass_tau : 2e-3f;
+  h->lo_budget = lo_budget;
   const uint64_t D = (uint64_t)d;
   int rc = 0;
   if (P > 1) {
@@ -1339,7 +1341,7 @@ inline int tc_ns_poly_next(TcHost& h, cudaStream_t s, int cur) {
   x.part_t = h.part_d + tc_ns_parts(h);
   rc = tc_launch_n<false, true, TC_EPI_NEXT>(h, s, h.tmXh_k[cur], h.tmBh_mn, x);
   if (rc) return rc;
-  ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d, h.e1_tau);
+  ns_tau_kernel<<<1, 256, 0, s>>>(h.st, h.part_d + tc_ns_parts(h), tc_ns_next_parts(h), d, h.e1_tau, h.lo_budget);
   if (h.prof) h.prof->count(K_OTHER);
   return cudaGetLastError() == cudaSuccess ? CONQUR_OK : CONQUR_ERR_CUDA;
 }

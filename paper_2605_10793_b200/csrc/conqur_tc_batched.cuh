@@ -12,7 +12,12 @@
 // second product so that they cannot reach M.
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..9 = epilogue (two warps per TMEM lane quarter,
-// one per half of the 128 columns).  Every wait is bounded.
+// one per half of the 128 columns), 10..13 = row norms (32 rows of the tile each; they run beside the first product
+// and fill issue slots the epilogue warps leave idle).  Every wait is bounded.
+//
+// Objective without fake-quantisation: sum_i ||y_i||_1 rnorm_i = <R, X_tilde^T S> (Section 3.2 with Eq. 2), so it is
+// taken once per problem from the cross-covariance accumulator on its way out instead of summing |y| element by
+// element in the epilogue.
 #pragma once
 #include "conqur_tc.cuh"
 
@@ -21,7 +26,8 @@ namespace conqur {
 constexpr int TCB_D = 128;                       // problem size this kernel is built for
 constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = two 64-column swizzled chunks of 16 KB
 constexpr int TCB_XSTAGES = 3;
-constexpr int TCB_THREADS = 320;                 // 2 + 8 warps
+constexpr int TCB_THREADS = 448;                 // 2 + 8 + 4 warps
+constexpr int TCB_NORM_WARP0 = 10;               // first of the four row-norm warps
 constexpr int TCB_EPI_THREADS = 256;
 constexpr int TCB_EPI_WARPS = TCB_EPI_THREADS / 32;
 constexpr int TCB_AUX_BYTES = 4096;
@@ -31,12 +37,11 @@ struct TcbAux {
   uint64_t rfull, rempty, mfull, mempty;
   uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
   uint64_t yfull[2], yempty[2], cready[2], cfree[2];
+  uint64_t nready[2];        // row norms of the tile in Y buffer b are in rn[b]
   uint32_t tmem_base;
   int abort_flag;
   double red_d[8];
-  int red_i[8];
-  int red_f[8];
-  float ss_x[2][2][128];     // [tile parity][column half][row]: half-row sums of squares exchanged between the two warps of a row
+  float rn[2][128];          // [tile parity][row]: 1 / ||x_row||, 0 for rows that are skipped or past the end
 };
 
 static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
@@ -52,6 +57,7 @@ struct TcbStepArgs {
   float* Mpart;               // S > 1: P * S partial cross-covariances (item order), summed into M by tcb_finish_kernel
   double* part_d;             // P * S objective partials (sum |y| * rnorm, or the quantised equivalent), item order
   DevState* st;               // P
+  const float* R;             // P x 128 x 128 fp32: the rotations (for the objective <R, X~^T S>)
   int8_t* signs;              // test hook: when set, the sign decisions (-1/0/+1) of this call, (P * n) x 128 row-major
 };
 
@@ -87,6 +93,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
       ptx::mbar_init(&aux->cready[b], TCB_EPI_WARPS); ptx::mbar_init(&aux->cfree[b], 1);
+      ptx::mbar_init(&aux->nready[b], 4);
     }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
@@ -182,6 +189,58 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (ok) ptx::umma_commit(&aux->mfull);
       }
     }
+  } else if (warp >= TCB_NORM_WARP0) {
+    // ---------------------------------------------------------------- a1: row norms from the tile in shared memory
+    const int r = (warp - TCB_NORM_WARP0) * 32 + lane;      // this lane's token inside every tile
+    int it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x) {
+      const int p = item / g.S, sp = item - p * g.S;
+      const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
+      int skipped = 0, nonfinite = 0;
+      for (int t = t_begin; t < t_end; ++t, ++it) {
+        const int yb = it & 1, xs = it % TCB_XSTAGES;
+        if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 34; break; }
+        // rn[yb] was last read by the epilogue of the tile two before this one
+        if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 35; break; }
+        uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;       // four chains; added in a fixed order
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, c));
+          const float a0 = __uint_as_float(w.x << 16), b0 = __uint_as_float(w.x & 0xffff0000u);
+          const float a1 = __uint_as_float(w.y << 16), b1 = __uint_as_float(w.y & 0xffff0000u);
+          const float a2 = __uint_as_float(w.z << 16), b2 = __uint_as_float(w.z & 0xffff0000u);
+          const float a3 = __uint_as_float(w.w << 16), b3 = __uint_as_float(w.w & 0xffff0000u);
+          s0 = fmaf(a0, a0, s0); s0 = fmaf(b0, b0, s0);
+          s1 = fmaf(a1, a1, s1); s1 = fmaf(b1, b1, s1);
+          s2 = fmaf(a2, a2, s2); s2 = fmaf(b2, b2, s2);
+          s3 = fmaf(a3, a3, s3); s3 = fmaf(b3, b3, s3);
+        }
+        const float ss = (s0 + s1) + (s2 + s3);
+        const bool valid = (t * 128 + r) < g.n;
+        const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
+        if (valid && !good) {
+          ++skipped;
+          if (!(ss == 0.f)) nonfinite = 1;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, c)) = make_uint4(0, 0, 0, 0);
+        }
+        aux->rn[yb][r] = good ? 1.0f / sqrtf(ss) : 0.f;
+        // a zeroed row must be visible to the second product (tensor-core proxy), rn to the epilogue warps
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&aux->nready[yb]);
+      }
+      if (!ok) break;
+      int wsk = skipped, wnf = nonfinite;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
+      if (lane == 0) {
+        if (wsk) atomicAdd(reinterpret_cast<unsigned long long*>(&g.st[p].step_skipped), (unsigned long long)wsk);
+        if (wnf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
+      }
+    }
   } else {
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;              // which 64 of the 128 columns this warp handles
@@ -193,37 +252,13 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int p = item / g.S, sp = item - p * g.S;
       const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
       double acc = 0.0;
-      int skipped = 0, nonfinite = 0;
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int yb = it & 1, xs = it % TCB_XSTAGES;
+        const int yb = it & 1;
         const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
-        if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 30; break; }
-        // a1: row norm from the tile in shared memory: each of the row's two warps sums its half of the columns and
-        // they swap the halves (named barriers 2..5, one per TMEM lane quarter; both warps have just passed the
-        // same wait, so both arrive).  The two halves are added in a fixed order.
-        uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
-        float ssh = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, half * 8 + c));
-          const uint32_t u[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float a = __uint_as_float(u[e] << 16), b = __uint_as_float(u[e] & 0xffff0000u);
-            ssh = fmaf(a, a, ssh); ssh = fmaf(b, b, ssh);
-          }
-        }
-        aux->ss_x[it & 1][half][r] = ssh;
-        asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
-        const float ss = aux->ss_x[it & 1][0][r] + aux->ss_x[it & 1][1][r];
+        if (!tc_wait(&aux->nready[yb], par2, abort_flag)) { ok = false; timeout_site = 30; break; }
+        const float rn = aux->rn[yb][r];
         const bool valid = (t * 128 + r) < g.n;
-        const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
-        if (valid && !good) {
-          if (half == 0) { ++skipped; if (!(ss == 0.f)) nonfinite = 1; }
-#pragma unroll
-          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, half * 8 + c)) = make_uint4(0, 0, 0, 0);
-        }
-        const float rn = good ? 1.0f / sqrtf(ss) : 0.f;
+        const bool good = rn > 0.f;
         const uint32_t rn_bits = bf16_bits(rn);
         if (!tc_wait(&aux->cfree[yb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
         if (!tc_wait(&aux->yfull[yb], par2, abort_flag)) { ok = false; timeout_site = 32; break; }
@@ -261,16 +296,14 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               w[i] = live ? (lo | (hi << 16)) : 0u;
             }
           } else {
-            // two elements per instruction: sign bits and a non-zero mask from the packed bf16 pair.  mag + 0x7fff sets
-            // bit 15 of a half exactly when the half is non-zero; the byte permute spreads that bit over the half.
+            // two elements per instruction: the sign bits and a non-zero mask (0xffff per half that is not +-0) of the
+            // packed bf16 pair; the objective comes from the accumulator at the end of the problem
             const uint32_t rn2 = live ? (rn_bits | (rn_bits << 16)) : 0u;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const float a = v[2 * i], b = v[2 * i + 1];
-              acc_t += fabsf(a) + fabsf(b);
-              const uint32_t pk = bf16x2_pack(a, b);
-              uint32_t nz;                                    // 0xffff per non-zero half (prmt: selector msb = replicate the byte's sign)
-              asm("prmt.b32 %0, %1, 0, 0xBB99;" : "=r"(nz) : "r"((pk & 0x7fff7fffu) + 0x7fff7fffu));
+              const uint32_t pk = bf16x2_pack(v[2 * i], v[2 * i + 1]);
+              uint32_t nz;
+              asm("set.neu.u32.bf16x2 %0, %1, %2;" : "=r"(nz) : "r"(pk), "r"(0u));
               w[i] = (rn2 | (pk & 0x80008000u)) & nz;
             }
           }
@@ -297,7 +330,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             so[1] = make_uint4(sb[4], sb[5], sb[6], sb[7]);
           }
         }
-        if (live) acc += (g.qs.bits > 0) ? (double)(rn * rq.delta) * (double)acc_t : (double)(acc_t * rn);
+        if (live && g.qs.bits > 0) acc += (double)(rn * rq.delta) * (double)acc_t;
         // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
         ptx::tc_fence_before();
         ptx::fence_proxy_async();
@@ -315,12 +348,24 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const uint32_t t_addr = tmem_base + 256u + ((uint32_t)(q * 32) << 16);
         // one item per problem: straight into M; several: into the item's partial (summed in item order afterwards)
         float* dst = (g.S == 1) ? g.M + ((long long)p * TCB_D + r) * TCB_D : g.Mpart + ((long long)item * TCB_D + r) * TCB_D;
+        const float* rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
+        float jacc = 0.f;
 #pragma unroll 1
         for (int cc = 0; cc < 2; ++cc) {
           const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
           float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
+          if (g.qs.bits == 0) {
+            // this item's share of the objective: <R, X~^T C'> over its rows of the accumulator (fp32 R)
+            const float4* r4 = reinterpret_cast<const float4*>(rrow + c * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 q4 = __ldg(r4 + i);
+              jacc = fmaf(v[4 * i], q4.x, jacc); jacc = fmaf(v[4 * i + 1], q4.y, jacc);
+              jacc = fmaf(v[4 * i + 2], q4.z, jacc); jacc = fmaf(v[4 * i + 3], q4.w, jacc);
+            }
+          }
           if (g.S == 1) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -333,24 +378,19 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
           }
         }
+        if (g.qs.bits == 0) acc = (double)jacc;
       }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&aux->mempty);
       // per-problem reductions in a fixed order (named barrier 1: the eight epilogue warps only)
       const double wsum = warp_sum_d(acc);
-      int wsk = skipped, wnf = nonfinite;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
-      if (lane == 0) { aux->red_d[ew] = wsum; aux->red_i[ew] = wsk; aux->red_f[ew] = wnf; }
+      if (lane == 0) aux->red_d[ew] = wsum;
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (ew == 0 && lane == 0) {
         double tot = 0.0;
-        int sk = 0, nf = 0;
-        for (int i = 0; i < 8; ++i) { tot += aux->red_d[i]; sk += aux->red_i[i]; nf |= aux->red_f[i]; }
+        for (int i = 0; i < 8; ++i) tot += aux->red_d[i];
         g.part_d[item] = tot;
-        if (sk) atomicAdd(reinterpret_cast<unsigned long long*>(&g.st[p].step_skipped), (unsigned long long)sk);
-        if (nf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
     }
@@ -452,6 +492,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   TcbStepArgs g{};
   g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
   g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0; g.signs = signs_out;
+  g.R = h.R + (size_t)p0 * TCB_D * TCB_D;
   // few problems: split each problem's tokens over several CTAs (partials land in the idle Newton-Schulz buffers,
   // 4 P matrices of 128 x 128 starting at Xa, and are summed in a fixed order)
   const int T = (int)((n + 127) / 128);

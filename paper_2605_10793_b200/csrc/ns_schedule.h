@@ -128,7 +128,7 @@ struct NsPlanParams {
   double final_err = 1e-6;
   int max_len = 100;
   int d = 0;                 // for seg_x; 0: always 2
-  double gap_budget = 1e-4;  // bound on the Procrustes gap given up by dropping the iterate's lo part
+  double gap_budget = 5e-4;  // worst-case bound on the Procrustes gap given up by dropping the iterate's lo part
 };
 
 // One endgame/lifting quintic for the interval [l, 1], rescaled; returns the lower end of its range.
