@@ -11,9 +11,13 @@
 // operand of the second product.  Rows with a zero or non-finite norm are zeroed in shared memory before the
 // second product so that they cannot reach M.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..9 = epilogue (two warps per TMEM lane quarter,
-// one per half of the 128 columns), 10..13 = row norms (32 rows of the tile each; they run beside the first product
-// and fill issue slots the epilogue warps leave idle).  Every wait is bounded.
+// Warp roles: 0 = TMA producer, 1 = issuer of the first product and TMEM owner, 2..17 = epilogue: two groups of
+// eight warps (two per TMEM lane quarter, one per half of the 128 columns) that take alternate tiles, so that one
+// group's waits and TMEM / shared-memory latencies overlap the other group's work; 18..21 = row norms (32 rows of
+// the tile each, beside the first product); 22 = issuer of the second product.  The two products have their own
+// issuing threads and Y has three TMEM buffers, so the first product runs up to three tiles ahead of the
+// epilogue.  Shared-memory bandwidth sets the floor of a tile: both products read both operands from it
+// (4 x 32 KB), TMA writes 32 KB, the norms read and the targets write 32 KB each.  Every wait is bounded.
 //
 // Objective without fake-quantisation: sum_i ||y_i||_1 rnorm_i = <R, X_tilde^T S> (Section 3.2 with Eq. 2), so it is
 // taken once per problem from the cross-covariance accumulator on its way out instead of summing |y| element by
@@ -25,26 +29,35 @@ namespace conqur {
 
 constexpr int TCB_D = 128;                       // problem size this kernel is built for
 constexpr int TCB_TILE_BYTES = 128 * 128 * 2;    // one 128 x 128 bf16 tile = two 64-column swizzled chunks of 16 KB
-constexpr int TCB_XSTAGES = 3;
-constexpr int TCB_THREADS = 448;                 // 2 + 8 + 4 warps
-constexpr int TCB_NORM_WARP0 = 10;               // first of the four row-norm warps
+constexpr int TCB_XSTAGES = 4;                   // a stage is held from the copy's issue until the second product has read it
+#ifndef TCB_EPI_GROUPS_N
+#define TCB_EPI_GROUPS_N 2
+#endif
+constexpr int TCB_EPI_GROUPS = TCB_EPI_GROUPS_N; // groups of eight epilogue warps taking tiles in turn
+constexpr int TCB_NORM_WARP0 = 2 + 8 * TCB_EPI_GROUPS;   // first of the four row-norm warps
+constexpr int TCB_MMA2_WARP = TCB_NORM_WARP0 + 4;        // issues the second product
+constexpr int TCB_THREADS = (TCB_MMA2_WARP + 1) * 32;
+constexpr int TCB_YBUF = 3;                      // Y accumulators in TMEM (128 columns each), then the M accumulator(s)
+constexpr int TCB_MBUF = (TCB_YBUF == 2) ? 2 : 1;   // 512 columns in all: 3 + 1 or 2 + 2
 constexpr int TCB_EPI_THREADS = 256;
 constexpr int TCB_EPI_WARPS = TCB_EPI_THREADS / 32;
-constexpr int TCB_AUX_BYTES = 4096;
+constexpr int TCB_AUX_BYTES = 2048;
 constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + TCB_AUX_BYTES + 1024;
 
 struct TcbAux {
-  uint64_t rfull, rempty, mfull, mempty;
+  uint64_t rfull, rempty, mfull[TCB_MBUF], mempty[TCB_MBUF];
+  uint64_t pdone;            // every epilogue warp has finished the problem (write-out and objective partial)
   uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
-  uint64_t yfull[2], yempty[2], cready[2], cfree[2];
-  uint64_t nready[2];        // row norms of the tile in Y buffer b are in rn[b]
+  uint64_t yfull[TCB_YBUF], yempty[TCB_YBUF], cready[2], cfree[2];
+  uint64_t nready[TCB_YBUF]; // row norms of the tile in Y buffer b are in rn[b]
   uint32_t tmem_base;
   int abort_flag;
-  double red_d[8];
-  float rn[2][128];          // [tile parity][row]: 1 / ||x_row||, 0 for rows that are skipped or past the end
+  double red_d[2][16];       // [problem parity][epilogue warp]: objective partials
+  float rn[TCB_YBUF][128];   // [Y buffer][row]: 1 / ||x_row||, 0 for rows that are skipped or past the end
 };
 
 static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
+static_assert(TCB_SMEM_BYTES <= 232448, "227 KB of dynamic shared memory per CTA");
 
 struct TcbStepArgs {
   int n, P;                   // P problems; M, part_d, st point at the first of them
@@ -88,13 +101,14 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
-    ptx::mbar_init(&aux->mfull, 1); ptx::mbar_init(&aux->mempty, TCB_EPI_WARPS);
+    for (int b = 0; b < TCB_MBUF; ++b) { ptx::mbar_init(&aux->mfull[b], 1); ptx::mbar_init(&aux->mempty[b], TCB_EPI_WARPS * TCB_EPI_GROUPS); }
+    ptx::mbar_init(&aux->pdone, TCB_EPI_WARPS * TCB_EPI_GROUPS);
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < TCB_YBUF; ++b) {
       ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
-      ptx::mbar_init(&aux->cready[b], TCB_EPI_WARPS); ptx::mbar_init(&aux->cfree[b], 1);
       ptx::mbar_init(&aux->nready[b], 4);
     }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->cready[b], TCB_EPI_WARPS); ptx::mbar_init(&aux->cfree[b], 1); }
     aux->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -105,7 +119,10 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
-  const uint32_t tmem_base = aux->tmem_base;     // columns [0,128) and [128,256): Y buffers; [256,384): M accumulator
+  // TMEM columns: the Y buffers, then the M accumulator(s) (with two, the next problem's second products can run
+  // while this problem's accumulator is written out)
+  const uint32_t tmem_base = aux->tmem_base;
+  constexpr uint32_t TM_M = 128u * TCB_YBUF;
   int timeout_site = 0;
 
   if (warp == 0) {
@@ -138,41 +155,22 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   } else if (warp == 1) {
+    // ---------------------------------------------------------------- first product: Y = X_tile R
     if (lane == 0) {
-      // instruction descriptors: bf16 x bf16 -> fp32, M = N = 128; first product A K-major / B MN-major, second both MN-major
-      const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-      const uint32_t idesc1 = idesc_base | (1u << 16);
-      const uint32_t idesc2 = idesc_base | (1u << 15) | (1u << 16);
-      const uint32_t sR_a = ptx::smem_u32(sR), sX_a = ptx::smem_u32(sX), sC_a = ptx::smem_u32(sC);
-      int xs = 0; uint32_t xph = 0;          // stage of the tile the first product reads
-      int xs2 = 0;                           // stage of the tile the second product reads (one tile behind)
-      int it = 0, it2 = 0;                   // tiles issued to the first / second product (over all problems)
-      int lp = 0;
+      // instruction descriptor: bf16 x bf16 -> fp32, M = N = 128; A K-major, B MN-major
+      const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24) | (1u << 16);
+      const uint32_t sR_a = ptx::smem_u32(sR), sX_a = ptx::smem_u32(sX);
+      int xs = 0; uint32_t xph = 0;
+      int it = 0, lp = 0;
       bool ok = true;
-      auto second_product = [&](bool first_of_problem) -> bool {
-        const int cb = it2 & 1;
-        if (!tc_wait(&aux->cready[cb], ((uint32_t)it2 >> 1) & 1u, abort_flag)) { timeout_site = 23; return false; }
-        ptx::tc_fence_after();
-        const uint32_t xa = sX_a + xs2 * TCB_TILE_BYTES, ca = sC_a + cb * TCB_TILE_BYTES;
-#pragma unroll
-        for (int j = 0; j < 8; ++j)          // 16 tokens per instruction: two 8-row groups, 2048 bytes per step
-          ptx::umma_bf16(tmem_base + 256, tc_smem_desc(xa + j * 2048, 16384, 1024), tc_smem_desc(ca + j * 2048, 16384, 1024),
-                         idesc2, (!first_of_problem || j > 0) ? 1u : 0u);
-        ptx::umma_commit(&aux->xempty[xs2]);
-        ptx::umma_commit(&aux->cfree[cb]);
-        if (++xs2 == TCB_XSTAGES) xs2 = 0;
-        ++it2;
-        return true;
-      };
       for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
         const int sp = item % g.S;
         const int T_item = (int)((long long)T * (sp + 1) / g.S) - (int)((long long)T * sp / g.S);
         if (!tc_wait(&aux->rfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 20; break; }
-        if (!tc_wait(&aux->mempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 21; break; }
-        for (int t = 0; t < T_item && ok; ++t) {
-          const int yb = it & 1;
+        for (int t = 0; t < T_item && ok; ++t, ++it) {
+          const int yb = it % TCB_YBUF;
           if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 22; break; }
-          if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
+          if (!tc_wait(&aux->yempty[yb], (((uint32_t)(it / TCB_YBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
           ptx::tc_fence_after();
           const uint32_t xa = sX_a + xs * TCB_TILE_BYTES;
 #pragma unroll
@@ -182,11 +180,40 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ptx::umma_commit(&aux->yfull[yb]);
           if (t == T_item - 1) ptx::umma_commit(&aux->rempty);     // R may be replaced once every first product has run
           if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
-          ++it;
-          if (t > 0) ok = second_product(t == 1);
         }
-        if (ok) ok = second_product(T_item == 1);
-        if (ok) ptx::umma_commit(&aux->mfull);
+      }
+    }
+  } else if (warp == TCB_MMA2_WARP) {
+    // ---------------------------------------------------------------- second product: M += X_tile^T C'
+    if (lane == 0) {
+      // both operands MN-major (contraction over the tokens, the slow dimension of both tiles)
+      const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24) |
+                              (1u << 15) | (1u << 16);
+      const uint32_t sX_a = ptx::smem_u32(sX), sC_a = ptx::smem_u32(sC);
+      int xs = 0; uint32_t xph = 0;
+      int it = 0, lp = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
+        const int sp = item % g.S;
+        const int T_item = (int)((long long)T * (sp + 1) / g.S) - (int)((long long)T * sp / g.S);
+        // the accumulator of the previous problem has been read out
+        const int mb = lp % TCB_MBUF;
+        if (!tc_wait(&aux->mempty[mb], (((uint32_t)(lp / TCB_MBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 21; break; }
+        for (int t = 0; t < T_item && ok; ++t, ++it) {
+          const int cb = it & 1;
+          if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 25; break; }
+          if (!tc_wait(&aux->cready[cb], ((uint32_t)it >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 23; break; }
+          ptx::tc_fence_after();
+          const uint32_t xa = sX_a + xs * TCB_TILE_BYTES, ca = sC_a + cb * TCB_TILE_BYTES;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)          // 16 tokens per instruction: two 8-row groups, 2048 bytes per step
+            ptx::umma_bf16(tmem_base + TM_M + mb * 128, tc_smem_desc(xa + j * 2048, 16384, 1024), tc_smem_desc(ca + j * 2048, 16384, 1024),
+                           idesc2, (t > 0 || j > 0) ? 1u : 0u);
+          ptx::umma_commit(&aux->xempty[xs]);
+          ptx::umma_commit(&aux->cfree[cb]);
+          if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
+        }
+        if (ok) ptx::umma_commit(&aux->mfull[mb]);
       }
     }
   } else if (warp >= TCB_NORM_WARP0) {
@@ -199,10 +226,10 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
       int skipped = 0, nonfinite = 0;
       for (int t = t_begin; t < t_end; ++t, ++it) {
-        const int yb = it & 1, xs = it % TCB_XSTAGES;
+        const int yb = it % TCB_YBUF, xs = it % TCB_XSTAGES;
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 34; break; }
-        // rn[yb] was last read by the epilogue of the tile two before this one
-        if (!tc_wait(&aux->yempty[yb], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 35; break; }
+        // rn[yb] was last read by the epilogue of the tile that used this Y buffer before
+        if (!tc_wait(&aux->yempty[yb], (((uint32_t)(it / TCB_YBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 35; break; }
         uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;       // four chains; added in a fixed order
 #pragma unroll
@@ -243,8 +270,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     }
   } else {
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;              // which 64 of the 128 columns this warp handles
-    const int ew = (warp - 2);                     // 0..7
+    const int grp = (warp - 2) >> 3;               // with two groups: group 0 takes the even tiles (and C' buffer 0), group 1 the odd ones
+    const int ew = (warp - 2) & 7;                 // 0..7 inside the group
+    const int half = ew >> 2;                      // which 64 of the 128 columns this warp handles
     const int r = q * 32 + lane;                   // token inside the tile; later: row of M
     int it = 0, lp = 0;
     bool ok = true;
@@ -253,18 +281,19 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
       double acc = 0.0;
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int yb = it & 1;
-        const uint32_t par2 = ((uint32_t)it >> 1) & 1u;
-        if (!tc_wait(&aux->nready[yb], par2, abort_flag)) { ok = false; timeout_site = 30; break; }
+        if (TCB_EPI_GROUPS == 2 && (it & 1) != grp) continue;
+        const int yb = it % TCB_YBUF, cb = it & 1;
+        const uint32_t par3 = ((uint32_t)(it / TCB_YBUF)) & 1u, par2 = ((uint32_t)it >> 1) & 1u;
+        if (!tc_wait(&aux->nready[yb], par3, abort_flag)) { ok = false; timeout_site = 30; break; }
         const float rn = aux->rn[yb][r];
         const bool valid = (t * 128 + r) < g.n;
         const bool good = rn > 0.f;
         const uint32_t rn_bits = bf16_bits(rn);
-        if (!tc_wait(&aux->cfree[yb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
-        if (!tc_wait(&aux->yfull[yb], par2, abort_flag)) { ok = false; timeout_site = 32; break; }
+        if (!tc_wait(&aux->cfree[cb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
+        if (!tc_wait(&aux->yfull[yb], par3, abort_flag)) { ok = false; timeout_site = 32; break; }
         ptx::tc_fence_after();
         const uint32_t t_addr = tmem_base + (uint32_t)(yb * 128) + ((uint32_t)(q * 32) << 16);
-        uint8_t* crow = sC + yb * TCB_TILE_BYTES;
+        uint8_t* crow = sC + cb * TCB_TILE_BYTES;
         RowQuant rq{0.f, 0.f, 0.f, 0.f};
         if (g.qs.bits > 0) {
           float vmax = -3.0e38f, vmin = 3.0e38f;   // the per-token scale needs the whole row
@@ -336,28 +365,34 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ptx::fence_proxy_async();
         __syncwarp();                              // one arrival per warp: every lane's fences precede it
         if (lane == 0) {
-          ptx::mbar_arrive(&aux->cready[yb]);
+          ptx::mbar_arrive(&aux->cready[cb]);
           ptx::mbar_arrive(&aux->yempty[yb]);
         }
       }
       if (!ok) break;
-      // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T)
-      if (!tc_wait(&aux->mfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 33; break; }
+      // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T).  Every
+      // epilogue warp takes part (with two groups each warp one 32 x 32 block, else two).
+      const int mb = lp % TCB_MBUF;
+      if (!tc_wait(&aux->mfull[mb], ((uint32_t)(lp / TCB_MBUF)) & 1u, abort_flag)) { ok = false; timeout_site = 33; break; }
       ptx::tc_fence_after();
       {
-        const uint32_t t_addr = tmem_base + 256u + ((uint32_t)(q * 32) << 16);
-        // one item per problem: straight into M; several: into the item's partial (summed in item order afterwards)
-        float* dst = (g.S == 1) ? g.M + ((long long)p * TCB_D + r) * TCB_D : g.Mpart + ((long long)item * TCB_D + r) * TCB_D;
+        const uint32_t t_addr = tmem_base + TM_M + (uint32_t)(mb * 128) + ((uint32_t)(q * 32) << 16);
+        // Every second product issued so far has finished and no new target tile exists before these warps return to
+        // the tiles, so the C' buffers are idle: each warp borrows 4 KB to turn its 32 x 32 block (a thread holds one
+        // row) into full 128-byte row segments.  One item per problem: added into M with fire-and-forget vector
+        // reductions (one addition per element and launch, so the result does not depend on any order); several:
+        // stored to the item's partial, summed in item order afterwards.
+        uint8_t* stg = sC + grp * TCB_TILE_BYTES + ew * 4096;
+        float* dst = (g.S == 1) ? g.M + ((long long)p * TCB_D + q * 32) * TCB_D : g.Mpart + ((long long)item * TCB_D + q * 32) * TCB_D;
         const float* rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
         float jacc = 0.f;
 #pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
+        for (int cc = grp; cc < 2; cc += TCB_EPI_GROUPS) {
           const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
-          float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
           if (g.qs.bits == 0) {
-            // this item's share of the objective: <R, X~^T C'> over its rows of the accumulator (fp32 R)
+            // this block's share of the objective: <R, X~^T C'> over its part of the accumulator (fp32 R)
             const float4* r4 = reinterpret_cast<const float4*>(rrow + c * 32);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -366,33 +401,25 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               jacc = fmaf(v[4 * i + 2], q4.z, jacc); jacc = fmaf(v[4 * i + 3], q4.w, jacc);
             }
           }
-          if (g.S == 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float4 o = d4[i];
-              o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
-              d4[i] = o;
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          }
+          if (g.S == 1) tc_red_block_f32(stg, lane, v, dst + c * 32, TCB_D, 32);
+          else tc_store_block_f32(stg, lane, v, dst + c * 32, TCB_D, 32);
         }
         if (g.qs.bits == 0) acc = (double)jacc;
       }
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&aux->mempty);
-      // per-problem reductions in a fixed order (named barrier 1: the eight epilogue warps only)
+      if (lane == 0) ptx::mbar_arrive(&aux->mempty[mb]);
+      // Per-problem reduction in a fixed order.  The barrier (bounded like every other wait) also keeps every warp
+      // off the C' buffers until all of them have finished staging.  The partials are double-buffered by problem
+      // parity: no warp can get two problems ahead of the thread that sums them.
       const double wsum = warp_sum_d(acc);
-      if (lane == 0) aux->red_d[ew] = wsum;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (ew == 0 && lane == 0) {
+      if (lane == 0) { aux->red_d[lp & 1][grp * 8 + ew] = wsum; ptx::mbar_arrive(&aux->pdone); }
+      if (!tc_wait(&aux->pdone, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 36; break; }
+      if (grp == 0 && ew == 0 && lane == 0) {
         double tot = 0.0;
-        for (int i = 0; i < 8; ++i) tot += aux->red_d[i];
+        for (int i = 0; i < 8 * TCB_EPI_GROUPS; ++i) tot += aux->red_d[lp & 1][i];
         g.part_d[item] = tot;
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
     }
   }
 
