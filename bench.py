@@ -8,7 +8,8 @@ its orthogonality check).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
   python bench.py --workload c1|c3|c4a|c4a_zp|c4b|a1_8b|fold|hadamard      other workloads, same line layout
-  python bench.py --profile-case path|heads|hadamard [--d ..] [--n ..]     a small bounded run for profiler captures
+  python bench.py --profile-case path|heads|heads-timeline|hadamard [--d ..] [--n ..]    small bounded runs for profiler
+                                                                            captures / the per-head kernel's timeline
 
 N > 1 (torchrun): N independent replicas, one per GPU, no data-path collective ("weak" scaling).
 --impl reference: times the float64 CPU oracle, as it stands, on the host cores.
@@ -387,6 +388,8 @@ def profile_case(args):
       path      --batches B batches of --n tokens at width --d through conqur_step (queued, one run of the two
                 products) and one conqur_update
       heads     the per-head kernels: --problems problems of d = 128, --n tokens each, two (step, update) rounds
+      heads-timeline  the per-head step kernel's own timestamps (conqur_debug_trace_heads): thread block 0, tiles of
+                its second problem, SM cycles relative to the first event shown
       hadamard  conqur_hadamard_rows on --n x --d bf16, three launches"""
     import torch
     from paper_2605_10793_b200 import binding as B
@@ -398,6 +401,29 @@ def profile_case(args):
         rc = B.conqur_hadamard_status()
         print(f"profile-case hadamard n={args.n} d={args.d} bf16: status={rc} |y|max={y.float().abs().max().item():.3f}")
         return 0 if rc == 0 else 1
+    if args.profile_case == "heads-timeline":
+        P, n, d = args.problems, args.n, 128
+        x = (torch.randn(P * n, d, device="cuda") * (1.0 + 20.0 * (torch.arange(d, device="cuda") < 2))).to(torch.bfloat16)
+        ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", batch=P)
+        for _ in range(3):
+            ctx.step_batched(x, n, d, n * d)
+        trace = torch.zeros(96 * 16, dtype=torch.int64, device="cuda")
+        ctx.debug_trace_heads(trace)
+        ctx.step_batched(x, n, d, n * d)
+        ctx.debug_trace_heads(None)
+        t = trace.cpu().numpy().reshape(96, 16)
+        tiles = (n + 127) // 128
+        names = ["copy", "mma1", "mma2", "norm>", "norm<", "epi>", "norms", "cfree", "y", "ld0", "st0", "ld1", "epi<", "out?", "out>", "out<"]
+        order = [0, 1, 2, 3, 4, 5, 6, 7, 8, 13, 14, 15, 9, 10, 11, 12]
+        first = tiles if 2 * tiles <= 96 else 0                       # the second problem of the block: steady state
+        t0 = t[first, 0]
+        print(f"profile-case heads-timeline P={P} n={n}: block 0, tiles {first}..{min(96, first + tiles) - 1} "
+              f"(problem boundary after tile {first + tiles - 1}), SM cycles since the first copy shown")
+        print(" tile " + " ".join(f"{nm:>7s}" for nm in names))
+        for i in range(first, min(96, first + tiles + 3)):
+            print(f"{i:5d} " + " ".join(f"{(t[i, e] - t0) if t[i, e] else 0:7d}" for e in order))
+        st = ctx.get_stats()
+        return 0 if st.status == 0 else 1
     if args.profile_case == "heads":
         P, n, d = args.problems, args.n, 128
         x = (torch.randn(P * n, d, device="cuda") * (1.0 + 20.0 * (torch.arange(d, device="cuda") < 2))).to(torch.bfloat16)
@@ -437,7 +463,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--distinct-cycles", type=int, default=0, help="cycles of distinct batches kept resident (0=all)")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-head and Walsh-Hadamard entries of the line")
-    ap.add_argument("--profile-case", default=None, choices=["path", "heads", "hadamard"],
+    ap.add_argument("--profile-case", default=None, choices=["path", "heads", "heads-timeline", "hadamard"],
                     help="run a small bounded case (for profiler captures) instead of the benchmark")
     ap.add_argument("--d", type=int, default=4096)
     ap.add_argument("--n", type=int, default=2048)

@@ -247,6 +247,15 @@ int conqur_debug_get_signs(conqur_ctx* ctx, int8_t* S_out_dev, int64_t capacity_
  * aligned, owned by the caller, valid until replaced; NULL switches the capture off.  Synchronises. */
 int conqur_debug_capture_signs(conqur_ctx* ctx, int8_t* S_dev, int64_t capacity_rows);
 
+/* Measurement hook for the fused per-head step kernel (tensor-core contexts with batch > 1; no counterpart in the
+ * paper): while a buffer is set, thread block 0 of every conqur_step_batched(_range) records SM-clock timestamps of
+ * its first 96 token tiles, 16 int64 slots per tile: 0 copy of the tile issued, 1 / 2 first / second product issued,
+ * 3 / 4 row norms begin / end, 5 epilogue reaches the tile, 6 norms available, 7 target buffer free, 8 rotated tile
+ * available, 13 / 14 / 15 first TMEM load back / first half written / second TMEM load back, 9 epilogue done;
+ * on a problem's last tile 10 / 11 / 12 accumulator awaited / being written out / written out.  trace_dev: device,
+ * capacity >= 96 * 16 int64, owned by the caller; NULL stops the recording.  Synchronises. */
+int conqur_debug_trace_heads(conqur_ctx* ctx, int64_t* trace_dev, int64_t capacity);
+
 /* Test hook (no counterpart in the paper): with CONQUR_DEBUG_CANARIES set, counts the guard bands behind the
  * workspace regions whose pattern has been overwritten (0 = all intact; a kernel of this library wrote past a region
  * otherwise).  Returns that count, or a negative status (CONQUR_ERR_INVALID_ARG when the context was created without

@@ -32,7 +32,7 @@ _live_contexts = None
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
     "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
-    "conqur_set_M", "conqur_debug_get_signs", "conqur_debug_capture_signs", "conqur_get_stats", "conqur_debug_check_canaries", "conqur_plan_schedule", "conqur_debug_gemm",
+    "conqur_set_M", "conqur_debug_get_signs", "conqur_debug_capture_signs", "conqur_get_stats", "conqur_debug_check_canaries", "conqur_debug_trace_heads", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
     "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows", "conqur_hadamard_status",
     "conqur_strerror",
@@ -120,6 +120,8 @@ def load() -> C.CDLL:
     lib.conqur_debug_get_signs.argtypes = [vp, vp, i64]
     lib.conqur_debug_capture_signs.restype = C.c_int
     lib.conqur_debug_capture_signs.argtypes = [vp, vp, i64]
+    lib.conqur_debug_trace_heads.restype = C.c_int
+    lib.conqur_debug_trace_heads.argtypes = [vp, vp, i64]
     lib.conqur_debug_check_canaries.restype = C.c_int
     lib.conqur_debug_check_canaries.argtypes = [vp]
     lib.conqur_get_stats.restype = C.c_int
@@ -470,6 +472,13 @@ class Context:
             out[name] = {"launches": int(pr.launches[i]), "timed": int(pr.timed_launches[i]),
                          "flops": float(pr.flops[i]), "ms": float(pr.ms[i])}
         return out
+
+    def debug_trace_heads(self, buf):
+        """Per-head tensor-core contexts: record the step kernel's timeline into `buf` (int64 CUDA tensor of at least
+        96 * 16 entries; None stops it).  See include/conqur.h for the slots."""
+        self._trace_buf = buf
+        ptr, cap = (0, 0) if buf is None else (buf.data_ptr(), buf.numel())
+        self._chk(load().conqur_debug_trace_heads(self.h, ptr, cap), "conqur_debug_trace_heads")
 
     def check_canaries(self) -> int:
         """Guard bands of the workspace that were overwritten (0 = intact); needs CONQUR_DEBUG_CANARIES."""

@@ -145,6 +145,7 @@ struct conqur_ctx {
   int pending_batches = 0;
   int8_t* sign_capture = nullptr;   // conqur_debug_capture_signs: where the fused per-head kernel writes its decisions
   int64_t sign_capture_rows = 0;
+  long long* heads_trace = nullptr;  // conqur_debug_trace_heads: timeline buffer of the fused per-head step kernel
   int n_sched, n_lift_init;   // device schedule: entry 0 = lifting quintic, 1 .. n_sched-1 = endgame; planned lifting steps
   std::vector<NsStep> sched;
   TcHost tc;                 // tensor maps etc. of the tensor-core mode
@@ -685,7 +686,7 @@ static int step_common(conqur_ctx* c, const void* X, int64_t n, int64_t ld, int6
   } else {
     if (g.P > 1 && c->sign_capture && (int64_t)np * n > c->sign_capture_rows) return CONQUR_ERR_INVALID_ARG;
     if (g.P > 1) {
-      rc = tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride, p0, np, c->sign_capture);
+      rc = tcb_step(c->tc, c->stream, X, g.in_dtype, n, ld, pstride, p0, np, c->sign_capture, c->heads_trace);
     } else {
       // stage the rows behind those already queued; run the products when the queue is full (at once if not deferring)
       if (c->pending_rows + n > c->L.n_rows) { rc = flush_pending(c); if (rc) return rc; }
@@ -826,6 +827,15 @@ extern "C" int conqur_debug_capture_signs(conqur_ctx* c, int8_t* S_dev, int64_t 
   CQ_CUDA(cudaStreamSynchronize(c->stream));           // no step in flight still writes to the previous buffer
   c->sign_capture = S_dev;
   c->sign_capture_rows = S_dev ? capacity_rows : 0;
+  return CONQUR_OK;
+}
+
+extern "C" int conqur_debug_trace_heads(conqur_ctx* c, int64_t* trace_dev, int64_t capacity) {
+  if (!c || capacity < 0) return CONQUR_ERR_INVALID_ARG;
+  if (c->cfg.mode != CONQUR_TC_BF16 || c->cfg.P == 1) return CONQUR_ERR_UNSUPPORTED;
+  if (trace_dev && capacity < (int64_t)TCB_TRACE_TILES * 16) return CONQUR_ERR_INVALID_ARG;
+  CQ_CUDA(cudaStreamSynchronize(c->stream));
+  c->heads_trace = reinterpret_cast<long long*>(trace_dev);
   return CONQUR_OK;
 }
 

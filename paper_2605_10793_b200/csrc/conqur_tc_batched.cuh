@@ -42,6 +42,11 @@ constexpr int TCB_MBUF = (TCB_YBUF == 2) ? 2 : 1;   // 512 columns in all: 3 + 1
 constexpr int TCB_EPI_THREADS = 256;
 constexpr int TCB_EPI_WARPS = TCB_EPI_THREADS / 32;
 constexpr int TCB_AUX_BYTES = 2048;
+// Timeline hook (conqur_debug_trace_heads): per tile 16 slots of clock64() values, see TCB_EV_* for the events.
+constexpr int TCB_TRACE_TILES = 96;
+enum { TCB_EV_TMA = 0, TCB_EV_MMA1 = 1, TCB_EV_MMA2 = 2, TCB_EV_NORM_BEGIN = 3, TCB_EV_NORM_END = 4, TCB_EV_EPI_BEGIN = 5,
+       TCB_EV_EPI_NORMS = 6, TCB_EV_EPI_CFREE = 7, TCB_EV_EPI_Y = 8, TCB_EV_EPI_END = 9, TCB_EV_OUT_WAIT = 10, TCB_EV_OUT_BEGIN = 11,
+       TCB_EV_OUT_END = 12, TCB_EV_EPI_LD0 = 13, TCB_EV_EPI_ST0 = 14, TCB_EV_EPI_LD1 = 15 };
 constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + TCB_AUX_BYTES + 1024;
 
 struct TcbAux {
@@ -71,6 +76,7 @@ struct TcbStepArgs {
   double* part_d;             // P * S objective partials (sum |y| * rnorm, or the quantised equivalent), item order
   DevState* st;               // P
   const float* R;             // P x 128 x 128 fp32: the rotations (for the objective <R, X~^T S>)
+  long long* trace;           // measurement hook: when set, CTA 0 records SM-clock timestamps of its first TCB_TRACE_TILES tiles
   int8_t* signs;              // test hook: when set, the sign decisions (-1/0/+1) of this call, (P * n) x 128 row-major
 };
 
@@ -124,11 +130,14 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const uint32_t tmem_base = aux->tmem_base;
   constexpr uint32_t TM_M = 128u * TCB_YBUF;
   int timeout_site = 0;
+  // one thread per role of CTA 0 stamps its events of the first tiles (nothing is recorded unless a buffer was given)
+  const bool tracing = g.trace != nullptr && blockIdx.x == 0 && lane == 0;
+#define TCB_TR(tile, ev) do { if (tracing && (tile) < TCB_TRACE_TILES) g.trace[(tile) * 16 + (ev)] = clock64(); } while (0)
 
   if (warp == 0) {
     if (lane == 0) {
       int xs = 0; uint32_t xph = 0;
-      int lp = 0;
+      int lp = 0, itp = 0;
       bool ok = true;
       int issued = 0;
       for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
@@ -145,6 +154,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           const int c1 = g.xp_outer_tokens ? p : t * 128, c2 = g.xp_outer_tokens ? t * 128 : p;
           tma_load_3d(dst, &tmX, &aux->xfull[xs], 0, c1, c2);
           tma_load_3d(dst + 16384, &tmX, &aux->xfull[xs], 64, c1, c2);
+          TCB_TR(itp, TCB_EV_TMA); ++itp;
           ++issued;
           if (++xs == TCB_XSTAGES) { xs = 0; xph ^= 1u; }
         }
@@ -172,6 +182,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 22; break; }
           if (!tc_wait(&aux->yempty[yb], (((uint32_t)(it / TCB_YBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 24; break; }
           ptx::tc_fence_after();
+          TCB_TR(it, TCB_EV_MMA1);
           const uint32_t xa = sX_a + xs * TCB_TILE_BYTES;
 #pragma unroll
           for (int j = 0; j < 8; ++j)        // 16 features per instruction: chunk j/4, 32 bytes per step inside the swizzled row
@@ -204,6 +215,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (!tc_wait(&aux->xfull[xs], xph, abort_flag)) { ok = false; timeout_site = 25; break; }
           if (!tc_wait(&aux->cready[cb], ((uint32_t)it >> 1) & 1u, abort_flag)) { ok = false; timeout_site = 23; break; }
           ptx::tc_fence_after();
+          TCB_TR(it, TCB_EV_MMA2);
           const uint32_t xa = sX_a + xs * TCB_TILE_BYTES, ca = sC_a + cb * TCB_TILE_BYTES;
 #pragma unroll
           for (int j = 0; j < 8; ++j)          // 16 tokens per instruction: two 8-row groups, 2048 bytes per step
@@ -230,6 +242,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 34; break; }
         // rn[yb] was last read by the epilogue of the tile that used this Y buffer before
         if (!tc_wait(&aux->yempty[yb], (((uint32_t)(it / TCB_YBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 35; break; }
+        if (warp == TCB_NORM_WARP0) TCB_TR(it, TCB_EV_NORM_BEGIN);
         uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;       // four chains; added in a fixed order
 #pragma unroll
@@ -257,6 +270,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         // a zeroed row must be visible to the second product (tensor-core proxy), rn to the epilogue warps
         ptx::fence_proxy_async();
         __syncwarp();
+        if (warp == TCB_NORM_WARP0) TCB_TR(it, TCB_EV_NORM_END);
         if (lane == 0) ptx::mbar_arrive(&aux->nready[yb]);
       }
       if (!ok) break;
@@ -284,14 +298,19 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (TCB_EPI_GROUPS == 2 && (it & 1) != grp) continue;
         const int yb = it % TCB_YBUF, cb = it & 1;
         const uint32_t par3 = ((uint32_t)(it / TCB_YBUF)) & 1u, par2 = ((uint32_t)it >> 1) & 1u;
+        const bool tr_epi = ew == 0;                       // the first warp of the tile's group stamps the epilogue
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_BEGIN);
         if (!tc_wait(&aux->nready[yb], par3, abort_flag)) { ok = false; timeout_site = 30; break; }
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_NORMS);
         const float rn = aux->rn[yb][r];
         const bool valid = (t * 128 + r) < g.n;
         const bool good = rn > 0.f;
         const uint32_t rn_bits = bf16_bits(rn);
         if (!tc_wait(&aux->cfree[cb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_CFREE);
         if (!tc_wait(&aux->yfull[yb], par3, abort_flag)) { ok = false; timeout_site = 32; break; }
         ptx::tc_fence_after();
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_Y);
         const uint32_t t_addr = tmem_base + (uint32_t)(yb * 128) + ((uint32_t)(q * 32) << 16);
         uint8_t* crow = sC + cb * TCB_TILE_BYTES;
         RowQuant rq{0.f, 0.f, 0.f, 0.f};
@@ -313,6 +332,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           const int c = half * 2 + cc;
           float v[32];
           ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+          if (tr_epi) TCB_TR(it, cc == 0 ? TCB_EV_EPI_LD0 : TCB_EV_EPI_LD1);
           uint32_t w[16];
           if (g.qs.bits > 0) {
 #pragma unroll
@@ -358,12 +378,14 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             so[0] = make_uint4(sb[0], sb[1], sb[2], sb[3]);
             so[1] = make_uint4(sb[4], sb[5], sb[6], sb[7]);
           }
+          if (tr_epi && cc == 0) TCB_TR(it, TCB_EV_EPI_ST0);
         }
         if (live && g.qs.bits > 0) acc += (double)(rn * rq.delta) * (double)acc_t;
         // hand the tile to the second product: shared-memory writes must be visible to the tensor-core proxy
         ptx::tc_fence_before();
         ptx::fence_proxy_async();
         __syncwarp();                              // one arrival per warp: every lane's fences precede it
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_END);
         if (lane == 0) {
           ptx::mbar_arrive(&aux->cready[cb]);
           ptx::mbar_arrive(&aux->yempty[yb]);
@@ -373,8 +395,10 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T).  Every
       // epilogue warp takes part (with two groups each warp one 32 x 32 block, else two).
       const int mb = lp % TCB_MBUF;
+      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_WAIT);
       if (!tc_wait(&aux->mfull[mb], ((uint32_t)(lp / TCB_MBUF)) & 1u, abort_flag)) { ok = false; timeout_site = 33; break; }
       ptx::tc_fence_after();
+      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_BEGIN);
       {
         const uint32_t t_addr = tmem_base + TM_M + (uint32_t)(mb * 128) + ((uint32_t)(q * 32) << 16);
         // Every second product issued so far has finished and no new target tile exists before these warps return to
@@ -408,6 +432,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
       ptx::tc_fence_before();
       __syncwarp();
+      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_END);
       if (lane == 0) ptx::mbar_arrive(&aux->mempty[mb]);
       // Per-problem reduction in a fixed order.  The barrier (bounded like every other wait) also keeps every warp
       // off the C' buffers until all of them have finished staging.  The partials are double-buffered by problem
@@ -492,7 +517,7 @@ inline int tcb_make_x_tmap(CUtensorMap* tm, const void* ptr, uint64_t n, uint64_
 // One streamed batch for all P problems.  X: device, bf16 or fp32 (fp32 is first rounded into the staging copy).
 // Problems [p0, p0 + np) of the context; X holds those np problems.
 inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int64_t n, int64_t ld, int64_t pstride, int p0,
-                    int np, int8_t* signs_out = nullptr) {
+                    int np, int8_t* signs_out = nullptr, long long* trace = nullptr) {
   static std::atomic<unsigned long long> attr_dev_mask{0};      // the attribute is per device
   const unsigned long long dev_bit = 1ull << (h.device & 63);
   if (!(attr_dev_mask.load(std::memory_order_acquire) & dev_bit)) {
@@ -519,7 +544,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   TcbStepArgs g{};
   g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
   g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0; g.signs = signs_out;
-  g.R = h.R + (size_t)p0 * TCB_D * TCB_D;
+  g.R = h.R + (size_t)p0 * TCB_D * TCB_D; g.trace = trace;
   // few problems: split each problem's tokens over several CTAs (partials land in the idle Newton-Schulz buffers,
   // 4 P matrices of 128 x 128 starting at Xa, and are summed in a fixed order)
   const int T = (int)((n + 127) / 128);
