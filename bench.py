@@ -397,7 +397,7 @@ def profile_case(args):
         x = torch.randn(args.n, args.d, device="cuda").to(torch.bfloat16)
         y = torch.empty_like(x)
         for _ in range(3):
-            B.conqur_hadamard_rows(x, out=y)
+            B.conqur_hadamard_rows(x, out=y, cuda_cores_only=args.cuda_cores_only)
         rc = B.conqur_hadamard_status()
         print(f"profile-case hadamard n={args.n} d={args.d} bf16: status={rc} |y|max={y.float().abs().max().item():.3f}")
         return 0 if rc == 0 else 1
@@ -470,6 +470,7 @@ def main():
     ap.add_argument("--problems", type=int, default=592)
     ap.add_argument("--batches", type=int, default=1, help="--profile-case path: batches queued before the products run")
     ap.add_argument("--no-graph", action="store_true", help="enqueue the update's launches directly (profiler launch lists)")
+    ap.add_argument("--cuda-cores-only", action="store_true", help="--profile-case hadamard: the CUDA-core kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
