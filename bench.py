@@ -275,6 +275,7 @@ def run_batched(args, g, w):
     peaks = _peaks()
     step_bytes = 2.0 * P * n * d
     ach = step_bytes / (step_ms * 1e-3) / 1e9
+    heads_traffic, heads_src = ncu_traffic("c4b.tcb_step")
     if not g.is_main:
         D.finish(g)
         return 0
@@ -290,9 +291,10 @@ def run_batched(args, g, w):
                 "d2h_bytes_per_step": 16 * P, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                     "traffic": 395.3e6 * (P * n) / (592 * 2048), "kernel": "tcb_step_kernel", "avg_launch_ms": step_ms,
-                     "traffic_note": "dram read+write of an ncu capture at 592 problems x 2048 tokens (395.3 MB for 310 MB of X; "
-                                     "profiles/tcb_kernels_d128_p592_n2048_ncu_full.md), scaled by the tokens processed",
+                     "traffic": (heads_traffic * (P * n) / (592 * 2048)) if heads_traffic else None, "kernel": "tcb_step_kernel",
+                     "avg_launch_ms": step_ms,
+                     "traffic_note": (f"dram read+write of an ncu capture at 592 problems x 2048 tokens ({heads_src}), scaled by the "
+                                      "tokens processed: the kernel streams its input once") if heads_src else "no capture",
                      "bytes_per_launch": step_bytes, "peak_source": peaks["source"],
                      "tensor_tflops": 4.0 * P * n * d * d / (step_ms * 1e-3) / 1e12},
         "cpu_baseline": None,

@@ -119,6 +119,8 @@ typedef struct {
   int64_t  n_skipped;       /* rows skipped (zero or non-finite norm) since init */
   double   last_J;          /* objective sum and token count consumed by the last update */
   int64_t  last_N;
+  int32_t  ns_lift_plan;    /* lifting steps the next update will start with (learnt from the updates so far; max over problems) */
+  int32_t  reserved;
 } conqur_stats;
 
 /* Bytes of device workspace conqur_init needs for (d, cfg).  Pure function; 0 on invalid arguments. */

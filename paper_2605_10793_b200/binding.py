@@ -54,7 +54,7 @@ class conqur_stats(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("status", C.c_int32), ("ns_steps_used", C.c_int32), ("updates", C.c_int32),
         ("orth_err", C.c_float), ("orth_fro", C.c_float), ("scale", C.c_float), ("n_skipped", C.c_int64),
-        ("last_J", C.c_double), ("last_N", C.c_int64),
+        ("last_J", C.c_double), ("last_N", C.c_int64), ("ns_lift_plan", C.c_int32), ("reserved", C.c_int32),
     ]
 
 

@@ -872,7 +872,7 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
   CQ_CUDA(cudaStreamSynchronize(c->stream));
   out->status = rc;
   out->ns_steps_used = 0; out->orth_err = 0.f; out->orth_fro = 0.f; out->n_skipped = 0;
-  out->last_J = 0.0; out->last_N = 0;
+  out->last_J = 0.0; out->last_N = 0; out->ns_lift_plan = 0; out->reserved = 0;
   out->updates = h[0].updates; out->scale = h[0].scale;
   for (int p = 0; p < P; ++p) {
     out->ns_steps_used = std::max(out->ns_steps_used, h[p].ns_steps_used);
@@ -882,6 +882,7 @@ extern "C" int conqur_get_stats(conqur_ctx* c, conqur_stats* out) {
     out->last_J += h[p].last_J;
     out->last_N += h[p].last_N;
     out->updates = std::min(out->updates, h[p].updates);
+    out->ns_lift_plan = std::max(out->ns_lift_plan, h[p].lift_init ? h[p].lift_plan : c->n_lift_init);
   }
   return CONQUR_OK;
 }

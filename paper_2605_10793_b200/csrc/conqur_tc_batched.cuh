@@ -294,6 +294,12 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int p = item / g.S, sp = item - p * g.S;
       const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
       double acc = 0.0;
+      if (g.qs.bits == 0) {
+        // the fp32 rotation rows the write-out will need for the objective: bring them into L2 now
+        const float* rr = g.R + ((long long)p * TCB_D + r) * TCB_D + (half * 2 + grp) * 32;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr));
+        if (TCB_EPI_GROUPS == 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + 32));
+      }
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
         if (TCB_EPI_GROUPS == 2 && (it & 1) != grp) continue;
         const int yb = it % TCB_YBUF, cb = it & 1;
