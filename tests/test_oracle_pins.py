@@ -536,3 +536,19 @@ def test_relative_quantisation_error_definition_and_bound(mode, clip):
     # the error is relative: scaling the activations changes nothing
     num2, den2 = O.token_diagnostics(3.0 * x, r, bits, mode, clip)[2:4]
     assert abs(num2 / den2 - num / den) < 1e-12
+    # ... and against a per-element search that uses none of the oracle's quantiser code: every code on the row's
+    # grid is tried and the nearest level taken (Appendix B: Q maps to the nearest grid point; ties do not change
+    # the distance), with the grid written out from the definition of the step and the code range
+    total = 0.0
+    for row in y:
+        if mode == "sym":
+            step = np.abs(row).max() / (2 ** (bits - 1) - 1)
+            levels = [step * k for k in range(-(2 ** (bits - 1) - 1), 2 ** (bits - 1))]
+        else:
+            lo, hi = clip * row.min(), clip * row.max()
+            step = (hi - lo) / (2 ** bits - 1)
+            zeta = -round(lo / step)                                   # integer zero-point
+            levels = [step * (k - zeta) for k in range(0, 2 ** bits)]
+        for v in row:
+            total += min((v - lv) ** 2 for lv in levels)
+    assert abs(num - total) <= 1e-10 * total
