@@ -71,7 +71,7 @@ typedef struct {
                                round half to even */
   int32_t  ns_steps;        /* Newton-Schulz steps planned before the re-projection loop;
                                0 = derive from ns_sigma_min_rel */
-  int32_t  ns_max_steps;    /* hard cap on Newton-Schulz steps per update; 0 = the planned schedule + 12 */
+  int32_t  ns_max_steps;    /* hard cap on Newton-Schulz steps per update; 0 = max(planned schedule + 12, 40) */
   float    orth_tol;        /* accept R when max|R^T R - I| <= orth_tol; 0 = default 1e-4 */
   float    prior_rel;       /* lam_rel >= 0: update is polar(M + lam R_prev),
                                lam = lam_rel * ||M||_F / sqrt(d); 0 = the paper's update */

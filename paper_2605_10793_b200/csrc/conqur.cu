@@ -603,7 +603,9 @@ extern "C" int conqur_init(conqur_ctx** out, int32_t d, const conqur_config* cfg
   c->n_sched = (int)c->sched.size();
   // ns_steps > 0: the caller's budget of steps; the lifting count starts from what the budget leaves after the endgame
   if (cfg->ns_steps > 0) c->n_lift_init = std::max(0, std::min(cfg->ns_steps, NS_SCHED_MAX) - (c->n_sched - 1));
-  if (g.ns_max_steps == 0) g.ns_max_steps = std::min(120, c->n_lift_init + c->n_sched - 1 + 12);
+  // generous: with the looped update graph steps that are not needed are never launched, and a lifting count learnt on
+  // easy updates must leave room for a hard one
+  if (g.ns_max_steps == 0) g.ns_max_steps = std::min(120, std::max(c->n_lift_init + c->n_sched - 1 + 12, 40));
   std::vector<SchedEntry> coef(NS_SCHED_MAX);
   for (int i = 0; i < NS_SCHED_MAX; ++i) {
     const NsStep& s = c->sched[std::min(i, c->n_sched - 1)];

@@ -43,6 +43,7 @@ struct DevState {
   int loop_passes;          // passes of the update graph's loop body in the update in flight
   long long loop_passes_total;   // ... since init (launch accounting)
   int lift_left;            // lifting steps still to run in the update in flight
+  int reentries;            // times the endgame ran out in the update in flight
   float growth;             // cumulative growth of the smallest singular values in the update in flight
   double diag_pr, diag_rho, diag_qnum, diag_qden;   // Section-4 diagnostics accumulated since the last update
   unsigned char seg_log[128];   // seg_x | seg_e << 4 of each step of the last update (launch accounting)

@@ -536,6 +536,7 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
 __device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
   if (!s->lift_init) { s->lift_plan = n_lift_init; s->lift_lo = -1; s->lift_hi = 127; s->lift_init = 1; }
   s->lift_left = s->lift_plan;
+  s->reentries = 0;
   s->loop_passes = 0;
   s->ns_idx = 1;                       // first endgame entry of the device schedule (entry 0 is the lifting quintic)
   s->growth = 1.0f;
@@ -614,8 +615,8 @@ static __global__ void ns_x0_kernel(const float* __restrict__ M, const float* __
 //     jumps to the last endgame entry fitted for an interval that still contains the spectrum;
 //   * if the endgame ran out without convergence (the lifting phase was too short for the smallest singular value):
 //     the last, order-3 convergent entry again while only a little is missing (||G - I||_F < 0.97: whatever lags has
-//     sigma^2 > 0.03 and doubles per step), otherwise two more lifting steps (safe to repeat: they never push a
-//     singular value below their floor) and the endgame again.
+//     sigma^2 > 0.03 and doubles per step), otherwise 2, then 4, 8, 16 more lifting steps (safe to repeat: they never
+//     push a singular value below their floor) and the endgame again.
 // The very first step also rescales: ||G_0||_F^(1/2) = (sum sigma^4)^(1/4) bounds the largest singular value of X_0
 // from above, far more tightly than the Frobenius norm X_0 was scaled by, and dividing X_0 by it is the same as
 // applying p(x / s): a / s, b / s^3, c / s^5.
@@ -656,7 +657,14 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
       s->lift_left -= 1;
     } else if (idx >= c.n_sched) {
       if (fro < 0.97f) { idx = c.n_sched - 1; }
-      else { lifting = true; s->lift_left = 1; idx = 1; }
+      else {
+        // 2, 4, 8, 16 more lifting steps, then the endgame again: a plan that was far too short (a much worse
+        // conditioned matrix than the ones the count was learnt on) still gets there within ns_max_steps
+        lifting = true;
+        s->lift_left = (2 << min(s->reentries, 3)) - 1;
+        s->reentries += 1;
+        idx = 1;
+      }
     }
     const SchedEntry e = c.sched[lifting ? 0 : idx];
     if (!lifting) idx += 1;

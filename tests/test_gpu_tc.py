@@ -260,3 +260,36 @@ def test_update_on_synthetic_spectra(mode, spectrum):
     tol = TOL[mode]
     assert rep["orth"] <= tol["orth"], rep
     assert rep["gap"] <= tol["gap"], (rep["gap"], st.ns_steps_used)
+
+
+@pytest.mark.parametrize("mode", ["tc", "exact"])
+def test_update_recovers_when_the_learnt_lifting_count_is_far_too_short(mode):
+    """The number of lifting steps an update starts with is learnt from the updates before it.  A context that has only
+    seen well-conditioned cross-covariances (and has learnt a short plan) is then given one with singular values down
+    to 1e-8 of the largest: the update must still deliver the polar factor (more steps, never a failure), and the
+    plan must climb."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    d = 512
+    rng = np.random.default_rng(9)
+    u, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    v, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    easy = (u * np.linspace(1.0, 0.3, d)) @ v.T
+    hard = (u * np.concatenate([np.ones(8), np.logspace(-3, -8, d - 8)])) @ v.T
+    ctx = B.Context(d=d, n_max=128, in_dtype="bf16", mode=mode)
+    plans, steps = [], []
+    for k in range(6):
+        ctx.set_M(torch.from_numpy(easy.astype(np.float32)).cuda(), 1.0, d)
+        ctx.update()
+        st = ctx.get_stats()
+        assert st.status == 0
+        plans.append(st.ns_lift_plan); steps.append(st.ns_steps_used)
+    assert plans[-1] <= 3 and steps[-1] < steps[0], (plans, steps)          # learnt: a handful of steps suffice
+    m32 = hard.astype(np.float32)
+    ctx.set_M(torch.from_numpy(m32).cuda(), 1.0, d)
+    ctx.update()
+    st = ctx.get_stats()
+    assert st.status == 0, (st.status, st.ns_steps_used)
+    assert st.ns_steps_used > steps[-1] and st.ns_lift_plan > plans[-1], (st.ns_steps_used, st.ns_lift_plan)
+    rep = update_parity(m32.astype(np.float64), ctx.get_R().cpu().numpy().astype(np.float64))
+    assert rep["orth"] <= TOL[mode]["orth"] and rep["gap"] <= TOL[mode]["gap"], (rep["orth"], rep["gap"], st.ns_steps_used)
