@@ -223,3 +223,56 @@ def test_token_sharded_wrapper_over_the_real_context_one_rank():
     assert int(row[0]) == 0 and row[1] == "True"
     assert float(row[2]) <= TOL["tc"]["J"] and float(row[3]) <= TOL["tc"]["gap"] and float(row[4]) <= TOL["tc"]["orth"]
     assert int(row[5]) == 3000
+
+
+def test_looped_update_graph_equals_direct_launches_bit_for_bit():
+    """After a context's first update the launch sequence is replayed from a captured graph whose middle is a
+    device-side loop over Newton-Schulz steps; CONQUR_DEBUG_NO_GRAPH enqueues every launch directly.  Same kernels,
+    same order, same data: rotations, statistics and step counts are identical over several cycles."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    d, n = 512, 1024
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2)
+    xs = [_dev(I.batch(w, b)) for b in range(6)]
+    out = []
+    for flags in (0, B.CONQUR_DEBUG_NO_GRAPH):
+        ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", defer_batches=2, debug_flags=flags)
+        ctx.set_R(_dev(I.initial_rotation(w), "f32"))
+        trace = []
+        for cyc in range(5):
+            ctx.step(xs[cyc % 6]); ctx.step(xs[(cyc + 1) % 6])
+            ctx.update()
+            st = ctx.get_stats()
+            assert st.status == 0
+            trace.append((ctx.get_R().clone(), int(st.ns_steps_used), int(st.ns_lift_plan), st.last_J))
+        out.append(trace)
+    for a, b in zip(*out):
+        assert torch.equal(a[0], b[0]) and a[1:] == b[1:]
+    launches = ctx.get_profile()["total_launches"]
+    assert launches > 0
+
+
+def test_per_head_step_timeline_hook():
+    """conqur_debug_trace_heads: thread block 0 stamps its first tiles; the events of a tile come in the order the
+    pipeline imposes (copy issued < first product < epilogue done < second product) and nothing is written once the
+    hook is switched off."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    P, n, d = 148, 512, 128                              # one problem per thread block, four tiles each
+    x = (torch.randn(P * n, d, device="cuda") * (1.0 + 20.0 * (torch.arange(d, device="cuda") < 2))).to(torch.bfloat16)
+    ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode="tc", batch=P)
+    trace = torch.zeros(96 * 16, dtype=torch.int64, device="cuda")
+    ctx.debug_trace_heads(trace)
+    ctx.step_batched(x, n, d, n * d)
+    ctx.debug_trace_heads(None)
+    t = trace.cpu().numpy().reshape(96, 16)
+    tiles = n // 128
+    used = t[:tiles]
+    assert (used[:, [0, 1, 2, 5, 9]] > 0).all()
+    assert (used[:, 0] < used[:, 1]).all() and (used[:, 1] < used[:, 9]).all() and (used[:, 9] < used[:, 2]).all()
+    assert not t[tiles:].any()                                       # block 0 worked on one problem only
+    trace.zero_()
+    ctx.step_batched(x, n, d, n * d)
+    torch.cuda.synchronize()
+    assert not trace.any().item()
+    assert ctx.get_stats().status == 0
