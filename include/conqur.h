@@ -69,14 +69,16 @@ typedef struct {
                                b in 2..8: per-token symmetric b-bit fake-quantisation of the
                                rotated row first (Appendix B, Q_sym), levels -(2^(b-1)-1)..(2^(b-1)-1),
                                round half to even */
-  int32_t  ns_steps;        /* Newton-Schulz steps planned before the re-projection loop;
+  int32_t  ns_steps;        /* Newton-Schulz steps a problem's FIRST update plans for (a budget, not a cap: the
+                               orthogonality check decides when the iteration ends, conqur_get_stats reports the steps
+                               used; later updates start from the count learnt so far, see conqur_update);
                                0 = derive from ns_sigma_min_rel */
   int32_t  ns_max_steps;    /* hard cap on Newton-Schulz steps per update; 0 = max(planned schedule + 12, 40) */
   float    orth_tol;        /* accept R when max|R^T R - I| <= orth_tol; 0 = default 1e-4 */
   float    prior_rel;       /* lam_rel >= 0: update is polar(M + lam R_prev),
                                lam = lam_rel * ||M||_F / sqrt(d); 0 = the paper's update */
-  float    ns_sigma_min_rel;/* assumed lower bound on sigma_min(M)/||M||_F used to plan the
-                               polynomial schedule; 0 = default 1e-9 */
+  float    ns_sigma_min_rel;/* assumed lower bound on sigma_min(M)/||M||_F from which the first update of a problem
+                               plans its number of lifting steps; 0 = default 1e-9 */
   int64_t  n_max;           /* largest n of any step call (sizes the workspace) */
   int32_t  batch;           /* P >= 1 independent problems of size d */
   int32_t  quant_mode;      /* CONQUR_QUANT_SYMMETRIC: Q_sym of Appendix B (delta = max|y| / (2^(b-1)-1));
@@ -189,6 +191,11 @@ int conqur_step_batched_range(conqur_ctx* ctx, const void* X_dev, int64_t n, int
  * R <- polar(M_eff) = U V^T of the SVD M_eff = U S V^T (Section 3.3), computed by
  * Newton-Schulz iterations and accepted only when max|R^T R - I| <= orth_tol;
  * then M, J, N <- 0 (Algorithm 1 starts every mini-batch with empty statistics).
+ * The iteration first lifts the small singular values with a fixed quintic, then converges with a short
+ * endgame.  How many lifting steps are needed depends on sigma_min(M), which nothing cheap bounds: each problem
+ * starts from the planned count and then learns it from its own updates (a count that fell short costs a few
+ * extra steps, never the result).  The rotation returned always passes the same orthogonality check; its last
+ * bits depend on the number of steps taken, i.e. on the context's history.
  * Host errors: CONQUR_ERR_EMPTY_UPDATE (no step since the last update),
  * CONQUR_ERR_RANK_DEFICIENT (tokens enqueued < d and prior_rel == 0).
  * If the iteration does not converge within ns_max_steps the old R and M are kept
