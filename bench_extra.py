@@ -136,7 +136,7 @@ def run_algorithm1(args, g, ClockSampler, peaks):
     dom = max(classes, key=lambda k: prof[k]["ms"])
     dn = max(1, prof[dom]["timed"])
     ach = prof[dom]["flops"] / (prof[dom]["ms"] * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
+    peak = peaks["bf16_tflops"]                      # launches timed alone between their own events: the burst figure
     st1, st2 = cal.ctx1.get_stats(), cal.ctx2.get_stats()
     if not g.is_main:
         D.finish(g)
@@ -155,8 +155,9 @@ def run_algorithm1(args, g, ClockSampler, peaks):
                 "d2h_bytes_per_step": 16, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
-                     "kernel": f"tc_gemm_kernel, {dom} epilogue at n={n}", "launches": dn,
-                     "avg_launch_ms": prof[dom]["ms"] / dn, "peak_source": f"{peaks['source']} sustained bf16"},
+                     "kernel": f"tc_gemm_kernel, {dom} epilogue over the {2 * L} queued site matrices of {n} rows", "launches": dn,
+                     "avg_launch_ms": prof[dom]["ms"] / dn, "peak_source": f"{peaks['source']} burst bf16",
+                     "frac_of_sustained": ach / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": ach / 2250.0},
         "cpu_baseline": None,
         "breakdown_ms": {"site_steps": float(parts[0]), "heads_update": float(parts[1]), "r1_update": float(parts[2]),
                          "head_steps_alone": float(head_steps_ms)},
@@ -265,7 +266,7 @@ def run_fold(args, g, ClockSampler, peaks):
     ms_e2e = D.max_over_ranks(g, e0.elapsed_time(e1) / Ke)
     flops = 3 * 2.0 * d * d * cols
     ach = flops / (ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
+    peak = peaks["bf16_tflops"]                      # launches timed alone between their own events: the burst figure
     if g.is_main:
         print(json.dumps({
             "metric": "weight elements folded/sec, R^T W with W 4096 x 14336 (whole call: split, three-pass product, status read)",
@@ -280,7 +281,8 @@ def run_fold(args, g, ClockSampler, peaks):
             "roofline": {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
                          "kernel": "tc_gemm_kernel, plain epilogue, 3 passes (timed with the two split kernels and the "
                                    "allocation of the output and scratch tensors of the call)",
-                         "avg_launch_ms": ms, "flops_per_launch": flops, "peak_source": f"{peaks['source']} sustained bf16"},
+                         "avg_launch_ms": ms, "flops_per_launch": flops, "peak_source": f"{peaks['source']} burst bf16",
+                         "frac_of_sustained": ach / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": ach / 2250.0},
             "cpu_baseline": None}))
     D.finish(g)
     return 0

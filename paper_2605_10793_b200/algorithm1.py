@@ -20,14 +20,18 @@ from . import binding as B
 
 class Calibrator:
     def __init__(self, d: int, n_heads: int, d_head: int, n_layers: int, n_max: int, *, in_dtype="bf16", mode="tc",
-                 quant_bits=0, quant_mode="sym", clip_ratio=0.0, prior_rel=0.0, record: Optional[str] = None):
-        """n_max: most tokens in one activation matrix.  record: None | "objective" | "full" (also keeps each
+                 quant_bits=0, quant_mode="sym", clip_ratio=0.0, prior_rel=0.0, record: Optional[str] = None,
+                 queue_sites: bool = True):
+        """n_max: most tokens in one activation matrix.  queue_sites (tensor-core mode): the R_1 context queues the 2L
+        activation matrices of a mini-batch and runs its two products once over all of them (the statistics are sums
+        over rows with R_1 fixed, Section 3.4); costs 4*d*n_max bytes of workspace per site.  record: None | "objective" | "full" (also keeps each
         cross-covariance, read before its update, and the sign decisions of every step; both synchronise and are
         meant for tests and logging)."""
         kw = dict(in_dtype=in_dtype, mode=mode, quant_bits=quant_bits, quant_mode=quant_mode, clip_ratio=clip_ratio,
                   prior_rel=prior_rel)
         self.d, self.n_heads, self.d_head, self.n_layers = d, n_heads, d_head, n_layers
-        self.ctx1 = B.Context(d=d, n_max=n_max, **kw)
+        queue = min(64, 2 * n_layers) if (queue_sites and mode == "tc") else 0
+        self.ctx1 = B.Context(d=d, n_max=n_max, defer_batches=queue, **kw)
         self.ctx2 = B.Context(d=d_head, n_max=n_max, batch=n_layers * n_heads, **kw)
         self.record = record
         self.log: List[Dict] = []
