@@ -749,6 +749,7 @@ extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tok
   if (!c || !J_sum || !n_tokens) return CONQUR_ERR_INVALID_ARG;
   { const int frc = flush_pending(c); if (frc) return frc; }
   const int P = c->cfg.P;
+  if (c->cfg.mode == CONQUR_TC_BF16) { const int orc = tcb_refresh_objective(c->tc, c->stream); if (orc) return orc; }
   std::vector<DevState> h(P);
   CQ_CUDA(cudaMemcpyAsync(h.data(), c->state(), sizeof(DevState) * P, cudaMemcpyDeviceToHost, c->stream));
   const int rc = sync_status(c);

@@ -426,13 +426,14 @@ static __global__ void splitk_reduce_add_kernel(float* __restrict__ M, const flo
   }
 }
 
-// Adds the step's objective partials (fixed order) and token counts to the running sums.
+// Adds the step's objective partials (fixed order; none when `partials` is null) and token counts to the running sums.
 static __global__ void finalize_step_kernel(DevState* st, const double* __restrict__ partials, int per_problem, int64_t n,
                                      double inv_sqrt_d, const double* __restrict__ part_diag = nullptr, int diag_blocks = 0) {
   const int p = blockIdx.x;
   __shared__ double red[8];
   double v = 0.0;
-  for (int i = threadIdx.x; i < per_problem; i += 256) v += partials[(int64_t)p * per_problem + i];
+  if (partials)
+    for (int i = threadIdx.x; i < per_problem; i += 256) v += partials[(int64_t)p * per_problem + i];
   const double tot = block_sum_d<256>(v, red);
   double dsum[4] = {0.0, 0.0, 0.0, 0.0};
   if (part_diag) {

@@ -70,6 +70,20 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+// Shared memory -> global through the copy engine (a box of the tensor map, whole), stored or added element by
+// element at the L2.  Asynchronous: the issuing thread commits the group and only waits until the source has been read.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, const void* smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tmap), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tmap, const void* smem_src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tmap), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
@@ -954,6 +968,7 @@ struct TcHost {
   float* part_f;
   // static tensor maps (d x d operands)
   CUtensorMap tmRb_mn;                       // R bf16 as MN-major B of the rotate product
+  CUtensorMap tmM_blk, tmMpart_blk;          // per-head case: fp32 M of all problems / the partials, 32 x 32 boxes
   CUtensorMap tmXh_mn[2], tmXh_k[2];         // iterate, stacked [hi; lo]
   CUtensorMap tmEh_k, tmEh_mn, tmBh_mn;
   Prof* prof;
@@ -990,6 +1005,24 @@ inline int tc_make_tmap(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     std::fprintf(stderr, "conqur: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+    return CONQUR_ERR_CUDA;
+  }
+  return CONQUR_OK;
+}
+
+// 2-D fp32 row-major tensor of 128 columns (rows x 128, contiguous rows); box = 32 rows x 32 columns, 128-byte swizzle.
+inline int tc_make_tmap_f32_blocks(CUtensorMap* tm, const void* ptr, uint64_t rows) {
+  PFN_encodeTiled fn = tc_encode_fn();
+  if (!fn) return CONQUR_ERR_CUDA;
+  const cuuint64_t dims[2] = {128, rows};
+  const cuuint64_t strides[1] = {128 * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "conqur: cuTensorMapEncodeTiled (fp32 blocks) failed (%d)\n", (int)r);
     return CONQUR_ERR_CUDA;
   }
   return CONQUR_OK;
@@ -1198,6 +1231,10 @@ inline int tc_init(TcHost* h, char* ws, const TcLayout& L, int d, int P, int64_t
   if (P > 1) {
     // all rotations stacked: problem p's R is rows [128 p, 128 p + 128); one box = 64 columns x all 128 rows
     rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, (uint64_t)P * D, D, D, 128);
+    // destinations of the per-head write-out: all cross-covariances stacked, and the partials of split problems
+    // (the idle Newton-Schulz buffers: 4 P matrices of 128 x 128 starting at Xa)
+    rc |= tc_make_tmap_f32_blocks(&h->tmM_blk, M, (uint64_t)P * D);
+    rc |= tc_make_tmap_f32_blocks(&h->tmMpart_blk, Xa, 4ull * (uint64_t)P * D);
     return rc ? CONQUR_ERR_CUDA : CONQUR_OK;
   }
   rc |= tc_make_tmap(&h->tmRb_mn, ws + L.Rb, D, D, D, 64);

@@ -41,6 +41,7 @@ constexpr int TCB_YBUF = 3;                      // Y accumulators in TMEM (128 
 constexpr int TCB_MBUF = (TCB_YBUF == 2) ? 2 : 1;   // 512 columns in all: 3 + 1 or 2 + 2
 constexpr int TCB_EPI_THREADS = 256;
 constexpr int TCB_EPI_WARPS = TCB_EPI_THREADS / 32;
+constexpr int TCB_PARTS = TCB_EPI_WARPS * TCB_EPI_GROUPS;   // objective partials per work item
 constexpr int TCB_AUX_BYTES = 2048;
 // Timeline hook (conqur_debug_trace_heads): per tile 16 slots of clock64() values, see TCB_EV_* for the events.
 constexpr int TCB_TRACE_TILES = 96;
@@ -51,13 +52,12 @@ constexpr int TCB_SMEM_BYTES = TCB_TILE_BYTES * (1 + TCB_XSTAGES + 2) + TCB_AUX_
 
 struct TcbAux {
   uint64_t rfull, rempty, mfull[TCB_MBUF], mempty[TCB_MBUF];
-  uint64_t pdone;            // every epilogue warp has finished the problem (write-out and objective partial)
+  uint64_t pdone[2];         // [epilogue group]: every warp of the group has finished the problem (write-out, objective partial)
   uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
   uint64_t yfull[TCB_YBUF], yempty[TCB_YBUF], cready[2], cfree[2];
   uint64_t nready[TCB_YBUF]; // row norms of the tile in Y buffer b are in rn[b]
   uint32_t tmem_base;
   int abort_flag;
-  double red_d[2][16];       // [problem parity][epilogue warp]: objective partials
   float rn[TCB_YBUF][128];   // [Y buffer][row]: 1 / ||x_row||, 0 for rows that are skipped or past the end
 };
 
@@ -73,9 +73,8 @@ struct TcbStepArgs {
   float* M;                   // P x 128 x 128 fp32 (without the 1/sqrt(d))
   int S;                      // token splits per problem: work item i = (problem i / S, tiles [T (i % S) / S, T (i % S + 1) / S))
   float* Mpart;               // S > 1: P * S partial cross-covariances (item order), summed into M by tcb_finish_kernel
-  double* part_d;             // P * S objective partials (sum |y| * rnorm, or the quantised equivalent), item order
+  double* part_d;             // fake-quantisation only: P * S * TCB_PARTS objective partials (one per epilogue warp), item order
   DevState* st;               // P
-  const float* R;             // P x 128 x 128 fp32: the rotations (for the objective <R, X~^T S>)
   long long* trace;           // measurement hook: when set, CTA 0 records SM-clock timestamps of its first TCB_TRACE_TILES tiles
   int8_t* signs;              // test hook: when set, the sign decisions (-1/0/+1) of this call, (P * n) x 128 row-major
 };
@@ -93,8 +92,54 @@ __device__ __forceinline__ uint32_t tcb_piece(int r, int c16) {
   return (uint32_t)((c16 >> 3) * 16384 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4));
 }
 
+// Work item -> problem and tile range [t_begin, t_end) of its T tiles (S items per problem).  T * S < 2^32: T <= 2^24
+// tiles and S is at most the number of SMs.  The common case S = 1 needs no division.
+__device__ __forceinline__ void tcb_item(int item, int T, int S, int& p, int& t_begin, int& t_end) {
+  if (S == 1) { p = item; t_begin = 0; t_end = T; return; }
+  p = item / S;
+  const unsigned sp = (unsigned)(item - p * S);
+  t_begin = (int)((unsigned)T * sp / (unsigned)S);
+  t_end = (int)((unsigned)T * (sp + 1u) / (unsigned)S);
+}
+
+// One warp's share of a problem's write-out: 32 x 32 fp32 blocks of the accumulator (TMEM address t_addr + 32 c, a
+// thread holds one row) for c = c0 .. c_end - 1.  Each block is laid into 4 KB of shared memory the way
+// the copy engine expects a 32 x 32 fp32 box (128-byte rows, 128-byte swizzle) and handed to it: added element by
+// element at the L2 (`add`; fire-and-forget, the warp only waits until the engine has read the staging area) or
+// stored.  Box (column 32 c, row y0) of tmOut.  Waits for the accumulator first (`bar`, `parity`; false when that
+// wait was abandoned) and arrives at `drained` once the warp's last block has left it.  Kept out of line: it runs once per problem and must not weigh on the tile loop.
+__device__ __noinline__ bool tcb_write_out(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t t_addr, uint8_t* stg,
+                                           int lane, const CUtensorMap* tmOut, int y0, bool add, int c0, int c_end, uint64_t* drained) {
+  if (!tc_wait(bar, parity, abort_flag)) return false;
+  ptx::tc_fence_after();
+#pragma unroll 1
+  for (int c = c0; c < c_end; ++c) {
+    float v[32];
+    ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+    if (c == c_end - 1) {                          // this warp's part of the accumulator is in registers
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(drained);
+    }
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
+      *reinterpret_cast<float4*>(stg + lane * 128 + ((p ^ (lane & 7)) << 4)) = make_float4(v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
+    ptx::fence_proxy_async();                      // the staged rows must be visible to the copy engine
+    __syncwarp();
+    if (lane == 0) {
+      if (add) ptx::tma_reduce_add_2d(tmOut, stg, c * 32, y0);
+      else ptx::tma_store_2d(tmOut, stg, c * 32, y0);
+      ptx::bulk_commit();
+      ptx::bulk_wait_read_all();                   // the staging area may be overwritten after this
+    }
+    __syncwarp();
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(TCB_THREADS, 1)
-tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR, const TcbStepArgs g) {
+tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
+                const __grid_constant__ CUtensorMap tmOut, const TcbStepArgs g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sR = smem;
@@ -107,8 +152,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->rfull, 1); ptx::mbar_init(&aux->rempty, 1);
-    for (int b = 0; b < TCB_MBUF; ++b) { ptx::mbar_init(&aux->mfull[b], 1); ptx::mbar_init(&aux->mempty[b], TCB_EPI_WARPS * TCB_EPI_GROUPS); }
-    ptx::mbar_init(&aux->pdone, TCB_EPI_WARPS * TCB_EPI_GROUPS);
+    for (int b = 0; b < TCB_MBUF; ++b) { ptx::mbar_init(&aux->mfull[b], 1); ptx::mbar_init(&aux->mempty[b], TCB_EPI_WARPS); }
+    for (int i = 0; i < TCB_EPI_GROUPS; ++i) ptx::mbar_init(&aux->pdone[i], TCB_EPI_WARPS);
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
     for (int b = 0; b < TCB_YBUF; ++b) {
       ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
@@ -120,6 +165,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     ptx::fence_proxy_async();
     ptx::prefetch_tmap(&tmX);
     ptx::prefetch_tmap(&tmR);
+    ptx::prefetch_tmap(&tmOut);
   }
   if (warp == 1) { ptx::tmem_alloc(&aux->tmem_base, 512); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
@@ -141,8 +187,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       bool ok = true;
       int issued = 0;
       for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
-        const int p = item / g.S, sp = item - p * g.S;
-        const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
+        int p, t_begin, t_end;
+        tcb_item(item, T, g.S, p, t_begin, t_end);
         if (!tc_wait(&aux->rempty, ((uint32_t)lp & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 11; break; }
         ptx::mbar_expect_tx(&aux->rfull, TCB_TILE_BYTES);
         ptx::tma_load_2d(sR, &tmR, &aux->rfull, 0, (g.p0 + p) * TCB_D);
@@ -174,8 +220,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int it = 0, lp = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
-        const int sp = item % g.S;
-        const int T_item = (int)((long long)T * (sp + 1) / g.S) - (int)((long long)T * sp / g.S);
+        int p_item, tb_item, te_item;
+        tcb_item(item, T, g.S, p_item, tb_item, te_item);
+        const int T_item = te_item - tb_item;
         if (!tc_wait(&aux->rfull, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 20; break; }
         for (int t = 0; t < T_item && ok; ++t, ++it) {
           const int yb = it % TCB_YBUF;
@@ -205,8 +252,9 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int it = 0, lp = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
-        const int sp = item % g.S;
-        const int T_item = (int)((long long)T * (sp + 1) / g.S) - (int)((long long)T * sp / g.S);
+        int p_item, tb_item, te_item;
+        tcb_item(item, T, g.S, p_item, tb_item, te_item);
+        const int T_item = te_item - tb_item;
         // the accumulator of the previous problem has been read out
         const int mb = lp % TCB_MBUF;
         if (!tc_wait(&aux->mempty[mb], (((uint32_t)(lp / TCB_MBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 21; break; }
@@ -234,8 +282,8 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     int it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x) {
-      const int p = item / g.S, sp = item - p * g.S;
-      const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
+      int p, t_begin, t_end;
+      tcb_item(item, T, g.S, p, t_begin, t_end);
       int skipped = 0, nonfinite = 0;
       for (int t = t_begin; t < t_end; ++t, ++it) {
         const int yb = it % TCB_YBUF, xs = it % TCB_XSTAGES;
@@ -289,19 +337,16 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int half = ew >> 2;                      // which 64 of the 128 columns this warp handles
     const int r = q * 32 + lane;                   // token inside the tile; later: row of M
     int it = 0, lp = 0;
+    uint32_t wo_count = 0;                         // write-outs this warp's group has done
     bool ok = true;
     for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x, ++lp) {
-      const int p = item / g.S, sp = item - p * g.S;
-      const int t_begin = (int)((long long)T * sp / g.S), t_end = (int)((long long)T * (sp + 1) / g.S);
+      int p, t_begin, t_end;
+      tcb_item(item, T, g.S, p, t_begin, t_end);
       double acc = 0.0;
-      if (g.qs.bits == 0) {
-        // the fp32 rotation rows the write-out will need for the objective: bring them into L2 now
-        const float* rr = g.R + ((long long)p * TCB_D + r) * TCB_D + (half * 2 + grp) * 32;
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr));
-        if (TCB_EPI_GROUPS == 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + 32));
-      }
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
         if (TCB_EPI_GROUPS == 2 && (it & 1) != grp) continue;
+        // the write-out's tensor map was last used a whole problem ago: fetch it again a few tiles before the end
+        if (lane == 0 && t + 2 * TCB_EPI_GROUPS >= t_end && t + TCB_EPI_GROUPS < t_end) ptx::prefetch_tmap(&tmOut);
         const int yb = it % TCB_YBUF, cb = it & 1;
         const uint32_t par3 = ((uint32_t)(it / TCB_YBUF)) & 1u, par2 = ((uint32_t)it >> 1) & 1u;
         const bool tr_epi = ew == 0;                       // the first warp of the tile's group stamps the epilogue
@@ -398,58 +443,34 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
       if (!ok) break;
-      // the problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T).  Every
-      // epilogue warp takes part (with two groups each warp one 32 x 32 block, else two).
-      const int mb = lp % TCB_MBUF;
-      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_WAIT);
-      if (!tc_wait(&aux->mfull[mb], ((uint32_t)(lp / TCB_MBUF)) & 1u, abort_flag)) { ok = false; timeout_site = 33; break; }
-      ptx::tc_fence_after();
-      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_BEGIN);
-      {
+      // The problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T).  With two
+      // groups, the one that owned the problem's last tile writes all of it out (each warp 32 rows x 64 columns) while
+      // the other goes straight on to the next problem's first tile, so the second products resume as soon as the
+      // accumulator has been read.
+      const int wo_grp = (TCB_EPI_GROUPS == 2) ? ((it - 1) & 1) : 0;
+      if (grp == wo_grp) {
+        const int mb = lp % TCB_MBUF;
+        if (ew == 0) TCB_TR(it - 1, TCB_EV_OUT_WAIT);
+        // Every second product issued so far has finished once the accumulator is complete, and this group's next
+        // target tile comes after the write-out, so its C' buffer is idle: each warp borrows 4 KB of it as staging
+        // area.  One item per problem: added into M (one addition per element and launch, so the result does not
+        // depend on any order); several: stored to the item's partial, summed in item order afterwards.
         const uint32_t t_addr = tmem_base + TM_M + (uint32_t)(mb * 128) + ((uint32_t)(q * 32) << 16);
-        // Every second product issued so far has finished and no new target tile exists before these warps return to
-        // the tiles, so the C' buffers are idle: each warp borrows 4 KB to turn its 32 x 32 block (a thread holds one
-        // row) into full 128-byte row segments.  One item per problem: added into M with fire-and-forget vector
-        // reductions (one addition per element and launch, so the result does not depend on any order); several:
-        // stored to the item's partial, summed in item order afterwards.
         uint8_t* stg = sC + grp * TCB_TILE_BYTES + ew * 4096;
-        float* dst = (g.S == 1) ? g.M + ((long long)p * TCB_D + q * 32) * TCB_D : g.Mpart + ((long long)item * TCB_D + q * 32) * TCB_D;
-        const float* rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
-        float jacc = 0.f;
-#pragma unroll 1
-        for (int cc = grp; cc < 2; cc += TCB_EPI_GROUPS) {
-          const int c = half * 2 + cc;
-          float v[32];
-          ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
-          if (g.qs.bits == 0) {
-            // this block's share of the objective: <R, X~^T C'> over its part of the accumulator (fp32 R)
-            const float4* r4 = reinterpret_cast<const float4*>(rrow + c * 32);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float4 q4 = __ldg(r4 + i);
-              jacc = fmaf(v[4 * i], q4.x, jacc); jacc = fmaf(v[4 * i + 1], q4.y, jacc);
-              jacc = fmaf(v[4 * i + 2], q4.z, jacc); jacc = fmaf(v[4 * i + 3], q4.w, jacc);
-            }
-          }
-          if (g.S == 1) tc_red_block_f32(stg, lane, v, dst + c * 32, TCB_D, 32);
-          else tc_store_block_f32(stg, lane, v, dst + c * 32, TCB_D, 32);
-        }
-        if (g.qs.bits == 0) acc = (double)jacc;
+        const int y0 = ((g.S == 1) ? (g.p0 + p) : item) * TCB_D + q * 32;
+        if (!tcb_write_out(&aux->mfull[mb], ((uint32_t)(lp / TCB_MBUF)) & 1u, abort_flag, t_addr, stg, lane, &tmOut, y0, g.S == 1,
+                           half * 2, half * 2 + 2, &aux->mempty[mb])) { ok = false; timeout_site = 33; break; }
+        if (ew == 0) TCB_TR(it - 1, TCB_EV_OUT_END);
+        // the group's warps stay off their C' buffer until all of them have finished staging in it (bounded wait)
+        if (lane == 0) ptx::mbar_arrive(&aux->pdone[grp]);
+        if (!tc_wait(&aux->pdone[grp], wo_count & 1u, abort_flag)) { ok = false; timeout_site = 36; break; }
+        ++wo_count;
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (grp == 0 && ew == 0) TCB_TR(it - 1, TCB_EV_OUT_END);
-      if (lane == 0) ptx::mbar_arrive(&aux->mempty[mb]);
-      // Per-problem reduction in a fixed order.  The barrier (bounded like every other wait) also keeps every warp
-      // off the C' buffers until all of them have finished staging.  The partials are double-buffered by problem
-      // parity: no warp can get two problems ahead of the thread that sums them.
-      const double wsum = warp_sum_d(acc);
-      if (lane == 0) { aux->red_d[lp & 1][grp * 8 + ew] = wsum; ptx::mbar_arrive(&aux->pdone); }
-      if (!tc_wait(&aux->pdone, (uint32_t)lp & 1u, abort_flag)) { ok = false; timeout_site = 36; break; }
-      if (grp == 0 && ew == 0 && lane == 0) {
-        double tot = 0.0;
-        for (int i = 0; i < 8 * TCB_EPI_GROUPS; ++i) tot += aux->red_d[lp & 1][i];
-        g.part_d[item] = tot;
+      // With fake-quantisation every warp leaves its objective partial of the problem (summed in a fixed order by the
+      // kernel that follows); without, the objective is <R, M> / sqrt(d) and is formed from M when it is read.
+      if (g.qs.bits > 0) {
+        const double wsum = warp_sum_d(acc);
+        if (lane == 0) g.part_d[(long long)item * TCB_PARTS + grp * 8 + ew] = wsum;
       }
     }
   }
@@ -464,6 +485,34 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
+}
+
+// Per-head problems without fake-quantisation: between two updates R is fixed and M = sum of X~^T S, so the objective
+// sum_rows <x~ R, s> / sqrt(d) equals <R, M> / sqrt(d) (Eq. 4 with the corner target); the step kernel does not
+// accumulate it.  It is formed from M by the update kernel and, for a read in between, by tcb_objective_kernel.
+inline bool tcb_objective_from_m(const TcHost& h) { return h.P > 1 && h.qs.bits == 0; }
+
+// st[p].J = <R_p, M_p> / sqrt(d), summed in a fixed order.  grid P, 256 threads.
+static __global__ void tcb_objective_kernel(DevState* st, const float* __restrict__ M, const float* __restrict__ R) {
+  const int p = blockIdx.x;
+  __shared__ double red[8];
+  const float4* m4 = reinterpret_cast<const float4*>(M + (size_t)p * TCB_D * TCB_D);
+  const float4* r4 = reinterpret_cast<const float4*>(R + (size_t)p * TCB_D * TCB_D);
+  double v = 0.0;
+  for (int i = threadIdx.x; i < TCB_D * TCB_D / 4; i += 256) {
+    const float4 m = m4[i], q = r4[i];
+    v += (double)m.x * q.x + (double)m.y * q.y + (double)m.z * q.z + (double)m.w * q.w;
+  }
+  const double tot = block_sum_d<256>(v, red);
+  if (threadIdx.x == 0) st[p].J = tot / sqrt((double)TCB_D);
+}
+
+inline int tcb_refresh_objective(TcHost& h, cudaStream_t s) {
+  if (!tcb_objective_from_m(h)) return CONQUR_OK;
+  tcb_objective_kernel<<<h.P, 256, 0, s>>>(h.st, h.M, h.R);
+  if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
+  if (h.prof) h.prof->count(K_OTHER);
+  return CONQUR_OK;
 }
 
 // M[p] += partial[p * S + 0] + ... + partial[p * S + S - 1], in that order.  grid (16, problems), 256 threads.
@@ -550,7 +599,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
   TcbStepArgs g{};
   g.n = (int)n; g.P = np; g.p0 = p0; g.qs = h.qs; g.xp_outer_tokens = outer_tokens;
   g.M = h.M + (size_t)p0 * TCB_D * TCB_D; g.part_d = h.part_d; g.st = h.st + p0; g.signs = signs_out;
-  g.R = h.R + (size_t)p0 * TCB_D * TCB_D; g.trace = trace;
+  g.trace = trace;
   // few problems: split each problem's tokens over several CTAs (partials land in the idle Newton-Schulz buffers,
   // 4 P matrices of 128 x 128 starting at Xa, and are summed in a fixed order)
   const int T = (int)((n + 127) / 128);
@@ -566,7 +615,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
     rec.e0 = h.prof->get_event(); rec.e1 = h.prof->get_event();
     cudaEventRecord(rec.e0, s);
   }
-  tcb_step_kernel<<<grid, TCB_THREADS, TCB_SMEM_BYTES, s>>>(tmX, h.tmRb_mn, g);
+  tcb_step_kernel<<<grid, TCB_THREADS, TCB_SMEM_BYTES, s>>>(tmX, h.tmRb_mn, S == 1 ? h.tmM_blk : h.tmMpart_blk, g);
   if (timed) { cudaEventRecord(rec.e1, s); h.prof->open.push_back(rec); }
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_ROTATE);
@@ -575,7 +624,7 @@ inline int tcb_step(TcHost& h, cudaStream_t s, const void* X, int in_dtype, int6
     if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
     if (h.prof) h.prof->count(K_OTHER);
   }
-  finalize_step_kernel<<<np, 256, 0, s>>>(g.st, h.part_d, S, n, 1.0 / std::sqrt((double)TCB_D));
+  finalize_step_kernel<<<np, 256, 0, s>>>(g.st, h.qs.bits > 0 ? h.part_d : nullptr, S * TCB_PARTS, n, 1.0 / std::sqrt((double)TCB_D));
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_OTHER);
   return CONQUR_OK;
@@ -614,7 +663,9 @@ static_assert(sizeof(TcbUpdAux) <= 4096, "the control block must fit its reserve
 
 struct TcbUpdArgs {
   int P;
+  int objective_from_m;        // 1: the objective consumed by this update is <R, M> / sqrt(d), formed here
   float* M; float* R;          // P x 128 x 128 fp32
+  __nv_bfloat16* Rb;           // P x 128 x 128: the rotations in bf16 (operand of the step kernel), rewritten with R
   DevState* st;
   NsControlParams ncp;
   float prior_rel, margin;
@@ -698,26 +749,33 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     DevState* const sg = g.st + p;                 // global copy: read once, written back once
     DevState* const s = &aux->state;
     if (threadIdx.x == 0) *s = *sg;
-    const float* Mrow = g.M + ((long long)p * TCB_D + r) * TCB_D;
-    const float* Rrow = g.R + ((long long)p * TCB_D + r) * TCB_D;
-    // ---- scale: lam = prior_rel ||M||_F / sqrt(d), X_0 = (M + lam R) / (||M + lam R||_F (1 + margin))
-    double ssq = 0.0;
-    for (int c = half * 64; c < half * 64 + 64; c += 4) {
-      const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
+    const float4* M4 = reinterpret_cast<const float4*>(g.M + (long long)p * TCB_D * TCB_D);
+    const float4* R4 = reinterpret_cast<const float4*>(g.R + (long long)p * TCB_D * TCB_D);
+    // ---- scale: lam = prior_rel ||M||_F / sqrt(d), X_0 = (M + lam R) / (||M + lam R||_F (1 + margin)), with
+    // ||M + lam R||^2 = ||M||^2 + 2 lam <M, R> + lam^2 ||R||^2; <R, M> / sqrt(d) is also the objective this update
+    // consumes where the step kernel does not accumulate it.  One coalesced pass, sums in double in a fixed order.
+    const bool need_r = g.objective_from_m || g.prior_rel > 0.f;
+    double ssq = 0.0, dot = 0.0, rsq = 0.0;
+#pragma unroll 8
+    for (int k = 0; k < TCB_D * TCB_D / 4 / TCBU_THREADS; ++k) {
+      const int i = k * TCBU_THREADS + threadIdx.x;
+      const float4 m = M4[i];
       ssq += (double)m.x * m.x + (double)m.y * m.y + (double)m.z * m.z + (double)m.w * m.w;
-    }
-    double fro2 = tcbu_block_sum(ssq, aux->red_d, warp, lane);
-    const float lam = g.prior_rel * (float)sqrt(fro2) * isd;
-    if (g.prior_rel > 0.f) {
-      ssq = 0.0;
-      for (int c = half * 64; c < half * 64 + 64; c += 4) {
-        const float4 m = *reinterpret_cast<const float4*>(Mrow + c);
-        const float4 q = *reinterpret_cast<const float4*>(Rrow + c);
-        const float a = fmaf(lam, q.x, m.x), b = fmaf(lam, q.y, m.y), cc = fmaf(lam, q.z, m.z), d4 = fmaf(lam, q.w, m.w);
-        ssq += (double)a * a + (double)b * b + (double)cc * cc + (double)d4 * d4;
+      if (need_r) {
+        const float4 q = R4[i];
+        dot += (double)m.x * q.x + (double)m.y * q.y + (double)m.z * q.z + (double)m.w * q.w;
+        rsq += (double)q.x * q.x + (double)q.y * q.y + (double)q.z * q.z + (double)q.w * q.w;
       }
-      fro2 = tcbu_block_sum(ssq, aux->red_d, warp, lane);
     }
+    const double m2 = tcbu_block_sum(ssq, aux->red_d, warp, lane);
+    if (need_r) {
+      dot = tcbu_block_sum(dot, aux->red_d, warp, lane);
+      rsq = tcbu_block_sum(rsq, aux->red_d, warp, lane);
+    }
+    if (g.objective_from_m && threadIdx.x == 0) s->J = dot * (double)isd;
+    const float lam = g.prior_rel * (float)sqrt(m2) * isd;
+    double fro2 = m2;
+    if (g.prior_rel > 0.f) fro2 = fmax(m2 + 2.0 * (double)lam * dot + (double)lam * (double)lam * rsq, 0.0);
     if (threadIdx.x == 0) {
       const float fro = (float)sqrt(fro2);
       const bool ok = (fro > 0.f) && (fro <= 3.0e38f) && (s->N > 0);
@@ -732,16 +790,20 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     __syncthreads();
     if (!aux->done) {
       const float x0s = aux->x0s;
-      for (int c16 = half * 8; c16 < half * 8 + 8; ++c16) {
-        uint32_t wh[4], wl[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int col = c16 * 8 + e * 2;
-          const float a = fmaf(lam, Rrow[col], Mrow[col]) * x0s, b = fmaf(lam, Rrow[col + 1], Mrow[col + 1]) * x0s;
-          bf16x2_split(a, b, wh[e], wl[e]);
+#pragma unroll 4
+      for (int k = 0; k < TCB_D * TCB_D / 4 / TCBU_THREADS; ++k) {
+        const int i = k * TCBU_THREADS + threadIdx.x;             // float4 i: row i / 32, columns 4 (i % 32)..+3
+        float4 a = M4[i];
+        if (lam != 0.f) {
+          const float4 q = R4[i];
+          a.x = fmaf(lam, q.x, a.x); a.y = fmaf(lam, q.y, a.y); a.z = fmaf(lam, q.z, a.z); a.w = fmaf(lam, q.w, a.w);
         }
-        *reinterpret_cast<uint4*>(sXh + tcb_piece(r, c16)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-        *reinterpret_cast<uint4*>(sXl + tcb_piece(r, c16)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+        uint32_t h0, h1, l0, l1;
+        bf16x2_split(a.x * x0s, a.y * x0s, h0, l0);
+        bf16x2_split(a.z * x0s, a.w * x0s, h1, l1);
+        const uint32_t off = tcb_piece(i >> 5, (i & 31) >> 1) + (uint32_t)(i & 1) * 8u;
+        *reinterpret_cast<uint2*>(sXh + off) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2*>(sXl + off) = make_uint2(l0, l1);
       }
       issue_products(issue_gram);
       bool gram_in_flight = true;
@@ -878,22 +940,24 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
     // ---- commit: R <- X, M <- 0, sums <- 0; or keep everything and latch the failure
     const bool converged = (aux->done == NS_DONE_CONVERGED);
     if (converged) {
-      float* Ro = g.R + ((long long)p * TCB_D + r) * TCB_D;
-      float* Mo = g.M + ((long long)p * TCB_D + r) * TCB_D;
-      for (int c16 = half * 8; c16 < half * 8 + 8; ++c16) {
-        const uint32_t off = tcb_piece(r, c16);
-        const uint4 h4 = *reinterpret_cast<const uint4*>(sXh + off), l4 = *reinterpret_cast<const uint4*>(sXl + off);
-        const uint32_t hh[4] = {h4.x, h4.y, h4.z, h4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
-        float o[8];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          o[2 * e] = __uint_as_float(hh[e] << 16) + __uint_as_float(ll[e] << 16);
-          o[2 * e + 1] = __uint_as_float(hh[e] & 0xffff0000u) + __uint_as_float(ll[e] & 0xffff0000u);
-        }
-        *reinterpret_cast<float4*>(Ro + c16 * 8) = make_float4(o[0], o[1], o[2], o[3]);
-        *reinterpret_cast<float4*>(Ro + c16 * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
-        *reinterpret_cast<float4*>(Mo + c16 * 8) = make_float4(0.f, 0.f, 0.f, 0.f);
-        *reinterpret_cast<float4*>(Mo + c16 * 8 + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      // coalesced: float4 i = row i / 32, columns 4 (i % 32)..+3; the bf16 copy the step kernel multiplies with is
+      // the round-to-nearest of the fp32 rotation
+      float4* Ro = reinterpret_cast<float4*>(g.R + (long long)p * TCB_D * TCB_D);
+      float4* Mo = reinterpret_cast<float4*>(g.M + (long long)p * TCB_D * TCB_D);
+      uint2* Rbo = reinterpret_cast<uint2*>(g.Rb + (long long)p * TCB_D * TCB_D);
+#pragma unroll 4
+      for (int k = 0; k < TCB_D * TCB_D / 4 / TCBU_THREADS; ++k) {
+        const int i = k * TCBU_THREADS + threadIdx.x;
+        const uint32_t off = tcb_piece(i >> 5, (i & 31) >> 1) + (uint32_t)(i & 1) * 8u;
+        const uint2 h2 = *reinterpret_cast<const uint2*>(sXh + off), l2 = *reinterpret_cast<const uint2*>(sXl + off);
+        float4 o;
+        o.x = __uint_as_float(h2.x << 16) + __uint_as_float(l2.x << 16);
+        o.y = __uint_as_float(h2.x & 0xffff0000u) + __uint_as_float(l2.x & 0xffff0000u);
+        o.z = __uint_as_float(h2.y << 16) + __uint_as_float(l2.y << 16);
+        o.w = __uint_as_float(h2.y & 0xffff0000u) + __uint_as_float(l2.y & 0xffff0000u);
+        Ro[i] = o;
+        Rbo[i] = make_uint2(bf16x2_pack(o.x, o.y), bf16x2_pack(o.z, o.w));
+        Mo[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
     if (threadIdx.x == 0) {
@@ -931,11 +995,13 @@ inline int tcb_update(TcHost& h, cudaStream_t s, const NsControlParams& ncp, flo
   }
   TcbUpdArgs g{};
   g.P = h.P; g.M = h.M; g.R = h.R; g.st = h.st; g.ncp = ncp; g.prior_rel = prior_rel; g.margin = margin;
+  g.objective_from_m = tcb_objective_from_m(h) ? 1 : 0;
+  g.Rb = reinterpret_cast<__nv_bfloat16*>(h.ws + h.L.Rb);
   const int grid = h.P < 2 * h.num_sms ? h.P : 2 * h.num_sms;
   tcb_update_kernel<<<grid, TCBU_THREADS, TCBU_SMEM_BYTES, s>>>(g);
   if (cudaGetLastError() != cudaSuccess) return CONQUR_ERR_CUDA;
   if (h.prof) h.prof->count(K_NS_RESID);
-  return tc_refresh_R(h, s, 0);
+  return CONQUR_OK;
 }
 
 }  // namespace conqur
