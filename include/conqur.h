@@ -212,6 +212,11 @@ int conqur_get_R(conqur_ctx* ctx, float* R_out_dev);
  * Objective accumulated since the last update, at the R those steps used:
  * J_sum[p] = sum_i ||y_i||_1/sqrt(d) (Section 3.2: the corner distance is 2N - 2J),
  * n_tokens[p] = rows used.  Host arrays of cfg.batch entries.  Synchronises.
+ * Per-head contexts (batch > 1) in tensor-core mode without fake-quantisation do not accumulate the sum row by row:
+ * with the rotation fixed between two updates, sum_i <x~_i R, s_i> = <R, sum_i x~_i^T s_i> = <R, M> (Eq. 4 with the
+ * corner target), so the objective is formed from the accumulated cross-covariance, here and by conqur_update (the
+ * value it consumes is reported as conqur_stats.last_J).  A rotation replaced by conqur_set_R between two updates is
+ * then the one the whole sum is evaluated with.
  */
 int conqur_get_objective(conqur_ctx* ctx, double* J_sum, int64_t* n_tokens);
 
@@ -237,7 +242,8 @@ int conqur_get_diagnostics(conqur_ctx* ctx, conqur_diagnostics* out);
 int conqur_get_M(conqur_ctx* ctx, float* M_out_dev);
 
 /* Overwrite the accumulated cross-covariance (same scaling as conqur_get_M) and the sums:
- * resume / teacher forcing.  J_sum, n_tokens: host arrays of cfg.batch entries. */
+ * resume / teacher forcing.  J_sum, n_tokens: host arrays of cfg.batch entries.  (Where the objective is formed from
+ * M, see conqur_get_objective, J_sum is stored but superseded by <R, M> / sqrt(d) at the next read.) */
 int conqur_set_M(conqur_ctx* ctx, const float* M_dev, const double* J_sum, const int64_t* n_tokens);
 
 /* Sign decisions of the last step call (tie-aware parity, Eq. 2: which corner each row was sent to): device int8,

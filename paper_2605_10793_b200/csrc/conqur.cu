@@ -360,7 +360,7 @@ int update_step(conqur_ctx* c, int k, int cur, bool last) {
   const int T = cdiv(d, SG_BM);
   const int parts = ns_parts(c);
   const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, d, use_shift, g.orth_tol,
-                            g.fro_tol, g.margin, g.lo_budget};
+                            g.fro_tol, g.margin, g.lo_budget, 1.0 / (double)d};
   float* X = cur ? Xb : Xa;
   float* Xn = cur ? Xa : Xb;
   c->tc.ns_k = k;
@@ -403,7 +403,7 @@ int update_impl(conqur_ctx* c) {
   if (g.mode == CONQUR_TC_BF16 && g.P > 1) {
     // many small problems: the whole iteration of a problem runs inside one CTA
     const NsControlParams ncp{c->at<SchedEntry>(c->L.sched), c->n_sched, c->n_lift_init, g.ns_max_steps, g.d, 1,
-                              g.orth_tol, g.fro_tol, g.margin, g.lo_budget};
+                              g.orth_tol, g.fro_tol, g.margin, g.lo_budget, 1.0 / (double)g.d};
     return tcb_update(c->tc, c->stream, ncp, g.prior_rel, g.margin);
   }
   int rc = update_prologue(c);

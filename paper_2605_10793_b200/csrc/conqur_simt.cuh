@@ -629,12 +629,35 @@ struct NsControlParams {
   int n_sched, n_lift_init, max_steps, d, use_shift;
   float tol, fro_tol, margin;
   float lo_budget;          // tensor-core mode: the iterate enters the last product as hi + lo while d 2^-8 / growth exceeds this
+  double inv_d;             // 1 / d (the decision runs on one thread between two products: no divisions there)
 };
 
 // The decision itself (one thread): tmx = max|G - I|, tsq = ||G - I||_F^2, ttr = tr G of step k.
-__device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double tsq, double ttr, int k, int cur_buf,
-                                                  const NsControlParams& c) {
-  const float fro = (float)sqrt(tsq);
+// The part of a problem's state the per-step decision reads and writes.  A kernel that iterates a problem in place keeps
+// it in registers between the steps (ns_ctl_load once, ns_ctl_store at the end).
+struct NsCtl {
+  float e_max, e_fro, tau, growth;
+  float coef[4];
+  int ns_done, ns_final_buf, ns_idx, lift_left, reentries, seg_x, seg_e, ns_steps_used;
+};
+__device__ __forceinline__ void ns_ctl_load(NsCtl& t, const DevState* s) {
+  t.e_max = s->e_max; t.e_fro = s->e_fro; t.tau = s->tau; t.growth = s->growth;
+  t.coef[0] = s->coef[0]; t.coef[1] = s->coef[1]; t.coef[2] = s->coef[2]; t.coef[3] = s->coef[3];
+  t.ns_done = s->ns_done; t.ns_final_buf = s->ns_final_buf; t.ns_idx = s->ns_idx; t.lift_left = s->lift_left;
+  t.reentries = s->reentries; t.seg_x = s->seg_x; t.seg_e = s->seg_e; t.ns_steps_used = s->ns_steps_used;
+}
+__device__ __forceinline__ void ns_ctl_store(const NsCtl& t, DevState* s) {
+  s->e_max = t.e_max; s->e_fro = t.e_fro; s->tau = t.tau; s->growth = t.growth;
+  s->coef[0] = t.coef[0]; s->coef[1] = t.coef[1]; s->coef[2] = t.coef[2]; s->coef[3] = t.coef[3];
+  s->ns_done = t.ns_done; s->ns_final_buf = t.ns_final_buf; s->ns_idx = t.ns_idx; s->lift_left = t.lift_left;
+  s->reentries = t.reentries; s->seg_x = t.seg_x; s->seg_e = t.seg_e; s->ns_steps_used = t.ns_steps_used;
+}
+
+// Returns the step's entry of the pass log (seg_x | seg_e << 4), or 0 when no step follows.
+__device__ __forceinline__ unsigned char ns_control_decide(NsCtl* s, float tmx, double tsq, double ttr, int k, int cur_buf,
+                                                           const NsControlParams& c) {
+  unsigned char log_entry = 0;
+  const float fro = sqrtf((float)tsq);
   s->e_max = tmx;
   s->e_fro = fro;
   if (!(tmx == tmx) || !(fro == fro)) {
@@ -684,7 +707,7 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
       // ||E_tau||_F^2 and tr E_tau from the statistics of G - I and tr G
       const double dd = (double)c.d;
       const double e2 = fmax(0.0, tsq + 2.0 * (1.0 - tau) * ttr + dd * (tau * tau - 1.0));
-      kappa = (cc * e2 + b1 * (ttr - dd * tau)) / dd;
+      kappa = (cc * e2 + b1 * (ttr - dd * tau)) * c.inv_d;
     }
     s->coef[0] = (float)(a + b * tau + cc * tau * tau + kappa);
     s->coef[1] = (float)b1;
@@ -695,10 +718,11 @@ __device__ __forceinline__ void ns_control_decide(DevState* s, float tmx, double
     const int seg_x = (!c.use_shift || (float)c.d * (1.0f / 256.0f) / s->growth > c.lo_budget) ? 2 : 1;
     s->growth *= (float)a;
     s->seg_x = seg_x;
-    if (k < 128) s->seg_log[k] = (unsigned char)(seg_x | (s->seg_e << 4));   // seg_e: what this step's residual product used
+    log_entry = (unsigned char)(seg_x | (s->seg_e << 4));           // seg_e: what this step's residual product used
     s->ns_idx = idx;
     s->ns_steps_used = k + 1;
   }
+  return log_entry;
 }
 
 static __global__ void ns_control_kernel(DevState* st, const float* __restrict__ part_max,
@@ -720,7 +744,13 @@ static __global__ void ns_control_kernel(DevState* st, const float* __restrict__
   const double tsq = block_sum_d<256>(sq, redd);
   const double ttr = block_sum_d<256>(tr, redd);
   const float tmx = block_max_f<256>(mx, redf);
-  if (threadIdx.x == 0) ns_control_decide(s, tmx, tsq, ttr, k, cur_buf, c);
+  if (threadIdx.x == 0) {
+    NsCtl t;
+    ns_ctl_load(t, s);
+    const unsigned char log_entry = ns_control_decide(&t, tmx, tsq, ttr, k, cur_buf, c);
+    ns_ctl_store(t, s);
+    if (log_entry && k < 128) s->seg_log[k] = log_entry;
+  }
 }
 
 // tau of the next residual product = mean sigma^2 of the new iterate = ||X||_F^2 / d (tensor-core mode), and how

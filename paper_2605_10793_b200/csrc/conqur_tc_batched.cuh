@@ -23,6 +23,8 @@
 // taken once per problem from the cross-covariance accumulator on its way out instead of summing |y| element by
 // element in the epilogue.
 #pragma once
+#include <type_traits>
+
 #include "conqur_tc.cuh"
 
 namespace conqur {
@@ -109,9 +111,11 @@ __device__ __forceinline__ void tcb_item(int item, int T, int S, int& p, int& t_
 // stored.  Box (column 32 c, row y0) of tmOut.  Waits for the accumulator first (`bar`, `parity`; false when that
 // wait was abandoned) and arrives at `drained` once the warp's last block has left it.  Kept out of line: it runs once per problem and must not weigh on the tile loop.
 __device__ __noinline__ bool tcb_write_out(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t t_addr, uint8_t* stg,
-                                           int lane, const CUtensorMap* tmOut, int y0, bool add, int c0, int c_end, uint64_t* drained) {
+                                           int lane, const CUtensorMap* tmOut, int y0, bool add, int c0, int c_end, uint64_t* drained,
+                                           long long* begun) {
   if (!tc_wait(bar, parity, abort_flag)) return false;
   ptx::tc_fence_after();
+  if (begun) *begun = clock64();                   // timeline hook
 #pragma unroll 1
   for (int c = c0; c < c_end; ++c) {
     float v[32];
@@ -459,7 +463,10 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         uint8_t* stg = sC + grp * TCB_TILE_BYTES + ew * 4096;
         const int y0 = ((g.S == 1) ? (g.p0 + p) : item) * TCB_D + q * 32;
         if (!tcb_write_out(&aux->mfull[mb], ((uint32_t)(lp / TCB_MBUF)) & 1u, abort_flag, t_addr, stg, lane, &tmOut, y0, g.S == 1,
-                           half * 2, half * 2 + 2, &aux->mempty[mb])) { ok = false; timeout_site = 33; break; }
+                           half * 2, half * 2 + 2, &aux->mempty[mb],
+                           (tracing && ew == 0 && it - 1 < TCB_TRACE_TILES) ? g.trace + (it - 1) * 16 + TCB_EV_OUT_BEGIN : nullptr)) {
+          ok = false; timeout_site = 33; break;
+        }
         if (ew == 0) TCB_TR(it - 1, TCB_EV_OUT_END);
         // the group's warps stay off their C' buffer until all of them have finished staging in it (bounded wait)
         if (lane == 0) ptx::mbar_arrive(&aux->pdone[grp]);
@@ -691,6 +698,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = threadIdx.x & 127;                 // the row this thread works on everywhere
   const int half = threadIdx.x >> 7;               // ... and which 64 of its 128 columns
+  const int c_diag = r >> 5;                       // the 32-column chunk holding the row's diagonal element (one per warp)
   if (threadIdx.x == 0) {
     ptx::mbar_init(&aux->mbar, 1);
     aux->abort_flag = 0;
@@ -745,6 +753,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         ptx::umma_bf16(tmem_base, desc_mn(aa[seg], j), desc_mn(bb[seg], j), idesc_mm, (seg > 0 || j > 0) ? 1u : 0u);
   };
 
+  NsCtl ctl{};                                     // thread 0 only
   for (int p = blockIdx.x; p < g.P && !timed_out; p += gridDim.x) {
     DevState* const sg = g.st + p;                 // global copy: read once, written back once
     DevState* const s = &aux->state;
@@ -786,6 +795,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       ns_arm_lifting(s, g.ncp.n_lift_init);
       s->tau = 1.0f / ((1.0f + g.margin) * (1.0f + g.margin) * (float)TCB_D);
       aux->done = s->ns_done; aux->tau = s->tau; aux->x0s = s->x0_scale; aux->lam = lam;
+      ns_ctl_load(ctl, s);                          // thread 0 keeps the decision's state in registers from here on
     }
     __syncthreads();
     if (!aux->done) {
@@ -815,8 +825,8 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         const float tau = aux->tau;
         float mx = 0.f, tr = 0.f;
         double sq = 0.0;
-#pragma unroll 1
-        for (int c = half * 2; c < half * 2 + 2; ++c) {
+        // (the diagonal lies in one 32-column chunk per warp, c_diag: only that chunk pays for finding it)
+        auto resid_chunk = [&](int c, auto has_diag) {
           float v[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), v);
           const int dcol = r - c * 32;
@@ -825,7 +835,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             float e1 = v[i];
-            if (i == dcol) { tr += v[i]; e1 -= 1.f; v[i] -= tau; }
+            if (decltype(has_diag)::value && i == dcol) { tr += v[i]; e1 -= 1.f; v[i] -= tau; }
             mx = fmaxf(mx, fabsf(e1));
             sq32 = fmaf(e1, e1, sq32);
           }
@@ -835,6 +845,10 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
             *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        };
+#pragma unroll 1
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
+          if (c == c_diag) resid_chunk(c, std::true_type{}); else resid_chunk(c, std::false_type{});
         }
         {
           const double wsq = warp_sum_d(sq), wtr = warp_sum_d((double)tr);
@@ -852,10 +866,11 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           double tsq = 0.0, ttr = 0.0;
           float tmx = 0.f;
           for (int i = 0; i < 8; ++i) { tsq += aux->red_d[i]; ttr += aux->red_t[i]; tmx = fmaxf(tmx, aux->red_f[i]); }
-          ns_control_decide(s, tmx, tsq, ttr, k, 0, ncp);
-          aux->done = s->ns_done;
-          aux->coef[0] = s->coef[0]; aux->coef[1] = s->coef[1]; aux->coef[2] = s->coef[2]; aux->coef[3] = s->coef[3];
-          aux->seg_x = s->seg_x;
+          const unsigned char log_entry = ns_control_decide(&ctl, tmx, tsq, ttr, k, 0, ncp);
+          if (log_entry && k < 128) s->seg_log[k] = log_entry;
+          aux->done = ctl.ns_done;
+          aux->coef[0] = ctl.coef[0]; aux->coef[1] = ctl.coef[1]; aux->coef[2] = ctl.coef[2]; aux->coef[3] = ctl.coef[3];
+          aux->seg_x = ctl.seg_x;
         }
         __syncthreads();
         if (!wait_products()) { timed_out = true; break; }
@@ -863,8 +878,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         const float cg = aux->coef[0], cb1 = aux->coef[1], cb2 = aux->coef[2], ck = aux->coef[3];
         const int seg_x = aux->seg_x;
         // ---- B = beta2 E E + beta1 E - kappa I (over E: the product that read it has finished)
-#pragma unroll 1
-        for (int c = half * 2; c < half * 2 + 2; ++c) {
+        auto poly_chunk = [&](int c, auto has_diag) {
           float gq[32], ee[32];
           ptx::tmem_ld32(t_row + (uint32_t)(c * 32), gq);
           ptx::tmem_ld32(t_row + 128u + (uint32_t)(c * 32), ee);
@@ -872,9 +886,10 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
           uint32_t w[16];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float e = (i == dcol) ? gq[i] - tau : gq[i];
+            const bool on_diag = decltype(has_diag)::value && i == dcol;
+            const float e = on_diag ? gq[i] - tau : gq[i];
             float b = fmaf(cb2, ee[i], cb1 * e);
-            if (i == dcol) b -= ck;
+            if (on_diag) b -= ck;
             ee[i] = b;
           }
 #pragma unroll
@@ -882,6 +897,10 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
             *reinterpret_cast<uint4*>(sEB + tcb_piece(r, c * 4 + q4)) = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        };
+#pragma unroll 1
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
+          if (c == c_diag) poly_chunk(c, std::true_type{}); else poly_chunk(c, std::false_type{});
         }
         // ---- X B
         issue_products([&] {
@@ -928,7 +947,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
         if (threadIdx.x == 0) {
           const double tx2 = ((aux->red_d[0] + aux->red_d[1]) + (aux->red_d[2] + aux->red_d[3])) +
                              ((aux->red_d[4] + aux->red_d[5]) + (aux->red_d[6] + aux->red_d[7]));
-          s->tau = (float)(tx2 / (double)TCB_D); aux->tau = s->tau;
+          ctl.tau = (float)(tx2 * (1.0 / (double)TCB_D)); aux->tau = ctl.tau;
         }
         __syncthreads();
       }
@@ -961,6 +980,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       }
     }
     if (threadIdx.x == 0) {
+      ns_ctl_store(ctl, s);
       ns_adapt_lift_plan(s, ncp.n_sched - 1, converged ? 1 : 0);
       if (converged) {
         s->last_J = s->J; s->last_N = s->N; s->J = 0.0; s->N = 0; s->updates += 1;
