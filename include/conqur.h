@@ -221,6 +221,18 @@ int conqur_get_R(conqur_ctx* ctx, float* R_out_dev);
 int conqur_get_objective(conqur_ctx* ctx, double* J_sum, int64_t* n_tokens);
 
 /*
+ * The same two arrays without stopping the stream: the values as of this point of the context's stream are copied to
+ * J_sum_host / n_tokens_host (host arrays of cfg.batch entries; page-locked memory for the copy to overlap) by copies
+ * enqueued on that stream, and the call returns at once.  The arrays hold the result, and must stay valid, once the
+ * stream has passed this point (an event recorded on the stream after the call, or any synchronising call).  For a
+ * training loop that logs the objective of every cycle without draining the queue: enqueue the read, then
+ * conqur_update, and look at the numbers one cycle later.  Runs the products of queued batches first, like
+ * conqur_get_objective.  Device-side conditions (CONQUR_ERR_NONFINITE ...) are reported by the next synchronising
+ * call, not here.
+ */
+int conqur_get_objective_async(conqur_ctx* ctx, double* J_sum_host, int64_t* n_tokens_host);
+
+/*
  * Diagnostics of Section 4 over the rows used since the last update, at the R those steps used (cfg.diagnostics = 1):
  *   sum_pr_over_d  sum_i PR(y_i)/d,  PR(y)/d = ||y||_2^4 / (d ||y||_4^4) in [1/d, 1]  (normalised participation ratio)
  *   sum_rho        sum_i rho(y_i),   rho(y) = ||y||_inf^2 / ||y||_2^2 in [1/d, 1]     (dynamic-range ratio, Appendix B)

@@ -31,7 +31,7 @@ _live_contexts = None
 
 EXPORTS = [
     "conqur_workspace_bytes", "conqur_init", "conqur_destroy", "conqur_set_R", "conqur_step",
-    "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_M",
+    "conqur_step_batched", "conqur_step_batched_range", "conqur_update", "conqur_get_R", "conqur_get_objective", "conqur_get_objective_async", "conqur_get_M",
     "conqur_set_M", "conqur_debug_get_signs", "conqur_debug_capture_signs", "conqur_get_stats", "conqur_debug_check_canaries", "conqur_debug_trace_heads", "conqur_plan_schedule", "conqur_debug_gemm",
     "conqur_set_profiling", "conqur_get_profile", "conqur_objective_noalloc", "conqur_debug_wait_timeout",
     "conqur_get_diagnostics", "conqur_fold_scratch_bytes", "conqur_fold_weight", "conqur_hadamard_rows", "conqur_hadamard_status",
@@ -112,6 +112,8 @@ def load() -> C.CDLL:
     lib.conqur_get_R.argtypes = [vp, vp]
     lib.conqur_get_objective.restype = C.c_int
     lib.conqur_get_objective.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.conqur_get_objective_async.restype = C.c_int
+    lib.conqur_get_objective_async.argtypes = [vp, vp, vp]
     lib.conqur_get_M.restype = C.c_int
     lib.conqur_get_M.argtypes = [vp, vp]
     lib.conqur_set_M.restype = C.c_int
@@ -428,6 +430,14 @@ class Context:
         if check:
             self._chk(rc, "conqur_get_objective")
         return (float(j[0]), int(n[0])) if self.batch == 1 else (j, n)
+
+    def get_objective_async(self, j_host, n_host):
+        """Enqueue the read of (J, N) into page-locked host tensors (float64 / int64, one entry per problem) on the
+        context's stream and return at once; the values are there once the stream has passed this point."""
+        t = self.torch
+        assert j_host.device.type == "cpu" and j_host.dtype == t.float64 and j_host.numel() == self.batch and j_host.is_contiguous()
+        assert n_host.device.type == "cpu" and n_host.dtype == t.int64 and n_host.numel() == self.batch and n_host.is_contiguous()
+        self._chk(load().conqur_get_objective_async(self.h, j_host.data_ptr(), n_host.data_ptr()), "conqur_get_objective_async")
 
     def get_diagnostics(self):
         """Section-4 diagnostics since the last update: list of dicts (one per problem)."""

@@ -31,7 +31,7 @@ inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 inline int cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, flags_agg, R, M, rnorm, rowmax, part_d, part_f, part_diag, sched;
+  size_t state, flags_agg, R, M, rnorm, rowmax, part_d, part_f, part_diag, sched, obj_out;
   size_t C;                 // exact: fp32 C' / Y (P x n_max x d); TC quant mode: fp32 Y
   size_t Xa, Xb, E, B;      // Newton-Schulz fp32 matrices (P x d x d each)
   size_t splitk;            // exact accumulate split-K partials
@@ -110,6 +110,7 @@ bool make_layout(int d, const conqur_config* c, Layout* L) {
   L->part_f = take(sizeof(float) * mp * P);
   L->part_diag = c->diagnostics ? take(sizeof(double) * 4 * mp * P) : 0;
   L->sched = take(sizeof(SchedEntry) * NS_SCHED_MAX);
+  L->obj_out = take(16 * P);                         // J (double) and N (int64) of every problem, for the asynchronous read
   L->acc_splits = 1;
   L->C = L->splitk = 0;
   // the four Newton-Schulz matrices form ONE region: a token-split per-head step borrows all of it as scratch
@@ -195,6 +196,9 @@ __global__ void clear_flags_kernel(DevState* st, int P, int* agg) {
 }
 __global__ void arm_check_kernel(DevState* st, int P) {
   for (int i = threadIdx.x; i < P; i += blockDim.x) { st[i].ns_done = 0; st[i].ns_steps_used = 0; }
+}
+__global__ void export_sums_kernel(const DevState* st, double* J, long long* N, int P) {
+  for (int i = threadIdx.x; i < P; i += blockDim.x) { J[i] = st[i].J; N[i] = st[i].N; }
 }
 __global__ void set_sums_kernel(DevState* st, const double* J, const long long* N, int P) {
   for (int i = threadIdx.x; i < P; i += blockDim.x) { st[i].J = J[i]; st[i].N = N[i]; }
@@ -755,6 +759,20 @@ extern "C" int conqur_get_objective(conqur_ctx* c, double* J_sum, int64_t* n_tok
   const int rc = sync_status(c);
   for (int p = 0; p < P; ++p) { J_sum[p] = h[p].J; n_tokens[p] = h[p].N; }
   return rc;
+}
+
+extern "C" int conqur_get_objective_async(conqur_ctx* c, double* J_sum_host, int64_t* n_tokens_host) {
+  if (!c || !J_sum_host || !n_tokens_host) return CONQUR_ERR_INVALID_ARG;
+  { const int frc = flush_pending(c); if (frc) return frc; }
+  const int P = c->cfg.P;
+  if (c->cfg.mode == CONQUR_TC_BF16) { const int orc = tcb_refresh_objective(c->tc, c->stream); if (orc) return orc; }
+  double* dJ = c->at<double>(c->L.obj_out);
+  long long* dN = reinterpret_cast<long long*>(dJ + P);
+  export_sums_kernel<<<1, 256, 0, c->stream>>>(c->state(), dJ, dN, P);
+  CQ_LAUNCHED(c, K_OTHER);
+  CQ_CUDA(cudaMemcpyAsync(J_sum_host, dJ, sizeof(double) * P, cudaMemcpyDeviceToHost, c->stream));
+  CQ_CUDA(cudaMemcpyAsync(n_tokens_host, dN, sizeof(long long) * P, cudaMemcpyDeviceToHost, c->stream));
+  return CONQUR_OK;
 }
 
 extern "C" int conqur_get_diagnostics(conqur_ctx* c, conqur_diagnostics* out) {

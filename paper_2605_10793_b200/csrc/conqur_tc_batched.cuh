@@ -781,7 +781,7 @@ __global__ void __launch_bounds__(TCBU_THREADS, 2) tcb_update_kernel(const TcbUp
       dot = tcbu_block_sum(dot, aux->red_d, warp, lane);
       rsq = tcbu_block_sum(rsq, aux->red_d, warp, lane);
     }
-    if (g.objective_from_m && threadIdx.x == 0) s->J = dot * (double)isd;
+    if (g.objective_from_m && threadIdx.x == 0) s->J = dot / sqrt((double)TCB_D);
     const float lam = g.prior_rel * (float)sqrt(m2) * isd;
     double fro2 = m2;
     if (g.prior_rel > 0.f) fro2 = fmax(m2 + 2.0 * (double)lam * dot + (double)lam * (double)lam * rsq, 0.0);

@@ -109,6 +109,37 @@ def test_queued_batches_equal_immediate_ones_and_the_oracle(quant):
     assert n3 == ref.N and abs(j3 - ref.J) <= TOL["tc"]["J"] * ref.J
 
 
+@pytest.mark.parametrize("mode,d,batch,defer", [("exact", 96, 1, 0), ("tc", 256, 1, 3), ("tc", 128, 5, 0), ("exact", 32, 3, 0)])
+def test_asynchronous_objective_read(mode, d, batch, defer):
+    """conqur_get_objective_async leaves (J, N) as of its point in the stream in page-locked host arrays without
+    stopping the stream: the values equal the synchronous read taken at the same point, also when an update that resets
+    the sums is enqueued behind it (the per-head tensor-core case forms J from M on the way)."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    n = 300
+    w = I.scaled(I.WORKLOADS["c2"], d=d, n=n, n_outlier=2, r0="qr")
+    ctx = B.Context(d=d, n_max=n, in_dtype="bf16", mode=mode, batch=batch, defer_batches=defer)
+    jh = torch.zeros(batch, dtype=torch.float64).pin_memory()
+    nh = torch.zeros(batch, dtype=torch.int64).pin_memory()
+    for cycle in range(2):
+        for b in range(2):
+            if batch == 1:
+                ctx.step(_dev(I.batch(w, 2 * cycle + b)))
+            else:
+                x = np.stack([I.batch(w, 10 * p + 2 * cycle + b) for p in range(batch)])
+                ctx.step_batched(_dev(x.reshape(batch * n, d)), n, d, n * d)
+        j_sync, n_sync = ctx.get_objective()
+        ctx.get_objective_async(jh, nh)
+        ctx.update()                                   # enqueued behind the read: resets the sums on the device
+        ctx.stream.synchronize()
+        assert np.array_equal(nh.numpy(), np.atleast_1d(n_sync)) and np.all(nh.numpy() == 2 * n)
+        assert np.array_equal(jh.numpy(), np.atleast_1d(j_sync)) and np.all(jh.numpy() > 0)
+        j0, n0 = ctx.get_objective()
+        assert np.all(np.atleast_1d(n0) == 0) and np.all(np.atleast_1d(j0) == 0.0)
+        st = ctx.get_stats()
+        assert st.status == 0 and abs(st.last_J - float(np.sum(jh.numpy()))) <= 1e-9 * st.last_J
+
+
 @pytest.mark.parametrize("mode", ["exact", "tc"])
 @pytest.mark.parametrize("bits", [2, 3, 8])
 @pytest.mark.parametrize("qmode,clip", [("sym", 1.0), ("zp", 0.9)])
