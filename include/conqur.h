@@ -170,6 +170,10 @@ int conqur_step(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld);
  * cfg.batch reads its n rows at X_dev + p*problem_stride + i*ld (elements), each
  * row normalised by its own d-slice norm.  problem_stride = d, ld = P*d is the
  * head-interleaved layout; problem_stride = n*ld is stacked problems.
+ * In tensor-core mode (d = 128) the fused kernel takes a row's norm from the rotated row, ||x R~|| with R~ the bf16
+ * copy of R its product uses: equal to ||x|| for an orthogonal R, here within ||R~ R~^T - I||_2 / 2 of it (about
+ * 1e-4 relative; the scale then enters the target tile rounded to bf16, 2^-9).  A uniform factor on the rows' scales
+ * does not change the rotation an update returns.
  */
 int conqur_step_batched(conqur_ctx* ctx, const void* X_dev, int64_t n, int64_t ld,
                         int64_t problem_stride);
@@ -277,8 +281,9 @@ int conqur_debug_capture_signs(conqur_ctx* ctx, int8_t* S_dev, int64_t capacity_
 /* Measurement hook for the fused per-head step kernel (tensor-core contexts with batch > 1; no counterpart in the
  * paper): while a buffer is set, thread block 0 of every conqur_step_batched(_range) records SM-clock timestamps of
  * its first 96 token tiles, 16 int64 slots per tile: 0 copy of the tile issued, 1 / 2 first / second product issued,
- * 3 / 4 row norms begin / end, 5 epilogue reaches the tile, 6 norms available, 7 target buffer free, 8 rotated tile
- * available, 13 / 14 / 15 first TMEM load back / first half written / second TMEM load back, 9 epilogue done;
+ * 5 epilogue reaches the tile, 8 rotated tile available, 3 / 4 pass over it for the rows' scales begins / ends, 6 scales
+ * available, 7 target buffer free, 13 / 14 / 15 first TMEM load back / first half written / second TMEM load back,
+ * 9 epilogue done;
  * on a problem's last tile 10 / 11 / 12 accumulator awaited / being written out / written out.  trace_dev: device,
  * capacity >= 96 * 16 int64, owned by the caller; NULL stops the recording.  Synchronises. */
 int conqur_debug_trace_heads(conqur_ctx* ctx, int64_t* trace_dev, int64_t capacity);

@@ -36,8 +36,7 @@ constexpr int TCB_XSTAGES = 4;                   // a stage is held from the cop
 #define TCB_EPI_GROUPS_N 2
 #endif
 constexpr int TCB_EPI_GROUPS = TCB_EPI_GROUPS_N; // groups of eight epilogue warps taking tiles in turn
-constexpr int TCB_NORM_WARP0 = 2 + 8 * TCB_EPI_GROUPS;   // first of the four row-norm warps
-constexpr int TCB_MMA2_WARP = TCB_NORM_WARP0 + 4;        // issues the second product
+constexpr int TCB_MMA2_WARP = 2 + 8 * TCB_EPI_GROUPS;    // issues the second product
 constexpr int TCB_THREADS = (TCB_MMA2_WARP + 1) * 32;
 constexpr int TCB_YBUF = 3;                      // Y accumulators in TMEM (128 columns each), then the M accumulator(s)
 constexpr int TCB_MBUF = (TCB_YBUF == 2) ? 2 : 1;   // 512 columns in all: 3 + 1 or 2 + 2
@@ -57,10 +56,8 @@ struct TcbAux {
   uint64_t pdone[2];         // [epilogue group]: every warp of the group has finished the problem (write-out, objective partial)
   uint64_t xfull[TCB_XSTAGES], xempty[TCB_XSTAGES];
   uint64_t yfull[TCB_YBUF], yempty[TCB_YBUF], cready[2], cfree[2];
-  uint64_t nready[TCB_YBUF]; // row norms of the tile in Y buffer b are in rn[b]
   uint32_t tmem_base;
   int abort_flag;
-  float rn[TCB_YBUF][128];   // [Y buffer][row]: 1 / ||x_row||, 0 for rows that are skipped or past the end
 };
 
 static_assert(sizeof(TcbAux) <= TCB_AUX_BYTES, "the barrier / exchange block must fit its reserved shared memory");
@@ -161,7 +158,6 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     for (int s = 0; s < TCB_XSTAGES; ++s) { ptx::mbar_init(&aux->xfull[s], 1); ptx::mbar_init(&aux->xempty[s], 1); }
     for (int b = 0; b < TCB_YBUF; ++b) {
       ptx::mbar_init(&aux->yfull[b], 1); ptx::mbar_init(&aux->yempty[b], TCB_EPI_WARPS);
-      ptx::mbar_init(&aux->nready[b], 4);
     }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&aux->cready[b], TCB_EPI_WARPS); ptx::mbar_init(&aux->cfree[b], 1); }
     aux->abort_flag = 0;
@@ -280,60 +276,6 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (ok) ptx::umma_commit(&aux->mfull[mb]);
       }
     }
-  } else if (warp >= TCB_NORM_WARP0) {
-    // ---------------------------------------------------------------- a1: row norms from the tile in shared memory
-    const int r = (warp - TCB_NORM_WARP0) * 32 + lane;      // this lane's token inside every tile
-    int it = 0;
-    bool ok = true;
-    for (int item = blockIdx.x; item < g.P * g.S && ok; item += gridDim.x) {
-      int p, t_begin, t_end;
-      tcb_item(item, T, g.S, p, t_begin, t_end);
-      int skipped = 0, nonfinite = 0;
-      for (int t = t_begin; t < t_end; ++t, ++it) {
-        const int yb = it % TCB_YBUF, xs = it % TCB_XSTAGES;
-        if (!tc_wait(&aux->xfull[xs], ((uint32_t)(it / TCB_XSTAGES)) & 1u, abort_flag)) { ok = false; timeout_site = 34; break; }
-        // rn[yb] was last read by the epilogue of the tile that used this Y buffer before
-        if (!tc_wait(&aux->yempty[yb], (((uint32_t)(it / TCB_YBUF)) & 1u) ^ 1u, abort_flag)) { ok = false; timeout_site = 35; break; }
-        if (warp == TCB_NORM_WARP0) TCB_TR(it, TCB_EV_NORM_BEGIN);
-        uint8_t* xrow = sX + xs * TCB_TILE_BYTES;
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;       // four chains; added in a fixed order
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const uint4 w = *reinterpret_cast<const uint4*>(xrow + tcb_piece(r, c));
-          const float a0 = __uint_as_float(w.x << 16), b0 = __uint_as_float(w.x & 0xffff0000u);
-          const float a1 = __uint_as_float(w.y << 16), b1 = __uint_as_float(w.y & 0xffff0000u);
-          const float a2 = __uint_as_float(w.z << 16), b2 = __uint_as_float(w.z & 0xffff0000u);
-          const float a3 = __uint_as_float(w.w << 16), b3 = __uint_as_float(w.w & 0xffff0000u);
-          s0 = fmaf(a0, a0, s0); s0 = fmaf(b0, b0, s0);
-          s1 = fmaf(a1, a1, s1); s1 = fmaf(b1, b1, s1);
-          s2 = fmaf(a2, a2, s2); s2 = fmaf(b2, b2, s2);
-          s3 = fmaf(a3, a3, s3); s3 = fmaf(b3, b3, s3);
-        }
-        const float ss = (s0 + s1) + (s2 + s3);
-        const bool valid = (t * 128 + r) < g.n;
-        const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
-        if (valid && !good) {
-          ++skipped;
-          if (!(ss == 0.f)) nonfinite = 1;
-#pragma unroll
-          for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, c)) = make_uint4(0, 0, 0, 0);
-        }
-        aux->rn[yb][r] = good ? 1.0f / sqrtf(ss) : 0.f;
-        // a zeroed row must be visible to the second product (tensor-core proxy), rn to the epilogue warps
-        ptx::fence_proxy_async();
-        __syncwarp();
-        if (warp == TCB_NORM_WARP0) TCB_TR(it, TCB_EV_NORM_END);
-        if (lane == 0) ptx::mbar_arrive(&aux->nready[yb]);
-      }
-      if (!ok) break;
-      int wsk = skipped, wnf = nonfinite;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
-      if (lane == 0) {
-        if (wsk) atomicAdd(reinterpret_cast<unsigned long long*>(&g.st[p].step_skipped), (unsigned long long)wsk);
-        if (wnf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
-      }
-    }
   } else {
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     const int grp = (warp - 2) >> 3;               // with two groups: group 0 takes the even tiles (and C' buffer 0), group 1 the odd ones
@@ -347,6 +289,7 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int p, t_begin, t_end;
       tcb_item(item, T, g.S, p, t_begin, t_end);
       double acc = 0.0;
+      int skipped = 0, nonfinite = 0;
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
         if (TCB_EPI_GROUPS == 2 && (it & 1) != grp) continue;
         // the write-out's tensor map was last used a whole problem ago: fetch it again a few tiles before the end
@@ -355,31 +298,56 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const uint32_t par3 = ((uint32_t)(it / TCB_YBUF)) & 1u, par2 = ((uint32_t)it >> 1) & 1u;
         const bool tr_epi = ew == 0;                       // the first warp of the tile's group stamps the epilogue
         if (tr_epi) TCB_TR(it, TCB_EV_EPI_BEGIN);
-        if (!tc_wait(&aux->nready[yb], par3, abort_flag)) { ok = false; timeout_site = 30; break; }
-        if (tr_epi) TCB_TR(it, TCB_EV_EPI_NORMS);
-        const float rn = aux->rn[yb][r];
-        const bool valid = (t * 128 + r) < g.n;
-        const bool good = rn > 0.f;
-        const uint32_t rn_bits = bf16_bits(rn);
-        if (!tc_wait(&aux->cfree[cb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
-        if (tr_epi) TCB_TR(it, TCB_EV_EPI_CFREE);
         if (!tc_wait(&aux->yfull[yb], par3, abort_flag)) { ok = false; timeout_site = 32; break; }
         ptx::tc_fence_after();
         if (tr_epi) TCB_TR(it, TCB_EV_EPI_Y);
         const uint32_t t_addr = tmem_base + (uint32_t)(yb * 128) + ((uint32_t)(q * 32) << 16);
         uint8_t* crow = sC + cb * TCB_TILE_BYTES;
-        RowQuant rq{0.f, 0.f, 0.f, 0.f};
-        if (g.qs.bits > 0) {
-          float vmax = -3.0e38f, vmin = 3.0e38f;   // the per-token scale needs the whole row
+        // a1: the row's scale, taken from the rotated row: ||x R~|| with R~ the bf16 copy of the orthogonal R the
+        // product uses.  It differs from ||x|| by at most ||R~ R~^T - I||_2 / 2 (about 1e-4 for a typical row at
+        // d = 128), an order below the rounding of the scale itself to bf16 in the target tile, and costs no pass
+        // over the input tile in shared memory, whose bandwidth bounds this kernel.  Every warp reads the whole
+        // row (both warps of a row pair get the same sum); with fake-quantisation the same pass finds the row's range.
+        if (tr_epi) TCB_TR(it, TCB_EV_NORM_BEGIN);
+        float ss;
+        float vmax = -3.0e38f, vmin = 3.0e38f;
+        {
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;       // four chains; added in a fixed order
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             float v[32];
             ptx::tmem_ld32(t_addr + (uint32_t)(c * 32), v);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) { vmax = fmaxf(vmax, v[i]); vmin = fminf(vmin, v[i]); }
+            for (int i = 0; i < 32; i += 4) {
+              s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1);
+              s2 = fmaf(v[i + 2], v[i + 2], s2); s3 = fmaf(v[i + 3], v[i + 3], s3);
+            }
+            if (g.qs.bits > 0) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) { vmax = fmaxf(vmax, v[i]); vmin = fminf(vmin, v[i]); }
+            }
           }
-          rq = row_quant(g.qs, vmax, vmin, good);
+          ss = (s0 + s1) + (s2 + s3);
         }
+        if (tr_epi) TCB_TR(it, TCB_EV_NORM_END);
+        const bool valid = (t * 128 + r) < g.n;
+        const bool good = valid && (ss > 0.f) && (ss <= 3.0e38f);
+        if (valid && !good) {
+          // the row takes no part; a non-finite one is also zeroed in the input tile for the second product (this
+          // warp's 64 columns; made visible to the tensor-core proxy by the fence before the tile is handed over)
+          if (half == 0) { ++skipped; if (!(ss == 0.f)) nonfinite = 1; }
+          uint8_t* xrow = sX + (it % TCB_XSTAGES) * TCB_TILE_BYTES;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(xrow + tcb_piece(r, half * 8 + c)) = make_uint4(0, 0, 0, 0);
+        }
+        const float rn = good ? 1.0f / sqrtf(ss) : 0.f;
+        const uint32_t rn_bits = bf16_bits(rn);
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_NORMS);
+        RowQuant rq{0.f, 0.f, 0.f, 0.f};
+        if (g.qs.bits > 0) rq = row_quant(g.qs, vmax, vmin, good);
+        // the target buffer is needed only now (the second product of the tile two back has read it)
+        if (!tc_wait(&aux->cfree[cb], par2 ^ 1u, abort_flag)) { ok = false; timeout_site = 31; break; }
+        if (tr_epi) TCB_TR(it, TCB_EV_EPI_CFREE);
         const bool live = (g.qs.bits == 0) ? good : (rq.inv > 0.f);
         float acc_t = 0.f;
 #pragma unroll 1
@@ -447,6 +415,15 @@ tcb_step_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
       if (!ok) break;
+      if (half == 0) {                               // rows skipped in this problem (counted once per row)
+        int wsk = skipped, wnf = nonfinite;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { wsk += __shfl_xor_sync(0xffffffffu, wsk, o); wnf |= __shfl_xor_sync(0xffffffffu, wnf, o); }
+        if (lane == 0) {
+          if (wsk) atomicAdd(reinterpret_cast<unsigned long long*>(&g.st[p].step_skipped), (unsigned long long)wsk);
+          if (wnf) atomicOr(&g.st[p].status_flags, STATUS_FLAG_NONFINITE);
+        }
+      }
       // The problem's cross-covariance: TMEM accumulator -> += global fp32 M (row r of M = feature r of X^T).  With two
       // groups, the one that owned the problem's last tile writes all of it out (each warp 32 rows x 64 columns) while
       // the other goes straight on to the next problem's first tile, so the second products resume as soon as the
