@@ -569,15 +569,6 @@ def main():
                 stage[slot].view(torch.int16).copy_(host[i % n_batches], non_blocking=True)
                 ready[slot].record(copy_stream)
 
-        total_b = K * cyc
-        D.barrier(g)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t_wall = time.perf_counter()
-        e0.record()
-        issued = 0
-        while issued < min(ring, total_b):
-            enqueue_copy(issued); issued += 1
         # the cycle's result (objective sum and token count) goes to page-locked host memory through the stream and is
         # looked at one cycle later, so the read never drains the queue
         res_j = [torch.zeros(1, dtype=torch.float64).pin_memory() for _ in range(2)]
@@ -589,6 +580,15 @@ def main():
             res_ev[c % 2].synchronize()
             objective_log.append((float(res_j[c % 2][0]), int(res_n[c % 2][0])))
 
+        total_b = K * cyc
+        D.barrier(g)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_wall = time.perf_counter()
+        e0.record()
+        issued = 0
+        while issued < min(ring, total_b):
+            enqueue_copy(issued); issued += 1
         for i in range(total_b):
             slot = i % ring
             main_stream.wait_event(ready[slot])
