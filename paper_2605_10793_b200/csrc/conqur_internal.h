@@ -37,9 +37,12 @@ struct DevState {
   int ns_idx;               // next entry of the polynomial schedule
   int seg_x;                // tensor-core mode: passes of the next-iterate product of the step in flight (1 or 2)
   int seg_e;                // tensor-core mode: passes of the next residual product (1 while the iterate is tiny, else 3)
-  // How many lifting steps an update starts with is learnt per problem from the updates before it (bisection between
-  // the largest count that fell short and the smallest that sufficed); see ns_adapt_lift_plan.
-  int lift_init, lift_plan, lift_lo, lift_hi;
+  // How many lifting steps an update starts with is learnt per problem from the updates before it: the count that
+  // keeps the running mean of the steps spent beyond plan + endgame below one; see ns_adapt_lift_plan.
+  int lift_init, lift_plan;
+  int lift_succ, lift_patience;   // updates in a row that needed no extra step / how many of them before one step fewer is tried
+  int lift_trial;                 // updates left of the trial period after such a descent
+  float lift_ema;                 // running mean of the extra steps at the current count
   int loop_passes;          // passes of the update graph's loop body in the update in flight
   long long loop_passes_total;   // ... since init (launch accounting)
   int lift_left;            // lifting steps still to run in the update in flight

@@ -535,7 +535,10 @@ static __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restri
 
 // Arm the lifting phase of an update: the count learnt so far, or the planned one on a problem's first update.
 __device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
-  if (!s->lift_init) { s->lift_plan = n_lift_init; s->lift_lo = -1; s->lift_hi = 127; s->lift_init = 1; }
+  if (!s->lift_init) {
+    s->lift_plan = n_lift_init; s->lift_succ = 0; s->lift_patience = 3; s->lift_trial = 0; s->lift_ema = 0.f;
+    s->lift_init = 1;
+  }
   s->lift_left = s->lift_plan;
   s->reentries = 0;
   s->loop_passes = 0;
@@ -543,28 +546,54 @@ __device__ __forceinline__ void ns_arm_lifting(DevState* s, int n_lift_init) {
   s->growth = 1.0f;
 }
 
-// After an update has converged in `steps_used` steps: learn how many lifting steps the next one should start with.
-// The plan was lift_plan lifting + n_endgame endgame steps.  Converging within it proves lift_plan sufficient; needing
-// more proves it short (the extra steps were the slower continuation of the endgame, so nothing is lost but time).
-// The count moves inside the bracket between the largest count known short and the smallest known sufficient; when
-// conditions change and a count that used to suffice falls short, the bracket reopens upwards.
+// After an update: learn how many lifting steps the next one should start with.  The plan was lift_plan lifting +
+// n_endgame endgame steps; an update that needed `extra` more ran them as the slower continuation of the endgame
+// (nothing is lost but time).  Measured on streams of the workloads, steps(count) is count + n_endgame once the count
+// suffices and erratic below (one lifting step short costs between nothing and five extra steps, depending on the
+// matrix), and which count suffices wanders by one or two from update to update.  One lifting step more costs exactly
+// one step per update, so the count that minimises the mean is the smallest whose mean shortfall stays below one:
+//   * the running mean of `extra` at the current count (weight 1/4 on the newest) above 1: one step more (at once by
+//     (extra + 1) / 2 when the count is far too short, extra >= 6);
+//   * lift_patience updates in a row without an extra step and a mean below 1/4: try one step fewer.  If the mean
+//     then exceeds 1 within the next 8 updates the descent did not pay: back up, and wait max(2, extra) times as
+//     long before the next try.
+// Before the first shortfall of a problem the count comes down by thirds per update (the planned count assumes a bound
+// on the smallest singular value that is usually far too pessimistic); the first shortfall ends that phase.
 __device__ __forceinline__ void ns_adapt_lift_plan(DevState* s, int n_endgame, int converged) {
   const int plan = s->lift_plan;
-  if (!converged) { s->lift_plan = min(plan + 2, 60); s->lift_lo = plan; s->lift_hi = 127; return; }
-  const int extra = s->ns_steps_used - (plan + n_endgame);
-  if (extra <= 0) {
-    s->lift_hi = min(s->lift_hi, plan);
-  } else {
-    s->lift_lo = max(s->lift_lo, plan);
-    if (s->lift_hi <= s->lift_lo) s->lift_hi = 127;
+  if (!converged) {
+    s->lift_plan = min(plan + 2, 60); s->lift_ema = 0.f; s->lift_succ = 0; s->lift_trial = 0;
+    return;
   }
-  // falling short costs about three steps per missing lifting step, one lifting step too many costs one: descend in
-  // thirds of the bracket, climb at once
-  int next;
-  if (s->lift_hi == 127) next = plan + max(1, (extra + 1) / 2);
-  else if (s->lift_hi - s->lift_lo > 1) next = s->lift_hi - max(1, (s->lift_hi - s->lift_lo - 1) / 3);
-  else next = s->lift_hi;
-  s->lift_plan = min(max(next, 0), 60);
+  const int extra = max(s->ns_steps_used - (plan + n_endgame), 0);
+  s->lift_ema = 0.75f * s->lift_ema + 0.25f * (float)extra;
+  s->lift_succ = extra == 0 ? s->lift_succ + 1 : 0;
+  if (s->lift_init == 1) {
+    // no update of this problem has fallen short yet: the planned count came from an assumed bound on the smallest
+    // singular value, usually far too pessimistic; come down by thirds until one does
+    // (lift_succ holds the last count that sufficed while this phase lasts)
+    if (extra == 0) {
+      s->lift_succ = plan;
+      s->lift_plan = plan > 0 ? plan - max(1, (plan + 1) / 3) : 0;
+      s->lift_ema = 0.f;
+      return;
+    }
+    s->lift_init = 2;
+    s->lift_plan = min(min(plan + max(1, (extra + 1) / 2), s->lift_succ > plan ? s->lift_succ : 60), 60);
+    s->lift_ema = 0.f; s->lift_succ = 0;
+    return;
+  }
+  const bool trial = s->lift_trial > 0;
+  if (trial) s->lift_trial -= 1;
+  if (s->lift_ema > 1.0f) {
+    const int up = (trial || extra < 6) ? 1 : (extra + 1) / 2;
+    s->lift_plan = min(plan + up, 60);
+    s->lift_ema = 0.f; s->lift_succ = 0; s->lift_trial = 0;
+    if (trial) s->lift_patience = min(128, s->lift_patience * max(2, extra));
+  } else if (s->lift_succ >= s->lift_patience && s->lift_ema < 0.25f && plan > 0) {
+    s->lift_plan = plan - 1;
+    s->lift_ema = 0.f; s->lift_succ = 0; s->lift_trial = 8;
+  }
 }
 
 // phase 0: lam = prior_rel * ||M_raw||_F / sqrt(d)      (reads partials of sumsq over M)
