@@ -293,3 +293,31 @@ def test_update_recovers_when_the_learnt_lifting_count_is_far_too_short(mode):
     assert st.ns_steps_used > steps[-1] and st.ns_lift_plan > plans[-1], (st.ns_steps_used, st.ns_lift_plan)
     rep = update_parity(m32.astype(np.float64), ctx.get_R().cpu().numpy().astype(np.float64))
     assert rep["orth"] <= TOL[mode]["orth"] and rep["gap"] <= TOL[mode]["gap"], (rep["orth"], rep["gap"], st.ns_steps_used)
+
+
+def test_lifting_count_comes_down_again_after_a_hard_update():
+    """One badly conditioned cross-covariance must not fix the lifting count for good: the count goes up for it, and
+    when the updates that follow need no extra steps it comes down again, one step at a time (every rotation on the
+    way passes the orthogonality gate)."""
+    from paper_2605_10793_b200 import binding as B
+    torch = _torch()
+    d = 256
+    rng = np.random.default_rng(11)
+    u, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    v, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    easy = torch.from_numpy(((u * np.linspace(1.0, 0.3, d)) @ v.T).astype(np.float32)).cuda()
+    hard = torch.from_numpy(((u * np.concatenate([np.ones(8), np.logspace(-3, -7, d - 8)])) @ v.T).astype(np.float32)).cuda()
+    ctx = B.Context(d=d, n_max=128, in_dtype="bf16", mode="tc")
+
+    def run(m):
+        ctx.set_M(m, 1.0, d)
+        ctx.update()
+        st = ctx.get_stats()
+        assert st.status == 0 and st.orth_err <= TOL["tc"]["orth"], (st.status, st.orth_err)
+        return st.ns_lift_plan, st.ns_steps_used
+
+    low = [run(easy) for _ in range(6)][-1][0]
+    peak = max(run(hard)[0] for _ in range(3))
+    assert peak >= low + 3, (low, peak)
+    plans = [run(easy)[0] for _ in range(24)]
+    assert plans[-1] <= peak - 3 and all(b <= a for a, b in zip(plans, plans[1:])), (low, peak, plans)
