@@ -3,25 +3,24 @@
 // A CTA owns one problem at a time and walks its tokens in tiles of 128 rows.  Per tile
 //   TMA            X tile (128 tokens x 128, bf16)              -> shared memory (read ONCE from HBM)
 //   tcgen05.mma    Y = X_tile R                                 -> TMEM          (R: bf16, resident in shared memory)
-//   epilogue       row norms from the X tile, sign / fake-quant of Y, objective partial,
-//                  C' = sgn(.) * rnorm as bf16                   -> shared memory
+//   epilogue       the rows' scales from a pass over Y (||x R~||, see the kernel), sign / fake-quant of Y,
+//                  C' = sgn(.) * scale as bf16                   -> shared memory
 //   tcgen05.mma    M += X_tile^T C'                              -> TMEM accumulator that lives for the whole problem
 // and after the last tile the accumulator is added to the problem's fp32 M in global memory.  The X tile in
-// shared memory serves three times: K-major operand of the first product, source of the row norms, MN-major
-// operand of the second product.  Rows with a zero or non-finite norm are zeroed in shared memory before the
-// second product so that they cannot reach M.
+// shared memory serves twice: K-major operand of the first product, MN-major operand of the second.  Rows with a
+// zero or non-finite scale are zeroed in shared memory before the second product so that they cannot reach M.
 //
 // Warp roles: 0 = TMA producer, 1 = issuer of the first product and TMEM owner, 2..17 = epilogue: two groups of
 // eight warps (two per TMEM lane quarter, one per half of the 128 columns) that take alternate tiles, so that one
-// group's waits and TMEM / shared-memory latencies overlap the other group's work; 18..21 = row norms (32 rows of
-// the tile each, beside the first product); 22 = issuer of the second product.  The two products have their own
-// issuing threads and Y has three TMEM buffers, so the first product runs up to three tiles ahead of the
-// epilogue.  Shared-memory bandwidth sets the floor of a tile: both products read both operands from it
-// (4 x 32 KB), TMA writes 32 KB, the norms read and the targets write 32 KB each.  Every wait is bounded.
+// group's waits and TMEM / shared-memory latencies overlap the other group's work; 18 = issuer of the second
+// product.  The two products have their own issuing threads and Y has three TMEM buffers, so the first product runs
+// up to three tiles ahead of the epilogue.  Shared-memory bandwidth sets the floor of a tile: both products read
+// both operands from it (4 x 32 KB), TMA writes 32 KB and the targets 32 KB.  Every wait is bounded.
 //
-// Objective without fake-quantisation: sum_i ||y_i||_1 rnorm_i = <R, X_tilde^T S> (Section 3.2 with Eq. 2), so it is
-// taken once per problem from the cross-covariance accumulator on its way out instead of summing |y| element by
-// element in the epilogue.
+// Objective without fake-quantisation: sum_i ||y_i||_1 rnorm_i = <R, X_tilde^T S> = <R, M> while R is fixed (Section
+// 3.2 with Eq. 2), so this kernel does not sum it: the update kernel forms it from M, and so does a read in between.
+// At the end of a problem the accumulator leaves through the copy engine (tensor reduce-add into M), handed over by
+// the epilogue group that owned the last tile while the other group goes on with the next problem.
 #pragma once
 #include <type_traits>
 
